@@ -1,0 +1,273 @@
+"""Pins for the oracle's basis fit, bit allocation, rate accounting and attention (CPU only)."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import spectra_inputs as si
+from oracle import codec, fit
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _tiny_side(side, n=1024):
+    wl = si.WORKLOADS["tiny"]
+    return si.draw_unit(wl, 0, 0, side, 0, n_tokens=n).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------- basis
+
+@pytest.mark.parametrize("mode", [fit.GAIN_ROTATE, fit.GAIN_SQRT, fit.GAIN_WHITEN])
+def test_basis_is_orthonormal_and_diagonalises(mode):
+    X = _tiny_side(si.SIDE_K)
+    f = fit.fit_basis(X, mode)
+    U, lam, C = f["U"], f["lam"], f["C"]
+    d = U.shape[0]
+    assert np.abs(U.T @ U - np.eye(d)).max() <= 1e-10
+    off = U.T @ C @ U - np.diag(lam)
+    assert np.abs(off).max() <= 1e-12 * np.abs(C).max() * d
+    assert (np.diff(lam) <= 1e-15 * lam[0]).all()
+    assert np.abs(f["W_enc"] @ f["W_dec"] - np.eye(d)).max() <= 1e-10
+    # each eigenvector's largest component is positive (sign convention)
+    assert (U[np.argmax(np.abs(U), axis=0), np.arange(d)] > 0).all()
+
+
+def test_basis_recovers_a_constructed_spectrum():
+    """X = sqrt(N) diag(sqrt(lam)) Q^T with N = d has X^T X / N = Q diag(lam) Q^T exactly."""
+    rng = np.random.default_rng(2)
+    d = 32
+    q, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    lam = np.sort(rng.random(d) + 0.05)[::-1] * np.arange(d, 0, -1)
+    X = np.sqrt(d) * np.sqrt(lam)[:, None] * q.T
+    f = fit.fit_basis(X, fit.GAIN_ROTATE)
+    assert np.allclose(f["lam"], lam, rtol=1e-10)
+    # eigenvectors equal the columns of Q up to sign
+    assert np.allclose(np.abs(f["U"].T @ q), np.eye(d), atol=1e-8)
+
+
+def test_latent_second_moment_identity_eq4():
+    """Eq. 4: with the square-root split the uncentred latent Y = X W_enc has Y^T Y / N = diag(sqrt(lam))."""
+    X = _tiny_side(si.SIDE_K)
+    f = fit.fit_basis(X, fit.GAIN_SQRT)
+    Y = X @ f["W_enc"]
+    S = Y.T @ Y / X.shape[0]
+    target = np.sqrt(f["lam"])
+    assert np.abs(S - np.diag(target)).max() <= 1e-9 * target[0]
+    # centred variances and means are the measured ones
+    Yc = Y - f["m_rot"][None, :]
+    assert np.allclose(Yc.mean(axis=0), 0, atol=1e-9)
+    assert np.allclose(Yc.var(axis=0), f["v_alloc"], rtol=1e-8, atol=1e-12)
+
+
+def test_whitening_split_gives_unit_variance():
+    X = _tiny_side(si.SIDE_V)
+    f = fit.fit_basis(X, fit.GAIN_WHITEN)
+    Yc = X @ f["W_enc"] - f["m_rot"][None, :]
+    assert np.allclose(Yc.var(axis=0), 1.0, rtol=1e-8)
+
+
+@pytest.mark.parametrize("mode", [fit.GAIN_ROTATE, fit.GAIN_SQRT, fit.GAIN_WHITEN])
+def test_score_is_invariant_under_the_shared_rotation(mode):
+    """q k^T = q' c^T with q' = W_dec q (appendix "Latent-space attention"), for every split of the spectrum."""
+    X = _tiny_side(si.SIDE_K, 256)
+    f = fit.fit_basis(X, mode)
+    rng = np.random.default_rng(4)
+    q = rng.standard_normal((5, X.shape[1]))
+    c = X @ f["W_enc"]                        # uncentred latent = (y + m')
+    qp = q @ f["W_dec"].T
+    a = q @ X.T
+    b = qp @ c.T
+    assert np.abs(a - b).max() <= 1e-10 * np.abs(a).max()
+
+
+def test_rotation_round_trip_through_fp32_matrices():
+    X = _tiny_side(si.SIDE_K, 64)
+    f = fit.fit_basis(_tiny_side(si.SIDE_K), fit.GAIN_SQRT)
+    we, wd, mr = f["W_enc"].astype(np.float32), f["W_dec"].astype(np.float32), f["m_rot"].astype(np.float32)
+    y = np.stack([codec.rotate_token(x, we, mr) for x in X.astype(np.float32)])
+    # independent fp64 statement of the same product
+    y_ref = X.astype(np.float32).astype(np.float64) @ we.astype(np.float64) - mr.astype(np.float64)
+    assert np.abs(y - y_ref).max() <= 1e-6 * np.abs(y_ref).max()
+    back = (y.astype(np.float64) + mr) @ wd.astype(np.float64)
+    assert np.abs(back - X).max() <= 2e-5 * np.abs(X).max()
+
+
+# ----------------------------------------------------------------------------- allocation
+
+def test_allocation_worked_example_from_eq5():
+    """v = [256, 16, 16, 1], mean rate 2: GM = 16, b = 2 + 0.5 log2(v / 16) = [4, 2, 2, 0]."""
+    v = np.array([256.0, 16.0, 16.0, 1.0])
+    assert np.allclose(fit.waterfill_closed_form(v, 2.0, 8), [4, 2, 2, 0])
+    assert list(fit.alloc_bits(v, 8, b_max=8)) == [4, 2, 2, 0]
+
+
+def test_allocation_matches_exhaustive_search():
+    rng = np.random.default_rng(9)
+    for _ in range(60):
+        v = (rng.random(4) ** 3 * 100 + 1e-6).astype(np.float32)
+        btot = int(rng.integers(0, 9))
+        b = fit.alloc_bits(v, btot, b_max=4)
+        assert b.sum() == min(btot, 16)
+        best = min((sum(float(v[j]) * 4.0 ** -c[j] for j in range(4)))
+                   for c in itertools.product(range(5), repeat=4) if sum(c) == min(btot, 16))
+        got = sum(float(v[j]) * 4.0 ** -int(b[j]) for j in range(4))
+        assert got <= best * (1 + 1e-12)
+
+
+def test_allocation_structure_on_a_decaying_spectrum():
+    d = 128
+    v = (np.arange(1, d + 1) ** -1.5).astype(np.float32)
+    for ratio in (4.0, 8.0, 12.0):
+        btot = fit.total_bits(d, ratio)
+        b = fit.alloc_bits(v, btot).astype(np.int64)
+        assert b.sum() == btot and b.max() <= 8
+        assert (np.diff(b) <= 0).all()                       # non-increasing along the energy order
+        dist = v.astype(np.float64) * 4.0 ** -b
+        # discrete water level: nobody below b_max would gain more from a bit than a holder would lose
+        assert dist[b < 8].max() <= 4 * dist[b > 0].min() * (1 + 1e-12)
+        # within one bit of the real-valued closed form (Eq. 5 with the clamp)
+        closed = fit.waterfill_closed_form(v, btot / d, 8)
+        inner = (closed > 0) & (closed < 8)
+        assert np.abs(b - closed)[inner].max() < 1.0
+    assert (fit.alloc_bits(v, fit.total_bits(d, 12.0)) == 0).any()   # the tail is dropped at low rate
+    assert fit.total_bits(128, 12.0) == 170 and fit.total_bits(128, 4.0) == 512 and fit.total_bits(128, 8.0) == 256
+
+
+def test_allocation_width_groups_and_clamp():
+    v = (np.arange(1, 129) ** -2.0).astype(np.float32)
+    b = fit.alloc_bits(v, 256, width_group=64)
+    assert len(set(b[:64])) == 1 and len(set(b[64:])) == 1 and b.sum() == 256 and b[0] >= b[64]
+    b = fit.alloc_bits(v, 256, width_group=2)
+    assert (b[0::2] == b[1::2]).all() and b.sum() == 256
+    assert list(fit.alloc_bits(np.ones(4), 100, b_max=8)) == [8, 8, 8, 8]
+    assert list(fit.alloc_bits(np.array([1.0, 1.0, 1.0, 1.0]), 2)) == [1, 1, 0, 0]     # ties: lowest index first
+
+
+# ----------------------------------------------------------------------------- rate accounting (paper's printed numbers)
+
+def _golden_lines(kind):
+    with open(os.path.join(GOLDEN, "paper_rate_accounting.txt")) as f:
+        return [line.split()[1:] for line in f if line.startswith(kind + " ")]
+
+
+def _printed(s):
+    return float(s[:-1]) * (1e3 if s.endswith("k") else 1e6)
+
+
+def test_effective_ratios_printed_in_the_paper():
+    for bits, g, printed in _golden_lines("ratio"):
+        widths = np.full(128, int(bits), np.uint8)
+        r = fit.effective_ratio(widths, int(g))
+        assert round(r, 2) == float(printed)
+    # zero-bit groups store nothing, not even metadata
+    w = np.zeros(128, np.uint8)
+    w[:64] = 4
+    assert fit.effective_bits_per_element(w, 64) == (64 * 4 + 32) / 128
+
+
+def test_capacity_table_printed_in_the_paper():
+    for layers, heads, hd, nbytes in _golden_lines("dense_bytes_per_token"):
+        assert int(layers) * int(heads) * int(hd) * 2 * 2 == int(nbytes)     # K and V, 2 bytes each
+    rows = _golden_lines("capacity")
+    assert len(rows) == 20
+    for budget, ratio, printed in rows:
+        got = fit.max_context_tokens(float(budget), float(ratio))
+        want = _printed(printed)
+        digits = 3 if want >= 1e5 else 2           # the table prints 2-3 significant digits
+        assert abs(got - want) <= 0.5 * 10 ** (np.floor(np.log10(want)) - digits + 1) * 1.0001
+
+
+# ----------------------------------------------------------------------------- attention
+
+def _coded_tiny(ratio=4.0, mode=fit.GAIN_SQRT, n=384, widths_override=None):
+    wl = si.WORKLOADS["tiny"]
+    out = {}
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        X = si.draw_unit(wl, 0, 0, side, 0)
+        f = fit.fit_basis(X.astype(np.float64), mode)
+        widths = fit.alloc_bits(f["v_alloc"], fit.total_bits(128, ratio)) if widths_override is None else \
+            np.full(128, widths_override, np.uint8)
+        tb = codec.tile_bytes(widths, 64)
+        cache = np.zeros(((n + 127) // 128) * tb, np.uint8)
+        we, wd, mr = (f[k].astype(np.float32) for k in ("W_enc", "W_dec", "m_rot"))
+        st, _ = codec.encode_unit(X[:n], we, mr, widths, 64, side, 0, cache, tb)
+        assert st == 0
+        out[name] = dict(X=X[:n], widths=widths, tb=tb, cache=cache, we=we, wd=wd, mr=mr)
+    return out
+
+
+def _attend(c, q, mode, n):
+    k, v = c["k"], c["v"]
+    return codec.attention_units(mode, q[None], [n], k["cache"], [0], [k["tb"]], v["cache"], [0], [v["tb"]],
+                                 k["wd"][None], k["mr"][None], k["widths"][None], v["wd"][None], v["mr"][None],
+                                 v["widths"][None], 64, 1.0 / np.sqrt(128.0))
+
+
+@pytest.mark.parametrize("mode", [fit.GAIN_ROTATE, fit.GAIN_SQRT, fit.GAIN_WHITEN])
+def test_latent_attention_equals_reconstruct_then_attend(mode):
+    n = 300                                      # ragged: two full tiles and a partial one
+    c = _coded_tiny(4.0, mode, n)
+    q = si.draw_queries(si.WORKLOADS["tiny"], 0, 0).astype(np.float64)
+    oa, la = _attend(c, q, "A", n)
+    ob, lb = _attend(c, q, "B", n)
+    assert np.abs(oa - ob).max() <= 1e-10 * np.abs(oa).max()
+    assert np.abs(la - lb).max() <= 1e-10
+
+
+def test_attention_at_eight_bits_matches_dense_textbook_attention():
+    n = 256
+    c = _coded_tiny(4.0, fit.GAIN_WHITEN, n, widths_override=8)
+    q = si.draw_queries(si.WORKLOADS["tiny"], 0, 0).astype(np.float64)
+    oa, la = _attend(c, q, "A", n)
+    K, V = c["k"]["X"].astype(np.float64), c["v"]["X"].astype(np.float64)
+    s = q @ K.T / np.sqrt(128.0)
+    p = np.exp(s - s.max(axis=1, keepdims=True))
+    lse = np.log(p.sum(axis=1)) + s.max(axis=1)
+    p /= p.sum(axis=1, keepdims=True)
+    assert np.allclose(p.sum(axis=1), 1.0)
+    dense = p @ V
+    assert np.abs(oa[0] - dense).max() <= 2e-2 * np.abs(dense).max()
+    assert np.abs(la[0] - lse).max() <= 5e-2
+
+
+def test_reconstruction_error_shrinks_with_rate_and_respects_step():
+    errs = []
+    for ratio in (12.0, 8.0, 4.0):
+        c = _coded_tiny(ratio, fit.GAIN_SQRT, 256)
+        k = c["k"]
+        _, xhat = codec.decode_unit(k["cache"], k["tb"], 256, k["wd"], k["mr"], k["widths"], 64, codec.SIDE_K)
+        errs.append(np.linalg.norm(xhat - k["X"]) / np.linalg.norm(k["X"]))
+    assert errs[0] > errs[1] > errs[2]
+    assert errs[2] < 0.1
+
+
+def test_importance_allocation_beats_uniform_at_low_rate():
+    """Observation 2, qualitatively: at 2 bits per channel, water-filled widths give a lower attention-output
+    error than uniform widths on the same data."""
+    n = 384
+    q = si.draw_queries(si.WORKLOADS["tiny"], 0, 0).astype(np.float64)
+    dense = _attend(_coded_tiny(4.0, fit.GAIN_WHITEN, n, widths_override=8), q, "A", n)[0]
+    wf = _attend(_coded_tiny(8.0, fit.GAIN_WHITEN, n), q, "A", n)[0]
+    un = _attend(_coded_tiny(8.0, fit.GAIN_WHITEN, n, widths_override=2), q, "A", n)[0]
+    assert np.linalg.norm(wf - dense) < np.linalg.norm(un - dense)
+
+
+def test_split_merge_of_partial_softmax_equals_unsplit():
+    """The log-sum-exp merge of partial (max, sum, accumulator) triples over any partition of the sequence
+    gives the unsplit softmax-weighted sum (textbook identity used by the sequence split)."""
+    rng = np.random.default_rng(21)
+    s = rng.standard_normal(1000) * 4
+    v = rng.standard_normal((1000, 8))
+    p = np.exp(s - s.max())
+    whole = (p[:, None] * v).sum(0) / p.sum()
+    cuts = [0, 17, 300, 301, 640, 1000]
+    parts = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        m = s[a:b].max()
+        e = np.exp(s[a:b] - m)
+        parts.append((m, e.sum(), (e[:, None] * v[a:b]).sum(0)))
+    M = max(m for m, _, _ in parts)
+    l = sum(np.exp(m - M) * li for m, li, _ in parts)
+    o = sum(np.exp(m - M) * oi for m, _, oi in parts)
+    assert np.abs(o / l - whole).max() <= 1e-12
