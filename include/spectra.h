@@ -1,0 +1,207 @@
+/*
+ * libspectra -- SPECTRA KV-cache codec, data-parallel hot path, for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every pointer marked "device" is caller-owned device memory (any allocator);
+ * pointers marked "host" are ordinary host memory.  The library allocates nothing and keeps
+ * no state between calls.  All work is enqueued on `stream` (a cudaStream_t passed as void*,
+ * NULL = the legacy default stream) and the calls return without synchronising.  Arguments
+ * are validated on the host before anything is launched; a non-zero return value means that
+ * nothing was enqueued.  Data-dependent anomalies (non-finite input, metadata beyond the
+ * fp16 range) are OR-ed into a caller-supplied device status word, never trapped.
+ *
+ * Vocabulary (paper notation).  A unit is one (sequence, kv-head) of one layer; a side is its
+ * keys (K) or values (V).  d = head_dim = 128.  Per unit-side the codec holds a decorrelating
+ * transform fitted from the cache's own second moment (Sec. 3.1, Eq. 3-4):
+ *     W_enc [d, d] (rotate + gain), W_dec [d, d] (its inverse), m' [d] (rotated mean),
+ * and integer per-channel bit widths b_j in [0, b_max] from reverse water-filling (Sec. 3.2,
+ * Eq. 5).  A token x (row vector) is stored as codes of y = x W_enc - m'.
+ *
+ * Parameter sets.  Transforms and widths usually depend on (layer, kv-head) only and are
+ * shared by the sequences of a batch: calls take `n_param_sets`, and unit u uses parameter
+ * set (u % n_param_sets).  With units ordered [sequence][kv-head] and n_param_sets = number
+ * of kv-heads this is "one set per head".
+ *
+ * Quantiser (Sec. 3.2: per-token min/max per group, one fp16 zero-point and scale per token
+ * per group, zero-bit channels dropped).  For each token and each scale group G of
+ * `scale_group` adjacent channels, over the channels with b_j > 0 only, in IEEE fp32,
+ * round-to-nearest-even, one rounding per operation, nothing fused:
+ *     lo = min y_j, hi = max y_j
+ *     lo16 = fp16 round-down(clamp(lo, +-65504));  lo_f = float(lo16)
+ *     R16  = fp16 round-up(min(hi - lo_f, 65504)); R_f  = float(R16)
+ *     L_j = 2^b_j - 1;  code_j = 0 if R_f == 0 else clamp(rint((y_j - lo_f) * (L_j / R_f)), 0, L_j)
+ *     reconstruction: yhat_j = lo_f if R_f == 0 else (float(code_j) * (R_f / L_j)) + lo_f;  b_j == 0: yhat_j = 0
+ *
+ * Packed tile format v1 (128 consecutive tokens of one unit-side; tiles of a unit-side are
+ * contiguous, tile t of unit u starts at cache + unit_offset[u] + t * spectra_tile_bytes()):
+ *   - A width b is split into its binary digits, sub-fields of 8, 4, 2 or 1 bits
+ *     (7 -> 4,2,1; 6 -> 4,2; 5 -> 4,1; 3 -> 2,1); the sub-field of size w holds code bits
+ *     [s, s+w), s = b & (w-1).
+ *   - A strip is one sub-field of one channel for the 128 tokens: 16*w bytes, seen as 8*w
+ *     little-endian 16-bit half-words; the i-th token of a half-word sits at bits [i*w, i*w+w).
+ *   - Strips are stored by class w = 8, 4, 2, 1 and, inside a class, by ascending channel.
+ *   - K side: token t is in half-word n = t*w/16.  Consecutive strips of a class are paired;
+ *     a pair takes 32*w bytes and its 32-bit word n is (half-word n of the first strip) |
+ *     (half-word n of the second) << 16.  An odd last strip is stored alone, half-words in order.
+ *   - V side: token t = 32a + 16h + i (a < 4, h < 2, i < 16) is in 32-bit word q = a*w + i*w/16
+ *     of its strip, low (h = 0) or high (h = 1) half-word, at bits [(i*w) % 16, +w).
+ *   - Then, for each scale group with a non-zero-width channel, ascending: lo16[128], R16[128]
+ *     (little-endian fp16, token order).
+ *   - tile bytes = 16 * sum_j b_j + 512 * (number of active scale groups); always a multiple of 16.
+ *   The K-side pairing puts two channels of one token 16 bits apart in a word, the V-side order
+ *   puts two tokens of one channel 16 bits apart: what the tensor-core operand registers of the
+ *   score and of the value contraction need, respectively.
+ */
+#ifndef SPECTRA_H_
+#define SPECTRA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* return codes */
+#define SPECTRA_OK 0
+#define SPECTRA_INVALID_ARG 1
+#define SPECTRA_UNSUPPORTED 2
+#define SPECTRA_WORKSPACE_TOO_SMALL 3
+#define SPECTRA_CAPACITY 4
+#define SPECTRA_CUDA_ERROR 5
+
+/* element types of caller tensors */
+#define SPECTRA_F32 0
+#define SPECTRA_BF16 1
+
+#define SPECTRA_SIDE_K 0
+#define SPECTRA_SIDE_V 1
+
+/* spectra_encode flags */
+#define SPECTRA_ROTATED_INPUT 1 /* x already holds y = x W_enc - m' in fp32; the rotation is skipped */
+
+/* bits of the device status word */
+#define SPECTRA_STATUS_NONFINITE 1 /* a non-finite coordinate reached the quantiser */
+#define SPECTRA_STATUS_F16_RANGE 2 /* a group minimum or range was saturated to the fp16 range */
+#define SPECTRA_STATUS_WAIT_TIMEOUT 4 /* a bounded wait on an on-chip copy gave up; the results are invalid */
+
+#define SPECTRA_GAIN_ROTATE 0 /* gamma = 1: a pure rotation */
+#define SPECTRA_GAIN_SQRT 1   /* gamma_j = lambda_j^(-1/4): the paper's square-root split (Eq. 3) */
+#define SPECTRA_GAIN_WHITEN 2 /* gamma_j = var_j^(-1/2): the pure-whitening split of the paper's footnote */
+
+typedef struct spectra_config {
+  int32_t head_dim;       /* 128 (other values: SPECTRA_UNSUPPORTED) */
+  int32_t tile_tokens;    /* 128 */
+  int32_t scale_group;    /* channels sharing one (lo16, R16) per token: 32, 64 (paper default) or 128 */
+  int32_t width_group;    /* adjacent channels sharing one width in spectra_alloc_bits: power of two, 1..scale_group */
+  int32_t b_max;          /* largest width, 1..8 */
+  int32_t gain_mode;      /* SPECTRA_GAIN_* (used by spectra_fit_basis only) */
+  int32_t layout_version; /* 1 */
+} spectra_config;
+
+/* ------------------------------------------------------------------------------------------------
+ * spectra_fit_basis -- Sec. 3.1, Eq. 3-4 and the appendix "G-Weighted SVD", restated on cache vectors:
+ * the right singular basis of the whitened weight is the eigenbasis of the uncentred second moment of
+ * the produced keys, so per unit-side
+ *     C = X^T X / N, mu = mean(X)            (fp32 products, fp64 accumulation)
+ *     C = U diag(lambda) U^T, lambda descending, each eigenvector's largest component positive (fp64 Jacobi)
+ *     m = mu U, var_j = max(lambda_j - m_j^2, 0), gains gamma per cfg->gain_mode (floor 1e-12 lambda_1)
+ *     W_enc = U diag(gamma), W_dec = diag(1/gamma) U^T, m' = m * gamma,
+ *     var_alloc = var * gamma^2 (ROTATE, SQRT) or var (WHITEN)
+ * x: device, element type x_dtype; unit u, token t, channel i at x[u*stride_unit + t*stride_token + i]
+ *    (strides in elements).  n_tokens >= 1.
+ * Outputs (device, fp32): w_enc, w_dec, basis_u [n_units, d, d] row-major; mean_rot, var_alloc, eigval
+ *    [n_units, d].  basis_u and eigval may be NULL.
+ * workspace: device, at least spectra_fit_workspace_bytes(cfg, n_units) bytes, 16-byte aligned.
+ */
+int spectra_fit_basis(const spectra_config* cfg, const void* x, int x_dtype, int64_t n_units, int64_t n_tokens,
+                      int64_t stride_unit, int64_t stride_token, float* w_enc, float* w_dec, float* mean_rot,
+                      float* var_alloc, float* eigval, float* basis_u, void* workspace, size_t workspace_bytes,
+                      void* stream);
+size_t spectra_fit_workspace_bytes(const spectra_config* cfg, int64_t n_units);
+
+/* ------------------------------------------------------------------------------------------------
+ * spectra_alloc_bits -- Sec. 3.2, Eq. 5 and the appendix "Reverse water-filling derivation": integer
+ * widths minimising sum_j v_j 4^(-b_j) subject to sum_j b_j <= Btot = floor(16 d / ratio), 0 <= b_j <= b_max,
+ * with cfg->width_group adjacent channels sharing one width taken from the group's mean variance.
+ * Realised as greedy marginal return (one bit at a time to the group with the largest v_G 4^(-b_G),
+ * ties to the lowest index), which is the exact integer optimum of that objective.
+ * var_alloc: device fp32 [n_units, d].  widths: device uint8 [n_units, d].  ratio > 0.
+ */
+int spectra_alloc_bits(const spectra_config* cfg, const float* var_alloc, int64_t n_units, double ratio,
+                       uint8_t* widths, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * spectra_encode -- Sec. 3.2-3.3 (Mode A streaming: each token is down-projected, quantised per token at
+ * the group widths and appended).  Appends n_new tokens to each of n_units unit-sides: unit u gets tokens
+ * x[u*stride_unit + i*stride_token + 0..d) for i < n_new at cache positions pos0[u] + i.
+ * Token slots of a touched tile that lie before pos0[u] are preserved, slots after the last appended token
+ * are written as zero, so a tile needs no initialisation when its slot 0 is appended first.
+ * x: device; x_dtype SPECTRA_F32 or SPECTRA_BF16; with SPECTRA_ROTATED_INPUT x must be SPECTRA_F32.
+ * pos0: device int32 [n_units].  w_enc: device fp32 [n_param_sets, d, d]; mean_rot [n_param_sets, d];
+ * widths: device uint8 [n_param_sets, d].  cache: device; unit_offset: device int64 [n_units], byte offset
+ * of the unit-side's first tile, multiple of 16.  status_word: device int32, OR-ed with SPECTRA_STATUS_* bits,
+ * may be NULL.
+ * The caller guarantees capacity: every touched tile lies inside its buffer.
+ */
+int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dtype, int flags, int64_t n_units,
+                   int64_t n_param_sets, const int32_t* pos0, int32_t n_new, int64_t stride_unit,
+                   int64_t stride_token, const float* w_enc, const float* mean_rot, const uint8_t* widths,
+                   uint8_t* cache, const int64_t* unit_offset, int32_t* status_word, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * spectra_decode -- Sec. 3.3 (Mode A reconstruction): xhat = (yhat + m') W_dec for tokens [0, n_tokens[u])
+ * of every unit-side; fp32 accumulation.  out: device, out_dtype SPECTRA_F32 or SPECTRA_BF16, element
+ * (u, t, i) at out[u*stride_unit + t*stride_token + i].  n_tokens: device int32 [n_units];
+ * max_tokens (host value) bounds it.  yhat_out (device fp32, same strides, may be NULL) receives the
+ * dequantised rotated coordinates.
+ */
+int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
+                   int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
+                   const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out, int out_dtype,
+                   float* yhat_out, int64_t stride_unit, int64_t stride_token, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * spectra_decode_attention -- appendix "Latent-space attention and memory" (Mode B): one decode query per
+ * (sequence, query head) attends to the whole coded cache of its kv-head without reconstructing it:
+ *     q' = softmax_scale * W_dec,K q      (the up-projection folded into the query, once per call)
+ *     s_t = q' . yhat^K_t                 (codes unpacked and dequantised in registers; the constant
+ *                                          q' . m'_K is dropped from the softmax and restored in lse)
+ *     o' = sum_t softmax(s)_t yhat^V_t    (online softmax, rotated value space, sequence split across CTAs)
+ *     out = (o' + m'_V) W_dec,V           (one lift per query head)
+ * Units are ordered u = sequence * n_kv_heads + kv_head; query head hq belongs to kv-head hq / (n_q_heads /
+ * n_kv_heads).  q: device [batch, n_q_heads, d], q_dtype.  seq_len: device int32 [batch] (tokens attended,
+ * <= max_seq_len; 0 gives a zero output row and lse = -inf).  cache_k/v with unit_offset_k/v: as in
+ * spectra_encode.  Parameter arrays as in spectra_encode/decode ([n_param_sets, ...]); mean_rot_k is read
+ * only when lse != NULL and may be NULL otherwise.  softmax_scale 0 means 1/sqrt(d).
+ * out: device [batch, n_q_heads, d], out_dtype.  lse: device fp32 [batch, n_q_heads] or NULL.
+ * workspace: device, >= spectra_attention_workspace_bytes(...), 16-byte aligned; scratch only, nothing is
+ * carried between calls.  status_word: device int32 or NULL.
+ */
+int spectra_decode_attention(const spectra_config* cfg, const void* q, int q_dtype, int32_t batch,
+                             int32_t n_kv_heads, int32_t n_q_heads, const int32_t* seq_len, int32_t max_seq_len,
+                             const uint8_t* cache_k, const int64_t* unit_offset_k, const uint8_t* cache_v,
+                             const int64_t* unit_offset_v, int64_t n_param_sets, const float* w_dec_k,
+                             const float* mean_rot_k, const uint8_t* widths_k, const float* w_dec_v,
+                             const float* mean_rot_v, const uint8_t* widths_v, float softmax_scale, void* out,
+                             int out_dtype, float* lse, void* workspace, size_t workspace_bytes,
+                             int32_t* status_word, void* stream);
+size_t spectra_attention_workspace_bytes(const spectra_config* cfg, int32_t batch, int32_t n_kv_heads,
+                                         int32_t n_q_heads, int32_t max_seq_len);
+
+/* ------------------------------------------------------------------------------------------------
+ * Helpers (host only, no device work).
+ * spectra_tile_bytes: size of one packed tile for the given widths (host uint8 [d]); 0 on bad arguments.
+ * spectra_config_default: fills cfg with head_dim 128, tile 128, scale_group 64, width_group 1, b_max 8,
+ *   SPECTRA_GAIN_SQRT, layout 1.
+ * spectra_total_bits: Btot = floor(16 d / ratio) clamped to b_max * d.
+ * spectra_status_string: name of a return code.
+ */
+size_t spectra_tile_bytes(const spectra_config* cfg, const uint8_t* widths_host);
+void spectra_config_default(spectra_config* cfg);
+int32_t spectra_total_bits(const spectra_config* cfg, double ratio);
+const char* spectra_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECTRA_H_ */

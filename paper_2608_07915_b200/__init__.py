@@ -1,0 +1,157 @@
+"""Thin Python binding of libspectra (the C ABI declared in include/spectra.h).
+
+Argument marshalling only: torch tensors supply device memory and the current CUDA stream; every
+step of the codec runs in the library's CUDA kernels.  There is no fallback: if the shared
+library is missing the first call raises.
+"""
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libspectra.so")
+_lib = None
+
+OK, INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CAPACITY, CUDA_ERROR = range(6)
+F32, BF16 = 0, 1
+SIDE_K, SIDE_V = 0, 1
+ROTATED_INPUT = 1
+STATUS_NONFINITE, STATUS_F16_RANGE, STATUS_WAIT_TIMEOUT = 1, 2, 4
+GAIN_ROTATE, GAIN_SQRT, GAIN_WHITEN = 0, 1, 2
+HEAD_DIM = 128
+TILE_TOKENS = 128
+
+EXPORTS = [
+    "spectra_fit_basis", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
+    "spectra_decode_attention", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
+    "spectra_total_bits", "spectra_status_string",
+]
+
+
+class SpectraError(RuntimeError):
+    pass
+
+
+class Config(C.Structure):
+    _fields_ = [("head_dim", C.c_int32), ("tile_tokens", C.c_int32), ("scale_group", C.c_int32),
+                ("width_group", C.c_int32), ("b_max", C.c_int32), ("gain_mode", C.c_int32),
+                ("layout_version", C.c_int32)]
+
+
+def lib():
+    """Loads libspectra.so; raises if it has not been built (no fallback path exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise SpectraError(f"{_LIB_PATH} is missing: build it with `python -m paper_2608_07915_b200.build`")
+        _lib = C.CDLL(_LIB_PATH)
+        _lib.spectra_fit_workspace_bytes.restype = C.c_size_t
+        _lib.spectra_attention_workspace_bytes.restype = C.c_size_t
+        _lib.spectra_tile_bytes.restype = C.c_size_t
+        _lib.spectra_total_bits.restype = C.c_int32
+        _lib.spectra_status_string.restype = C.c_char_p
+        _lib.spectra_config_default.restype = None
+    return _lib
+
+
+def default_config(**overrides):
+    cfg = Config()
+    lib().spectra_config_default(C.byref(cfg))
+    for k, v in overrides.items():
+        setattr(cfg, k, int(v))
+    return cfg
+
+
+def status_string(code):
+    return lib().spectra_status_string(C.c_int(code)).decode()
+
+
+def _check(rc, what):
+    if rc != OK:
+        raise SpectraError(f"{what}: {status_string(rc)}")
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t):
+    import torch
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise SpectraError(f"unsupported tensor dtype {t.dtype}")
+
+
+def tile_bytes(cfg, widths_host):
+    """widths_host: 128 integers (any sequence).  Bytes of one packed tile."""
+    arr = (C.c_uint8 * HEAD_DIM)(*[int(w) for w in widths_host])
+    n = lib().spectra_tile_bytes(C.byref(cfg), arr)
+    if n == 0 and any(int(w) for w in widths_host):
+        raise SpectraError("spectra_tile_bytes: bad arguments")
+    return int(n)
+
+
+def total_bits(cfg, ratio):
+    return int(lib().spectra_total_bits(C.byref(cfg), C.c_double(ratio)))
+
+
+def fit_workspace_bytes(cfg, n_units):
+    return int(lib().spectra_fit_workspace_bytes(C.byref(cfg), C.c_int64(n_units)))
+
+
+def attention_workspace_bytes(cfg, batch, n_kv_heads, n_q_heads, max_seq_len):
+    return int(lib().spectra_attention_workspace_bytes(C.byref(cfg), C.c_int32(batch), C.c_int32(n_kv_heads),
+                                                       C.c_int32(n_q_heads), C.c_int32(max_seq_len)))
+
+
+def fit_basis(cfg, x, n_units, n_tokens, stride_unit, stride_token, w_enc, w_dec, mean_rot, var_alloc,
+              eigval=None, basis_u=None, workspace=None):
+    rc = lib().spectra_fit_basis(C.byref(cfg), _ptr(x), C.c_int(_dtype_code(x)), C.c_int64(n_units),
+                                 C.c_int64(n_tokens), C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(w_enc),
+                                 _ptr(w_dec), _ptr(mean_rot), _ptr(var_alloc), _ptr(eigval), _ptr(basis_u),
+                                 _ptr(workspace), C.c_size_t(0 if workspace is None else workspace.numel() *
+                                                             workspace.element_size()), _stream())
+    _check(rc, "spectra_fit_basis")
+
+
+def alloc_bits(cfg, var_alloc, n_units, ratio, widths):
+    rc = lib().spectra_alloc_bits(C.byref(cfg), _ptr(var_alloc), C.c_int64(n_units), C.c_double(ratio), _ptr(widths),
+                                  _stream())
+    _check(rc, "spectra_alloc_bits")
+
+
+def encode(cfg, side, x, flags, n_units, n_param_sets, pos0, n_new, stride_unit, stride_token, w_enc, mean_rot,
+           widths, cache, unit_offset, status_word=None):
+    rc = lib().spectra_encode(C.byref(cfg), C.c_int(side), _ptr(x), C.c_int(_dtype_code(x)), C.c_int(flags),
+                              C.c_int64(n_units), C.c_int64(n_param_sets), _ptr(pos0), C.c_int32(n_new),
+                              C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(w_enc), _ptr(mean_rot),
+                              _ptr(widths), _ptr(cache), _ptr(unit_offset), _ptr(status_word), _stream())
+    _check(rc, "spectra_encode")
+
+
+def decode(cfg, side, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec, mean_rot, widths, out,
+           yhat_out, stride_unit, stride_token):
+    out_code = _dtype_code(out) if out is not None else F32
+    rc = lib().spectra_decode(C.byref(cfg), C.c_int(side), _ptr(cache), _ptr(unit_offset), C.c_int64(n_units),
+                              C.c_int64(n_param_sets), _ptr(n_tokens), C.c_int32(max_tokens), _ptr(w_dec),
+                              _ptr(mean_rot), _ptr(widths), _ptr(out), C.c_int(out_code), _ptr(yhat_out),
+                              C.c_int64(stride_unit), C.c_int64(stride_token), _stream())
+    _check(rc, "spectra_decode")
+
+
+def decode_attention(cfg, q, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k, cache_v,
+                     unit_offset_v, n_param_sets, w_dec_k, mean_rot_k, widths_k, w_dec_v, mean_rot_v, widths_v,
+                     softmax_scale, out, lse, workspace, status_word=None):
+    rc = lib().spectra_decode_attention(
+        C.byref(cfg), _ptr(q), C.c_int(_dtype_code(q)), C.c_int32(batch), C.c_int32(n_kv_heads), C.c_int32(n_q_heads),
+        _ptr(seq_len), C.c_int32(max_seq_len), _ptr(cache_k), _ptr(unit_offset_k), _ptr(cache_v),
+        _ptr(unit_offset_v), C.c_int64(n_param_sets), _ptr(w_dec_k), _ptr(mean_rot_k), _ptr(widths_k), _ptr(w_dec_v),
+        _ptr(mean_rot_v), _ptr(widths_v), C.c_float(softmax_scale), _ptr(out), C.c_int(_dtype_code(out)), _ptr(lse),
+        _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()), _ptr(status_word), _stream())
+    _check(rc, "spectra_decode_attention")

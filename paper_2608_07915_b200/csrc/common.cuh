@@ -1,0 +1,150 @@
+// Shared device/host helpers of libspectra: configuration checks, the per-unit strip table that
+// describes a packed tile, and the mapping between (strip, token) and storage bits.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/spectra.h"
+
+namespace spectra {
+
+constexpr int kD = 128;          // head_dim
+constexpr int kTile = 128;       // tokens per tile
+constexpr int kMaxStrips = 384;  // 128 channels x at most 3 sub-fields
+constexpr int kMaxGroups = 4;    // scale groups per token (scale_group >= 32)
+
+inline int check_config(const spectra_config* c) {
+  if (!c) return SPECTRA_INVALID_ARG;
+  if (c->head_dim != kD || c->tile_tokens != kTile || c->layout_version != 1) return SPECTRA_UNSUPPORTED;
+  if (c->scale_group != 32 && c->scale_group != 64 && c->scale_group != 128) return SPECTRA_UNSUPPORTED;
+  if (c->b_max < 1 || c->b_max > 8) return SPECTRA_INVALID_ARG;
+  int wg = c->width_group;
+  if (wg < 1 || wg > c->scale_group || (wg & (wg - 1))) return SPECTRA_INVALID_ARG;
+  if (c->gain_mode < 0 || c->gain_mode > 2) return SPECTRA_INVALID_ARG;
+  return SPECTRA_OK;
+}
+
+inline int launch_status() { return cudaGetLastError() == cudaSuccess ? SPECTRA_OK : SPECTRA_CUDA_ERROR; }
+
+// Description of one unit-side's tile, built in shared memory from the 128 widths.
+// Strips are numbered in storage order: class 8 first, then 4, 2, 1; ascending channel inside a class.
+struct StripTable {
+  int n_strips;
+  int class_first[5];             // first strip index of class c (w = 8 >> c); class_first[4] = n_strips
+  int class_off[5];               // byte offset of the class region; class_off[4] = payload bytes
+  int n_groups;                   // d / scale_group
+  int n_act;                      // active scale groups
+  int meta_off[kMaxGroups];       // byte offset of lo16[128] of group g (R16 follows 256 bytes later), -1 if inactive
+  int tile_bytes;
+  uint8_t chan[kMaxStrips];
+  uint8_t shift[kMaxStrips];
+  uint8_t width[kD];
+};
+
+// Called by all threads of a CTA (at least one full warp); includes the closing __syncthreads().
+__device__ inline void build_strip_table(StripTable& T, const uint8_t* __restrict__ widths_global, int scale_group) {
+  const int tid = threadIdx.x;
+  if (tid < kD) T.width[tid] = widths_global[tid];
+  __syncthreads();
+  if (tid < 32) {
+    const int lane = tid;
+    int count = 0, off = 0;
+#pragma unroll
+    for (int c = 0; c < 4; c++) {
+      const int w = 8 >> c;
+      if (lane == 0) { T.class_first[c] = count; T.class_off[c] = off; }
+      int first = count;
+      for (int word = 0; word < kD / 32; word++) {
+        const int j = word * 32 + lane;
+        const int b = T.width[j];
+        const bool present = (b & w) != 0;
+        const unsigned m = __ballot_sync(0xffffffffu, present);
+        if (present) {
+          const int k = count + __popc(m & ((1u << lane) - 1u));
+          T.chan[k] = (uint8_t)j;
+          T.shift[k] = (uint8_t)(b & (w - 1));
+        }
+        count += __popc(m);
+      }
+      off += 16 * w * (count - first);
+    }
+    int n_groups = kD / scale_group;
+    int n_act = 0;
+    for (int g = 0; g < n_groups; g++) {
+      bool any = false;
+      for (int j = g * scale_group + lane; j < (g + 1) * scale_group; j += 32) any |= T.width[j] != 0;
+      const bool act = __any_sync(0xffffffffu, any);
+      if (lane == 0) T.meta_off[g] = act ? off + 512 * n_act : -1;
+      n_act += act ? 1 : 0;
+    }
+    if (lane == 0) {
+      T.n_strips = count; T.class_first[4] = count; T.class_off[4] = off;
+      T.n_groups = n_groups; T.n_act = n_act; T.tile_bytes = off + 512 * n_act;
+      for (int g = n_groups; g < kMaxGroups; g++) T.meta_off[g] = -1;
+    }
+  }
+  __syncthreads();
+}
+
+__device__ inline int strip_class(const StripTable& T, int k) {
+  return (k >= T.class_first[1]) + (k >= T.class_first[2]) + (k >= T.class_first[3]);
+}
+
+// Storage position of the field of token t in strip k: byte offset of its half-word and the bit inside it.
+__device__ inline void locate_field(const StripTable& T, int side, int k, int t, int& byte_off, int& bit) {
+  const int c = strip_class(T, k);
+  const int w = 8 >> c;
+  const int i_in = k - T.class_first[c];
+  const int cnt = T.class_first[c + 1] - T.class_first[c];
+  if (side == SPECTRA_SIDE_V) {
+    const int a = t >> 5, h = (t >> 4) & 1, i = t & 15;
+    byte_off = T.class_off[c] + 16 * w * i_in + 4 * (a * w + ((i * w) >> 4)) + 2 * h;
+    bit = (i * w) & 15;
+  } else {
+    const int n = (t * w) >> 4;
+    bit = (t * w) & 15;
+    if ((i_in | 1) < cnt) byte_off = T.class_off[c] + 32 * w * (i_in >> 1) + 4 * n + 2 * (i_in & 1);
+    else byte_off = T.class_off[c] + 16 * w * i_in + 2 * n;
+  }
+}
+
+// Inverse map: the half-word at payload byte offset `off` (even) belongs to strip k and holds the
+// 16/w tokens first_token + e * token_step... (always consecutive tokens): returns k (or -1), sets w and first token.
+__device__ inline int halfword_owner(const StripTable& T, int side, int off, int& w, int& first_token) {
+  int c = (off >= T.class_off[1]) + (off >= T.class_off[2]) + (off >= T.class_off[3]);
+  w = 8 >> c;
+  const int rel = off - T.class_off[c];
+  const int cnt = T.class_first[c + 1] - T.class_first[c];
+  const int per = 16 / w;  // tokens per half-word
+  if (side == SPECTRA_SIDE_V) {
+    const int i_in = rel / (16 * w);
+    const int r = rel - i_in * 16 * w;
+    const int q = r >> 2, h = (r >> 1) & 1;
+    const int a = q / w, m = q - a * w;
+    first_token = 32 * a + 16 * h + m * per;
+    return T.class_first[c] + i_in;
+  }
+  const int paired_bytes = 32 * w * (cnt >> 1);
+  if (rel < paired_bytes) {
+    const int p = rel / (32 * w);
+    const int r = rel - p * 32 * w;
+    first_token = (r >> 2) * per;
+    return T.class_first[c] + 2 * p + ((r >> 1) & 1);
+  }
+  first_token = ((rel - paired_bytes) >> 1) * per;
+  return T.class_first[c] + cnt - 1;
+}
+
+__device__ inline float load_as_float(const void* p, int dtype, int64_t idx) {
+  if (dtype == SPECTRA_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx]);
+  return reinterpret_cast<const float*>(p)[idx];
+}
+
+__device__ inline void store_from_float(void* p, int dtype, int64_t idx, float v) {
+  if (dtype == SPECTRA_BF16) reinterpret_cast<__nv_bfloat16*>(p)[idx] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(p)[idx] = v;
+}
+
+}  // namespace spectra

@@ -1,0 +1,310 @@
+// spectra_fit_basis (second-moment accumulation + fp64 Jacobi eigensolver + transform assembly) and
+// spectra_alloc_bits (greedy integer reverse water-filling).
+#include "common.cuh"
+
+namespace spectra {
+
+// ------------------------------------------------------------------------------------------------
+// Moments: S = sum_t x_t^T x_t and s = sum_t x_t.  Each CTA takes a chunk of tokens, forms the
+// chunk's products in fp32 (each thread an 8x8 block of S) and adds them to the fp64 totals.
+constexpr int kMomChunk = 256;
+
+struct FitWorkspace {   // per unit, all fp64
+  double S[kD * kD];
+  double VT[kD * kD];   // rows are eigenvectors (transposed so that plane rotations touch contiguous rows)
+  double s[kD];
+};
+
+__global__ void __launch_bounds__(256) moments_kernel(const void* x, int x_dtype, int64_t n_tokens,
+                                                      int64_t stride_unit, int64_t stride_token, FitWorkspace* ws) {
+  __shared__ float xs[32][kD + 4];
+  const int u = blockIdx.y;
+  const int64_t t_begin = (int64_t)blockIdx.x * kMomChunk;
+  const int64_t t_end = min(t_begin + (int64_t)kMomChunk, n_tokens);
+  const int tid = threadIdx.x;
+  const int r0 = (tid / 16) * 8, c0 = (tid % 16) * 8;
+  float acc[8][8];
+#pragma unroll
+  for (int a = 0; a < 8; a++)
+#pragma unroll
+    for (int b = 0; b < 8; b++) acc[a][b] = 0.f;
+  float colsum = 0.f;  // threads 0..127: sum of channel tid
+  for (int64_t t0 = t_begin; t0 < t_end; t0 += 32) {
+    __syncthreads();
+    for (int idx = tid; idx < 32 * kD; idx += blockDim.x) {
+      const int tt = idx / kD, i = idx - tt * kD;
+      xs[tt][i] = t0 + tt < t_end ? load_as_float(x, x_dtype, (int64_t)u * stride_unit + (t0 + tt) * stride_token + i)
+                                  : 0.f;
+    }
+    __syncthreads();
+    for (int tt = 0; tt < 32; tt++) {
+      float xr[8], xc[8];
+#pragma unroll
+      for (int a = 0; a < 8; a++) { xr[a] = xs[tt][r0 + a]; xc[a] = xs[tt][c0 + a]; }
+#pragma unroll
+      for (int a = 0; a < 8; a++)
+#pragma unroll
+        for (int b = 0; b < 8; b++) acc[a][b] = fmaf(xr[a], xc[b], acc[a][b]);
+      if (tid < kD) colsum += xs[tt][tid];
+    }
+  }
+  FitWorkspace& W = ws[u];
+#pragma unroll
+  for (int a = 0; a < 8; a++)
+#pragma unroll
+    for (int b = 0; b < 8; b++) atomicAdd(&W.S[(r0 + a) * kD + c0 + b], (double)acc[a][b]);
+  if (tid < kD) atomicAdd(&W.s[tid], (double)colsum);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Eigensolver: cyclic two-sided Jacobi in fp64, round-robin ordering (127 rounds of 64 disjoint
+// plane rotations per sweep), one CTA of 512 threads per matrix, matrix in shared memory.
+constexpr int kLdJ = kD + 1;
+constexpr int kMaxSweeps = 30;
+
+struct EigSmem {
+  double A[kD * kLdJ];
+  double c[64], s[64];
+  int pp[64], qq[64];
+  double red[16];
+  double lam[kD];
+  int order[kD];
+  double mu[kD], m[kD], gam[kD];
+};
+
+struct FitOut {
+  float* w_enc; float* w_dec; float* mean_rot; float* var_alloc; float* eigval; float* basis_u;
+  int gain_mode; int64_t n_tokens;
+};
+
+__device__ inline double block_sum_512(double v, double* red) {
+#pragma unroll
+  for (int s = 16; s; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int i = 0; i < 16; i++) t += red[i];
+  return t;
+}
+
+__global__ void __launch_bounds__(512, 1) eigen_kernel(FitWorkspace* ws, FitOut o) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  EigSmem& E = *reinterpret_cast<EigSmem*>(smem_raw);
+  const int u = blockIdx.x, tid = threadIdx.x;
+  FitWorkspace& W = ws[u];
+  const double inv_n = 1.0 / (double)o.n_tokens;
+  for (int idx = tid; idx < kD * kD; idx += 512) {
+    const int r = idx / kD, c = idx - r * kD;
+    // symmetrise: the two triangles were accumulated by different threads in the same order, but keep it exact
+    E.A[r * kLdJ + c] = 0.5 * (W.S[r * kD + c] + W.S[c * kD + r]) * inv_n;
+    W.VT[idx] = r == c ? 1.0 : 0.0;
+  }
+  if (tid < kD) E.mu[tid] = W.s[tid] * inv_n;
+  __syncthreads();
+  double fro = 0.0;
+  for (int idx = tid; idx < kD * kD; idx += 512) { const double v = E.A[(idx / kD) * kLdJ + idx % kD]; fro += v * v; }
+  fro = block_sum_512(fro, E.red);
+  const double tol2 = 1e-28 * fro;   // (1e-14 ||C||_F)^2
+
+  const int pair = tid >> 3, sub = tid & 7;
+  for (int sweep = 0; sweep < kMaxSweeps; sweep++) {
+    double off = 0.0;
+    for (int idx = tid; idx < kD * kD; idx += 512) {
+      const int r = idx / kD, c = idx - r * kD;
+      if (r != c) { const double v = E.A[r * kLdJ + c]; off += v * v; }
+    }
+    off = block_sum_512(off, E.red);
+    if (off <= tol2) break;
+    for (int round = 0; round < kD - 1; round++) {
+      if (tid < 64) {
+        int p, q;
+        if (tid == 0) { p = kD - 1; q = round; }
+        else { p = (round + tid) % (kD - 1); q = (round - tid + (kD - 1)) % (kD - 1); }
+        if (p > q) { const int t = p; p = q; q = t; }
+        const double app = E.A[p * kLdJ + p], aqq = E.A[q * kLdJ + q], apq = E.A[p * kLdJ + q];
+        double c = 1.0, s = 0.0;
+        if (apq != 0.0 && fabs(apq) > 1e-300) {
+          const double tau = (aqq - app) / (2.0 * apq);
+          const double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
+          c = 1.0 / sqrt(1.0 + t * t);
+          s = t * c;
+        }
+        E.c[tid] = c; E.s[tid] = s; E.pp[tid] = p; E.qq[tid] = q;
+      }
+      __syncthreads();
+      const int p = E.pp[pair], q = E.qq[pair];
+      const double c = E.c[pair], s = E.s[pair];
+      // rows: A <- J^T A ; eigenvector rows: VT <- J^T VT
+      for (int k = sub; k < kD; k += 8) {
+        const double ap = E.A[p * kLdJ + k], aq = E.A[q * kLdJ + k];
+        E.A[p * kLdJ + k] = c * ap - s * aq;
+        E.A[q * kLdJ + k] = s * ap + c * aq;
+        const double vp = W.VT[p * kD + k], vq = W.VT[q * kD + k];
+        W.VT[p * kD + k] = c * vp - s * vq;
+        W.VT[q * kD + k] = s * vp + c * vq;
+      }
+      __syncthreads();
+      // columns: A <- A J
+      for (int k = sub; k < kD; k += 8) {
+        const double ap = E.A[k * kLdJ + p], aq = E.A[k * kLdJ + q];
+        E.A[k * kLdJ + p] = c * ap - s * aq;
+        E.A[k * kLdJ + q] = s * ap + c * aq;
+      }
+      __syncthreads();
+    }
+  }
+  // ---- order eigenvalues (descending, ties by index), fix signs, assemble the transform
+  if (tid < kD) E.lam[tid] = E.A[tid * kLdJ + tid];
+  __syncthreads();
+  if (tid < kD) {
+    const double l = E.lam[tid];
+    int rank = 0;
+    for (int k = 0; k < kD; k++) rank += (E.lam[k] > l) || (E.lam[k] == l && k < tid);
+    E.order[rank] = tid;
+  }
+  __syncthreads();
+  if (tid < kD) {
+    // output column j = tid comes from Jacobi row order[j]
+    const int src = E.order[tid];
+    const double* v = W.VT + src * kD;
+    int kmax = 0; double amax = -1.0;
+    for (int k = 0; k < kD; k++) { const double a = fabs(v[k]); if (a > amax) { amax = a; kmax = k; } }
+    const double sign = v[kmax] < 0.0 ? -1.0 : 1.0;
+    double m = 0.0;
+    for (int k = 0; k < kD; k++) m += E.mu[k] * v[k];
+    m *= sign;
+    const double lam = fmax(E.lam[src], 0.0);
+    E.m[tid] = m;
+    E.gam[tid] = sign;            // stash the sign; replaced by the gain below
+    E.A[tid * kLdJ + tid] = lam;  // sorted eigenvalue j now on the diagonal slot j (diagonal no longer needed)
+  }
+  __syncthreads();
+  if (tid < kD) {
+    const double lam = E.A[tid * kLdJ + tid];
+    const double lam1 = E.A[0];
+    const double m = E.m[tid];
+    const double var = fmax(lam - m * m, 0.0);
+    const double floor_v = 1e-12 * lam1;
+    double g = 1.0;
+    if (o.gain_mode == SPECTRA_GAIN_SQRT) g = 1.0 / sqrt(sqrt(fmax(lam, floor_v)));
+    else if (o.gain_mode == SPECTRA_GAIN_WHITEN) g = 1.0 / sqrt(fmax(var, floor_v));
+    const double sign = E.gam[tid];
+    const int64_t base = (int64_t)u * kD;
+    o.mean_rot[base + tid] = (float)(m * g);
+    o.var_alloc[base + tid] = (float)(o.gain_mode == SPECTRA_GAIN_WHITEN ? var : var * g * g);
+    if (o.eigval) o.eigval[base + tid] = (float)lam;
+    const double* v = W.VT + E.order[tid] * kD;
+    const int64_t mb = (int64_t)u * kD * kD;
+    for (int k = 0; k < kD; k++) {
+      const double ukj = sign * v[k];                       // U[k][j], j = tid
+      o.w_enc[mb + k * kD + tid] = (float)(ukj * g);        // W_enc = U diag(gamma)
+      o.w_dec[mb + tid * kD + k] = (float)(ukj / g);        // W_dec = diag(1/gamma) U^T
+      if (o.basis_u) o.basis_u[mb + k * kD + tid] = (float)ukj;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Allocation: one warp per unit.  Lane l holds groups l, l+32, l+64, l+96 (when present).
+__global__ void __launch_bounds__(128) alloc_kernel(const float* __restrict__ var_alloc, int64_t n_units, int btot,
+                                                    int b_max, int wg, uint8_t* __restrict__ widths) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t u = (int64_t)blockIdx.x * 4 + warp;
+  if (u >= n_units) return;
+  const int ng = kD / wg;
+  double v[4];
+  int b[4];
+#pragma unroll
+  for (int r = 0; r < 4; r++) {
+    const int g = lane + 32 * r;
+    b[r] = 0; v[r] = -1.0;
+    if (g < ng) {
+      float acc = var_alloc[u * kD + g * wg];
+      for (int j = 1; j < wg; j++) acc = __fadd_rn(acc, var_alloc[u * kD + g * wg + j]);
+      v[r] = (double)(wg == 1 ? acc : __fdiv_rn(acc, (float)wg));
+    }
+  }
+  int steps = btot / wg;
+  if (steps > ng * b_max) steps = ng * b_max;
+  for (int it = 0; it < steps; it++) {
+    double best = -1.0; int best_g = 1 << 30;
+#pragma unroll
+    for (int r = 0; r < 4; r++) {
+      const int g = lane + 32 * r;
+      if (g < ng && b[r] < b_max) {
+        const double val = scalbn(v[r], -2 * b[r]);
+        if (val > best || (val == best && g < best_g)) { best = val; best_g = g; }
+      }
+    }
+#pragma unroll
+    for (int s = 16; s; s >>= 1) {
+      const double ob = __shfl_xor_sync(0xffffffffu, best, s);
+      const int og = __shfl_xor_sync(0xffffffffu, best_g, s);
+      if (ob > best || (ob == best && og < best_g)) { best = ob; best_g = og; }
+    }
+#pragma unroll
+    for (int r = 0; r < 4; r++) if (lane + 32 * r == best_g) b[r]++;
+  }
+#pragma unroll
+  for (int r = 0; r < 4; r++) {
+    const int g = lane + 32 * r;
+    if (g < ng) for (int j = 0; j < wg; j++) widths[u * kD + g * wg + j] = (uint8_t)b[r];
+  }
+}
+
+}  // namespace spectra
+
+using namespace spectra;
+
+extern "C" size_t spectra_fit_workspace_bytes(const spectra_config* cfg, int64_t n_units) {
+  if (check_config(cfg) || n_units < 0) return 0;
+  return sizeof(FitWorkspace) * (size_t)n_units;
+}
+
+extern "C" int spectra_fit_basis(const spectra_config* cfg, const void* x, int x_dtype, int64_t n_units,
+                                 int64_t n_tokens, int64_t stride_unit, int64_t stride_token, float* w_enc,
+                                 float* w_dec, float* mean_rot, float* var_alloc, float* eigval, float* basis_u,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (n_units < 0 || n_tokens < 1) return SPECTRA_INVALID_ARG;
+  if (x_dtype != SPECTRA_F32 && x_dtype != SPECTRA_BF16) return SPECTRA_INVALID_ARG;
+  if (n_units == 0) return SPECTRA_OK;
+  if (!x || !w_enc || !w_dec || !mean_rot || !var_alloc || !workspace) return SPECTRA_INVALID_ARG;
+  if (workspace_bytes < sizeof(FitWorkspace) * (size_t)n_units) return SPECTRA_WORKSPACE_TOO_SMALL;
+  if (n_units > 65535) return SPECTRA_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  FitWorkspace* ws = reinterpret_cast<FitWorkspace*>(workspace);
+  if (cudaMemsetAsync(ws, 0, sizeof(FitWorkspace) * (size_t)n_units, st) != cudaSuccess) return SPECTRA_CUDA_ERROR;
+  dim3 grid((unsigned)((n_tokens + kMomChunk - 1) / kMomChunk), (unsigned)n_units);
+  moments_kernel<<<grid, 256, 0, st>>>(x, x_dtype, n_tokens, stride_unit, stride_token, ws);
+  if (launch_status()) return SPECTRA_CUDA_ERROR;
+  if (cudaFuncSetAttribute(eigen_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(EigSmem)) !=
+      cudaSuccess)
+    return SPECTRA_CUDA_ERROR;
+  FitOut o{w_enc, w_dec, mean_rot, var_alloc, eigval, basis_u, cfg->gain_mode, n_tokens};
+  eigen_kernel<<<(unsigned)n_units, 512, sizeof(EigSmem), st>>>(ws, o);
+  return launch_status();
+}
+
+extern "C" int32_t spectra_total_bits(const spectra_config* cfg, double ratio) {
+  if (check_config(cfg) || !(ratio > 0.0)) return -1;
+  double bits = 16.0 * kD / ratio + 1e-9;
+  int64_t b = (int64_t)bits;
+  const int64_t cap = (int64_t)cfg->b_max * kD;
+  return (int32_t)(b > cap ? cap : b);
+}
+
+extern "C" int spectra_alloc_bits(const spectra_config* cfg, const float* var_alloc, int64_t n_units, double ratio,
+                                  uint8_t* widths, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (n_units < 0 || !(ratio > 0.0)) return SPECTRA_INVALID_ARG;
+  if (n_units == 0) return SPECTRA_OK;
+  if (!var_alloc || !widths) return SPECTRA_INVALID_ARG;
+  const int btot = spectra_total_bits(cfg, ratio);
+  alloc_kernel<<<(unsigned)((n_units + 3) / 4), 128, 0, (cudaStream_t)stream>>>(var_alloc, n_units, btot, cfg->b_max,
+                                                                                cfg->width_group, widths);
+  return launch_status();
+}
