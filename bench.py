@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the SPECTRA coded-KV decode path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama32] [--impl ours|reference]
+
+A step is one decode step of the whole model shape: in every layer, append one new token per sequence to the
+coded K and V caches (rotate, quantise, pack) and run coded-cache decode attention over the grown cache.
+Calibration (basis fit, bit allocation) and the prefill encode happen once during set-up and are reported
+separately.  Prints one JSON line.  With --impl reference the CPU oracle is timed instead (a deliberately plain
+program: a reported baseline, not a target).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "coded_kv_decode_attention_kv_tokens_per_s"
+UNIT = "KV tokens/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            parts = [s.strip() for s in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def _dist_setup(n_gpus):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    return rank, world, local
+
+
+def _barrier(world):
+    import torch
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def _max_over_ranks(x, world):
+    import torch
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle legs
+
+class OracleSample:
+    """A bounded sample of the workload built and run by the oracle alone (numpy generator, oracle fit,
+    allocation and encode): `heads` kv-heads of layer 0, sequence 0, n_tokens cached tokens."""
+
+    def __init__(self, wl, n_tokens):
+        import spectra_inputs as si
+        from oracle import codec as oc
+        from oracle import fit as ofit
+        self.wl, self.n, self.oc = wl, n_tokens, oc
+        H, d = wl.kv_heads, wl.head_dim
+        self.G = wl.q_heads // H
+        self.par = {}
+        cap_tiles = (n_tokens + 1 + 127) // 128
+        for side in (si.SIDE_K, si.SIDE_V):
+            X = np.stack([si.draw_unit(wl, 0, h, side, 0, n_tokens=n_tokens) for h in range(H)])
+            fits = [ofit.fit_basis(X[h][:min(wl.n_fit, n_tokens)].astype(np.float64), ofit.GAIN_SQRT) for h in range(H)]
+            widths = np.stack([ofit.alloc_bits(f["v_alloc"].astype(np.float32), ofit.total_bits(d, wl.ratio))
+                               for f in fits])
+            tb = np.array([oc.tile_bytes(w, 64) for w in widths], np.int64)
+            off = np.concatenate([[0], np.cumsum(tb * cap_tiles)[:-1]]).astype(np.int64)
+            cache = np.zeros(int((tb * cap_tiles).sum()), np.uint8)
+            we = np.stack([f["W_enc"] for f in fits]).astype(np.float32)
+            wd = np.stack([f["W_dec"] for f in fits]).astype(np.float32)
+            mr = np.stack([f["m_rot"] for f in fits]).astype(np.float32)
+            oc.encode_units(X, we, mr, widths, 64, side, 0, cache, off, tb)
+            self.par[side] = dict(we=we, wd=wd, mr=mr, widths=widths, tb=tb, off=off, cache=cache)
+        self.q = si.draw_queries(wl, 0, 0).reshape(H, self.G, d).astype(np.float64)
+        self.new = {side: np.stack([si.draw_unit(wl, 0, h, side, 0, n_tokens=1, start=n_tokens) for h in range(H)])
+                    for side in (si.SIDE_K, si.SIDE_V)}
+
+    def step(self):
+        """One decode step on the sample: append one token per unit (both sides), then latent-space attention
+        over n+1 tokens.  Returns (seconds, token_heads, threads)."""
+        oc = self.oc
+        k, v = self.par[0], self.par[1]
+        H = self.wl.kv_heads
+        t0 = time.perf_counter()
+        for side in (0, 1):
+            p = self.par[side]
+            oc.encode_units(self.new[side], p["we"], p["mr"], p["widths"], 64, side, self.n, p["cache"], p["off"],
+                            p["tb"])
+        oc.attention_units("B", self.q, [self.n + 1] * H, k["cache"], k["off"], k["tb"], v["cache"], v["off"],
+                           v["tb"], k["wd"], k["mr"], k["widths"], v["wd"], v["mr"], v["widths"], 64,
+                           1.0 / np.sqrt(128.0))
+        dt = time.perf_counter() - t0
+        return dt, H * (self.n + 1), min(oc.num_threads(), H)
+
+
+def _oracle_rate(wl, seconds_budget, reps=1):
+    """Sizes a sample so that `reps` oracle steps take about seconds_budget; returns (times, token_heads, threads,
+    description)."""
+    probe = OracleSample(wl, 512)
+    dt, th, threads = probe.step()
+    per_th = dt / th
+    n = int(max(128, min(wl.n_tokens, (seconds_budget / reps / per_th / wl.kv_heads) // 128 * 128)))
+    sample = OracleSample(wl, n)
+    times = []
+    for _ in range(reps):
+        dt, th, threads = sample.step()
+        times.append(dt)
+    desc = (f"layer 0, sequence 0, {wl.kv_heads} kv-heads x {n} cached tokens, built and run by the oracle alone; "
+            f"one step = append 1 token per unit + Mode B attention; token-heads/s divided by layers*kv_heads")
+    return times, th, threads, desc
+
+
+def run_reference(args, wl):
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    reps = args.warmup + args.steps
+    times, th, threads, desc = _oracle_rate(wl, 90.0, reps)
+    t = float(np.mean(times[args.warmup:]))
+    value = th / t / (wl.layers * wl.kv_heads)          # same unit as the GPU arm: KV tokens/s of the full model
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "note": "CPU oracle on a bounded sample; value scaled to the full model "
+                                                "shape"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------- GPU arm
+
+def run_ours(args, wl):
+    import torch
+
+    import paper_2608_07915_b200 as sp
+    from paper_2608_07915_b200 import harness
+    rank, world, local = _dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    steps, warmup = args.steps, max(args.warmup, 3)
+    hbm_gbs, peak_kind = _peaks()
+    model = harness.CodedModelCache(wl, layers=args.layers or None, extra_tokens=steps + warmup + 8 + 2 * steps)
+    t0 = time.perf_counter()
+    model.build(time_phases=True)
+    setup_s = time.perf_counter() - t0
+    L, B, H, Hq, d, U = model.layers, model.batch, model.H, model.Hq, model.d, model.n_units
+    dt = torch.bfloat16
+    gen = torch.Generator(device="cuda").manual_seed(1234 + rank)
+    n_in = 4                                           # distinct input sets, cycled
+    q_dev = torch.randn((n_in, L, B, Hq, d), generator=gen, device="cuda").to(dt)
+    nk_dev = torch.randn((n_in, L, U, d), generator=gen, device="cuda").to(dt)
+    nv_dev = torch.randn((n_in, L, U, d), generator=gen, device="cuda").to(dt)
+    out_dev = torch.zeros((L, B, Hq, d), dtype=dt, device="cuda")
+    q_host, nk_host, nv_host = (t.cpu().pin_memory() for t in (q_dev, nk_dev, nv_dev))
+    out_host = torch.zeros((L, B, Hq, d), dtype=dt).pin_memory()
+    q_stage, nk_stage, nv_stage = (torch.empty_like(t[0]) for t in (q_dev, nk_dev, nv_dev))
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    attn_events = []
+
+    def mark(layer, which):
+        e = ev(); e.record(); attn_events.append(e)
+
+    def step_resident(i, timed=False):
+        model.decode_step(q_dev[i % n_in], nk_dev[i % n_in], nv_dev[i % n_in], out_dev, mark if timed else None)
+
+    def step_e2e(i):
+        q_stage.copy_(q_host[i % n_in], non_blocking=True)
+        nk_stage.copy_(nk_host[i % n_in], non_blocking=True)
+        nv_stage.copy_(nv_host[i % n_in], non_blocking=True)
+        model.decode_step(q_stage, nk_stage, nv_stage, out_dev)
+        out_host.copy_(out_dev, non_blocking=True)
+
+    # ---- device-resident timing
+    for i in range(warmup):
+        step_resident(i)
+    _barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    e_start, e_end = ev(), ev()
+    e_start.record()
+    for i in range(steps):
+        step_resident(i, timed=True)
+    e_end.record()
+    _barrier(world)
+    clocks = sampler.stop()
+    ms_step = _max_over_ranks(e_start.elapsed_time(e_end) / steps, world)
+    attn_ms = [attn_events[2 * j].elapsed_time(attn_events[2 * j + 1]) for j in range(len(attn_events) // 2)]
+    attn_ms_avg = float(np.mean(attn_ms))
+    n_ctx = int(model.seq_len.max().item())
+    kv_tokens = B * n_ctx
+
+    # ---- end to end: pinned host inputs copied in, outputs copied out, every step
+    for i in range(2):
+        step_e2e(i)
+    _barrier(world)
+    e0, e1 = ev(), ev()
+    e0.record()
+    for i in range(steps):
+        step_e2e(i)
+    e1.record()
+    _barrier(world)
+    ms_e2e = _max_over_ranks(e0.elapsed_time(e1) / steps, world)
+    status = int(model.status.item())
+
+    bytes_call = model.attention_bytes(layer=0)
+    achieved = bytes_call / (attn_ms_avg * 1e-3) / 1e9
+    h2d = sum(t[0].numel() * t.element_size() for t in (q_host, nk_host, nv_host))
+    d2h = out_host.numel() * out_host.element_size()
+    line = {
+        "metric": METRIC, "value": world * kv_tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "layers": L, "batch": B, "kv_heads": H, "q_heads": Hq, "head_dim": d,
+                   "context": n_ctx, "ratio": wl.ratio, "cache_dtype_replaced": "bf16",
+                   "coded_cache_gb": model.coded_bytes() / 1e9, "parallelism": f"replicas{world}",
+                   "l2": "coded cache per step far exceeds L2; no flush needed" if model.coded_bytes() > 4e8
+                   else "WARNING: coded cache fits L2"},
+        "e2e": {"value": world * kv_tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+        "gpu_launches": steps * L * (2 + sp.ATTENTION_LAUNCHES),
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "spectra_decode_attention (one layer call)", "achieved": achieved,
+                     "peak": hbm_gbs, "unit": "GB/s", "frac": achieved / hbm_gbs, "peak_kind": peak_kind,
+                     "traffic": None, "bytes_per_launch": bytes_call, "ms_per_launch": attn_ms_avg},
+        "phases": {"setup_s": setup_s, "fit_alloc_ms_total": model.timings["fit_alloc_ms"],
+                   "prefill_encode_ms_total": model.timings["prefill_encode_ms"],
+                   "prefill_encode_tokens_per_s": L * 2 * U * wl.n_tokens / max(model.timings["prefill_encode_ms"],
+                                                                               1e-9) * 1e3 / 2},
+        "status_word": status,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        times, th, threads, desc = _oracle_rate(wl, 15.0, 1)
+        line["cpu_baseline"] = {"value": th / times[0] / (wl.layers * wl.kv_heads), "unit": UNIT, "cores": threads,
+                                "kind": "oracle", "sample": desc}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="llama32")
+    ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers than the workload (invalid as a result)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    import spectra_inputs as si
+    wl = si.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -19,6 +19,7 @@ STATUS_NONFINITE, STATUS_F16_RANGE, STATUS_WAIT_TIMEOUT = 1, 2, 4
 GAIN_ROTATE, GAIN_SQRT, GAIN_WHITEN = 0, 1, 2
 HEAD_DIM = 128
 TILE_TOKENS = 128
+ATTENTION_LAUNCHES = 2   # kernels one spectra_decode_attention call enqueues
 
 EXPORTS = [
     "spectra_fit_basis", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
