@@ -172,7 +172,11 @@ int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, co
  * n_kv_heads).  q: device [batch, n_q_heads, d], q_dtype.  seq_len: device int32 [batch] (tokens attended,
  * <= max_seq_len; 0 gives a zero output row and lse = -inf).  cache_k/v with unit_offset_k/v: as in
  * spectra_encode.  Parameter arrays as in spectra_encode/decode ([n_param_sets, ...]); mean_rot_k is read
- * only when lse != NULL and may be NULL otherwise.  softmax_scale 0 means 1/sqrt(d).
+ * only when lse != NULL and may be NULL otherwise.  widths_k_host / widths_v_host: HOST copies of the two width
+ * arrays ([n_param_sets, d], the same values the caller already needs for spectra_tile_bytes); read during the
+ * call only.  They let the host size shared-memory rings and pick the kernel variant without a device
+ * round-trip.  With both NULL, or a GQA group above 4, or scale_group != 64, a slower CUDA-core kernel runs.
+ * softmax_scale 0 means 1/sqrt(d).
  * out: device [batch, n_q_heads, d], out_dtype.  lse: device fp32 [batch, n_q_heads] or NULL.
  * workspace: device, >= spectra_attention_workspace_bytes(...), 16-byte aligned; scratch only, nothing is
  * carried between calls.  status_word: device int32 or NULL.
@@ -182,9 +186,10 @@ int spectra_decode_attention(const spectra_config* cfg, const void* q, int q_dty
                              const uint8_t* cache_k, const int64_t* unit_offset_k, const uint8_t* cache_v,
                              const int64_t* unit_offset_v, int64_t n_param_sets, const float* w_dec_k,
                              const float* mean_rot_k, const uint8_t* widths_k, const float* w_dec_v,
-                             const float* mean_rot_v, const uint8_t* widths_v, float softmax_scale, void* out,
-                             int out_dtype, float* lse, void* workspace, size_t workspace_bytes,
-                             int32_t* status_word, void* stream);
+                             const float* mean_rot_v, const uint8_t* widths_v, const uint8_t* widths_k_host,
+                             const uint8_t* widths_v_host, float softmax_scale, void* out, int out_dtype,
+                             float* lse, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                             void* stream);
 size_t spectra_attention_workspace_bytes(const spectra_config* cfg, int32_t batch, int32_t n_kv_heads,
                                          int32_t n_q_heads, int32_t max_seq_len);
 

@@ -1,5 +1,5 @@
 // spectra_decode_attention entry point and host-side helpers of the library.
-#include "attention_generic.cuh"
+#include "attention_mma.cuh"
 
 using namespace spectra;
 
@@ -14,6 +14,72 @@ int generic_splits(int n_units, int max_seq_len) {
   return splits;
 }
 
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return sms;
+}
+
+// Workspace carve-up of the tensor-core path.
+struct FastLayout {
+  size_t desc_off, prefix_off, warp_off, rec_off, total;
+  int total_warps, rec_stride;
+};
+
+FastLayout fast_layout(int64_t n_units, int total_warps, int vs_max) {
+  FastLayout L{};
+  L.total_warps = total_warps;
+  L.rec_stride = kFastGqa * (kRecHead + vs_max);
+  size_t off = 0;
+  L.desc_off = off; off = align_up(off + sizeof(UnitDesc) * (size_t)n_units, 256);
+  L.prefix_off = off; off = align_up(off + sizeof(int32_t) * (size_t)(n_units + 1), 256);
+  L.warp_off = off; off = align_up(off + sizeof(int32_t) * (size_t)total_warps, 256);
+  L.rec_off = off; off = align_up(off + sizeof(float) * (size_t)L.rec_stride * (size_t)(total_warps + n_units), 256);
+  L.total = off;
+  return L;
+}
+
+// What the host learns from the widths: tile sizes, V strip and block counts.
+struct WidthFacts { int max_tile_k = 0, max_tile_v = 0, max_vstrips = 0, max_vblocks = 0; bool ok = true; };
+
+WidthFacts width_facts(const uint8_t* wk, const uint8_t* wv, int64_t n_sets) {
+  WidthFacts F;
+  for (int64_t s = 0; s < n_sets; s++) {
+    for (int side = 0; side < 2; side++) {
+      const uint8_t* w = (side ? wv : wk) + s * kD;
+      int bits = 0, cnt[4] = {0, 0, 0, 0}, act[2] = {0, 0};
+      for (int j = 0; j < kD; j++) {
+        if (w[j] > 8) { F.ok = false; return F; }
+        bits += w[j];
+        act[j / 64] |= w[j] != 0;
+        for (int c = 0; c < 4; c++) cnt[c] += (w[j] & (8 >> c)) != 0;
+      }
+      const int tb = 16 * bits + 512 * (act[0] + act[1]);
+      if (side == 0) F.max_tile_k = tb > F.max_tile_k ? tb : F.max_tile_k;
+      else {
+        F.max_tile_v = tb > F.max_tile_v ? tb : F.max_tile_v;
+        const int strips = cnt[0] + cnt[1] + cnt[2] + cnt[3];
+        const int blocks = (cnt[0] + 15) / 16 + (cnt[1] + 15) / 16 + (cnt[2] + 15) / 16 + (cnt[3] + 15) / 16;
+        F.max_vstrips = strips > F.max_vstrips ? strips : F.max_vstrips;
+        F.max_vblocks = blocks > F.max_vblocks ? blocks : F.max_vblocks;
+      }
+    }
+  }
+  return F;
+}
+
+template <int NVB>
+int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {
+  if (cudaFuncSetAttribute(attention_mma_kernel<NVB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+      cudaSuccess)
+    return SPECTRA_CUDA_ERROR;
+  attention_mma_kernel<NVB><<<grid, kFastWarps * 32, smem, st>>>(a, f);
+  return launch_status();
+}
+
 }  // namespace
 
 extern "C" size_t spectra_attention_workspace_bytes(const spectra_config* cfg, int32_t batch, int32_t n_kv_heads,
@@ -22,7 +88,11 @@ extern "C" size_t spectra_attention_workspace_bytes(const spectra_config* cfg, i
   const int64_t n_units = (int64_t)batch * n_kv_heads;
   if (n_units == 0) return 16;
   const int splits = generic_splits((int)n_units, max_seq_len);
-  return (size_t)n_units * splits * (n_q_heads / n_kv_heads) * kPartialStride * sizeof(float) + 16;
+  const size_t generic = (size_t)n_units * splits * (n_q_heads / n_kv_heads) * kPartialStride * sizeof(float) + 16;
+  int sms = sm_count();
+  if (sms <= 0) sms = 160;
+  const size_t fast = fast_layout(n_units, sms * 2 * kFastWarps, kMaxStrips).total;
+  return generic > fast ? generic : fast;
 }
 
 extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q, int q_dtype, int32_t batch,
@@ -31,6 +101,7 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
                                         const uint8_t* cache_v, const int64_t* unit_offset_v, int64_t n_param_sets,
                                         const float* w_dec_k, const float* mean_rot_k, const uint8_t* widths_k,
                                         const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
+                                        const uint8_t* widths_k_host, const uint8_t* widths_v_host,
                                         float softmax_scale, void* out, int out_dtype, float* lse, void* workspace,
                                         size_t workspace_bytes, int32_t* status_word, void* stream) {
   int rc = check_config(cfg);
@@ -46,6 +117,7 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
       !mean_rot_v || !widths_k || !widths_v || !out || !workspace)
     return SPECTRA_INVALID_ARG;
   if (lse && !mean_rot_k) return SPECTRA_INVALID_ARG;
+  if ((widths_k_host == nullptr) != (widths_v_host == nullptr)) return SPECTRA_INVALID_ARG;
   const int64_t n_units = (int64_t)batch * n_kv_heads;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   if (workspace_bytes < spectra_attention_workspace_bytes(cfg, batch, n_kv_heads, n_q_heads, max_seq_len))
@@ -63,6 +135,45 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
   a.n_splits = generic_splits((int)n_units, max_seq_len);
   a.status = status_word;
   cudaStream_t st = (cudaStream_t)stream;
+
+  // ---- tensor-core path: GQA group <= 4, scale group 64, host copy of the widths available
+  if (widths_k_host && gqa <= kFastGqa && cfg->scale_group == 64) {
+    const WidthFacts F = width_facts(widths_k_host, widths_v_host, n_param_sets);
+    if (!F.ok) return SPECTRA_INVALID_ARG;
+    const int sms = sm_count();
+    if (sms <= 0) return SPECTRA_CUDA_ERROR;
+    const int slot_k = (int)align_up((size_t)(F.max_tile_k > 16 ? F.max_tile_k : 16), 128);
+    const int slot_v = (int)align_up((size_t)(F.max_tile_v > 16 ? F.max_tile_v : 16), 128);
+    const size_t pair = (size_t)slot_k + slot_v;
+    const size_t budget = 200 * 1024;
+    int ctas_per_sm = 2 * kFastWarps * pair <= budget ? 2 : 1;
+    int depth = (int)(budget / ((size_t)ctas_per_sm * kFastWarps * pair));
+    if (depth > 4) depth = 4;
+    if (depth >= 1 && F.max_vblocks <= 24 && F.max_vblocks >= 0) {
+      FastLayout L = fast_layout(n_units, sms * ctas_per_sm * kFastWarps, F.max_vstrips);
+      if (L.total > workspace_bytes) return SPECTRA_WORKSPACE_TOO_SMALL;
+      char* ws = reinterpret_cast<char*>(workspace);
+      FastArgs f{};
+      f.desc = reinterpret_cast<UnitDesc*>(ws + L.desc_off);
+      f.tile_prefix = reinterpret_cast<int32_t*>(ws + L.prefix_off);
+      f.warp_unit = reinterpret_cast<int32_t*>(ws + L.warp_off);
+      f.records = reinterpret_cast<float*>(ws + L.rec_off);
+      f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = F.max_vstrips;
+      f.n_units = (int)n_units; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
+      attention_prep_kernel<<<(unsigned)n_units + 1, 128, sizeof(PrepSmem), st>>>(a, f);
+      if (launch_status()) return SPECTRA_CUDA_ERROR;
+      const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64;
+      const int grid = sms * ctas_per_sm;
+      if (F.max_vblocks <= 10) rc = launch_fast_main<10>(a, f, grid, smem, st);
+      else if (F.max_vblocks <= 16) rc = launch_fast_main<16>(a, f, grid, smem, st);
+      else rc = launch_fast_main<24>(a, f, grid, smem, st);
+      if (rc) return rc;
+      attention_mma_combine_kernel<<<(unsigned)n_units, 128, 0, st>>>(a, f);
+      return launch_status();
+    }
+  }
+
+  // ---- generic path
   if (cudaFuncSetAttribute(attention_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)sizeof(GenericSmem)) != cudaSuccess)
     return SPECTRA_CUDA_ERROR;

@@ -35,6 +35,7 @@ class CodedModelCache:
         self.seq_len = torch.zeros(self.batch, dtype=torch.int32, device=device)
         self.pos0 = torch.zeros(self.n_units, dtype=torch.int32, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.tensor_path = True                          # pass host widths to spectra_decode_attention
         self.keep_raw_units = keep_raw_units or {}      # {(layer, side): [unit indices]} raw vectors kept on host
         self.raw = {}
         self.timings = {}
@@ -109,7 +110,8 @@ class CodedModelCache:
         k, v = self.side[layer]
         sp.decode_attention(self.cfg, q, self.batch, self.H, self.Hq, self.seq_len, self.cap_tokens, k.cache,
                             k.unit_offset, v.cache, v.unit_offset, self.H, k.w_dec, k.m_rot, k.widths, v.w_dec,
-                            v.m_rot, v.widths, 0.0, out, lse, self.workspace, self.status)
+                            v.m_rot, v.widths, 0.0, out, lse, self.workspace, self.status,
+                            k.widths_host if self.tensor_path else None, v.widths_host if self.tensor_path else None)
 
     def decode_step(self, q_all, new_k_all, new_v_all, out_all, on_attend=None):
         """q_all [layers, batch, Hq, d]; new_*_all [layers, n_units, d]; out_all like q_all.  Appends one token

@@ -239,7 +239,7 @@ def _oracle_attention(wl_group, q, n_tokens, K, V, cache_k, cache_v, mode="B"):
 
 
 def _gpu_attention(sp, cfg, q_dev, batch, n_kv, n_q, seq_len, max_len, K, V, cache_k, cache_v, want_lse=True,
-                   out_dtype=None):
+                   out_dtype=None, host_widths=True):
     pk, pv = K["params"], V["params"]
     dk, dv = H.dev_params(pk), H.dev_params(pv)
     out = torch.zeros((batch, n_q, 128), dtype=out_dtype or torch.float32, device="cuda")
@@ -249,15 +249,16 @@ def _gpu_attention(sp, cfg, q_dev, batch, n_kv, n_q, seq_len, max_len, K, V, cac
     sp.decode_attention(cfg, q_dev, batch, n_kv, n_q, H.to_dev(np.asarray(seq_len, np.int32)), max_len,
                         H.to_dev(cache_k), H.to_dev(K["off"]), H.to_dev(cache_v), H.to_dev(V["off"]), pk.n_sets,
                         dk["w_dec"], dk["m_rot"], dk["widths"], dv["w_dec"], dv["m_rot"], dv["widths"], 0.0, out, lse,
-                        ws, status)
+                        ws, status, pk.widths if host_widths else None, pv.widths if host_widths else None)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     return out.float().cpu().numpy(), None if lse is None else lse.cpu().numpy()
 
 
+@pytest.mark.parametrize("host_widths", [True, False], ids=["tensor", "generic"])
 @pytest.mark.parametrize("ratio", [4.0, 8.0, 12.0])
 @pytest.mark.parametrize("n", [1024, 1000, 77])
-def test_tiny_attention_matches_oracle(sp, ratio, n):
+def test_tiny_attention_matches_oracle(sp, ratio, n, host_widths):
     wl, S = _tiny_setup(sp, ratio)
     cfg = sp.default_config()
     caches = {}
@@ -269,7 +270,8 @@ def test_tiny_attention_matches_oracle(sp, ratio, n):
     q = si.draw_queries(wl, 0, 0)                                                 # [4, 128]
     ref_b, lse_b = _oracle_attention(4, q[None].astype(np.float64), [n], S["k"], S["v"], caches["k"], caches["v"])
     ref_a, _ = _oracle_attention(4, q[None].astype(np.float64), [n], S["k"], S["v"], caches["k"], caches["v"], "A")
-    got, lse = _gpu_attention(sp, cfg, H.to_dev(q[None]), 1, 1, 4, [n], n, S["k"], S["v"], caches["k"], caches["v"])
+    got, lse = _gpu_attention(sp, cfg, H.to_dev(q[None]), 1, 1, 4, [n], n, S["k"], S["v"], caches["k"], caches["v"],
+                              host_widths=host_widths)
     assert H.rel_err_per_vector(got[0], ref_b[0]) <= TOL
     assert H.rel_err_per_vector(got[0], ref_a[0]) <= TOL
     assert np.abs(lse[0] - lse_b[0]).max() <= 2e-3
