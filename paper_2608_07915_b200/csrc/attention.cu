@@ -1,5 +1,5 @@
 // spectra_decode_attention entry point and host-side helpers of the library.
-#include "attention_mma.cuh"
+#include "attention_tc_main.cuh"
 
 using namespace spectra;
 

@@ -1,0 +1,366 @@
+// Fused coded-cache decode attention for GQA groups of up to 4 query heads and scale_group 64.
+//
+// Three kernels per call:
+//   prep    (one CTA per unit)  folds W_dec,K and the softmax scale into the query (q'), turns it into
+//           tensor-core B fragments per 16-strip chunk of the K tile, and lays out the per-unit descriptor;
+//           one extra CTA builds the tile prefix sums and each warp's starting unit.
+//   main    persistent, one warp = one worker.  The (unit, tile) space is flattened and cut into equal
+//           contiguous ranges, one per warp.  A warp streams its K and V tiles into its own shared-memory
+//           ring with 1-D bulk copies (cp.async.bulk + mbarrier), and per 64-token half tile
+//             - unpacks K codes straight into mma.sync A fragments (rows = tokens, k = strips), multiplies by
+//               the q' fragments (columns = head x {hi, lo} halves of an fp16 split), applies the per-token
+//               group scales, runs the online softmax with warp shuffles,
+//             - transposes the probabilities (times the V group ranges) with movmatrix into B fragments,
+//             - unpacks V codes into A fragments (rows = strips, k = tokens) and accumulates the output in the
+//               rotated value space in registers.
+//           At the end of a unit the warp writes one partial record (max, sum, accumulators per V strip).
+//   combine (one CTA per unit)  merges the records (log-sum-exp), folds strips back into channels, adds the
+//           rotated mean and lifts the result once with W_dec,V.
+//
+// Codes enter the MMA as fp16 numbers 2^w + code, built with one shift and one logic op per pair: the field is
+// moved to the top of the fp16 mantissa and OR-ed with the exponent of 2^w.  The constant 2^w is removed
+// analytically (K: precomputed per head and group; V: an extra all-ones MMA row sum).
+#pragma once
+#include "attention_generic.cuh"
+
+namespace spectra {
+
+constexpr int kFastGqa = 4;
+constexpr int kKcMax = 28;       // upper bound of 16-strip chunks in a K tile (384 strips in 4 classes)
+constexpr int kFastWarps = 4;    // warps per CTA of the main kernel
+constexpr int kRecHead = 4;      // floats of a record's per-head header: m, l, plo0, plo1
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct alignas(16) UnitDesc {
+  int32_t tbk, tbv;
+  int32_t kmeta[2], vmeta[2];   // byte offset of lo16[128] of scale group g (R16 256 bytes later), -1 if inactive
+  uint32_t kcls[4], vcls[4];    // per class: strips | strips of scale group 0 << 8 | (byte offset / 16) << 16
+  uint32_t vfirst[4];           // index of the first V strip of each class
+  int32_t n_vstrips, pad0;
+  float kscale[4];              // 2^-e_h
+  float kcorr[4][2];            // sum_k 2^w_k (B_hi + B_lo) per head and scale group
+  float qlo[4][2];              // sum of q' over the active channels of a scale group
+  float qconst[4];              // q' . m'_K (natural-log units)
+  uint2 kB[kKcMax][2][32];      // [chunk][scale group][lane] -> (b0, b1)
+};
+
+struct FastArgs {
+  UnitDesc* desc; int32_t* tile_prefix; int32_t* warp_unit; float* records;
+  int total_warps; int rec_stride; int vs_max; int n_units;
+  int depth; int slot_k, slot_v;
+};
+
+// ------------------------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after a fixed number of polls (each poll itself blocks for a bounded hardware interval).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (int it = 0; it < (1 << 20); ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t a) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+
+__device__ __forceinline__ float2 h2f2(uint32_t x) {
+  __half2 h;
+  *reinterpret_cast<uint32_t*>(&h) = x;
+  return __half22float2(h);
+}
+
+// ------------------------------------------------------------------------------------------------ prep kernel
+struct PrepSmem {
+  StripTable tk, tv;
+  alignas(16) float qraw[kFastGqa][kD];
+  alignas(16) float qrot[kFastGqa][kD];
+  __half bhi[kFastGqa][kMaxStrips];
+  __half blo[kFastGqa][kMaxStrips];
+  float red[kFastGqa][4];
+  int escale[kFastGqa];
+  int scan[128];
+};
+
+__device__ inline uint32_t pack_cls(const StripTable& T, int c) {
+  const int first = T.class_first[c], n = T.class_first[c + 1] - first;
+  int n_g0 = 0;
+  for (int k = first; k < first + n; k++) n_g0 += T.chan[k] < 64;
+  return (uint32_t)n | ((uint32_t)n_g0 << 8) | ((uint32_t)(T.class_off[c] / 16) << 16);
+}
+
+__global__ void __launch_bounds__(128) attention_prep_kernel(AttnArgs p, FastArgs f) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  PrepSmem& S = *reinterpret_cast<PrepSmem*>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if ((int)blockIdx.x == f.n_units) {
+    // ---- tile prefix sums over units and each worker warp's first unit
+    const int n_units = f.n_units;
+    const int per = (n_units + 127) / 128;
+    int local = 0;
+    for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (p.seq_len[i / p.n_kv] + kTile - 1) / kTile;
+    S.scan[tid] = local;
+    __syncthreads();
+    if (tid == 0) {
+      int run = 0;
+      for (int i = 0; i < 128; i++) { const int v = S.scan[i]; S.scan[i] = run; run += v; }
+      f.tile_prefix[n_units] = run;
+    }
+    __syncthreads();
+    int run = S.scan[tid];
+    for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) {
+      f.tile_prefix[i] = run;
+      run += (p.seq_len[i / p.n_kv] + kTile - 1) / kTile;
+    }
+    __syncthreads();
+    __threadfence_block();
+    const long long total = f.tile_prefix[n_units];
+    for (int gw = tid; gw < f.total_warps; gw += 128) {
+      const long long g0 = (long long)gw * total / f.total_warps;
+      int lo = 0, hi = n_units;             // first unit whose end is beyond g0
+      while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (f.tile_prefix[mid + 1] > g0) hi = mid; else lo = mid + 1;
+      }
+      f.warp_unit[gw] = lo;
+    }
+    return;
+  }
+  const int u = blockIdx.x;
+  const int b = u / p.n_kv, hk = u - b * p.n_kv;
+  const int ps = (int)(u % p.n_param_sets);
+  const int G = p.gqa;
+  build_strip_table(S.tk, p.widths_k + (int64_t)ps * kD, 64);
+  build_strip_table(S.tv, p.widths_v + (int64_t)ps * kD, 64);
+  const StripTable& TK = S.tk;
+  const StripTable& TV = S.tv;
+  UnitDesc& D = f.desc[u];
+  for (int idx = tid; idx < kFastGqa * kD; idx += 128) {
+    const int h = idx / kD, i = idx - h * kD;
+    S.qraw[h][i] = h < G ? load_as_float(p.q, p.q_dtype, ((int64_t)b * p.n_q + hk * G + h) * kD + i) : 0.f;
+  }
+  __syncthreads();
+  const float* wk = p.w_dec_k + (int64_t)ps * kD * kD;
+  for (int j = warp; j < kD; j += 4) {
+    const float4 wrow = *reinterpret_cast<const float4*>(wk + j * kD + lane * 4);
+#pragma unroll
+    for (int h = 0; h < kFastGqa; h++) {
+      const float4 qv = *reinterpret_cast<const float4*>(&S.qraw[h][lane * 4]);
+      float acc = wrow.x * qv.x + wrow.y * qv.y + wrow.z * qv.z + wrow.w * qv.w;
+#pragma unroll
+      for (int s = 16; s; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+      if (lane == 0) S.qrot[h][j] = acc * p.scale * kLog2e;   // scores live in the log2 domain
+    }
+  }
+  __syncthreads();
+  // per-head power-of-two normalisation so that the fp16 hi/lo split of q'' = q' 2^shift / L is well conditioned
+  const int nk = TK.n_strips;
+  {
+    const int h = warp;  // one warp per head
+    float mx = 0.f;
+    for (int k = lane; k < nk; k += 32) {
+      const int c = TK.chan[k];
+      mx = fmaxf(mx, fabsf(S.qrot[h][c] * (float)(1 << TK.shift[k]) / (float)((1 << TK.width[c]) - 1)));
+    }
+#pragma unroll
+    for (int s = 16; s; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+    int e = 0;
+    if (mx > 0.f && isfinite(mx)) { int ex; frexpf(mx, &ex); e = 10 - ex; }
+    e = max(-100, min(100, e));
+    if (lane == 0) { S.escale[h] = e; D.kscale[h] = ldexpf(1.f, 24 - e); }
+    float corr0 = 0.f, corr1 = 0.f;
+    for (int k = lane; k < nk; k += 32) {
+      const int c = TK.chan[k];
+      const float v = ldexpf(S.qrot[h][c] * (float)(1 << TK.shift[k]) / (float)((1 << TK.width[c]) - 1), e);
+      const __half hi = __float2half_rn(v);
+      const __half lo = __float2half_rn(v - __half2float(hi));
+      S.bhi[h][k] = hi; S.blo[h][k] = lo;
+      const float off = (float)(1 << (8 >> strip_class(TK, k)));    // 2^w
+      const float t = off * (__half2float(hi) + __half2float(lo));
+      if (c < 64) corr0 += t; else corr1 += t;
+    }
+    float q0 = 0.f, q1 = 0.f, qc = 0.f;
+    for (int j = lane; j < kD; j += 32) {
+      const float v = S.qrot[h][j];
+      if (TK.width[j]) { if (j < 64) q0 += v; else q1 += v; }
+      if (p.mean_rot_k) qc += v * p.mean_rot_k[(int64_t)ps * kD + j];
+    }
+#pragma unroll
+    for (int s = 16; s; s >>= 1) {
+      corr0 += __shfl_xor_sync(0xffffffffu, corr0, s); corr1 += __shfl_xor_sync(0xffffffffu, corr1, s);
+      q0 += __shfl_xor_sync(0xffffffffu, q0, s); q1 += __shfl_xor_sync(0xffffffffu, q1, s);
+      qc += __shfl_xor_sync(0xffffffffu, qc, s);
+    }
+    if (lane == 0) {
+      D.kcorr[h][0] = corr0; D.kcorr[h][1] = corr1; D.qlo[h][0] = q0; D.qlo[h][1] = q1;
+      D.qconst[h] = qc / kLog2e;
+    }
+  }
+  __syncthreads();
+  // B fragments: chunk = 16 consecutive strips of a class; column n = head (n >> 1), hi (n & 1 == 0) or lo half
+  int chunk0 = 0;
+  for (int c = 0; c < 4; c++) {
+    const int first = TK.class_first[c], n = TK.class_first[c + 1] - first;
+    const int nch = (n + 15) / 16;
+    for (int idx = tid; idx < nch * 2 * 32; idx += 128) {
+      const int ci = idx / 64, g = (idx >> 5) & 1, ln = idx & 31;
+      const int gid = ln >> 2, tg = ln & 3, h = gid >> 1, part = gid & 1;
+      uint32_t r[2];
+#pragma unroll
+      for (int half = 0; half < 2; half++) {
+        uint32_t v = 0;
+#pragma unroll
+        for (int e = 0; e < 2; e++) {
+          const int krow = 2 * tg + 8 * half + e;
+          const int k = first + 16 * ci + krow;
+          uint16_t bits = 0;
+          if (16 * ci + krow < n && h < G && (TK.chan[k] >= 64 ? 1 : 0) == g)
+            bits = __half_as_ushort(part ? S.blo[h][k] : S.bhi[h][k]);
+          v |= (uint32_t)bits << (16 * e);
+        }
+        r[half] = v;
+      }
+      if (chunk0 + ci < kKcMax) D.kB[chunk0 + ci][g][ln] = make_uint2(r[0], r[1]);
+    }
+    chunk0 += nch;
+  }
+  if (tid < 4) {
+    D.kcls[tid] = pack_cls(TK, tid);
+    D.vcls[tid] = pack_cls(TV, tid);
+    D.vfirst[tid] = TV.class_first[tid];
+  }
+  if (tid == 0) {
+    D.tbk = TK.tile_bytes; D.tbv = TV.tile_bytes;
+    D.kmeta[0] = TK.meta_off[0]; D.kmeta[1] = TK.meta_off[1];
+    D.vmeta[0] = TV.meta_off[0]; D.vmeta[1] = TV.meta_off[1];
+    D.n_vstrips = TV.n_strips; D.pad0 = 0;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ combine kernel
+struct CombineSmem {
+  StripTable tv;
+  float o[kD];
+  float orot[kD];
+};
+
+__global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, FastArgs f) {
+  __shared__ CombineSmem S;
+  const int tid = threadIdx.x;
+  const int u = blockIdx.x;
+  const int b = u / p.n_kv, hk = u - b * p.n_kv;
+  const int ps = (int)(u % p.n_param_sets);
+  const int G = p.gqa;
+  build_strip_table(S.tv, p.widths_v + (int64_t)ps * kD, 64);
+  const StripTable& TV = S.tv;
+  const long long total = f.tile_prefix[f.n_units];
+  const long long ta = f.tile_prefix[u], tb = f.tile_prefix[u + 1];
+  const float* wv = p.w_dec_v + (int64_t)ps * kD * kD;
+  // workers whose ranges intersect this unit: the largest gw with floor(gw * total / W) <= tile
+  int gw_first = 0, gw_last = -1;
+  if (tb > ta) {
+    gw_first = (int)(((ta + 1) * f.total_warps + total - 1) / total) - 1;
+    gw_last = (int)(((tb - 1 + 1) * (long long)f.total_warps + total - 1) / total) - 1;
+  }
+  // a worker whose range is empty wrote no record
+  auto nonempty = [&](int gw) {
+    return (long long)(gw + 1) * total / f.total_warps > (long long)gw * total / f.total_warps;
+  };
+  for (int h = 0; h < G; h++) {
+    const int64_t hoff = (int64_t)h * (kRecHead + f.vs_max);
+    float M = -INFINITY;
+    for (int gw = gw_first; gw <= gw_last; gw++)
+      if (nonempty(gw)) M = fmaxf(M, f.records[(int64_t)(gw + u) * f.rec_stride + hoff]);
+    float L = 0.f, P0 = 0.f, P1 = 0.f;
+    for (int gw = gw_first; gw <= gw_last; gw++) {
+      if (!nonempty(gw)) continue;
+      const float* rec = f.records + (int64_t)(gw + u) * f.rec_stride + hoff;
+      const float e = rec[0] == -INFINITY ? 0.f : exp2f(rec[0] - M);
+      L += e * rec[1]; P0 += e * rec[2]; P1 += e * rec[3];
+    }
+    __syncthreads();
+    S.o[tid] = 0.f;
+    __syncthreads();
+    for (int k = tid; k < TV.n_strips; k += 128) {
+      float acc = 0.f;
+      for (int gw = gw_first; gw <= gw_last; gw++) {
+        if (!nonempty(gw)) continue;
+        const float* rec = f.records + (int64_t)(gw + u) * f.rec_stride + hoff;
+        const float e = rec[0] == -INFINITY ? 0.f : exp2f(rec[0] - M);
+        acc += e * rec[kRecHead + k];
+      }
+      const int c = TV.chan[k];
+      atomicAdd(&S.o[c], acc * 16777216.f * (float)(1 << TV.shift[k]) / (float)((1 << TV.width[c]) - 1));   // codes entered the MMA as code * 2^-24
+    }
+    __syncthreads();
+    const bool live = L > 0.f;
+    float v = 0.f;
+    if (live) {
+      v = S.o[tid];
+      if (TV.width[tid]) v += tid < 64 ? P0 : P1;
+      v = v / L + p.mean_rot_v[(int64_t)ps * kD + tid];
+    }
+    S.orot[tid] = v;
+    __syncthreads();
+    float outv = 0.f;
+    for (int j = 0; j < kD; j++) outv = fmaf(S.orot[j], wv[j * kD + tid], outv);
+    const int64_t oidx = ((int64_t)b * p.n_q + hk * G + h) * kD + tid;
+    store_from_float(p.out, p.out_dtype, oidx, live ? outv : 0.f);
+    if (p.lse && tid == 0)
+      p.lse[(int64_t)b * p.n_q + hk * G + h] = live ? (M + log2f(L)) / kLog2e + f.desc[u].qconst[h] : -INFINITY;
+  }
+}
+
+}  // namespace spectra
