@@ -43,7 +43,7 @@ FastLayout fast_layout(int64_t n_units, int total_warps, int vs_max) {
 }
 
 // What the host learns from the widths: tile sizes, V strip and block counts.
-struct WidthFacts { int max_tile_k = 0, max_tile_v = 0, max_vstrips = 0, max_vblocks = 0; bool ok = true; };
+struct WidthFacts { int max_tile_k = 0, max_tile_v = 0, max_vstrips = 0, max_vblocks = 0; int vb[4] = {0, 0, 0, 0}; bool ok = true; };
 
 WidthFacts width_facts(const uint8_t* wk, const uint8_t* wv, int64_t n_sets) {
   WidthFacts F;
@@ -65,19 +65,35 @@ WidthFacts width_facts(const uint8_t* wk, const uint8_t* wv, int64_t n_sets) {
         const int blocks = (cnt[0] + 15) / 16 + (cnt[1] + 15) / 16 + (cnt[2] + 15) / 16 + (cnt[3] + 15) / 16;
         F.max_vstrips = strips > F.max_vstrips ? strips : F.max_vstrips;
         F.max_vblocks = blocks > F.max_vblocks ? blocks : F.max_vblocks;
+        for (int c = 0; c < 4; c++) F.vb[c] = (cnt[c] + 15) / 16 > F.vb[c] ? (cnt[c] + 15) / 16 : F.vb[c];
       }
     }
   }
   return F;
 }
 
-template <int NVB>
+template <int Q8, int Q4, int Q2, int Q1>
 int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {
-  if (cudaFuncSetAttribute(attention_mma_kernel<NVB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-      cudaSuccess)
+  if (cudaFuncSetAttribute(attention_mma_kernel<Q8, Q4, Q2, Q1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem) != cudaSuccess)
     return SPECTRA_CUDA_ERROR;
-  attention_mma_kernel<NVB><<<grid, kFastWarps * 32, smem, st>>>(a, f);
+  attention_mma_kernel<Q8, Q4, Q2, Q1><<<grid, kFastWarps * 32, smem, st>>>(a, f);
   return launch_status();
+}
+
+// Quota tuples (V blocks of 16 strips per class 8, 4, 2, 1) the main kernel is built for, smallest first.
+// They cover the width profiles that reverse water-filling produces at 4x to 12x on decaying spectra; anything
+// else runs on the CUDA-core kernel.
+constexpr int kQuotas[][4] = {{0, 1, 8, 2}, {0, 1, 3, 6}, {0, 1, 6, 4}, {0, 8, 2, 2}, {0, 7, 3, 4}};
+constexpr int kNumQuotas = sizeof(kQuotas) / sizeof(kQuotas[0]);
+
+int pick_quota(const int (&vb)[4]) {
+  for (int i = 0; i < kNumQuotas; i++) {
+    bool fits = true;
+    for (int c = 0; c < 4; c++) fits = fits && vb[c] <= kQuotas[i][c];
+    if (fits) return i;
+  }
+  return -1;
 }
 
 }  // namespace
@@ -149,7 +165,8 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
     int ctas_per_sm = 2 * kFastWarps * pair <= budget ? 2 : 1;
     int depth = (int)(budget / ((size_t)ctas_per_sm * kFastWarps * pair));
     if (depth > 4) depth = 4;
-    if (depth >= 1 && F.max_vblocks <= 24 && F.max_vblocks >= 0) {
+    const int quota = pick_quota(F.vb);
+    if (depth >= 1 && quota >= 0) {
       FastLayout L = fast_layout(n_units, sms * ctas_per_sm * kFastWarps, F.max_vstrips);
       if (L.total > workspace_bytes) return SPECTRA_WORKSPACE_TOO_SMALL;
       char* ws = reinterpret_cast<char*>(workspace);
@@ -164,9 +181,13 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
       if (launch_status()) return SPECTRA_CUDA_ERROR;
       const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64;
       const int grid = sms * ctas_per_sm;
-      if (F.max_vblocks <= 10) rc = launch_fast_main<10>(a, f, grid, smem, st);
-      else if (F.max_vblocks <= 16) rc = launch_fast_main<16>(a, f, grid, smem, st);
-      else rc = launch_fast_main<24>(a, f, grid, smem, st);
+      switch (quota) {
+        case 0: rc = launch_fast_main<0, 1, 8, 2>(a, f, grid, smem, st); break;
+        case 1: rc = launch_fast_main<0, 1, 3, 6>(a, f, grid, smem, st); break;
+        case 2: rc = launch_fast_main<0, 1, 6, 4>(a, f, grid, smem, st); break;
+        case 3: rc = launch_fast_main<0, 8, 2, 2>(a, f, grid, smem, st); break;
+        default: rc = launch_fast_main<0, 7, 3, 4>(a, f, grid, smem, st); break;
+      }
       if (rc) return rc;
       attention_mma_combine_kernel<<<(unsigned)n_units, 128, 0, st>>>(a, f);
       return launch_status();

@@ -6,6 +6,10 @@
 // codes into A fragments; fields above bit 10 are first brought down by one shift of the whole word.  The
 // position-dependent power of two is folded into the B operand (exact): on the K side the four MMAs of a chunk
 // take the tokens whose fields share a position, on the V side the probabilities get one scaled copy per class.
+//
+// The V accumulators live in registers, one 16-strip block per accumulator.  Their number and their class must be
+// compile-time facts, so the kernel is instantiated for a few "quota" tuples (blocks per class 8, 4, 2, 1); the
+// host picks the smallest tuple that covers the widths of the call.
 #pragma once
 #include "attention_tc_common.cuh"
 
@@ -16,15 +20,14 @@ namespace spectra {
 template <int W> struct Unpack;
 template <> struct Unpack<8> {   // 4 words, 2 tokens each (bits 0 and 8)
   static constexpr int NW = 4;
-  static constexpr uint32_t kMask = 0x00FF00FFu;
   static __device__ __forceinline__ uint32_t get(const uint32_t (&w)[NW], const uint32_t (&ws)[NW], int ii) {
-    return ((ii & 1) ? ws[ii >> 1] : w[ii >> 1]) & kMask;
+    return ((ii & 1) ? ws[ii >> 1] : w[ii >> 1]) & 0x00FF00FFu;
   }
   static __device__ __forceinline__ void shifted(const uint32_t (&w)[NW], uint32_t (&ws)[NW]) {
 #pragma unroll
     for (int i = 0; i < NW; i++) ws[i] = w[i] >> 8;
   }
-  static __host__ __device__ constexpr int peff(int u) { return 0; }
+  static __host__ __device__ constexpr int peff(int u) { return 0 * u; }
 };
 template <> struct Unpack<4> {   // 2 words, 4 tokens each (bits 0, 4, 8, 12)
   static constexpr int NW = 2;
@@ -80,25 +83,8 @@ __device__ __forceinline__ void ld_halfwords(const unsigned char* p, uint32_t (&
   else w[0] = *reinterpret_cast<const uint16_t*>(p);
 }
 
-// Four MMAs of one 16-strip chunk: MMA u takes tokens u (row gid) and u + 4 (row gid + 8) of the pass.
-template <int W, bool G0, bool G1>
-__device__ __forceinline__ void k_chunk_mma(const uint32_t (&wa)[Unpack<W>::NW], const uint32_t (&wb)[Unpack<W>::NW],
-                                            uint2 b0, uint2 b1, float (&acc)[2][4][4]) {
-  using U = Unpack<W>;
-  uint32_t was[U::NW], wbs[U::NW];
-  U::shifted(wa, was);
-  U::shifted(wb, wbs);
-#pragma unroll
-  for (int u = 0; u < 4; u++) {
-    const uint32_t a0 = U::get(wa, was, u), a1 = U::get(wa, was, u + 4);
-    const uint32_t a2 = U::get(wb, wbs, u), a3 = U::get(wb, wbs, u + 4);
-    if constexpr (G0) mma16816(acc[0][u], a0, a1, a2, a3, hmul2_pow2(b0.x, U::peff(u)), hmul2_pow2(b0.y, U::peff(u)));
-    if constexpr (G1) mma16816(acc[1][u], a0, a1, a2, a3, hmul2_pow2(b1.x, U::peff(u)), hmul2_pow2(b1.y, U::peff(u)));
-  }
-}
-
-// One class of the K tile for one half tile.  Chunks are 16 strips (8 interleaved pairs); chunks whose strips all
-// belong to one scale group and that are complete take the straight path, the others the guarded one.
+// One class of the K tile for one half tile.  A chunk is 16 strips = 8 interleaved pairs; MMA u of a chunk takes
+// tokens u (row gid) and u + 4 (row gid + 8) of the pass, pair slots tig and tig + 4 as its k columns.
 template <int W>
 __device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls, const uint2* __restrict__ kB,
                                         int& chunk_id, int hp, int gid, int tig, int lane, float (&acc)[2][4][4]) {
@@ -106,106 +92,110 @@ __device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls
   constexpr int NW = U::NW;
   const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
   if (n == 0) return;
-  const unsigned char* base = ktile + (cls >> 16) * 16 + 32 * W * tig + 4 * W * gid + (W == 1 ? 0 : 4 * NW * hp);
-  const int full0 = n_g0 >> 4;                 // complete chunks inside scale group 0
-  const int first1 = (n_g0 + 15) >> 4;         // first chunk that lies inside scale group 1
-  const int full_end = n >> 4;                 // complete chunks overall
-  int ci = 0;
-  for (; ci < full0; ci++, chunk_id++) {
-    uint32_t wa[NW], wb[NW];
-    ld_words<NW>(base + 256 * W * ci, wa);
-    ld_words<NW>(base + 256 * W * ci + 128 * W, wb);
-    if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-    const uint2 b0 = __ldg(kB + (chunk_id * 2 + 0) * 32 + lane);
-    k_chunk_mma<W, true, false>(wa, wb, b0, b0, acc);
-  }
-  for (; ci * 16 < n; ci++, chunk_id++) {
-    if (ci >= first1 && ci < full_end) {       // complete chunk inside scale group 1
-      uint32_t wa[NW], wb[NW];
-      ld_words<NW>(base + 256 * W * ci, wa);
-      ld_words<NW>(base + 256 * W * ci + 128 * W, wb);
-      if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-      const uint2 b1 = __ldg(kB + (chunk_id * 2 + 1) * 32 + lane);
-      k_chunk_mma<W, false, true>(wa, wb, b1, b1, acc);
-      continue;
-    }
-    // guarded path: chunk straddles the scale groups and/or is the incomplete last chunk of the class
+  const unsigned char* cbase = ktile + (cls >> 16) * 16;
+  const int thr = 4 * W * gid + (W == 1 ? 0 : 4 * NW * hp);    // this thread's token block inside a pair
+  const int n_ch = (n + 15) >> 4;
+#pragma unroll 1
+  for (int ci = 0; ci < n_ch; ci++, chunk_id++) {
     const int ns = min(16, n - 16 * ci);
+    const unsigned char* cb = cbase + 256 * W * ci;
     uint32_t wa[NW], wb[NW];
+    if (ns == 16) {
+      ld_words<NW>(cb + 32 * W * tig + thr, wa);
+      ld_words<NW>(cb + 32 * W * (tig + 4) + thr, wb);
+    } else if (!(ns & 1)) {
+      // incomplete chunk of whole pairs: slots past the end re-read the last pair (their B rows are zero)
+      const int last = (ns >> 1) - 1;
+      ld_words<NW>(cb + 32 * W * min(tig, last) + thr, wa);
+      ld_words<NW>(cb + 32 * W * min(tig + 4, last) + thr, wb);
+    } else {
+      // the class has an odd number of strips: its last strip is stored alone, half-words in order
 #pragma unroll
-    for (int i = 0; i < NW; i++) { wa[i] = 0u; wb[i] = 0u; }
-    const unsigned char* cb = ktile + (cls >> 16) * 16 + 256 * W * ci;
+      for (int i = 0; i < NW; i++) { wa[i] = 0u; wb[i] = 0u; }
+      const int thr_h = 2 * W * gid + (W == 1 ? 0 : 2 * NW * hp);
+#pragma unroll
+      for (int half = 0; half < 2; half++) {
+        const int ps = tig + 4 * half;
+        uint32_t (&wd)[NW] = half ? wb : wa;
+        if (2 * ps + 1 < ns) ld_words<NW>(cb + 32 * W * ps + thr, wd);
+        else if (2 * ps < ns) ld_halfwords<NW>(cb + 32 * W * ps + thr_h, wd);
+      }
+    }
+    if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
+    uint32_t was[NW], wbs[NW];
+    U::shifted(wa, was);
+    U::shifted(wb, wbs);
+    uint32_t a[4][4];
+#pragma unroll
+    for (int u = 0; u < 4; u++) {
+      a[u][0] = U::get(wa, was, u); a[u][1] = U::get(wa, was, u + 4);
+      a[u][2] = U::get(wb, wbs, u); a[u][3] = U::get(wb, wbs, u + 4);
+    }
+    if (16 * ci < n_g0) {                    // strips of scale group 0 in this chunk
+      const uint2 b = __ldg(kB + (chunk_id * 2 + 0) * 32 + lane);
+#pragma unroll
+      for (int u = 0; u < 4; u++)
+        mma16816(acc[0][u], a[u][0], a[u][1], a[u][2], a[u][3], hmul2_pow2(b.x, U::peff(u)), hmul2_pow2(b.y, U::peff(u)));
+    }
+    if (16 * ci + ns > n_g0) {               // strips of scale group 1 in this chunk
+      const uint2 b = __ldg(kB + (chunk_id * 2 + 1) * 32 + lane);
+#pragma unroll
+      for (int u = 0; u < 4; u++)
+        mma16816(acc[1][u], a[u][0], a[u][1], a[u][2], a[u][3], hmul2_pow2(b.x, U::peff(u)), hmul2_pow2(b.y, U::peff(u)));
+    }
+  }
+}
+
+// One class of the V tile for one half tile, at most Q blocks of 16 strips, accumulators acc_o[OFF .. OFF + Q).
+// The probabilities first get the class's position scales; MMA u of a block contracts the token pairs of B
+// fragments u and u + 4.
+template <int W, int Q, int OFF, int NACC>
+__device__ __forceinline__ void v_class(const unsigned char* vtile, uint32_t cls, int hp, int gid, int tig,
+                                        const uint32_t (&pb)[8], float (&acc_o)[NACC][4]) {
+  if constexpr (Q > 0) {
+    using U = Unpack<W>;
+    constexpr int NW = U::NW;
+    const int n = cls & 0xff;
+    if (n == 0) return;
+    uint32_t pw[8];
+#pragma unroll
+    for (int ii = 0; ii < 8; ii++) pw[ii] = hmul2_pow2(pb[ii], U::peff(ii));
+    const unsigned char* cbase = vtile + (cls >> 16) * 16 + 4 * W * tig + (W == 1 ? 0 : 4 * NW * hp);
+#pragma unroll
+    for (int bi = 0; bi < Q; bi++) {
+      if (16 * bi < n) {
+        uint32_t wa[NW], wb[NW], was[NW], wbs[NW];
+        if (16 * bi + 16 <= n) {
+          ld_words<NW>(cbase + 16 * W * (16 * bi + gid), wa);
+          ld_words<NW>(cbase + 16 * W * (16 * bi + gid + 8), wb);
+        } else {                               // rows past the end repeat the last strip; their results are unused
+          ld_words<NW>(cbase + 16 * W * min(16 * bi + gid, n - 1), wa);
+          ld_words<NW>(cbase + 16 * W * min(16 * bi + gid + 8, n - 1), wb);
+        }
+        if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
+        U::shifted(wa, was);
+        U::shifted(wb, wbs);
+#pragma unroll
+        for (int u = 0; u < 4; u++)
+          mma16816(acc_o[OFF + bi], U::get(wa, was, u), U::get(wb, wbs, u), U::get(wa, was, u + 4),
+                   U::get(wb, wbs, u + 4), pw[u], pw[u + 4]);
+      }
+    }
+  }
+}
+
+// Writes one class's accumulators into a partial record: row r of the class goes to strip index first + r, taking
+// the column of the scale group the strip belongs to.
+template <int Q, int OFF, int NACC>
+__device__ __forceinline__ void store_class(float* rec, uint32_t cls, int first, int gid, const float (&acc_o)[NACC][4]) {
+  const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
+#pragma unroll
+  for (int bi = 0; bi < Q; bi++) {
 #pragma unroll
     for (int half = 0; half < 2; half++) {
-      const int ps = tig + 4 * half;
-      uint32_t (&wd)[NW] = half ? wb : wa;
-      if (2 * ps + 1 < ns) ld_words<NW>(cb + 32 * W * ps + 4 * W * gid + (W == 1 ? 0 : 4 * NW * hp), wd);
-      else if (2 * ps < ns) ld_halfwords<NW>(cb + 32 * W * ps + 2 * W * gid + (W == 1 ? 0 : 2 * NW * hp), wd);
+      const int r = 16 * bi + gid + 8 * half;
+      if (r < n) rec[kRecHead + first + r] = r >= n_g0 ? acc_o[OFF + bi][2 * half + 1] : acc_o[OFF + bi][2 * half];
     }
-    if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-    const bool has0 = 16 * ci < n_g0, has1 = 16 * ci + ns > n_g0;
-    uint2 b0 = make_uint2(0u, 0u), b1 = make_uint2(0u, 0u);
-    if (has0) b0 = __ldg(kB + (chunk_id * 2 + 0) * 32 + lane);
-    if (has1) b1 = __ldg(kB + (chunk_id * 2 + 1) * 32 + lane);
-    k_chunk_mma<W, true, true>(wa, wb, b0, b1, acc);   // a group without strips in the chunk has zero B
-  }
-}
-
-// A fragments of one 16-strip block of the V tile for one half tile (rows gid and gid + 8).
-template <int W>
-__device__ __forceinline__ void v_block_frags(const unsigned char* cbase, int row0, int n, int hp,
-                                              uint32_t (&a)[4][4]) {
-  using U = Unpack<W>;
-  constexpr int NW = U::NW;
-  uint32_t wa[NW], wb[NW], was[NW], wbs[NW];
-  ld_words<NW>(cbase + 16 * W * min(row0, n - 1), wa);       // rows past the end repeat the last strip: unused
-  ld_words<NW>(cbase + 16 * W * min(row0 + 8, n - 1), wb);
-  if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-  U::shifted(wa, was);
-  U::shifted(wb, wbs);
-#pragma unroll
-  for (int u = 0; u < 4; u++) {
-    a[u][0] = U::get(wa, was, u); a[u][1] = U::get(wb, wbs, u);
-    a[u][2] = U::get(wa, was, u + 4); a[u][3] = U::get(wb, wbs, u + 4);
-  }
-}
-
-template <int NVB>
-__device__ __forceinline__ void v_accumulate(float (&acc_o)[NVB][4], int mb, const uint32_t (&a)[4][4],
-                                             const uint32_t (&pw)[8]) {
-  switch (mb) {
-#define SPECTRA_VCASE(K)                                                                        \
-  case K:                                                                                       \
-    if constexpr (K < NVB) {                                                                    \
-      _Pragma("unroll") for (int u = 0; u < 4; u++)                                             \
-          mma16816(acc_o[K < NVB ? K : 0], a[u][0], a[u][1], a[u][2], a[u][3], pw[u], pw[u + 4]); \
-    }                                                                                           \
-    break;
-    SPECTRA_VCASE(0) SPECTRA_VCASE(1) SPECTRA_VCASE(2) SPECTRA_VCASE(3) SPECTRA_VCASE(4) SPECTRA_VCASE(5)
-    SPECTRA_VCASE(6) SPECTRA_VCASE(7) SPECTRA_VCASE(8) SPECTRA_VCASE(9) SPECTRA_VCASE(10) SPECTRA_VCASE(11)
-    SPECTRA_VCASE(12) SPECTRA_VCASE(13) SPECTRA_VCASE(14) SPECTRA_VCASE(15) SPECTRA_VCASE(16) SPECTRA_VCASE(17)
-    SPECTRA_VCASE(18) SPECTRA_VCASE(19) SPECTRA_VCASE(20) SPECTRA_VCASE(21) SPECTRA_VCASE(22) SPECTRA_VCASE(23)
-#undef SPECTRA_VCASE
-    default: break;
-  }
-}
-
-// One class of the V tile for one half tile: the probabilities get the class's position scales, then every block
-// of 16 strips is unpacked and accumulated into its own register accumulator.
-template <int W, int NVB>
-__device__ __forceinline__ void v_class(const unsigned char* vtile, uint32_t cls, int& mb, int hp, int gid, int tig,
-                                        const uint32_t (&pb)[8], float (&acc_o)[NVB][4]) {
-  using U = Unpack<W>;
-  const int n = cls & 0xff;
-  if (n == 0) return;
-  uint32_t pw[8];
-#pragma unroll
-  for (int ii = 0; ii < 8; ii++) pw[ii] = hmul2_pow2(pb[ii], U::peff(ii));
-  const unsigned char* cbase = vtile + (cls >> 16) * 16 + 4 * W * tig + (W == 1 ? 0 : 4 * U::NW * hp);
-  for (int bi = 0; bi * 16 < n; bi++, mb++) {
-    uint32_t a[4][4];
-    v_block_frags<W>(cbase, 16 * bi + gid, n, hp, a);
-    v_accumulate<NVB>(acc_o, mb, a, pw);
   }
 }
 
@@ -224,8 +214,9 @@ struct TileCursor {   // walks the flattened (unit, tile) space; all fields are 
   }
 };
 
-template <int NVB>
+template <int Q8, int Q4, int Q2, int Q1>
 __global__ void __launch_bounds__(kFastWarps * 32, 2) attention_mma_kernel(AttnArgs p, FastArgs f) {
+  constexpr int NACC = Q8 + Q4 + Q2 + Q1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gid = lane >> 2, tig = lane & 3;
@@ -271,7 +262,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 2) attention_mma_kernel(AttnA
     for (int j = 0; j < min(D, count); j++) { start_k(j); start_v(j); }
   issued_k = issued_v = min(D, count);
 
-  float acc_o[NVB][4];
+  float acc_o[NACC][4];
   float m_run = -INFINITY, l_run = 0.f, plo0 = 0.f, plo1 = 0.f;
   uint32_t kcls[4], vcls[4];
   int kmeta0 = -1, kmeta1 = -1, vmeta0 = -1, vmeta1 = -1;
@@ -294,7 +285,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 2) attention_mma_kernel(AttnA
       kB = &d.kB[0][0][0];
       n_seq = p.seq_len[cons.u / p.n_kv];
 #pragma unroll
-      for (int mb = 0; mb < NVB; mb++)
+      for (int mb = 0; mb < NACC; mb++)
 #pragma unroll
         for (int e = 0; e < 4; e++) acc_o[mb][e] = 0.f;
       m_run = -INFINITY; l_run = 0.f; plo0 = 0.f; plo1 = 0.f;
@@ -318,33 +309,33 @@ __global__ void __launch_bounds__(kFastWarps * 32, 2) attention_mma_kernel(AttnA
       k_class<2>(ktile, kcls[2], kB, chunk_id, hp, gid, tig, lane, acc);
       k_class<1>(ktile, kcls[3], kB, chunk_id, hp, gid, tig, lane, acc);
 
-      // per-token group minimum and range of the K tile (fp16), this thread's 8 tokens
+      // per-token group minimum and range of the K tile (fp16), this thread's 8 tokens: token ii is MMA u = ii & 3,
+      // row gid (ii < 4) or gid + 8; the fp16 pair r holds tokens 2r and 2r + 1
       const int tok_off = 2 * (gid * 16 + 8 * hp);
       uint32_t klo0[4] = {0, 0, 0, 0}, kr0[4] = {0, 0, 0, 0}, klo1[4] = {0, 0, 0, 0}, kr1[4] = {0, 0, 0, 0};
       if (kmeta0 >= 0) { ld_words<4>(ktile + kmeta0 + tok_off, klo0); ld_words<4>(ktile + kmeta0 + 256 + tok_off, kr0); }
       if (kmeta1 >= 0) { ld_words<4>(ktile + kmeta1 + tok_off, klo1); ld_words<4>(ktile + kmeta1 + 256 + tok_off, kr1); }
+      if (hp == 1 && issued_k < count) {     // the K slot is free: refill it with the tile D positions ahead
+        __syncwarp();
+        if (lane == 0) { fence_async_smem(); start_k(issued_k % D); }
+        issued_k++;
+      }
       float s[8];
       float mx = -INFINITY;
       const int tok0 = cons.t * kTile + gid * 16 + 8 * hp;
 #pragma unroll
-      for (int ii = 0; ii < 8; ii++) {
-        const int u = ii & 3, cb = (ii >> 2) * 2;             // token ii: MMA u, row gid (ii < 4) or gid + 8
-        const float a0 = acc[0][u][cb] + acc[0][u][cb + 1];   // hi + lo halves of q'
-        const float a1 = acc[1][u][cb] + acc[1][u][cb + 1];
-        const float2 lo0 = h2f2(klo0[ii >> 1]), r0 = h2f2(kr0[ii >> 1]);
-        const float2 lo1 = h2f2(klo1[ii >> 1]), r1 = h2f2(kr1[ii >> 1]);
-        const float l0 = (ii & 1) ? lo0.y : lo0.x, rr0 = (ii & 1) ? r0.y : r0.x;
-        const float l1 = (ii & 1) ? lo1.y : lo1.x, rr1 = (ii & 1) ? r1.y : r1.x;
-        float v = kscale * (rr0 * a0 + rr1 * a1) + l0 * qlo0 + l1 * qlo1;
-        if (tok0 + ii >= n_seq) v = -INFINITY;
-        s[ii] = v;
-        mx = fmaxf(mx, v);
-      }
-      if (hp == 1) {           // the K slot is free: refill it with the tile D positions ahead
-        if (issued_k < count) {
-          __syncwarp();
-          if (lane == 0) { fence_async_smem(); start_k(issued_k % D); }
-          issued_k++;
+      for (int r = 0; r < 4; r++) {
+        const float2 lo0 = h2f2(klo0[r]), r0 = h2f2(kr0[r]), lo1 = h2f2(klo1[r]), r1 = h2f2(kr1[r]);
+#pragma unroll
+        for (int e = 0; e < 2; e++) {
+          const int ii = 2 * r + e, u = ii & 3, cb = (ii >> 2) * 2;
+          const float a0 = acc[0][u][cb] + acc[0][u][cb + 1];   // hi + lo halves of q'
+          const float a1 = acc[1][u][cb] + acc[1][u][cb + 1];
+          float v = kscale * ((e ? r0.y : r0.x) * a0 + (e ? r1.y : r1.x) * a1) + (e ? lo0.y : lo0.x) * qlo0 +
+                    (e ? lo1.y : lo1.x) * qlo1;
+          if (tok0 + ii >= n_seq) v = -INFINITY;
+          s[ii] = v;
+          mx = fmaxf(mx, v);
         }
       }
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
@@ -355,7 +346,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 2) attention_mma_kernel(AttnA
         m_run = mx;
         l_run *= alpha; plo0 *= alpha; plo1 *= alpha;
 #pragma unroll
-        for (int mb = 0; mb < NVB; mb++)
+        for (int mb = 0; mb < NACC; mb++)
 #pragma unroll
           for (int e = 0; e < 4; e++) acc_o[mb][e] *= alpha;
       }
@@ -365,29 +356,30 @@ __global__ void __launch_bounds__(kFastWarps * 32, 2) attention_mma_kernel(AttnA
       if (vmeta1 >= 0) { ld_words<4>(vtile + vmeta1 + tok_off, vlo1); ld_words<4>(vtile + vmeta1 + 256 + tok_off, vr1); }
       // probabilities times the V group ranges, as fp16 pairs (group 0, group 1), transposed into B fragments
       uint32_t pb[8];
+      const float m_use = m_run == -INFINITY ? 0.f : m_run;
 #pragma unroll
-      for (int ii = 0; ii < 8; ii++) {
-        const float pr = m_run == -INFINITY ? 0.f : fast_exp2(s[ii] - m_run);
-        const float2 lo0 = h2f2(vlo0[ii >> 1]), r0 = h2f2(vr0[ii >> 1]);
-        const float2 lo1 = h2f2(vlo1[ii >> 1]), r1 = h2f2(vr1[ii >> 1]);
-        l_run += pr;
-        plo0 = fmaf(pr, (ii & 1) ? lo0.y : lo0.x, plo0);
-        plo1 = fmaf(pr, (ii & 1) ? lo1.y : lo1.x, plo1);
-        const __half2 pk = __floats2half2_rn(pr * ((ii & 1) ? r0.y : r0.x), pr * ((ii & 1) ? r1.y : r1.x));
-        pb[ii] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pk));
+      for (int r = 0; r < 4; r++) {
+        const float2 lo0 = h2f2(vlo0[r]), r0 = h2f2(vr0[r]), lo1 = h2f2(vlo1[r]), r1 = h2f2(vr1[r]);
+#pragma unroll
+        for (int e = 0; e < 2; e++) {
+          const int ii = 2 * r + e;
+          const float pr = fast_exp2(s[ii] - m_use);
+          l_run += pr;
+          plo0 = fmaf(pr, e ? lo0.y : lo0.x, plo0);
+          plo1 = fmaf(pr, e ? lo1.y : lo1.x, plo1);
+          const __half2 pk = __floats2half2_rn(pr * (e ? r0.y : r0.x), pr * (e ? r1.y : r1.x));
+          pb[ii] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pk));
+        }
       }
       // ------------------------------------------------------------ P~ x V codes
-      int mb = 0;
-      v_class<8, NVB>(vtile, vcls[0], mb, hp, gid, tig, pb, acc_o);
-      v_class<4, NVB>(vtile, vcls[1], mb, hp, gid, tig, pb, acc_o);
-      v_class<2, NVB>(vtile, vcls[2], mb, hp, gid, tig, pb, acc_o);
-      v_class<1, NVB>(vtile, vcls[3], mb, hp, gid, tig, pb, acc_o);
-      if (hp == 1) {
-        if (issued_v < issued_k) {
-          __syncwarp();
-          if (lane == 0) { fence_async_smem(); start_v(issued_v % D); }
-          issued_v++;
-        }
+      v_class<8, Q8, 0, NACC>(vtile, vcls[0], hp, gid, tig, pb, acc_o);
+      v_class<4, Q4, Q8, NACC>(vtile, vcls[1], hp, gid, tig, pb, acc_o);
+      v_class<2, Q2, Q8 + Q4, NACC>(vtile, vcls[2], hp, gid, tig, pb, acc_o);
+      v_class<1, Q1, Q8 + Q4 + Q2, NACC>(vtile, vcls[3], hp, gid, tig, pb, acc_o);
+      if (hp == 1 && issued_v < issued_k) {
+        __syncwarp();
+        if (lane == 0) { fence_async_smem(); start_v(issued_v % D); }
+        issued_v++;
       }
     }
     // ------------------------------------------------------------ end of this warp's share of the unit?
@@ -403,26 +395,10 @@ __global__ void __launch_bounds__(kFastWarps * 32, 2) attention_mma_kernel(AttnA
       float* rec = f.records + (int64_t)(gw + cons.u) * f.rec_stride + tig * (kRecHead + f.vs_max);
       if (gid == 0) { rec[0] = m_run; rec[1] = l; rec[2] = q0; rec[3] = q1; }
       const UnitDesc& d = f.desc[cons.u];
-      int mbase = 0;
-#pragma unroll
-      for (int c = 0; c < 4; c++) {
-        const uint32_t cls = vcls[c];
-        const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
-        const int first = d.vfirst[c];
-        const int nblk = (n + 15) >> 4;
-#pragma unroll
-        for (int mb = 0; mb < NVB; mb++) {
-          const int bi = mb - mbase;
-          if (bi >= 0 && bi < nblk) {
-#pragma unroll
-            for (int half = 0; half < 2; half++) {
-              const int r = 16 * bi + gid + 8 * half;
-              if (r < n) rec[kRecHead + first + r] = r >= n_g0 ? acc_o[mb][2 * half + 1] : acc_o[mb][2 * half];
-            }
-          }
-        }
-        mbase += nblk;
-      }
+      store_class<Q8, 0, NACC>(rec, vcls[0], d.vfirst[0], gid, acc_o);
+      store_class<Q4, Q8, NACC>(rec, vcls[1], d.vfirst[1], gid, acc_o);
+      store_class<Q2, Q8 + Q4, NACC>(rec, vcls[2], d.vfirst[2], gid, acc_o);
+      store_class<Q1, Q8 + Q4 + Q2, NACC>(rec, vcls[3], d.vfirst[3], gid, acc_o);
       fresh = true;
     }
     cons.next(f);
