@@ -1,5 +1,6 @@
 // spectra_decode_attention entry point and host-side helpers of the library.
 #include "attention_tc_main.cuh"
+#include "attention_tc_combine.cuh"
 
 using namespace spectra;
 
@@ -107,7 +108,7 @@ extern "C" size_t spectra_attention_workspace_bytes(const spectra_config* cfg, i
   const size_t generic = (size_t)n_units * splits * (n_q_heads / n_kv_heads) * kPartialStride * sizeof(float) + 16;
   int sms = sm_count();
   if (sms <= 0) sms = 160;
-  const size_t fast = fast_layout(n_units, sms * 2 * kFastWarps, kMaxStrips).total;
+  const size_t fast = fast_layout(n_units, sms * 3 * kFastWarps, kMaxStrips).total;
   return generic > fast ? generic : fast;
 }
 
@@ -162,7 +163,7 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
     const int slot_v = (int)align_up((size_t)(F.max_tile_v > 16 ? F.max_tile_v : 16), 128);
     const size_t pair = (size_t)slot_k + slot_v;
     const size_t budget = 200 * 1024;
-    int ctas_per_sm = 2 * kFastWarps * pair <= budget ? 2 : 1;
+    int ctas_per_sm = 3 * kFastWarps * pair <= budget ? 3 : (2 * kFastWarps * pair <= budget ? 2 : 1);
     int depth = (int)(budget / ((size_t)ctas_per_sm * kFastWarps * pair));
     if (depth > 4) depth = 4;
     const int quota = pick_quota(F.vb);
@@ -177,7 +178,7 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
       f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = F.max_vstrips;
       f.n_units = (int)n_units; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
-      attention_prep_kernel<<<(unsigned)n_units + 1, 128, sizeof(PrepSmem), st>>>(a, f);
+      attention_prep_kernel<<<(unsigned)n_units + 1, kPrepThreads, sizeof(PrepSmem), st>>>(a, f);
       if (launch_status()) return SPECTRA_CUDA_ERROR;
       const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64;
       const int grid = sms * ctas_per_sm;
@@ -189,7 +190,7 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
         default: rc = launch_fast_main<0, 7, 3, 4>(a, f, grid, smem, st); break;
       }
       if (rc) return rc;
-      attention_mma_combine_kernel<<<(unsigned)n_units, 128, 0, st>>>(a, f);
+      attention_mma_combine_kernel<<<(unsigned)(n_units * gqa), 128, 0, st>>>(a, f);
       return launch_status();
     }
   }

@@ -41,6 +41,8 @@ struct alignas(16) UnitDesc {
   float kcorr[4][2];            // sum_k 2^w_k (B_hi + B_lo) per head and scale group
   float qlo[4][2];              // sum of q' over the active channels of a scale group
   float qconst[4];              // q' . m'_K (natural-log units)
+  uint8_t vchan[kMaxStrips];    // channel of V strip k
+  float vcoef[kMaxStrips];      // 2^24 * 2^shift / (2^width - 1): turns the strip's accumulator into its share of yhat
   uint2 kB[kKcMax][2][32];      // [chunk][scale group][lane] -> (b0, b1)
 };
 
@@ -141,17 +143,22 @@ __device__ inline uint32_t pack_cls(const StripTable& T, int c) {
   return (uint32_t)n | ((uint32_t)n_g0 << 8) | ((uint32_t)(T.class_off[c] / 16) << 16);
 }
 
-__global__ void __launch_bounds__(128) attention_prep_kernel(AttnArgs p, FastArgs f) {
+constexpr int kPrepThreads = 512;
+
+__global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p, FastArgs f) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   PrepSmem& S = *reinterpret_cast<PrepSmem*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kWarps = kPrepThreads / 32;
   if ((int)blockIdx.x == f.n_units) {
     // ---- tile prefix sums over units and each worker warp's first unit
     const int n_units = f.n_units;
     const int per = (n_units + 127) / 128;
     int local = 0;
-    for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (p.seq_len[i / p.n_kv] + kTile - 1) / kTile;
-    S.scan[tid] = local;
+    if (tid < 128) {
+      for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (p.seq_len[i / p.n_kv] + kTile - 1) / kTile;
+      S.scan[tid] = local;
+    }
     __syncthreads();
     if (tid == 0) {
       int run = 0;
@@ -159,20 +166,28 @@ __global__ void __launch_bounds__(128) attention_prep_kernel(AttnArgs p, FastArg
       f.tile_prefix[n_units] = run;
     }
     __syncthreads();
-    int run = S.scan[tid];
-    for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) {
-      f.tile_prefix[i] = run;
-      run += (p.seq_len[i / p.n_kv] + kTile - 1) / kTile;
+    if (tid < 128) {
+      int run = S.scan[tid];
+      for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) {
+        f.tile_prefix[i] = run;
+        run += (p.seq_len[i / p.n_kv] + kTile - 1) / kTile;
+      }
     }
     __syncthreads();
     __threadfence_block();
-    const long long total = f.tile_prefix[n_units];
-    for (int gw = tid; gw < f.total_warps; gw += 128) {
+    __shared__ int sprefix[4097];          // units of one call; larger calls search the global copy
+    const bool in_smem = n_units <= 4096;
+    if (in_smem)
+      for (int i = tid; i <= n_units; i += kPrepThreads) sprefix[i] = f.tile_prefix[i];
+    __syncthreads();
+    const int* pre = in_smem ? sprefix : f.tile_prefix;
+    const long long total = pre[n_units];
+    for (int gw = tid; gw < f.total_warps; gw += kPrepThreads) {
       const long long g0 = (long long)gw * total / f.total_warps;
       int lo = 0, hi = n_units;             // first unit whose end is beyond g0
       while (lo < hi) {
         const int mid = (lo + hi) >> 1;
-        if (f.tile_prefix[mid + 1] > g0) hi = mid; else lo = mid + 1;
+        if (pre[mid + 1] > g0) hi = mid; else lo = mid + 1;
       }
       f.warp_unit[gw] = lo;
     }
@@ -187,13 +202,13 @@ __global__ void __launch_bounds__(128) attention_prep_kernel(AttnArgs p, FastArg
   const StripTable& TK = S.tk;
   const StripTable& TV = S.tv;
   UnitDesc& D = f.desc[u];
-  for (int idx = tid; idx < kFastGqa * kD; idx += 128) {
+  for (int idx = tid; idx < kFastGqa * kD; idx += kPrepThreads) {
     const int h = idx / kD, i = idx - h * kD;
     S.qraw[h][i] = h < G ? load_as_float(p.q, p.q_dtype, ((int64_t)b * p.n_q + hk * G + h) * kD + i) : 0.f;
   }
   __syncthreads();
   const float* wk = p.w_dec_k + (int64_t)ps * kD * kD;
-  for (int j = warp; j < kD; j += 4) {
+  for (int j = warp; j < kD; j += kWarps) {
     const float4 wrow = *reinterpret_cast<const float4*>(wk + j * kD + lane * 4);
 #pragma unroll
     for (int h = 0; h < kFastGqa; h++) {
@@ -207,7 +222,7 @@ __global__ void __launch_bounds__(128) attention_prep_kernel(AttnArgs p, FastArg
   __syncthreads();
   // per-head power-of-two normalisation so that the fp16 hi/lo split of q'' = q' 2^shift / L is well conditioned
   const int nk = TK.n_strips;
-  {
+  if (warp < kFastGqa) {
     const int h = warp;  // one warp per head
     float mx = 0.f;
     for (int k = lane; k < nk; k += 32) {
@@ -254,7 +269,7 @@ __global__ void __launch_bounds__(128) attention_prep_kernel(AttnArgs p, FastArg
   for (int c = 0; c < 4; c++) {
     const int first = TK.class_first[c], n = TK.class_first[c + 1] - first;
     const int nch = (n + 15) / 16;
-    for (int idx = tid; idx < nch * 2 * 32; idx += 128) {
+    for (int idx = tid; idx < nch * 2 * 32; idx += kPrepThreads) {
       const int ci = idx / 64, g = (idx >> 5) & 1, ln = idx & 31;
       const int gid = ln >> 2, tg = ln & 3, h = gid >> 1, part = gid & 1;
       uint32_t r[2];
@@ -276,90 +291,19 @@ __global__ void __launch_bounds__(128) attention_prep_kernel(AttnArgs p, FastArg
     }
     chunk0 += nch;
   }
-  if (tid < 4) {
-    D.kcls[tid] = pack_cls(TK, tid);
-    D.vcls[tid] = pack_cls(TV, tid);
-    D.vfirst[tid] = TV.class_first[tid];
-  }
+  if (tid >= 64 && tid < 68) D.kcls[tid - 64] = pack_cls(TK, tid - 64);      // spread over different warps
+  if (tid >= 96 && tid < 100) D.vcls[tid - 96] = pack_cls(TV, tid - 96);
+  if (tid >= 128 && tid < 132) D.vfirst[tid - 128] = TV.class_first[tid - 128];
   if (tid == 0) {
     D.tbk = TK.tile_bytes; D.tbv = TV.tile_bytes;
     D.kmeta[0] = TK.meta_off[0]; D.kmeta[1] = TK.meta_off[1];
     D.vmeta[0] = TV.meta_off[0]; D.vmeta[1] = TV.meta_off[1];
     D.n_vstrips = TV.n_strips; D.pad0 = 0;
   }
-}
-
-// ------------------------------------------------------------------------------------------------ combine kernel
-struct CombineSmem {
-  StripTable tv;
-  float o[kD];
-  float orot[kD];
-};
-
-__global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, FastArgs f) {
-  __shared__ CombineSmem S;
-  const int tid = threadIdx.x;
-  const int u = blockIdx.x;
-  const int b = u / p.n_kv, hk = u - b * p.n_kv;
-  const int ps = (int)(u % p.n_param_sets);
-  const int G = p.gqa;
-  build_strip_table(S.tv, p.widths_v + (int64_t)ps * kD, 64);
-  const StripTable& TV = S.tv;
-  const long long total = f.tile_prefix[f.n_units];
-  const long long ta = f.tile_prefix[u], tb = f.tile_prefix[u + 1];
-  const float* wv = p.w_dec_v + (int64_t)ps * kD * kD;
-  // workers whose ranges intersect this unit: the largest gw with floor(gw * total / W) <= tile
-  int gw_first = 0, gw_last = -1;
-  if (tb > ta) {
-    gw_first = (int)(((ta + 1) * f.total_warps + total - 1) / total) - 1;
-    gw_last = (int)(((tb - 1 + 1) * (long long)f.total_warps + total - 1) / total) - 1;
-  }
-  // a worker whose range is empty wrote no record
-  auto nonempty = [&](int gw) {
-    return (long long)(gw + 1) * total / f.total_warps > (long long)gw * total / f.total_warps;
-  };
-  for (int h = 0; h < G; h++) {
-    const int64_t hoff = (int64_t)h * (kRecHead + f.vs_max);
-    float M = -INFINITY;
-    for (int gw = gw_first; gw <= gw_last; gw++)
-      if (nonempty(gw)) M = fmaxf(M, f.records[(int64_t)(gw + u) * f.rec_stride + hoff]);
-    float L = 0.f, P0 = 0.f, P1 = 0.f;
-    for (int gw = gw_first; gw <= gw_last; gw++) {
-      if (!nonempty(gw)) continue;
-      const float* rec = f.records + (int64_t)(gw + u) * f.rec_stride + hoff;
-      const float e = rec[0] == -INFINITY ? 0.f : exp2f(rec[0] - M);
-      L += e * rec[1]; P0 += e * rec[2]; P1 += e * rec[3];
-    }
-    __syncthreads();
-    S.o[tid] = 0.f;
-    __syncthreads();
-    for (int k = tid; k < TV.n_strips; k += 128) {
-      float acc = 0.f;
-      for (int gw = gw_first; gw <= gw_last; gw++) {
-        if (!nonempty(gw)) continue;
-        const float* rec = f.records + (int64_t)(gw + u) * f.rec_stride + hoff;
-        const float e = rec[0] == -INFINITY ? 0.f : exp2f(rec[0] - M);
-        acc += e * rec[kRecHead + k];
-      }
-      const int c = TV.chan[k];
-      atomicAdd(&S.o[c], acc * 16777216.f * (float)(1 << TV.shift[k]) / (float)((1 << TV.width[c]) - 1));   // codes entered the MMA as code * 2^-24
-    }
-    __syncthreads();
-    const bool live = L > 0.f;
-    float v = 0.f;
-    if (live) {
-      v = S.o[tid];
-      if (TV.width[tid]) v += tid < 64 ? P0 : P1;
-      v = v / L + p.mean_rot_v[(int64_t)ps * kD + tid];
-    }
-    S.orot[tid] = v;
-    __syncthreads();
-    float outv = 0.f;
-    for (int j = 0; j < kD; j++) outv = fmaf(S.orot[j], wv[j * kD + tid], outv);
-    const int64_t oidx = ((int64_t)b * p.n_q + hk * G + h) * kD + tid;
-    store_from_float(p.out, p.out_dtype, oidx, live ? outv : 0.f);
-    if (p.lse && tid == 0)
-      p.lse[(int64_t)b * p.n_q + hk * G + h] = live ? (M + log2f(L)) / kLog2e + f.desc[u].qconst[h] : -INFINITY;
+  for (int k = tid; k < TV.n_strips; k += kPrepThreads) {
+    const int c = TV.chan[k];
+    D.vchan[k] = (uint8_t)c;
+    D.vcoef[k] = 16777216.f * (float)(1 << TV.shift[k]) / (float)((1 << TV.width[c]) - 1);
   }
 }
 

@@ -215,7 +215,7 @@ struct TileCursor {   // walks the flattened (unit, tile) space; all fields are 
 };
 
 template <int Q8, int Q4, int Q2, int Q1>
-__global__ void __launch_bounds__(kFastWarps * 32, 2) attention_mma_kernel(AttnArgs p, FastArgs f) {
+__global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnArgs p, FastArgs f) {
   constexpr int NACC = Q8 + Q4 + Q2 + Q1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

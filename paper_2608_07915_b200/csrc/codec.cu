@@ -2,6 +2,7 @@
 // One CTA of 128 threads owns one (unit-side, tile); no other CTA touches that tile, so the
 // read-modify-write of a partly filled tail tile needs no atomics.
 #include "common.cuh"
+#include "encode_append.cuh"
 
 namespace spectra {
 
@@ -245,6 +246,12 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
   if (!x || !pos0 || !widths || !cache || !unit_offset) return SPECTRA_INVALID_ARG;
   if (!(flags & SPECTRA_ROTATED_INPUT) && (!w_enc || !mean_rot)) return SPECTRA_INVALID_ARG;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
+  if (n_new <= kAppendMaxTokens) {   // decode-step appends: one light CTA per unit-side
+    AppendArgs ap{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
+                  w_enc, mean_rot, widths, cache, unit_offset, status_word};
+    encode_append_kernel<<<(unsigned)n_units, 128, 0, (cudaStream_t)stream>>>(ap);
+    return launch_status();
+  }
   EncodeArgs a{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
                w_enc, mean_rot, widths, cache, unit_offset, status_word};
   if (cudaFuncSetAttribute(encode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CodecSmem)) !=
