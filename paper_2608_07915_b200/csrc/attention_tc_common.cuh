@@ -26,7 +26,7 @@
 namespace spectra {
 
 constexpr int kFastGqa = 4;
-constexpr int kKcMax = 28;       // upper bound of 16-strip chunks in a K tile (384 strips in 4 classes)
+constexpr int kKcMax = 32;       // upper bound of 16-strip chunks in a K tile (two runs per class)
 constexpr int kFastWarps = 4;    // warps per CTA of the main kernel
 constexpr int kRecHead = 4;      // floats of a record's per-head header: m, l, plo0, plo1
 constexpr float kLog2e = 1.4426950408889634f;
@@ -43,7 +43,7 @@ struct alignas(16) UnitDesc {
   float qconst[4];              // q' . m'_K (natural-log units)
   uint8_t vchan[kMaxStrips];    // channel of V strip k
   float vcoef[kMaxStrips];      // 2^24 * 2^shift / (2^width - 1): turns the strip's accumulator into its share of yhat
-  uint2 kB[kKcMax][2][32];      // [chunk][scale group][lane] -> (b0, b1)
+  uint2 kB[kKcMax][4][32];      // [chunk][MMA u of the chunk][lane] -> (b0, b1)
 };
 
 struct FastArgs {
@@ -264,32 +264,42 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
     }
   }
   __syncthreads();
-  // B fragments: chunk = 16 consecutive strips of a class; column n = head (n >> 1), hi (n & 1 == 0) or lo half
+  // B fragments.  Each class is walked as two runs, one per scale group: run 0 = strips [0, n_g0), run 1 = strips
+  // [n_g0 rounded down to a pair, n); a chunk is 16 consecutive strips of a run and contributes to that run's
+  // scale group only (rows of the other group, or past the end, are zero).  Column n = head (n >> 1), hi
+  // (n & 1 == 0) or lo half of the fp16 split.  Variant u carries the factor 2^-p_eff(u) of the unpacking.
   int chunk0 = 0;
   for (int c = 0; c < 4; c++) {
     const int first = TK.class_first[c], n = TK.class_first[c + 1] - first;
-    const int nch = (n + 15) / 16;
-    for (int idx = tid; idx < nch * 2 * 32; idx += kPrepThreads) {
-      const int ci = idx / 64, g = (idx >> 5) & 1, ln = idx & 31;
+    int n_g0 = 0;
+    for (int k = first; k < first + n; k++) n_g0 += TK.chan[k] < 64;      // every thread: at most 128 steps
+    const int s1 = n_g0 & ~1;
+    const int nch0 = (n_g0 + 15) / 16, nch1 = n > n_g0 ? (n - s1 + 15) / 16 : 0;
+    const int w = 8 >> c;
+    for (int idx = tid; idx < (nch0 + nch1) * 4 * 32; idx += kPrepThreads) {
+      const int ch = idx >> 7, u4 = (idx >> 5) & 3, ln = idx & 31;
+      const int run = ch >= nch0 ? 1 : 0;
+      const int start = run ? s1 + 16 * (ch - nch0) : 16 * ch;
       const int gid = ln >> 2, tg = ln & 3, h = gid >> 1, part = gid & 1;
+      const int pe = w == 8 ? 0 : (w == 4 ? 4 * (u4 & 1) : (w == 2 ? 2 * u4 : u4));
+      const __half scale = __ushort_as_half((unsigned short)((15 - pe) << 10));
       uint32_t r[2];
 #pragma unroll
       for (int half = 0; half < 2; half++) {
         uint32_t v = 0;
 #pragma unroll
         for (int e = 0; e < 2; e++) {
-          const int krow = 2 * tg + 8 * half + e;
-          const int k = first + 16 * ci + krow;
+          const int strip = start + 2 * tg + 8 * half + e;
           uint16_t bits = 0;
-          if (16 * ci + krow < n && h < G && (TK.chan[k] >= 64 ? 1 : 0) == g)
-            bits = __half_as_ushort(part ? S.blo[h][k] : S.bhi[h][k]);
+          if (strip < n && h < G && (TK.chan[first + strip] >= 64 ? 1 : 0) == run)
+            bits = __half_as_ushort(__hmul(part ? S.blo[h][first + strip] : S.bhi[h][first + strip], scale));
           v |= (uint32_t)bits << (16 * e);
         }
         r[half] = v;
       }
-      if (chunk0 + ci < kKcMax) D.kB[chunk0 + ci][g][ln] = make_uint2(r[0], r[1]);
+      if (chunk0 + ch < kKcMax) D.kB[chunk0 + ch][u4][ln] = make_uint2(r[0], r[1]);
     }
-    chunk0 += nch;
+    chunk0 += nch0 + nch1;
   }
   if (tid >= 64 && tid < 68) D.kcls[tid - 64] = pack_cls(TK, tid - 64);      // spread over different warps
   if (tid >= 96 && tid < 100) D.vcls[tid - 96] = pack_cls(TV, tid - 96);

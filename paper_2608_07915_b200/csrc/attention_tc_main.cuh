@@ -83,29 +83,50 @@ __device__ __forceinline__ void ld_halfwords(const unsigned char* p, uint32_t (&
   else w[0] = *reinterpret_cast<const uint16_t*>(p);
 }
 
-// One class of the K tile for one half tile.  A chunk is 16 strips = 8 interleaved pairs; MMA u of a chunk takes
-// tokens u (row gid) and u + 4 (row gid + 8) of the pass, pair slots tig and tig + 4 as its k columns.
+// Four MMAs of one chunk into one scale group's accumulators: MMA u takes tokens u (row gid) and u + 4 (row
+// gid + 8) of the pass, pair slots tig and tig + 4 as its k columns, and B variant u (scaled by 2^-p_eff(u)).
 template <int W>
-__device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls, const uint2* __restrict__ kB,
-                                        int& chunk_id, int hp, int gid, int tig, int lane, float (&acc)[2][4][4]) {
+__device__ __forceinline__ void k_chunk(uint32_t (&wa)[Unpack<W>::NW], uint32_t (&wb)[Unpack<W>::NW], int hp,
+                                        const uint2* __restrict__ kb, float (&acc)[4][4]) {
   using U = Unpack<W>;
   constexpr int NW = U::NW;
-  const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
-  if (n == 0) return;
-  const unsigned char* cbase = ktile + (cls >> 16) * 16;
+  if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
+  uint32_t was[NW], wbs[NW];
+  U::shifted(wa, was);
+  U::shifted(wb, wbs);
+#pragma unroll
+  for (int u = 0; u < 4; u++) {
+    const uint2 b = __ldg(kb + u * 32);
+    mma16816(acc[u], U::get(wa, was, u), U::get(wa, was, u + 4), U::get(wb, wbs, u), U::get(wb, wbs, u + 4), b.x, b.y);
+  }
+}
+
+// One run of a class of the K tile for one half tile: strips [start, end) of the class (start even), all of one
+// scale group.  Chunks of 16 strips = 8 interleaved pairs; `n` = strips in the class (an odd n means that the last
+// strip is stored alone).
+template <int W>
+__device__ __forceinline__ void k_run(const unsigned char* cbase, int n, int start, int end, const uint2* __restrict__& kb,
+                                      int hp, int gid, int tig, float (&acc)[4][4]) {
+  using U = Unpack<W>;
+  constexpr int NW = U::NW;
   const int thr = 4 * W * gid + (W == 1 ? 0 : 4 * NW * hp);    // this thread's token block inside a pair
-  const int n_ch = (n + 15) >> 4;
+  const unsigned char* pa = cbase + 16 * W * start + 32 * W * tig + thr;
+  int s = start;
 #pragma unroll 1
-  for (int ci = 0; ci < n_ch; ci++, chunk_id++) {
-    const int ns = min(16, n - 16 * ci);
-    const unsigned char* cb = cbase + 256 * W * ci;
+  for (; s + 16 <= end && s + 16 <= (n & ~1); s += 16, pa += 256 * W, kb += 4 * 32) {   // complete chunks
     uint32_t wa[NW], wb[NW];
-    if (ns == 16) {
-      ld_words<NW>(cb + 32 * W * tig + thr, wa);
-      ld_words<NW>(cb + 32 * W * (tig + 4) + thr, wb);
-    } else if (!(ns & 1)) {
-      // incomplete chunk of whole pairs: slots past the end re-read the last pair (their B rows are zero)
-      const int last = (ns >> 1) - 1;
+    ld_words<NW>(pa, wa);
+    ld_words<NW>(pa + 128 * W, wb);
+    k_chunk<W>(wa, wb, hp, kb, acc);
+  }
+#pragma unroll 1
+  for (; s < end; s += 16, kb += 4 * 32) {                     // the tail of the run
+    const int avail = min(16, n - s);                          // strips stored from s on (B rows past `end` are zero)
+    const unsigned char* cb = cbase + 16 * W * s;
+    uint32_t wa[NW], wb[NW];
+    if (!(avail & 1)) {
+      // whole pairs only: slots past the end re-read the last pair
+      const int last = (avail >> 1) - 1;
       ld_words<NW>(cb + 32 * W * min(tig, last) + thr, wa);
       ld_words<NW>(cb + 32 * W * min(tig + 4, last) + thr, wb);
     } else {
@@ -117,33 +138,24 @@ __device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls
       for (int half = 0; half < 2; half++) {
         const int ps = tig + 4 * half;
         uint32_t (&wd)[NW] = half ? wb : wa;
-        if (2 * ps + 1 < ns) ld_words<NW>(cb + 32 * W * ps + thr, wd);
-        else if (2 * ps < ns) ld_halfwords<NW>(cb + 32 * W * ps + thr_h, wd);
+        if (2 * ps + 1 < avail) ld_words<NW>(cb + 32 * W * ps + thr, wd);
+        else if (2 * ps < avail) ld_halfwords<NW>(cb + 32 * W * ps + thr_h, wd);
       }
     }
-    if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-    uint32_t was[NW], wbs[NW];
-    U::shifted(wa, was);
-    U::shifted(wb, wbs);
-    uint32_t a[4][4];
-#pragma unroll
-    for (int u = 0; u < 4; u++) {
-      a[u][0] = U::get(wa, was, u); a[u][1] = U::get(wa, was, u + 4);
-      a[u][2] = U::get(wb, wbs, u); a[u][3] = U::get(wb, wbs, u + 4);
-    }
-    if (16 * ci < n_g0) {                    // strips of scale group 0 in this chunk
-      const uint2 b = __ldg(kB + (chunk_id * 2 + 0) * 32 + lane);
-#pragma unroll
-      for (int u = 0; u < 4; u++)
-        mma16816(acc[0][u], a[u][0], a[u][1], a[u][2], a[u][3], hmul2_pow2(b.x, U::peff(u)), hmul2_pow2(b.y, U::peff(u)));
-    }
-    if (16 * ci + ns > n_g0) {               // strips of scale group 1 in this chunk
-      const uint2 b = __ldg(kB + (chunk_id * 2 + 1) * 32 + lane);
-#pragma unroll
-      for (int u = 0; u < 4; u++)
-        mma16816(acc[1][u], a[u][0], a[u][1], a[u][2], a[u][3], hmul2_pow2(b.x, U::peff(u)), hmul2_pow2(b.y, U::peff(u)));
-    }
+    k_chunk<W>(wa, wb, hp, kb, acc);
   }
+}
+
+// One class of the K tile for one half tile: run 0 = the strips of scale group 0, run 1 = those of group 1
+// (starting at the pair that holds its first strip).
+template <int W>
+__device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls, const uint2* __restrict__& kb,
+                                        int hp, int gid, int tig, float (&acc)[2][4][4]) {
+  const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
+  if (n == 0) return;
+  const unsigned char* cbase = ktile + (cls >> 16) * 16;
+  if (n_g0 > 0) k_run<W>(cbase, n, 0, n_g0, kb, hp, gid, tig, acc[0]);
+  if (n > n_g0) k_run<W>(cbase, n, n_g0 & ~1, n, kb, hp, gid, tig, acc[1]);
 }
 
 // One class of the V tile for one half tile, at most Q blocks of 16 strips, accumulators acc_o[OFF .. OFF + Q).
@@ -303,11 +315,11 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
         for (int u = 0; u < 4; u++)
 #pragma unroll
           for (int e = 0; e < 4; e++) acc[g][u][e] = 0.f;
-      int chunk_id = 0;
-      k_class<8>(ktile, kcls[0], kB, chunk_id, hp, gid, tig, lane, acc);
-      k_class<4>(ktile, kcls[1], kB, chunk_id, hp, gid, tig, lane, acc);
-      k_class<2>(ktile, kcls[2], kB, chunk_id, hp, gid, tig, lane, acc);
-      k_class<1>(ktile, kcls[3], kB, chunk_id, hp, gid, tig, lane, acc);
+      const uint2* kb = kB + lane;       // walks the B fragment table in chunk order
+      k_class<8>(ktile, kcls[0], kb, hp, gid, tig, acc);
+      k_class<4>(ktile, kcls[1], kb, hp, gid, tig, acc);
+      k_class<2>(ktile, kcls[2], kb, hp, gid, tig, acc);
+      k_class<1>(ktile, kcls[3], kb, hp, gid, tig, acc);
 
       // per-token group minimum and range of the K tile (fp16), this thread's 8 tokens: token ii is MMA u = ii & 3,
       // row gid (ii < 4) or gid + 8; the fp16 pair r holds tokens 2r and 2r + 1

@@ -20,7 +20,6 @@ struct AppendArgs {
 __global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
   __shared__ float xs[kAppendMaxTokens][kD];
   __shared__ float red_lo[4], red_hi[4];
-  __shared__ int red_any[4];
   __shared__ int cls_cnt[4][4];          // [class][warp]: strips of the class owned by the warp's channels
   __shared__ int grp_act[kMaxGroups];
   const int u = blockIdx.x;
