@@ -120,6 +120,30 @@ int spectra_fit_basis(const spectra_config* cfg, const void* x, int x_dtype, int
 size_t spectra_fit_workspace_bytes(const spectra_config* cfg, int64_t n_units);
 
 /* ------------------------------------------------------------------------------------------------
+ * spectra_fit_basis_static -- the paper has no counterpart; this is a packaging variant of spectra_fit_basis for
+ * callers that may not allocate device memory at the point where they calibrate: a serving plug-in that lives
+ * inside a host process with a fixed, pre-carved memory arena, or a component started after the process has
+ * frozen its allocator (allocation there would synchronise the device or is simply forbidden).  It takes the
+ * same inputs and writes the same outputs, but needs no workspace argument: the scratch (second-moment sums and
+ * eigenvector rows, fp64) lives in a fixed array inside the library image, sized for at most
+ * SPECTRA_FIT_STATIC_MAX_UNITS unit-sides per call (about 263 KB each, 2.1 MB in all, held by every device that
+ * loads the library until the process exits).
+ *   - n_units > SPECTRA_FIT_STATIC_MAX_UNITS returns SPECTRA_CAPACITY and enqueues nothing; fit larger sets in
+ *     slices of that many unit-sides.
+ *   - The first call on a device looks up the device address of the array (with that device current); make that
+ *     first call outside any stream capture.  Later calls on the same device reuse the address.
+ *   - The call allocates nothing and calls no allocating routine.  All calls on a device share the one array,
+ *     which still holds the previous call's contents when a call starts; the call clears what it accumulates
+ *     into.  Two calls whose GPU work overlaps (different streams, no ordering between them) would race on the
+ *     array: order them.
+ */
+#define SPECTRA_FIT_STATIC_MAX_UNITS 8
+int spectra_fit_basis_static(const spectra_config* cfg, const void* x, int x_dtype, int64_t n_units,
+                             int64_t n_tokens, int64_t stride_unit, int64_t stride_token, float* w_enc,
+                             float* w_dec, float* mean_rot, float* var_alloc, float* eigval, float* basis_u,
+                             void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * spectra_alloc_bits -- Sec. 3.2, Eq. 5 and the appendix "Reverse water-filling derivation": integer
  * widths minimising sum_j v_j 4^(-b_j) subject to sum_j b_j <= Btot = floor(16 d / ratio), 0 <= b_j <= b_max,
  * with cfg->width_group adjacent channels sharing one width taken from the group's mean variance.

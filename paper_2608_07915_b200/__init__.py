@@ -22,7 +22,7 @@ TILE_TOKENS = 128
 ATTENTION_LAUNCHES = 3   # kernels one spectra_decode_attention call enqueues
 
 EXPORTS = [
-    "spectra_fit_basis", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
+    "spectra_fit_basis", "spectra_fit_basis_static", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
     "spectra_decode_attention", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
     "spectra_total_bits", "spectra_status_string",
 ]
@@ -119,6 +119,21 @@ def fit_basis(cfg, x, n_units, n_tokens, stride_unit, stride_token, w_enc, w_dec
                                  _ptr(workspace), C.c_size_t(0 if workspace is None else workspace.numel() *
                                                              workspace.element_size()), _stream())
     _check(rc, "spectra_fit_basis")
+
+
+FIT_STATIC_MAX_UNITS = 8
+
+
+def fit_basis_static(cfg, x, n_units, n_tokens, stride_unit, stride_token, w_enc, w_dec, mean_rot, var_alloc,
+                     eigval=None, basis_u=None):
+    """spectra_fit_basis without a workspace argument, for callers that cannot allocate device memory when they
+    calibrate: the scratch is a fixed array inside the library (at most FIT_STATIC_MAX_UNITS unit-sides per call).
+    Make the first call on a device outside stream capture; do not overlap two calls on one device."""
+    rc = lib().spectra_fit_basis_static(C.byref(cfg), _ptr(x), C.c_int(_dtype_code(x)), C.c_int64(n_units),
+                                        C.c_int64(n_tokens), C.c_int64(stride_unit), C.c_int64(stride_token),
+                                        _ptr(w_enc), _ptr(w_dec), _ptr(mean_rot), _ptr(var_alloc), _ptr(eigval),
+                                        _ptr(basis_u), _stream())
+    _check(rc, "spectra_fit_basis_static")
 
 
 def alloc_bits(cfg, var_alloc, n_units, ratio, widths):

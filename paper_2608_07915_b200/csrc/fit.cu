@@ -288,6 +288,37 @@ extern "C" int spectra_fit_basis(const spectra_config* cfg, const void* x, int x
   return launch_status();
 }
 
+// ------------------------------------------------------------------------------------------------
+// Variant without a caller workspace: the scratch is a fixed array in the library image.
+static __device__ __align__(256) unsigned char g_fit_static_scratch[sizeof(FitWorkspace) * SPECTRA_FIT_STATIC_MAX_UNITS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_fit_static_addr[kMaxDevices];   // device address of the array, per device, looked up on first use
+}  // namespace
+
+extern "C" int spectra_fit_basis_static(const spectra_config* cfg, const void* x, int x_dtype, int64_t n_units,
+                                        int64_t n_tokens, int64_t stride_unit, int64_t stride_token, float* w_enc,
+                                        float* w_dec, float* mean_rot, float* var_alloc, float* eigval,
+                                        float* basis_u, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (n_units < 0) return SPECTRA_INVALID_ARG;
+  if (n_units > SPECTRA_FIT_STATIC_MAX_UNITS) return SPECTRA_CAPACITY;
+  if (n_units == 0) return SPECTRA_OK;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPECTRA_CUDA_ERROR;
+  if (!g_fit_static_addr[dev]) {
+    // In host code the array's name is only a handle; the kernels need its address on the current device.
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_fit_static_scratch) != cudaSuccess || !ptr) return SPECTRA_CUDA_ERROR;
+    g_fit_static_addr[dev] = ptr;
+  }
+  return spectra_fit_basis(cfg, x, x_dtype, n_units, n_tokens, stride_unit, stride_token, w_enc, w_dec, mean_rot,
+                           var_alloc, eigval, basis_u, g_fit_static_addr[dev],
+                           sizeof(FitWorkspace) * (size_t)n_units, stream);
+}
+
 extern "C" int32_t spectra_total_bits(const spectra_config* cfg, double ratio) {
   if (check_config(cfg) || !(ratio > 0.0)) return -1;
   double bits = 16.0 * kD / ratio + 1e-9;
