@@ -44,7 +44,7 @@ class CodedModelCache:
             dtype=torch.uint8, device=device)
 
     # ------------------------------------------------------------------ set-up (calibrate + prefill encode)
-    def _draw_layer_side(self, layer, side):
+    def draw_layer_side(self, layer, side):
         wl = self.wl
         dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
         x = torch.empty((self.batch, self.H, self.n_tokens, self.d), dtype=dt, device=self.device)
@@ -52,7 +52,10 @@ class CodedModelCache:
             x[:, h] = si.draw_unit_torch(wl, layer, h, side, self.batch, self.n_tokens, self.device)
         return x
 
-    def build(self, time_phases=False):
+    def build(self, time_phases=False, params_override=None):
+        """params_override: optional {(layer, side): dict(w_enc, w_dec, m_rot, widths)} of numpy arrays [H, ...]; the
+        library's own fit and allocation are skipped for those layer-sides (used by parity tests, which hand the
+        same parameters to both implementations)."""
         cfg, H, d, N = self.cfg, self.H, self.d, self.n_tokens
         n_fit = min(self.wl.n_fit, N)
         f32 = dict(dtype=torch.float32, device=self.device)
@@ -61,15 +64,22 @@ class CodedModelCache:
         t_fit = t_enc = 0.0
         for layer in range(self.layers):
             for side in (si.SIDE_K, si.SIDE_V):
-                x = self._draw_layer_side(layer, side)
+                x = self.draw_layer_side(layer, side)
                 ls = LayerSide()
                 ls.w_enc, ls.w_dec = (torch.zeros((H, d, d), **f32) for _ in range(2))
                 ls.m_rot, ls.var = (torch.zeros((H, d), **f32) for _ in range(2))
                 ls.widths = torch.zeros((H, d), dtype=torch.uint8, device=self.device)
                 e0, e1, e2 = ev(), ev(), ev()
                 e0.record()
-                sp.fit_basis(cfg, x, H, n_fit, N * d, d, ls.w_enc, ls.w_dec, ls.m_rot, ls.var, None, None, fit_ws)
-                sp.alloc_bits(cfg, ls.var, H, self.wl.ratio, ls.widths)
+                ov = (params_override or {}).get((layer, side))
+                if ov is not None:
+                    ls.w_enc.copy_(torch.from_numpy(np.ascontiguousarray(ov["w_enc"], np.float32)))
+                    ls.w_dec.copy_(torch.from_numpy(np.ascontiguousarray(ov["w_dec"], np.float32)))
+                    ls.m_rot.copy_(torch.from_numpy(np.ascontiguousarray(ov["m_rot"], np.float32)))
+                    ls.widths.copy_(torch.from_numpy(np.ascontiguousarray(ov["widths"], np.uint8)))
+                else:
+                    sp.fit_basis(cfg, x, H, n_fit, N * d, d, ls.w_enc, ls.w_dec, ls.m_rot, ls.var, None, None, fit_ws)
+                    sp.alloc_bits(cfg, ls.var, H, self.wl.ratio, ls.widths)
                 e1.record()
                 ls.widths_host = ls.widths.cpu().numpy()
                 ls.tile_bytes = np.array([sp.tile_bytes(cfg, w) for w in ls.widths_host], np.int64)

@@ -1,0 +1,103 @@
+"""Parity at the workloads' full context lengths, in the launch configuration bench.py times (the harness the
+benchmark uses), on sampled units the oracle can compute one by one.
+
+Both sides get the same transforms and widths (fitted by the oracle from the same raw vectors); the GPU encodes
+every unit of the layer, appends one token per sequence and attends; the oracle does the same for the sampled
+(sequence, kv-head) units from the raw vectors alone.  Checked: code mismatches (rare +-1 ties only), and the
+attention output of the decode step (2e-3, max |diff| / max |oracle| per vector).
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import spectra_inputs as si
+from oracle import codec as oc
+from oracle import fit as ofit
+from tests import helpers as H
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3
+
+CASES = {
+    # name: (workload, batch used here, sampled (sequence, kv-head) units)
+    "llama1_4x_32k": ("llama1", 1, [(0, 0), (0, 5)]),
+    "llama32_8x_32k_batch8": ("llama32", 8, [(0, 0), (3, 5), (7, 7)]),
+    "qwen28_12x_64k": ("qwen28", 2, [(0, 1), (1, 3)]),
+    "long_8x_128k": ("long128k", 1, [(0, 2)]),
+}
+
+
+@pytest.mark.parametrize("case", list(CASES))
+def test_full_context_decode_step_matches_oracle(case):
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2608_07915_b200 as sp
+    from paper_2608_07915_b200 import harness
+    name, batch, sampled = CASES[case]
+    wl = si.WORKLOADS[name]
+    Hk, G, d, N = wl.kv_heads, wl.group, wl.head_dim, wl.n_tokens
+    model = harness.CodedModelCache(wl, layers=1, batch=batch, extra_tokens=128)
+    # raw vectors (generator output, not codec output): fit tokens of sequence 0 for every head, and the sampled units
+    params, raw = {}, {}
+    for side in (si.SIDE_K, si.SIDE_V):
+        x = model.draw_layer_side(0, side)                                     # [batch, H, N, d]
+        fits = [ofit.fit_basis(x[0, h, :wl.n_fit].float().cpu().numpy().astype(np.float64), ofit.GAIN_SQRT)
+                for h in range(Hk)]
+        widths = np.stack([ofit.alloc_bits(f["v_alloc"].astype(np.float32), ofit.total_bits(d, wl.ratio))
+                           for f in fits])
+        params[(0, side)] = dict(w_enc=np.stack([f["W_enc"] for f in fits]), w_dec=np.stack([f["W_dec"] for f in fits]),
+                                 m_rot=np.stack([f["m_rot"] for f in fits]), widths=widths)
+        for (s, h) in sampled:
+            raw[(side, s, h)] = x[s, h].float().cpu().numpy()
+        del x
+    model.build(params_override=params)          # same generator seeds: the harness redraws the same vectors
+    assert int(model.status.item()) == 0
+    # one decode step on the GPU
+    gen = torch.Generator(device="cuda").manual_seed(99)
+    q = torch.randn((1, batch, wl.q_heads, d), generator=gen, device="cuda").to(torch.bfloat16)
+    nk = torch.randn((1, batch * Hk, d), generator=gen, device="cuda").to(torch.bfloat16)
+    nv = torch.randn((1, batch * Hk, d), generator=gen, device="cuda").to(torch.bfloat16)
+    out = torch.zeros((1, batch, wl.q_heads, d), dtype=torch.float32, device="cuda")
+    model.decode_step(q, nk, nv, out)
+    torch.cuda.synchronize()
+    assert int(model.status.item()) == 0
+    got = out[0].cpu().numpy().reshape(batch, Hk, G, d)
+    qh = q[0].float().cpu().numpy().reshape(batch, Hk, G, d).astype(np.float64)
+    new = {si.SIDE_K: nk[0].float().cpu().numpy(), si.SIDE_V: nv[0].float().cpu().numpy()}
+    n_tiles = (N + 1 + 127) // 128
+    for (s, h) in sampled:
+        u = s * Hk + h
+        caches = {}
+        for side in (si.SIDE_K, si.SIDE_V):
+            P = params[(0, side)]
+            pr = H.Params(P["w_enc"][[h]], P["w_dec"][[h]], P["m_rot"][[h]], P["widths"][[h]], 64)
+            tb = int(pr.tile_bytes[0])
+            c = np.zeros(n_tiles * tb, np.uint8)
+            xs = np.concatenate([raw[(side, s, h)], new[side][u][None]], axis=0)
+            assert H.oracle_encode(pr, side, xs[None], [0], c, np.zeros(1, np.int64)) == 0
+            caches[side] = (pr, tb, c)
+            # the GPU's bytes for this unit: codes equal up to rare +-1 ties (metadata flips counted apart)
+            ls = model.side[0][side]
+            a = int(ls.unit_offset_host[u])
+            g = ls.cache[a:a + n_tiles * tb].cpu().numpy()
+            sample_t = np.unique(np.concatenate([np.arange(0, N + 1, 97), [N - 1, N]]))
+            bad = tot = meta_diff = 0
+            for t in sample_t:
+                cr, lr, rr = oc.unpack_token(c[(t // 128) * tb:(t // 128 + 1) * tb], pr.widths[0], 64, side, int(t % 128))
+                cg, lg, rg = oc.unpack_token(g[(t // 128) * tb:(t // 128 + 1) * tb], pr.widths[0], 64, side, int(t % 128))
+                if not (np.array_equal(lr, lg) and np.array_equal(rr, rg)):
+                    meta_diff += 1
+                    continue
+                diff = np.abs(cr.astype(np.int64) - cg.astype(np.int64))
+                assert diff.max() <= 1
+                bad += int((diff != 0).sum()); tot += int((pr.widths[0] > 0).sum())
+            assert bad <= max(2, 1e-4 * tot * 5), (bad, tot)      # sample of ~340 tokens: allow the tie budget x5
+            assert meta_diff <= max(1, 0.01 * sample_t.size)
+        (pk, tbk, ck), (pv, tbv, cv) = caches[si.SIDE_K], caches[si.SIDE_V]
+        ref, _ = oc.attention_units("B", qh[s, h][None], [N + 1], ck, [0], [tbk], cv, [0], [tbv], pk.w_dec, pk.m_rot,
+                                    pk.widths, pv.w_dec, pv.m_rot, pv.widths, 64, 1.0 / np.sqrt(128.0))
+        # bf16 queries on the GPU side are exactly the fp32 values the oracle used
+        assert H.rel_err_per_vector(got[s, h], ref[0]) <= TOL, (case, s, h)
