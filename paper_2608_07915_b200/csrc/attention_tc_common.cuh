@@ -197,8 +197,7 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
   const int G = p.gqa;
-  build_strip_table(S.tk, p.widths_k + (int64_t)ps * kD, 64);
-  build_strip_table(S.tv, p.widths_v + (int64_t)ps * kD, 64);
+  build_strip_tables(S.tk, p.widths_k + (int64_t)ps * kD, S.tv, p.widths_v + (int64_t)ps * kD, 64);
   const StripTable& TK = S.tk;
   const StripTable& TV = S.tv;
   UnitDesc& D = f.desc[u];

@@ -211,6 +211,13 @@ __device__ __forceinline__ void store_class(float* rec, uint32_t cls, int first,
   }
 }
 
+// Two floats to packed fp16 (low = a), saturating at the largest finite value instead of producing infinity.
+__device__ __forceinline__ uint32_t pack_half2_sat(float a, float b) {
+  uint32_t d;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(b), "f"(a));
+  return d;
+}
+
 struct TileCursor {   // walks the flattened (unit, tile) space; all fields are warp-uniform
   int u, t, nt;
   __device__ __forceinline__ void seek_unit(const FastArgs& f) {
@@ -282,6 +289,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
   const uint2* kB = nullptr;
   int n_seq = 0;
   bool fresh = true, ok = true;
+  float boost = 0.f;          // power-of-two lift of the probabilities (see below); -1 = not chosen yet
 
   for (int j = 0; j < count && ok; j++) {
     const int slot = j % D;
@@ -302,6 +310,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
         for (int e = 0; e < 4; e++) acc_o[mb][e] = 0.f;
       m_run = -INFINITY; l_run = 0.f; plo0 = 0.f; plo1 = 0.f;
       fresh = false;
+      boost = -1.f;
     }
 
 #pragma unroll 1
@@ -368,7 +377,23 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
       if (vmeta1 >= 0) { ld_words<4>(vtile + vmeta1 + tok_off, vlo1); ld_words<4>(vtile + vmeta1 + 256 + tok_off, vr1); }
       // probabilities times the V group ranges, as fp16 pairs (group 0, group 1), transposed into B fragments
       uint32_t pb[8];
-      const float m_use = m_run == -INFINITY ? 0.f : m_run;
+      if (boost < 0.f) {
+        // First half tile of this warp's share of the unit.  Probabilities are exp2(s - max) <= 1 and enter the
+        // tensor core as fp16 times the V group range; with tens of thousands of tokens the typical probability is
+        // far below the fp16 normal range.  Lift everything by 2^boost (the record's maximum is lowered by the same
+        // amount, so the merge is unaffected), leaving room for group ranges 8x larger than in this half tile.
+        float rmax = 0.f;
+#pragma unroll
+        for (int r = 0; r < 4; r++) {
+          const float2 a = h2f2(vr0[r]), b = h2f2(vr1[r]);
+          rmax = fmaxf(rmax, fmaxf(fmaxf(a.x, a.y), fmaxf(b.x, b.y)));
+        }
+#pragma unroll
+        for (int sft = 1; sft <= 16; sft <<= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, sft));
+        const int e = (int)((__float_as_uint(rmax) >> 23) & 0xff) - 126;     // rmax < 2^e
+        boost = (float)max(0, min(13, 13 - e));
+      }
+      const float m_use = (m_run == -INFINITY ? 0.f : m_run) - boost;
 #pragma unroll
       for (int r = 0; r < 4; r++) {
         const float2 lo0 = h2f2(vlo0[r]), r0 = h2f2(vr0[r]), lo1 = h2f2(vlo1[r]), r1 = h2f2(vr1[r]);
@@ -379,8 +404,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
           l_run += pr;
           plo0 = fmaf(pr, e ? lo0.y : lo0.x, plo0);
           plo1 = fmaf(pr, e ? lo1.y : lo1.x, plo1);
-          const __half2 pk = __floats2half2_rn(pr * (e ? r0.y : r0.x), pr * (e ? r1.y : r1.x));
-          pb[ii] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&pk));
+          pb[ii] = movmatrix_trans(pack_half2_sat(pr * (e ? r0.y : r0.x), pr * (e ? r1.y : r1.x)));
         }
       }
       // ------------------------------------------------------------ P~ x V codes
@@ -405,7 +429,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
         q1 += __shfl_xor_sync(0xffffffffu, q1, sft);
       }
       float* rec = f.records + (int64_t)(gw + cons.u) * f.rec_stride + tig * (kRecHead + f.vs_max);
-      if (gid == 0) { rec[0] = m_run; rec[1] = l; rec[2] = q0; rec[3] = q1; }
+      if (gid == 0) { rec[0] = m_run - boost; rec[1] = l; rec[2] = q0; rec[3] = q1; }
       const UnitDesc& d = f.desc[cons.u];
       store_class<Q8, 0, NACC>(rec, vcls[0], d.vfirst[0], gid, acc_o);
       store_class<Q4, Q8, NACC>(rec, vcls[1], d.vfirst[1], gid, acc_o);

@@ -3,6 +3,7 @@
 // read-modify-write of a partly filled tail tile needs no atomics.
 #include "common.cuh"
 #include "encode_append.cuh"
+#include "encode_tc.cuh"
 
 namespace spectra {
 
@@ -250,6 +251,19 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
     AppendArgs ap{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
                   w_enc, mean_rot, widths, cache, unit_offset, status_word};
     encode_append_kernel<<<(unsigned)n_units, 128, 0, (cudaStream_t)stream>>>(ap);
+    return launch_status();
+  }
+  if (x_dtype == SPECTRA_BF16 && !(flags & SPECTRA_ROTATED_INPUT) && cfg->scale_group == 64 &&
+      stride_token % 8 == 0 && stride_unit % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+    // bf16 bulk encode: rotation on the tensor cores
+    EncodeTcArgs ta{reinterpret_cast<const __nv_bfloat16*>(x), side, n_param_sets, pos0, n_new, stride_unit,
+                    stride_token, w_enc, mean_rot, widths, cache, unit_offset, status_word};
+    if (cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)sizeof(EncodeTcSmem)) != cudaSuccess)
+      return SPECTRA_CUDA_ERROR;
+    const unsigned tiles = (unsigned)((n_new + 2 * kTile - 2) / kTile);
+    dim3 grid((tiles + kTcTilesPerCta - 1) / kTcTilesPerCta, (unsigned)n_units);
+    encode_tc_kernel<<<grid, kTcThreads, sizeof(EncodeTcSmem), (cudaStream_t)stream>>>(ta);
     return launch_status();
   }
   EncodeArgs a{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,

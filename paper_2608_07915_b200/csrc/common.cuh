@@ -43,13 +43,9 @@ struct StripTable {
   uint8_t width[kD];
 };
 
-// Called by all threads of a CTA (at least one full warp); includes the closing __syncthreads().
-__device__ inline void build_strip_table(StripTable& T, const uint8_t* __restrict__ widths_global, int scale_group) {
-  const int tid = threadIdx.x;
-  if (tid < kD) T.width[tid] = widths_global[tid];
-  __syncthreads();
-  if (tid < 32) {
-    const int lane = tid;
+// The scan itself, run by one full warp after T.width has been filled.
+__device__ inline void strip_table_scan(StripTable& T, int scale_group, int lane) {
+  {
     int count = 0, off = 0;
 #pragma unroll
     for (int c = 0; c < 4; c++) {
@@ -85,6 +81,26 @@ __device__ inline void build_strip_table(StripTable& T, const uint8_t* __restric
       for (int g = n_groups; g < kMaxGroups; g++) T.meta_off[g] = -1;
     }
   }
+}
+
+// Called by all threads of a CTA (at least one full warp); includes the closing __syncthreads().
+__device__ inline void build_strip_table(StripTable& T, const uint8_t* __restrict__ widths_global, int scale_group) {
+  const int tid = threadIdx.x;
+  if (tid < kD) T.width[tid] = widths_global[tid];
+  __syncthreads();
+  if (tid < 32) strip_table_scan(T, scale_group, tid);
+  __syncthreads();
+}
+
+// Two tables at once (at least 256 threads): warp 0 scans the first, warp 1 the second.
+__device__ inline void build_strip_tables(StripTable& A, const uint8_t* __restrict__ wa, StripTable& B,
+                                          const uint8_t* __restrict__ wb, int scale_group) {
+  const int tid = threadIdx.x;
+  if (tid < kD) A.width[tid] = wa[tid];
+  else if (tid < 2 * kD) B.width[tid - kD] = wb[tid - kD];
+  __syncthreads();
+  if (tid < 32) strip_table_scan(A, scale_group, tid);
+  else if (tid < 64) strip_table_scan(B, scale_group, tid - 32);
   __syncthreads();
 }
 

@@ -76,9 +76,16 @@ __global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
     float y;
     if (rotated) y = xs[t][j];
     else {
+      // all 128 loads of the column are issued before the FMA chain consumes them (latency-bound otherwise)
+      float wcol[kD / 4];
       float a0 = 0.f;
-#pragma unroll 8
-      for (int i = 0; i < kD; i++) a0 = fmaf(xs[t][i], __ldg(w + i * kD + j), a0);
+#pragma unroll
+      for (int blk = 0; blk < 4; blk++) {
+#pragma unroll
+        for (int i = 0; i < kD / 4; i++) wcol[i] = __ldg(w + (blk * (kD / 4) + i) * kD + j);
+#pragma unroll
+        for (int i = 0; i < kD / 4; i++) a0 = fmaf(xs[t][blk * (kD / 4) + i], wcol[i], a0);
+      }
       y = __fsub_rn(a0, mr);
     }
     if (b && !isfinite(y)) status |= SPECTRA_STATUS_NONFINITE;
