@@ -24,6 +24,9 @@ if ROOT not in sys.path:
 import numpy as np
 
 METRIC = "coded_kv_decode_attention_kv_tokens_per_s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (one layer of the workload),
+# from the ncu capture summarised in profiles/attention_mma_kernel_llama32_2layer.md (same per-launch shape)
+NCU_TRAFFIC_BYTES = {"llama32": 173.1e6}
 UNIT = "KV tokens/s"
 
 
@@ -36,52 +39,52 @@ def _peaks():
 
 
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and clock-event reasons of one GPU in a background thread (NVML, read-only)."""
 
-    def __init__(self, gpu_index):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.p = None
-        self.gpu_index = gpu_index
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40}
+
+    def __init__(self, gpu_index, period_s=0.01):
+        import threading
+        self.idx, self.period = gpu_index, period_s
+        self.sm, self.reasons, self.max_sm = [], set(), None
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._ok = False
+
+    def _run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            # honour CUDA_VISIBLE_DEVICES when it lists indices
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            phys = self.idx
+            if vis and all(v.strip().isdigit() for v in vis.split(",")):
+                phys = int(vis.split(",")[self.idx])
+            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_sm = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            self._ok = True
+            while not self._stop.is_set():
+                self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                try:
+                    mask = int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                except Exception:
+                    mask = int(pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+                for name, bit in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                time.sleep(self.period)
+        except Exception:
+            self._ok = False
 
     def start(self):
-        try:
-            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
-                                      stderr=subprocess.DEVNULL)
-        except OSError:
-            self.p = None
+        self._thread.start()
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.p is None:
-            return out
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.p.kill()
-        self.f.flush()
-        self.f.seek(0)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.f:
-            parts = [s.strip() for s in line.split(",")]
-            if len(parts) < 9:
-                continue
-            try:
-                sm.append(float(parts[1])); mx.append(float(parts[2]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        self.f.close()
-        os.unlink(self.f.name)
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
-                       samples=len(sm))
+        self._stop.set()
+        self._thread.join(timeout=5)
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_sm, "reasons": sorted(self.reasons), "samples": len(self.sm)}
+        if self.sm:
+            out["sm_mhz"] = float(np.median(self.sm))
         return out
 
 
@@ -107,12 +110,12 @@ def _barrier(world):
     torch.cuda.synchronize()
 
 
-def _max_over_ranks(x, world):
+def _max_over_ranks(x, world, device="cuda"):
     import torch
     if world == 1:
         return x
     import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    t = torch.tensor([x], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
 
@@ -321,7 +324,7 @@ def run_ours(args, wl):
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "spectra_decode_attention (one layer call)", "achieved": achieved,
                      "peak": hbm_gbs, "unit": "GB/s", "frac": achieved / hbm_gbs, "peak_kind": peak_kind,
-                     "traffic": None, "bytes_per_launch": bytes_call, "ms_per_launch": attn_ms_avg},
+                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "bytes_per_launch": bytes_call, "ms_per_launch": attn_ms_avg},
         "phases": {"setup_s": setup_s, "fit_alloc_ms_total": model.timings["fit_alloc_ms"],
                    "prefill_encode_ms_total": model.timings["prefill_encode_ms"],
                    "prefill_encode_tokens_per_s": L * 2 * U * wl.n_tokens / max(model.timings["prefill_encode_ms"],
