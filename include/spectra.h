@@ -31,30 +31,25 @@
  *     L_j = 2^b_j - 1;  code_j = 0 if R_f == 0 else clamp(rint((y_j - lo_f) * (L_j / R_f)), 0, L_j)
  *     reconstruction: yhat_j = lo_f if R_f == 0 else (float(code_j) * (R_f / L_j)) + lo_f;  b_j == 0: yhat_j = 0
  *
- * Packed tile format v2 (128 consecutive tokens of one unit-side; tiles of a unit-side are
- * contiguous, tile t of unit u starts at cache + unit_offset[u] + t * spectra_tile_bytes();
- * tile bit n = bit n % 8 of byte n / 8):
+ * Packed tile format v1 (128 consecutive tokens of one unit-side; tiles of a unit-side are
+ * contiguous, tile t of unit u starts at cache + unit_offset[u] + t * spectra_tile_bytes()):
  *   - A width b is split into its binary digits, sub-fields of 8, 4, 2 or 1 bits
  *     (7 -> 4,2,1; 6 -> 4,2; 5 -> 4,1; 3 -> 2,1); the sub-field of size w holds code bits
  *     [s, s+w), s = b & (w-1).
- *   - A strip is one sub-field of one channel for the 128 tokens.  Strips are ordered by class
- *     w = 8, 4, 2, 1 and, inside a class, by ascending channel.  B = sum_j b_j.
- *   - K side, token-major: the fields of one token in strip order form its token string of B bits
- *     (strip k at string bits [o_k, o_k + w_k), o_k = widths of the strips before it; a field never
- *     crosses a 16-bit boundary of the string).  With F = B / 32 and r = B % 32: string bits
- *     [32 i, 32 i + 32), i < F, are the little-endian 32-bit word at byte 4 * (128 i + t) (word-major,
- *     token-minor); the last r string bits of the 128 tokens are packed densely behind the words:
- *     string bit 32 F + u of token t is tile bit 4096 F + r t + u.
- *   - V side, strip-major: strip k is 16 * w_k bytes at byte 16 * o_k; token t = 32a + 16h + i
- *     (a < 4, h < 2, i < 16) is in 32-bit word q = a*w + i*w/16 of its strip, low (h = 0) or high
- *     (h = 1) half-word, at bits [(i*w) % 16, +w).
+ *   - A strip is one sub-field of one channel for the 128 tokens: 16*w bytes, seen as 8*w
+ *     little-endian 16-bit half-words; the i-th token of a half-word sits at bits [i*w, i*w+w).
+ *   - Strips are stored by class w = 8, 4, 2, 1 and, inside a class, by ascending channel.
+ *   - K side: token t is in half-word n = t*w/16.  Consecutive strips of a class are paired;
+ *     a pair takes 32*w bytes and its 32-bit word n is (half-word n of the first strip) |
+ *     (half-word n of the second) << 16.  An odd last strip is stored alone, half-words in order.
+ *   - V side: token t = 32a + 16h + i (a < 4, h < 2, i < 16) is in 32-bit word q = a*w + i*w/16
+ *     of its strip, low (h = 0) or high (h = 1) half-word, at bits [(i*w) % 16, +w).
  *   - Then, for each scale group with a non-zero-width channel, ascending: lo16[128], R16[128]
  *     (little-endian fp16, token order).
  *   - tile bytes = 16 * sum_j b_j + 512 * (number of active scale groups); always a multiple of 16.
- *   The two orders are what the tensor-core contractions read without a transpose: the score
- *   contraction runs over channels with one token per accumulator row (a thread unpacks the string
- *   of its token), the value contraction runs over tokens with one strip per accumulator row (a
- *   thread unpacks its strip; tokens t and t + 16 are the two halves of an operand register).
+ *   The K-side pairing puts two channels of one token 16 bits apart in a word, the V-side order
+ *   puts two tokens of one channel 16 bits apart: what the tensor-core operand registers of the
+ *   score and of the value contraction need, respectively.
  */
 #ifndef SPECTRA_H_
 #define SPECTRA_H_
@@ -100,7 +95,7 @@ typedef struct spectra_config {
   int32_t width_group;    /* adjacent channels sharing one width in spectra_alloc_bits: power of two, 1..scale_group */
   int32_t b_max;          /* largest width, 1..8 */
   int32_t gain_mode;      /* SPECTRA_GAIN_* (used by spectra_fit_basis only) */
-  int32_t layout_version; /* 2 */
+  int32_t layout_version; /* 1 */
 } spectra_config;
 
 /* ------------------------------------------------------------------------------------------------

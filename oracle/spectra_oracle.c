@@ -21,26 +21,23 @@
  * written operation, no fused multiply-add (compile with -ffp-contract=off).  Rotations,
  * softmax and attention sums are fp64.
  *
- * Packed tile format v2 (128 tokens of one unit-side; tile bit n = bit n%8 of byte n/8):
+ * Packed tile format v1 (128 tokens of one unit-side):
  *   width b in 0..8 is split into its binary digits, "sub-fields" of 8, 4, 2 or 1 bits
  *   (7 -> 4,2,1; 6 -> 4,2; 5 -> 4,1; 3 -> 2,1); the sub-field of size w holds code bits
  *   [s, s+w) with s = b & (w-1).  A "strip" is one sub-field of one channel for all 128
- *   tokens.  Strips are ordered by class w = 8, 4, 2, 1, and inside a class by ascending
- *   channel.  B = sum_j b_j.
- *     K side (token-major): the fields of one token, in strip order, form its "token
- *             string" of B bits (strip k at string bits [o_k, o_k + w_k), o_k = sum of the
- *             widths of the strips before it).  With F = B / 32 and r = B % 32: string
- *             bits [32 i, 32 i + 32), i < F, are the little-endian 32-bit word at byte
- *             4 * (128 i + t) of the tile (word-major, token-minor); the last r string
- *             bits of the 128 tokens are packed densely after the words: string bit
- *             32 F + u of token t is tile bit 4096 F + r t + u.
- *     V side (strip-major): strip k is 16*w bytes at the byte offset 16 * (sum of the widths
- *             of the strips before it); token t = 32*a + 16*h + i (a in 0..3, h in 0..1,
- *             i in 0..15) is in 32-bit word q = a*w + i*w/16 of its strip, in the low
- *             (h = 0) or high (h = 1) half-word, at bits [(i*w)%16, +w).
- *   After the payload (16 B bytes on either side), for every scale group that has a
- *   non-zero-width channel, in ascending order: lo16[128] then R16[128] (little-endian
- *   fp16, token order).
+ *   tokens: 128*w bits = 16*w bytes, seen as 8*w little-endian 16-bit half-words; inside
+ *   a half-word the field of the i-th token it holds sits at bits [i*w, i*w+w).
+ *   Strips are stored by class w = 8, 4, 2, 1, and inside a class by ascending channel.
+ *   The half-word order differs by side:
+ *     K side: token t is in half-word n = t*w/16 of its strip.  Consecutive strips of a
+ *             class are paired; a pair occupies 32*w bytes, 32-bit word n = (half-word n
+ *             of the first strip) | (half-word n of the second strip) << 16.  An odd last
+ *             strip of a class is stored alone, half-words in order (16*w bytes).
+ *     V side: token t = 32*a + 16*h + i (a in 0..3, h in 0..1, i in 0..15) is in 32-bit
+ *             word q = a*w + i*w/16 of its strip, in the low (h = 0) or high (h = 1)
+ *             half-word, at bits [(i*w)%16, +w).
+ *   After the strips, for every scale group that has a non-zero-width channel, in
+ *   ascending order: lo16[128] then R16[128] (little-endian fp16, token order).
  *   tile bytes = 16 * sum_j b_j + 512 * (number of active scale groups).
  */
 #include <math.h>
@@ -108,44 +105,53 @@ int spo_subfields(int b, int* w_out, int* shift_out) {
 
 typedef struct {
   int chan, w, shift;
-  int mode;        /* 3: V side, strip-major; 4: K side, token-major */
-  int64_t base;    /* V: byte offset of the strip in the tile; K: bit offset of the field in the token string */
-  int64_t total;   /* B = sum of all widths (bits of a token string) */
+  int mode;        /* 0: alone, natural order; 1: K pair, low half; 2: K pair, high half; 3: V order */
+  int64_t base;    /* byte offset in the tile of the strip (mode 0, 3) or of its pair (1, 2) */
 } spo_strip;
 
-/* Enumerate the strips of a tile.  Returns their number; *payload_bytes gets the size of the payload region. */
+/* Enumerate the strips of a tile.  Returns their number; *payload_bytes gets the size of the strip region. */
 static int spo_strips(const uint8_t* widths, int d, int side, spo_strip* out, int64_t* payload_bytes) {
   int n = 0;
-  int64_t bits = 0;                              /* widths of the strips so far */
+  int64_t off = 0;
   for (int w = 8; w >= 1; w >>= 1) {
+    int first = n;
     for (int j = 0; j < d; j++) {
       if (widths[j] & w) {
         out[n].chan = j; out[n].w = w; out[n].shift = widths[j] & (w - 1);
-        if (side == SPO_SIDE_V) { out[n].mode = 3; out[n].base = 16 * bits; }
-        else { out[n].mode = 4; out[n].base = bits; }
-        bits += w;
         n++;
       }
     }
+    int cnt = n - first;
+    for (int i = 0; i < cnt; i++) {
+      spo_strip* s = &out[first + i];
+      if (side == SPO_SIDE_V) {
+        s->mode = 3; s->base = off + (int64_t)16 * w * i;
+      } else if ((i | 1) < cnt) {               /* has a partner */
+        s->mode = 1 + (i & 1); s->base = off + (int64_t)32 * w * (i / 2);
+      } else {                                   /* odd last strip */
+        s->mode = 0; s->base = off + (int64_t)16 * w * i;
+      }
+    }
+    off += (int64_t)16 * w * cnt;
   }
-  for (int i = 0; i < n; i++) out[i].total = bits;
-  *payload_bytes = 16 * bits;
+  *payload_bytes = off;
   return n;
 }
 
-/* Tile bit offset of the lowest bit of the field of token t of a strip (the field's w bits are consecutive
- * tile bits: a field never crosses a 32-bit word of a token string, nor a half-word of a V strip). */
-static int64_t spo_locate(const spo_strip* s, int t) {
+/* Where the field of token t of a strip lives: byte offset of its half-word, bit offset inside it. */
+static void spo_locate(const spo_strip* s, int t, int64_t* byte_off, int* bit_off) {
   int w = s->w;
   if (s->mode == 3) {
     int a = t / 32, h = (t % 32) / 16, i = t % 16;
     int q = a * w + (i * w) / 16;
-    return 8 * (s->base + 4 * (int64_t)q + 2 * h) + (i * w) % 16;
+    *byte_off = s->base + 4 * (int64_t)q + 2 * h;
+    *bit_off = (i * w) % 16;
+  } else {
+    int n = (t * w) / 16;
+    *bit_off = (t * w) % 16;
+    if (s->mode == 0) *byte_off = s->base + 2 * (int64_t)n;
+    else *byte_off = s->base + 4 * (int64_t)n + 2 * (s->mode - 1);
   }
-  int64_t F = s->total / 32, r = s->total % 32;
-  int64_t o = s->base;
-  if (o < 32 * F) return 32 * (128 * (o / 32) + t) + o % 32;
-  return 4096 * F + r * t + (o - 32 * F);
 }
 
 static int spo_active_groups(const uint8_t* widths, int d, int gs, int* active /* [d/gs] */) {
@@ -254,22 +260,6 @@ void spo_dequantise_token(const uint16_t* codes, const uint16_t* lo16, const uin
 static void spo_put16(uint8_t* p, uint16_t v) { p[0] = (uint8_t)(v & 0xff); p[1] = (uint8_t)(v >> 8); }
 static uint16_t spo_get16(const uint8_t* p) { return (uint16_t)(p[0] | (p[1] << 8)); }
 
-static void spo_put_bits(uint8_t* tile, int64_t bit, int w, unsigned v) {
-  for (int k = 0; k < w; k++) {
-    int64_t n = bit + k;
-    uint8_t m = (uint8_t)(1u << (n % 8));
-    if ((v >> k) & 1u) tile[n / 8] |= m; else tile[n / 8] &= (uint8_t)~m;
-  }
-}
-static unsigned spo_get_bits(const uint8_t* tile, int64_t bit, int w) {
-  unsigned v = 0;
-  for (int k = 0; k < w; k++) {
-    int64_t n = bit + k;
-    v |= (unsigned)((tile[n / 8] >> (n % 8)) & 1u) << k;
-  }
-  return v;
-}
-
 /* Write token slot t (0..127) of a tile.  Overwrites exactly that token's bits and metadata. */
 void spo_pack_token(uint8_t* tile, const uint8_t* widths, int d, int gs, int side, int t, const uint16_t* codes,
                     const uint16_t* lo16, const uint16_t* R16) {
@@ -277,8 +267,13 @@ void spo_pack_token(uint8_t* tile, const uint8_t* widths, int d, int gs, int sid
   int64_t payload;
   int n = spo_strips(widths, d, side, st, &payload);
   for (int k = 0; k < n; k++) {
-    unsigned field = ((unsigned)codes[st[k].chan] >> st[k].shift) & ((1u << st[k].w) - 1u);
-    spo_put_bits(tile, spo_locate(&st[k], t), st[k].w, field);
+    int64_t bo; int bit;
+    spo_locate(&st[k], t, &bo, &bit);
+    uint16_t field = (uint16_t)((codes[st[k].chan] >> st[k].shift) & ((1u << st[k].w) - 1u));
+    uint16_t hw = spo_get16(tile + bo);
+    uint16_t mask = (uint16_t)(((1u << st[k].w) - 1u) << bit);
+    hw = (uint16_t)((hw & ~mask) | (uint16_t)(field << bit));
+    spo_put16(tile + bo, hw);
   }
   for (int g = 0; g < d / gs; g++) {
     int64_t mo = spo_meta_offset(widths, d, gs, g);
@@ -295,7 +290,10 @@ void spo_unpack_token(const uint8_t* tile, const uint8_t* widths, int d, int gs,
   int n = spo_strips(widths, d, side, st, &payload);
   for (int j = 0; j < d; j++) codes[j] = 0;
   for (int k = 0; k < n; k++) {
-    unsigned field = spo_get_bits(tile, spo_locate(&st[k], t), st[k].w);
+    int64_t bo; int bit;
+    spo_locate(&st[k], t, &bo, &bit);
+    uint16_t hw = spo_get16(tile + bo);
+    uint16_t field = (uint16_t)((hw >> bit) & ((1u << st[k].w) - 1u));
     codes[st[k].chan] |= (uint16_t)(field << st[k].shift);
   }
   for (int g = 0; g < d / gs; g++) {

@@ -26,27 +26,25 @@ int sm_count() {
 
 // Workspace carve-up of the tensor-core path.
 struct FastLayout {
-  size_t ctx_off, desc_off, prefix_off, worker_off, rec_off, total;
-  int workers, rec_stride;
+  size_t desc_off, prefix_off, warp_off, rec_off, total;
+  int total_warps, rec_stride;
 };
 
-FastLayout fast_layout(int64_t n_units, int workers, int vs_max) {
+FastLayout fast_layout(int64_t n_units, int total_warps, int vs_max) {
   FastLayout L{};
-  L.workers = workers;
+  L.total_warps = total_warps;
   L.rec_stride = kFastGqa * (kRecHead + vs_max);
   size_t off = 0;
-  L.ctx_off = off; off = align_up(off + sizeof(UnitCtx) * (size_t)n_units, 256);
   L.desc_off = off; off = align_up(off + sizeof(UnitDesc) * (size_t)n_units, 256);
   L.prefix_off = off; off = align_up(off + sizeof(int32_t) * (size_t)(n_units + 1), 256);
-  L.worker_off = off; off = align_up(off + sizeof(int32_t) * (size_t)workers, 256);
-  L.rec_off = off; off = align_up(off + sizeof(float) * (size_t)L.rec_stride * (size_t)(workers + n_units), 256);
+  L.warp_off = off; off = align_up(off + sizeof(int32_t) * (size_t)total_warps, 256);
+  L.rec_off = off; off = align_up(off + sizeof(float) * (size_t)L.rec_stride * (size_t)(total_warps + n_units), 256);
   L.total = off;
   return L;
 }
 
-// What the host learns from the widths: tile sizes, and whether every parameter set fits the tensor-core path
-// (operand columns of the score MMA, accumulator rows, groups and sets of the value MMA).
-struct WidthFacts { int max_tile_k = 0, max_tile_v = 0, max_vstrips = 0; bool valid = true, fits = true; };
+// What the host learns from the widths: tile sizes, V strip and block counts.
+struct WidthFacts { int max_tile_k = 0, max_tile_v = 0, max_vstrips = 0, max_vblocks = 0; int vb[4] = {0, 0, 0, 0}; bool ok = true; };
 
 WidthFacts width_facts(const uint8_t* wk, const uint8_t* wv, int64_t n_sets) {
   WidthFacts F;
@@ -55,29 +53,48 @@ WidthFacts width_facts(const uint8_t* wk, const uint8_t* wv, int64_t n_sets) {
       const uint8_t* w = (side ? wv : wk) + s * kD;
       int bits = 0, cnt[4] = {0, 0, 0, 0}, act[2] = {0, 0};
       for (int j = 0; j < kD; j++) {
-        if (w[j] > 8) { F.valid = false; return F; }
+        if (w[j] > 8) { F.ok = false; return F; }
         bits += w[j];
         act[j / 64] |= w[j] != 0;
         for (int c = 0; c < 4; c++) cnt[c] += (w[j] & (8 >> c)) != 0;
       }
-      const int cfirst[5] = {0, cnt[0], cnt[0] + cnt[1], cnt[0] + cnt[1] + cnt[2], cnt[0] + cnt[1] + cnt[2] + cnt[3]};
       const int tb = 16 * bits + 512 * (act[0] + act[1]);
-      if (side == 0) {
-        F.max_tile_k = tb > F.max_tile_k ? tb : F.max_tile_k;
-        const int n_words = (bits + 31) / 32;
-        int cols = 0;
-        for (int i = 0; i < n_words && i < kKWordsMax; i++) cols += shape_slots(k_word_shape(cfirst, bits, i));
-        if (n_words > kKWordsMax || (cols + 7) / 8 > kKStepsMax) F.fits = false;
-      } else {
+      if (side == 0) F.max_tile_k = tb > F.max_tile_k ? tb : F.max_tile_k;
+      else {
         F.max_tile_v = tb > F.max_tile_v ? tb : F.max_tile_v;
-        F.max_vstrips = cfirst[4] > F.max_vstrips ? cfirst[4] : F.max_vstrips;
-        int row_first[4], grp[8];
-        const int rows = v_row_plan(cfirst, row_first);
-        if (rows > kVRowsMax || v_groups(cfirst, row_first, grp) > kVGroupsMax) F.fits = false;
+        const int strips = cnt[0] + cnt[1] + cnt[2] + cnt[3];
+        const int blocks = (cnt[0] + 15) / 16 + (cnt[1] + 15) / 16 + (cnt[2] + 15) / 16 + (cnt[3] + 15) / 16;
+        F.max_vstrips = strips > F.max_vstrips ? strips : F.max_vstrips;
+        F.max_vblocks = blocks > F.max_vblocks ? blocks : F.max_vblocks;
+        for (int c = 0; c < 4; c++) F.vb[c] = (cnt[c] + 15) / 16 > F.vb[c] ? (cnt[c] + 15) / 16 : F.vb[c];
       }
     }
   }
   return F;
+}
+
+template <int Q8, int Q4, int Q2, int Q1>
+int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {
+  if (cudaFuncSetAttribute(attention_mma_kernel<Q8, Q4, Q2, Q1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem) != cudaSuccess)
+    return SPECTRA_CUDA_ERROR;
+  attention_mma_kernel<Q8, Q4, Q2, Q1><<<grid, kFastWarps * 32, smem, st>>>(a, f);
+  return launch_status();
+}
+
+// Quota tuples (V blocks of 16 strips per class 8, 4, 2, 1) the main kernel is built for, smallest first.
+// They cover the width profiles that reverse water-filling produces at 4x to 12x on decaying spectra; anything
+// else runs on the CUDA-core kernel.
+constexpr int kQuotas[][4] = {{0, 1, 8, 2}, {0, 1, 3, 6}, {0, 1, 6, 4}, {0, 8, 2, 2}, {0, 7, 3, 4}};
+constexpr int kNumQuotas = sizeof(kQuotas) / sizeof(kQuotas[0]);
+
+int pick_quota(const int (&vb)[4]) {
+  for (int i = 0; i < kNumQuotas; i++) {
+    bool fits = true;
+    for (int c = 0; c < 4; c++) fits = fits && vb[c] <= kQuotas[i][c];
+    if (fits) return i;
+  }
+  return -1;
 }
 
 }  // namespace
@@ -91,7 +108,7 @@ extern "C" size_t spectra_attention_workspace_bytes(const spectra_config* cfg, i
   const size_t generic = (size_t)n_units * splits * (n_q_heads / n_kv_heads) * kPartialStride * sizeof(float) + 16;
   int sms = sm_count();
   if (sms <= 0) sms = 160;
-  const size_t fast = fast_layout(n_units, sms, kVRowsMax).total;
+  const size_t fast = fast_layout(n_units, sms * 3 * kFastWarps, kMaxStrips).total;
   return generic > fast ? generic : fast;
 }
 
@@ -136,40 +153,43 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
   a.status = status_word;
   cudaStream_t st = (cudaStream_t)stream;
 
-  // ---- tensor-core path: GQA group <= 4, scale group 64, host copy of the widths available, plans that fit
+  // ---- tensor-core path: GQA group <= 4, scale group 64, host copy of the widths available
   if (widths_k_host && gqa <= kFastGqa && cfg->scale_group == 64) {
     const WidthFacts F = width_facts(widths_k_host, widths_v_host, n_param_sets);
-    if (!F.valid) return SPECTRA_INVALID_ARG;
+    if (!F.ok) return SPECTRA_INVALID_ARG;
     const int sms = sm_count();
     if (sms <= 0) return SPECTRA_CUDA_ERROR;
     const int slot_k = (int)align_up((size_t)(F.max_tile_k > 16 ? F.max_tile_k : 16), 128);
     const int slot_v = (int)align_up((size_t)(F.max_tile_v > 16 ? F.max_tile_v : 16), 128);
-    const size_t fixed = align_up(sizeof(MainSmem), 128) + 128;
-    const size_t budget = 220 * 1024;
-    int depth = fixed < budget ? (int)((budget - fixed) / ((size_t)slot_k + slot_v)) : 0;
-    if (depth > kMaxStages) depth = kMaxStages;
-    if (F.fits && depth >= 2) {
-      FastLayout L = fast_layout(n_units, sms, F.max_vstrips);
+    const size_t pair = (size_t)slot_k + slot_v;
+    const size_t budget = 200 * 1024;
+    int ctas_per_sm = 3 * kFastWarps * pair <= budget ? 3 : (2 * kFastWarps * pair <= budget ? 2 : 1);
+    int depth = (int)(budget / ((size_t)ctas_per_sm * kFastWarps * pair));
+    if (depth > 4) depth = 4;
+    const int quota = pick_quota(F.vb);
+    if (depth >= 1 && quota >= 0) {
+      FastLayout L = fast_layout(n_units, sms * ctas_per_sm * kFastWarps, F.max_vstrips);
       if (L.total > workspace_bytes) return SPECTRA_WORKSPACE_TOO_SMALL;
       char* ws = reinterpret_cast<char*>(workspace);
       FastArgs f{};
-      f.ctx = reinterpret_cast<UnitCtx*>(ws + L.ctx_off);
       f.desc = reinterpret_cast<UnitDesc*>(ws + L.desc_off);
       f.tile_prefix = reinterpret_cast<int32_t*>(ws + L.prefix_off);
-      f.worker_unit = reinterpret_cast<int32_t*>(ws + L.worker_off);
+      f.warp_unit = reinterpret_cast<int32_t*>(ws + L.warp_off);
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
-      f.total_warps = L.workers; f.rec_stride = L.rec_stride; f.vs_max = F.max_vstrips;
+      f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = F.max_vstrips;
       f.n_units = (int)n_units; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
       attention_prep_kernel<<<(unsigned)n_units + 1, kPrepThreads, sizeof(PrepSmem), st>>>(a, f);
       if (launch_status()) return SPECTRA_CUDA_ERROR;
-      // the shared-memory size also keeps a second CTA off the SM: each CTA takes all tensor-memory columns
-      size_t smem = fixed + (size_t)depth * ((size_t)slot_k + slot_v);
-      if (smem < 120 * 1024) smem = 120 * 1024;
-      if (cudaFuncSetAttribute(attention_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-          cudaSuccess)
-        return SPECTRA_CUDA_ERROR;
-      attention_umma_kernel<<<sms, kMainThreads, smem, st>>>(a, f);
-      if (launch_status()) return SPECTRA_CUDA_ERROR;
+      const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64;
+      const int grid = sms * ctas_per_sm;
+      switch (quota) {
+        case 0: rc = launch_fast_main<0, 1, 8, 2>(a, f, grid, smem, st); break;
+        case 1: rc = launch_fast_main<0, 1, 3, 6>(a, f, grid, smem, st); break;
+        case 2: rc = launch_fast_main<0, 1, 6, 4>(a, f, grid, smem, st); break;
+        case 3: rc = launch_fast_main<0, 8, 2, 2>(a, f, grid, smem, st); break;
+        default: rc = launch_fast_main<0, 7, 3, 4>(a, f, grid, smem, st); break;
+      }
+      if (rc) return rc;
       attention_mma_combine_kernel<<<(unsigned)(n_units * gqa), 128, 0, st>>>(a, f);
       return launch_status();
     }
@@ -205,7 +225,7 @@ extern "C" size_t spectra_tile_bytes(const spectra_config* cfg, const uint8_t* w
 extern "C" void spectra_config_default(spectra_config* cfg) {
   if (!cfg) return;
   cfg->head_dim = kD; cfg->tile_tokens = kTile; cfg->scale_group = 64; cfg->width_group = 1; cfg->b_max = 8;
-  cfg->gain_mode = SPECTRA_GAIN_SQRT; cfg->layout_version = 2;
+  cfg->gain_mode = SPECTRA_GAIN_SQRT; cfg->layout_version = 1;
 }
 
 extern "C" const char* spectra_status_string(int code) {

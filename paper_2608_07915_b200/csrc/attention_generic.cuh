@@ -122,7 +122,11 @@ __global__ void __launch_bounds__(128) attention_generic_kernel(AttnArgs p) {
 #pragma unroll
         for (int h = 0; h < kMaxGqa; h++) acc[g][h] = 0.f;
       for (int k = 0; k < TK.n_strips; k++) {
-        const float f = (float)read_field(S.tile_k, field_bit(TK, SPECTRA_SIDE_K, k, t), 8 >> strip_class(TK, k));
+        int bo, bit;
+        locate_field(TK, SPECTRA_SIDE_K, k, t, bo, bit);
+        const int w = 8 >> strip_class(TK, k);
+        const unsigned hw = *reinterpret_cast<const uint16_t*>(S.tile_k + bo);
+        const float f = (float)((hw >> bit) & ((1u << w) - 1u));
         const int g = TK.chan[k] / gs;
 #pragma unroll
         for (int gg = 0; gg < kMaxGroups; gg++)

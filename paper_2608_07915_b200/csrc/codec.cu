@@ -131,9 +131,25 @@ __global__ void __launch_bounds__(128, 1) encode_kernel(EncodeArgs p) {
   if (status && p.status) atomicOr(p.status, status);
   __syncthreads();
 
-  // pack the payload (K: token strings, V: strips)
+  // pack: one half-word of the payload at a time, in storage order
   uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
-  pack_tile_payload(T, p.side, S.codes, kLdC, slot_lo, slot_hi, tile_ptr, tid, blockDim.x);
+  const int payload = T.class_off[4];
+  for (int off = 2 * tid; off < payload; off += 2 * blockDim.x) {
+    int w, first;
+    const int k = halfword_owner(T, p.side, off, w, first);
+    const int chan = T.chan[k], shift = T.shift[k];
+    const int per = 16 / w;
+    const unsigned fmask = (1u << w) - 1u;
+    unsigned hw = 0, keep = 0;
+    for (int e = 0; e < per; e++) {
+      const int tok = first + e;
+      if (tok < slot_lo) keep |= fmask << (e * w);
+      else if (tok < slot_hi) hw |= (((unsigned)S.codes[tok * kLdC + chan] >> shift) & fmask) << (e * w);
+    }
+    uint16_t* dst = reinterpret_cast<uint16_t*>(tile_ptr + off);
+    if (keep) hw |= (unsigned)(*dst) & keep;
+    *dst = (uint16_t)hw;
+  }
   for (int g = 0; g < T.n_groups; g++) {
     if (T.meta_off[g] < 0 || t < slot_lo) continue;
     uint16_t* lo_dst = reinterpret_cast<uint16_t*>(tile_ptr + T.meta_off[g]) + t;
@@ -169,7 +185,11 @@ __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
   const int t = tid;
   for (int j = 0; j < kD; j += 4) *reinterpret_cast<uint32_t*>(&S.codes[t * kLdC + j]) = 0u;
   for (int k = 0; k < T.n_strips; k++) {
-    const unsigned field = read_field(tile_ptr, field_bit(T, p.side, k, t), 8 >> strip_class(T, k));
+    int bo, bit;
+    locate_field(T, p.side, k, t, bo, bit);
+    const int w = 8 >> strip_class(T, k);
+    const unsigned hw = *reinterpret_cast<const uint16_t*>(tile_ptr + bo);
+    const unsigned field = (hw >> bit) & ((1u << w) - 1u);
     S.codes[t * kLdC + T.chan[k]] |= (uint8_t)(field << T.shift[k]);
   }
   __syncthreads();

@@ -1,9 +1,8 @@
 // Append path of spectra_encode for a handful of new tokens per unit-side (the decode step appends one).
 // One CTA of 128 threads per unit-side, thread j = rotated channel j.  No staging of whole tiles: the thread
 // rotates its channel, the CTA reduces the per-group minimum and maximum, every thread quantises its own code and
-// writes its sub-fields into the tail tile: V side with 16-bit read-modify-writes (different strips never share a
-// half-word), K side by assembling the token string in shared memory and storing its words.  The CTA owns the
-// unit-side, so global memory needs no atomics.
+// writes its sub-fields into the tail tile with 16-bit read-modify-writes.  Different strips never share a
+// half-word, and the CTA owns the unit-side, so no atomics are needed.
 #pragma once
 #include "common.cuh"
 
@@ -23,7 +22,6 @@ __global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
   __shared__ float red_lo[4], red_hi[4];
   __shared__ int cls_cnt[4][4];          // [class][warp]: strips of the class owned by the warp's channels
   __shared__ int grp_act[kMaxGroups];
-  __shared__ unsigned tok_string[kD * 8 / 32 + 1];   // K side: the token string being assembled
   const int u = blockIdx.x;
   const int ps = (int)(u % p.n_param_sets);
   const int j = threadIdx.x, lane = j & 31, warp = j >> 5;
@@ -43,14 +41,14 @@ __global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
   }
   if (b) grp_act[j / gs] = 1;
   __syncthreads();
-  int cls_off[4], my_rank[4];
+  int cls_n[4], cls_off[4], my_rank[4];
   int off = 0;
 #pragma unroll
   for (int c = 0; c < 4; c++) {
     int before = 0, n = 0;
 #pragma unroll
     for (int w = 0; w < 4; w++) { if (w < warp) before += cls_cnt[c][w]; n += cls_cnt[c][w]; }
-    cls_off[c] = off; my_rank[c] = before + rank_in_warp[c];
+    cls_n[c] = n; cls_off[c] = off; my_rank[c] = before + rank_in_warp[c];
     off += 16 * (8 >> c) * n;
   }
   const int payload = off;
@@ -136,45 +134,27 @@ __global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
       for (int i = j; i < tile_bytes / 16; i += 128) reinterpret_cast<uint4*>(tile)[i] = make_uint4(0, 0, 0, 0);
       __syncthreads();
     }
-    if (p.side == SPECTRA_SIDE_V) {
 #pragma unroll
-      for (int c = 0; c < 4; c++) {
-        const int wd = 8 >> c;
-        if (b & wd) {
-          const int shift = b & (wd - 1);
-          const unsigned field = ((unsigned)code >> shift) & ((1u << wd) - 1u);
-          const int k = my_rank[c];
+    for (int c = 0; c < 4; c++) {
+      const int wd = 8 >> c;
+      if (b & wd) {
+        const int shift = b & (wd - 1);
+        const unsigned field = ((unsigned)code >> shift) & ((1u << wd) - 1u);
+        const int k = my_rank[c], n = cls_n[c];
+        int bo, bit;
+        if (p.side == SPECTRA_SIDE_V) {
           const int a = slot >> 5, h = (slot >> 4) & 1, i = slot & 15;
-          const int bo = cls_off[c] + 16 * wd * k + 4 * (a * wd + ((i * wd) >> 4)) + 2 * h;
-          const int bit = (i * wd) & 15;
-          uint16_t* dst = reinterpret_cast<uint16_t*>(tile + bo);
-          const unsigned below = (1u << bit) - 1u;            // earlier tokens of the half-word are kept
-          *dst = (uint16_t)(((unsigned)(*dst) & below) | (field << bit));
+          bo = cls_off[c] + 16 * wd * k + 4 * (a * wd + ((i * wd) >> 4)) + 2 * h;
+          bit = (i * wd) & 15;
+        } else {
+          const int hw = (slot * wd) >> 4;
+          bit = (slot * wd) & 15;
+          if ((k | 1) < n) bo = cls_off[c] + 32 * wd * (k >> 1) + 4 * hw + 2 * (k & 1);
+          else bo = cls_off[c] + 16 * wd * k + 2 * hw;
         }
-      }
-    } else {
-      const int B = payload >> 4, F = B >> 5, r = B & 31;
-      if (j <= F) tok_string[j] = 0u;
-      __syncthreads();
-#pragma unroll
-      for (int c = 0; c < 4; c++) {
-        const int wd = 8 >> c;
-        if (b & wd) {
-          const int shift = b & (wd - 1);
-          const unsigned field = ((unsigned)code >> shift) & ((1u << wd) - 1u);
-          const int o = (cls_off[c] >> 4) + my_rank[c] * wd;  // offset of the field in the token string
-          atomicOr(&tok_string[o >> 5], field << (o & 31));
-        }
-      }
-      __syncthreads();
-      if (j < F) reinterpret_cast<uint32_t*>(tile)[kTile * j + slot] = tok_string[j];
-      else if (j == F && r) {                                 // the remainder bits, packed densely behind the words
-        uint32_t* tail = reinterpret_cast<uint32_t*>(tile + 512 * F);
-        const int bitpos = r * slot, q = bitpos >> 5, sh = bitpos & 31;
-        const unsigned long long m = (unsigned long long)((1u << r) - 1u) << sh;
-        const unsigned long long v = (unsigned long long)tok_string[F] << sh;
-        tail[q] = (tail[q] & ~(unsigned)m) | (unsigned)v;
-        if (m >> 32) tail[q + 1] = (tail[q + 1] & ~(unsigned)(m >> 32)) | (unsigned)(v >> 32);
+        uint16_t* dst = reinterpret_cast<uint16_t*>(tile + bo);
+        const unsigned below = (1u << bit) - 1u;              // earlier tokens of the half-word are kept
+        *dst = (uint16_t)(((unsigned)(*dst) & below) | (field << bit));
       }
     }
     if (meta_off >= 0 && (j % gs) == 0) {                     // one writer per scale group

@@ -178,9 +178,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_tc_kernel(EncodeTcArgs p
       }
     }
     __syncthreads();
-    // ---- pack the payload (K: token strings, V: strips)
+    // ---- pack: one half-word of the payload at a time, in storage order
     uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
-    pack_tile_payload(T, p.side, S.codes, kLdCode, slot_lo, slot_hi, tile_ptr, tid, kTcThreads);
+    const int payload = T.class_off[4];
+    for (int off = 2 * tid; off < payload; off += 2 * kTcThreads) {
+      int w, first;
+      const int k = halfword_owner(T, p.side, off, w, first);
+      const int chan = T.chan[k], shift = T.shift[k];
+      const int per = 16 / w;
+      const unsigned fmask = (1u << w) - 1u;
+      unsigned hw = 0, keep = 0;
+      for (int e = 0; e < per; e++) {
+        const int tok = first + e;
+        if (tok < slot_lo) keep |= fmask << (e * w);
+        else if (tok < slot_hi) hw |= (((unsigned)S.codes[tok * kLdCode + chan] >> shift) & fmask) << (e * w);
+      }
+      uint16_t* dst = reinterpret_cast<uint16_t*>(tile_ptr + off);
+      if (keep) hw |= (unsigned)(*dst) & keep;
+      *dst = (uint16_t)hw;
+    }
     for (int idx = tid; idx < 2 * kTile; idx += kTcThreads) {
       const int g = idx / kTile, t = idx - g * kTile;
       if (T.meta_off[g] < 0 || t < slot_lo) continue;

@@ -35,7 +35,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_config_default_and_host_helpers(lib):
     cfg = sp.default_config()
     assert (cfg.head_dim, cfg.tile_tokens, cfg.scale_group, cfg.width_group, cfg.b_max, cfg.layout_version) == \
-        (128, 128, 64, 1, 8, 2)
+        (128, 128, 64, 1, 8, 1)
     assert sp.total_bits(cfg, 4.0) == 512 and sp.total_bits(cfg, 8.0) == 256 and sp.total_bits(cfg, 12.0) == 170
     assert sp.total_bits(cfg, 1.0) == 1024                      # clamped to b_max * d
     w = [4] * 128

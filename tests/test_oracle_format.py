@@ -101,11 +101,8 @@ def _positions(widths, side):
 
 
 @pytest.mark.parametrize("side", [codec.SIDE_K, codec.SIDE_V])
-@pytest.mark.parametrize("extra", [[], [3], [8, 8, 8, 5]])
-def test_layout_is_a_bijection_onto_the_payload(side, extra):
-    # every sub-field class, odd and even strip counts; token strings of 32, 35 and 61 bits (whole words, words plus
-    # a remainder)
-    widths = np.array([7, 5, 3, 0, 1, 8, 2, 6] + extra, np.uint8)
+def test_layout_is_a_bijection_onto_the_payload(side):
+    widths = np.array([7, 5, 3, 0, 1, 8, 2, 6], np.uint8)     # every sub-field class, odd and even strip counts
     seen = _positions(widths, side)
     payload_bits = 128 * int(widths.sum())
     assert len(seen) == payload_bits
@@ -146,16 +143,6 @@ def test_packer_reproduces_handworked_tiles():
     for off, val in gold[("B", "K")].items():
         expect[off] = val
     assert np.array_equal(tile, expect)
-    wc = np.array([8, 8, 8, 8, 4, 2, 1, 0], np.uint8)
-    for side, name in ((codec.SIDE_K, "K"), (codec.SIDE_V, "V")):
-        tile = np.zeros(codec.tile_bytes(wc, 8), np.uint8)
-        assert tile.size == 1136
-        codec.pack_token(tile, wc, 8, side, 3, np.array([0x12, 0x34, 0x56, 0x78, 0xA, 2, 1, 0], np.uint16),
-                         np.zeros(1, np.uint16), np.zeros(1, np.uint16))
-        expect = np.zeros_like(tile)
-        for off, val in gold[("C", name)].items():
-            expect[off] = val
-        assert np.array_equal(tile, expect)
 
 
 @pytest.mark.parametrize("side", [codec.SIDE_K, codec.SIDE_V])
