@@ -134,13 +134,21 @@ struct PrepSmem {
   float red[kFastGqa][4];
   int escale[kFastGqa];
   int scan[128];
+  int ng0[2][4];      // strips of scale group 0 per class: [K, V][class]
 };
 
-__device__ inline uint32_t pack_cls(const StripTable& T, int c) {
+__device__ inline uint32_t pack_cls(const StripTable& T, int c, int n_g0) {
   const int first = T.class_first[c], n = T.class_first[c + 1] - first;
-  int n_g0 = 0;
-  for (int k = first; k < first + n; k++) n_g0 += T.chan[k] < 64;
   return (uint32_t)n | ((uint32_t)n_g0 << 8) | ((uint32_t)(T.class_off[c] / 16) << 16);
+}
+
+// Strips of class c whose channel lies in scale group 0 (channels < 64), counted by one warp.
+__device__ inline int count_group0(const StripTable& T, int c, int lane) {
+  int cnt = 0;
+  for (int k = T.class_first[c] + lane; k < T.class_first[c + 1]; k += 32) cnt += T.chan[k] < 64;
+#pragma unroll
+  for (int s = 16; s; s >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, s);
+  return cnt;
 }
 
 constexpr int kPrepThreads = 512;
@@ -207,16 +215,27 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
   }
   __syncthreads();
   const float* wk = p.w_dec_k + (int64_t)ps * kD * kD;
-  for (int j = warp; j < kD; j += kWarps) {
-    const float4 wrow = *reinterpret_cast<const float4*>(wk + j * kD + lane * 4);
+  {
+    float4 wrow[kD / kWarps];
 #pragma unroll
-    for (int h = 0; h < kFastGqa; h++) {
-      const float4 qv = *reinterpret_cast<const float4*>(&S.qraw[h][lane * 4]);
-      float acc = wrow.x * qv.x + wrow.y * qv.y + wrow.z * qv.z + wrow.w * qv.w;
+    for (int r = 0; r < kD / kWarps; r++)          // all row loads of this warp in flight together
+      wrow[r] = *reinterpret_cast<const float4*>(wk + (warp + kWarps * r) * kD + lane * 4);
 #pragma unroll
-      for (int s = 16; s; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-      if (lane == 0) S.qrot[h][j] = acc * p.scale * kLog2e;   // scores live in the log2 domain
+    for (int r = 0; r < kD / kWarps; r++) {
+#pragma unroll
+      for (int h = 0; h < kFastGqa; h++) {
+        const float4 qv = *reinterpret_cast<const float4*>(&S.qraw[h][lane * 4]);
+        float acc = wrow[r].x * qv.x + wrow[r].y * qv.y + wrow[r].z * qv.z + wrow[r].w * qv.w;
+#pragma unroll
+        for (int s = 16; s; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+        if (lane == 0) S.qrot[h][warp + kWarps * r] = acc * p.scale * kLog2e;   // scores live in the log2 domain
+      }
     }
+  }
+  if (warp >= 8) {                                  // meanwhile: group-0 strip counts per class (warps 8..15)
+    const int side = (warp - 8) >> 2, c = (warp - 8) & 3;
+    const int cnt = count_group0(side ? TV : TK, c, lane);
+    if (lane == 0) S.ng0[side][c] = cnt;
   }
   __syncthreads();
   // per-head power-of-two normalisation so that the fp16 hi/lo split of q'' = q' 2^shift / L is well conditioned
@@ -270,8 +289,7 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
   int chunk0 = 0;
   for (int c = 0; c < 4; c++) {
     const int first = TK.class_first[c], n = TK.class_first[c + 1] - first;
-    int n_g0 = 0;
-    for (int k = first; k < first + n; k++) n_g0 += TK.chan[k] < 64;      // every thread: at most 128 steps
+    const int n_g0 = S.ng0[0][c];
     const int s1 = n_g0 & ~1;
     const int nch0 = (n_g0 + 15) / 16, nch1 = n > n_g0 ? (n - s1 + 15) / 16 : 0;
     const int w = 8 >> c;
@@ -300,8 +318,8 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
     }
     chunk0 += nch0 + nch1;
   }
-  if (tid >= 64 && tid < 68) D.kcls[tid - 64] = pack_cls(TK, tid - 64);      // spread over different warps
-  if (tid >= 96 && tid < 100) D.vcls[tid - 96] = pack_cls(TV, tid - 96);
+  if (tid >= 64 && tid < 68) D.kcls[tid - 64] = pack_cls(TK, tid - 64, S.ng0[0][tid - 64]);
+  if (tid >= 96 && tid < 100) D.vcls[tid - 96] = pack_cls(TV, tid - 96, S.ng0[1][tid - 96]);
   if (tid >= 128 && tid < 132) D.vfirst[tid - 128] = TV.class_first[tid - 128];
   if (tid == 0) {
     D.tbk = TK.tile_bytes; D.tbv = TV.tile_bytes;
