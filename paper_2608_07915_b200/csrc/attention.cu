@@ -108,7 +108,8 @@ extern "C" size_t spectra_attention_workspace_bytes(const spectra_config* cfg, i
   const size_t generic = (size_t)n_units * splits * (n_q_heads / n_kv_heads) * kPartialStride * sizeof(float) + 16;
   int sms = sm_count();
   if (sms <= 0) sms = 160;
-  const size_t fast = fast_layout(n_units, sms * 3 * kFastWarps, kMaxStrips).total;
+  const int npass = (n_q_heads / n_kv_heads + kFastGqa - 1) / kFastGqa;
+  const size_t fast = fast_layout(n_units * npass, sms * 3 * kFastWarps, kMaxStrips).total;
   return generic > fast ? generic : fast;
 }
 
@@ -153,8 +154,11 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
   a.status = status_word;
   cudaStream_t st = (cudaStream_t)stream;
 
-  // ---- tensor-core path: GQA group <= 4, scale group 64, host copy of the widths available
-  if (widths_k_host && gqa <= kFastGqa && cfg->scale_group == 64) {
+  // ---- tensor-core path: scale group 64, host copy of the widths available; a GQA group of more than 4 query
+  // heads is taken in passes of 4 (each pass is a unit of its own that reads the same tiles)
+  const int npass = (gqa + kFastGqa - 1) / kFastGqa;
+  const int64_t n_vunits = n_units * npass;
+  if (widths_k_host && cfg->scale_group == 64 && n_vunits <= 65534) {
     const WidthFacts F = width_facts(widths_k_host, widths_v_host, n_param_sets);
     if (!F.ok) return SPECTRA_INVALID_ARG;
     const int sms = sm_count();
@@ -168,7 +172,7 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
     if (depth > 4) depth = 4;
     const int quota = pick_quota(F.vb);
     if (depth >= 1 && quota >= 0) {
-      FastLayout L = fast_layout(n_units, sms * ctas_per_sm * kFastWarps, F.max_vstrips);
+      FastLayout L = fast_layout(n_vunits, sms * ctas_per_sm * kFastWarps, F.max_vstrips);
       if (L.total > workspace_bytes) return SPECTRA_WORKSPACE_TOO_SMALL;
       char* ws = reinterpret_cast<char*>(workspace);
       FastArgs f{};
@@ -177,8 +181,8 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
       f.warp_unit = reinterpret_cast<int32_t*>(ws + L.warp_off);
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
       f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = F.max_vstrips;
-      f.n_units = (int)n_units; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
-      attention_prep_kernel<<<(unsigned)n_units + 1, kPrepThreads, sizeof(PrepSmem), st>>>(a, f);
+      f.n_units = (int)n_vunits; f.npass = npass; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
+      attention_prep_kernel<<<(unsigned)n_vunits + 1, kPrepThreads, sizeof(PrepSmem), st>>>(a, f);
       if (launch_status()) return SPECTRA_CUDA_ERROR;
       const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64;
       const int grid = sms * ctas_per_sm;
@@ -190,7 +194,7 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
         default: rc = launch_fast_main<0, 7, 3, 4>(a, f, grid, smem, st); break;
       }
       if (rc) return rc;
-      attention_mma_combine_kernel<<<(unsigned)(n_units * gqa), 128, 0, st>>>(a, f);
+      attention_mma_combine_kernel<<<(unsigned)(n_vunits * kFastGqa), 128, 0, st>>>(a, f);
       return launch_status();
     }
   }

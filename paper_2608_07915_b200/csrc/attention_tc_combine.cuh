@@ -1,4 +1,4 @@
-// Combine kernel of the tensor-core decode attention: one CTA of 128 threads per (unit, query head).
+// Combine kernel of the tensor-core decode attention: one CTA of 128 threads per (unit of the tensor path, head slot).
 // Merges the partial records the worker warps wrote for the unit (log-sum-exp over the sequence split), folds the
 // per-strip accumulators back into channels of the rotated value space, adds the rotated mean and lifts the result
 // once through W_dec,V:  out = (o' / l + m'_V) W_dec,V.
@@ -15,17 +15,19 @@ __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, 
   __shared__ float s_o[kD];
   __shared__ float s_part[4][kMaxStrips];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int G = p.gqa;
-  const int u = blockIdx.x / G, h = blockIdx.x - u * G;
+  const int vu = blockIdx.x / kFastGqa, h = blockIdx.x - vu * kFastGqa;   // unit of the tensor path, head slot of its pass
+  const int u = vu / f.npass, h0 = kFastGqa * (vu - u * f.npass);
+  if (h0 + h >= p.gqa) return;
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
-  const UnitDesc& D = f.desc[u];
+  const UnitDesc& D = f.desc[vu];
   const long long total = f.tile_prefix[f.n_units];
-  const long long ta = f.tile_prefix[u], tb = f.tile_prefix[u + 1];
-  const int64_t oidx = ((int64_t)b * p.n_q + hk * G + h) * kD + tid;
+  const long long ta = f.tile_prefix[vu], tb = f.tile_prefix[vu + 1];
+  const int64_t hidx = (int64_t)b * p.n_q + hk * p.gqa + h0 + h;         // query head in the caller's order
+  const int64_t oidx = hidx * kD + tid;
   if (tb <= ta) {                                            // empty sequence
     store_from_float(p.out, p.out_dtype, oidx, 0.f);
-    if (p.lse && tid == 0) p.lse[(int64_t)b * p.n_q + hk * G + h] = -INFINITY;
+    if (p.lse && tid == 0) p.lse[hidx] = -INFINITY;
     return;
   }
   // workers whose tile ranges intersect this unit: the largest gw with floor(gw * total / W) <= tile
@@ -34,7 +36,7 @@ __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, 
   const int gw_last = (int)((tb * W + total - 1) / total) - 1;
   const int nrec = gw_last - gw_first + 1;
   const int64_t hoff = (int64_t)h * (kRecHead + f.vs_max);
-  auto rec_ptr = [&](int r) { return f.records + (int64_t)(gw_first + r + u) * f.rec_stride + hoff; };
+  auto rec_ptr = [&](int r) { return f.records + (int64_t)(gw_first + r + vu) * f.rec_stride + hoff; };
   auto nonempty = [&](int r) {
     const long long gw = gw_first + r;
     return (gw + 1) * total / W > gw * total / W;
@@ -121,7 +123,7 @@ __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, 
   }
   store_from_float(p.out, p.out_dtype, oidx, live ? (o0 + o1) + (o2 + o3) : 0.f);
   if (p.lse && tid == 0)
-    p.lse[(int64_t)b * p.n_q + hk * G + h] = live ? (M + log2f(L)) / kLog2e + D.qconst[h] : -INFINITY;
+    p.lse[hidx] = live ? (M + log2f(L)) / kLog2e + D.qconst[h] : -INFINITY;
 }
 
 }  // namespace spectra

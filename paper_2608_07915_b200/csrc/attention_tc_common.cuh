@@ -48,7 +48,9 @@ struct alignas(16) UnitDesc {
 
 struct FastArgs {
   UnitDesc* desc; int32_t* tile_prefix; int32_t* warp_unit; float* records;
-  int total_warps; int rec_stride; int vs_max; int n_units;
+  int total_warps; int rec_stride; int vs_max;
+  int n_units;       // units of the tensor path: (sequence, kv-head, pass); a pass takes up to 4 query heads of the group
+  int npass;
   int depth; int slot_k, slot_v;
 };
 
@@ -164,7 +166,7 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
     const int per = (n_units + 127) / 128;
     int local = 0;
     if (tid < 128) {
-      for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (p.seq_len[i / p.n_kv] + kTile - 1) / kTile;
+      for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (p.seq_len[(i / f.npass) / p.n_kv] + kTile - 1) / kTile;
       S.scan[tid] = local;
     }
     __syncthreads();
@@ -178,7 +180,7 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
       int run = S.scan[tid];
       for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) {
         f.tile_prefix[i] = run;
-        run += (p.seq_len[i / p.n_kv] + kTile - 1) / kTile;
+        run += (p.seq_len[(i / f.npass) / p.n_kv] + kTile - 1) / kTile;
       }
     }
     __syncthreads();
@@ -201,17 +203,18 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
     }
     return;
   }
-  const int u = blockIdx.x;
+  const int vu = blockIdx.x;
+  const int u = vu / f.npass, h0 = kFastGqa * (vu - u * f.npass);   // cache unit, first query head of this pass
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
-  const int G = p.gqa;
+  const int G = min(kFastGqa, p.gqa - h0);                          // query heads of this pass
   build_strip_tables(S.tk, p.widths_k + (int64_t)ps * kD, S.tv, p.widths_v + (int64_t)ps * kD, 64);
   const StripTable& TK = S.tk;
   const StripTable& TV = S.tv;
-  UnitDesc& D = f.desc[u];
+  UnitDesc& D = f.desc[vu];
   for (int idx = tid; idx < kFastGqa * kD; idx += kPrepThreads) {
     const int h = idx / kD, i = idx - h * kD;
-    S.qraw[h][i] = h < G ? load_as_float(p.q, p.q_dtype, ((int64_t)b * p.n_q + hk * G + h) * kD + i) : 0.f;
+    S.qraw[h][i] = h < G ? load_as_float(p.q, p.q_dtype, ((int64_t)b * p.n_q + hk * p.gqa + h0 + h) * kD + i) : 0.f;
   }
   __syncthreads();
   const float* wk = p.w_dec_k + (int64_t)ps * kD * kD;

@@ -267,9 +267,9 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
     const UnitDesc& d = f.desc[prod.u];
     const uint32_t tbk = d.tbk, tbv = d.tbv;
     mbar_expect_tx(bars + 8 * slot, tbk);
-    bulk_load(smem_u32(ring_k + slot * f.slot_k), p.cache_k + p.off_k[prod.u] + (int64_t)prod.t * tbk, tbk,
+    bulk_load(smem_u32(ring_k + slot * f.slot_k), p.cache_k + p.off_k[prod.u / f.npass] + (int64_t)prod.t * tbk, tbk,
               bars + 8 * slot);
-    v_src = p.cache_v + p.off_v[prod.u] + (int64_t)prod.t * tbv;
+    v_src = p.cache_v + p.off_v[prod.u / f.npass] + (int64_t)prod.t * tbv;
     v_bytes = tbv;
     prod.next(f);
   };
@@ -303,7 +303,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
       kmeta0 = d.kmeta[0]; kmeta1 = d.kmeta[1]; vmeta0 = d.vmeta[0]; vmeta1 = d.vmeta[1];
       kscale = d.kscale[tig]; qlo0 = d.qlo[tig][0]; qlo1 = d.qlo[tig][1];
       kB = &d.kB[0][0][0];
-      n_seq = p.seq_len[cons.u / p.n_kv];
+      n_seq = p.seq_len[(cons.u / f.npass) / p.n_kv];
 #pragma unroll
       for (int mb = 0; mb < NACC; mb++)
 #pragma unroll
