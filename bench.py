@@ -242,13 +242,14 @@ def run_ours(args, wl):
         e = ev(); e.record(); attn_events.append(e)
 
     def step_resident(i, timed=False):
-        model.decode_step(q_dev[i % n_in], nk_dev[i % n_in], nv_dev[i % n_in], out_dev, mark if timed else None)
+        model.decode_step(q_dev[i % n_in], nk_dev[i % n_in], nv_dev[i % n_in], out_dev, mark if timed else None,
+                          fused=args.fused)
 
     def step_e2e(i):
         q_stage.copy_(q_host[i % n_in], non_blocking=True)
         nk_stage.copy_(nk_host[i % n_in], non_blocking=True)
         nv_stage.copy_(nv_host[i % n_in], non_blocking=True)
-        model.decode_step(q_stage, nk_stage, nv_stage, out_dev)
+        model.decode_step(q_stage, nk_stage, nv_stage, out_dev, fused=args.fused)
         out_host.copy_(out_dev, non_blocking=True)
 
     # ---- device-resident timing
@@ -320,9 +321,10 @@ def run_ours(args, wl):
                    else "WARNING: coded cache fits L2"},
         "e2e": {"value": world * kv_tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
-        "gpu_launches": steps * L * (2 + sp.ATTENTION_LAUNCHES),
+        "gpu_launches": steps * L * (sp.STEP_LAUNCHES if args.fused else 2 + sp.ATTENTION_LAUNCHES),
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "spectra_decode_attention (one layer call)", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": "spectra_decode_step (one layer call: append + attention)" if args.fused
+                     else "spectra_decode_attention (one layer call)", "achieved": achieved,
                      "peak": hbm_gbs, "unit": "GB/s", "frac": achieved / hbm_gbs, "peak_kind": peak_kind,
                      "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "bytes_per_launch": bytes_call, "ms_per_launch": attn_ms_avg},
         "phases": {"setup_s": setup_s, "fit_alloc_ms_total": model.timings["fit_alloc_ms"],
@@ -351,6 +353,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers than the workload (invalid as a result)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--unfused", dest="fused", action="store_false",
+                    help="per layer: spectra_encode (K, V) + spectra_decode_attention instead of spectra_decode_step")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="launch the timed steps directly instead of replaying them as CUDA graphs")
     args = ap.parse_args()

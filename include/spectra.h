@@ -199,7 +199,8 @@ int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, co
  * only when lse != NULL and may be NULL otherwise.  widths_k_host / widths_v_host: HOST copies of the two width
  * arrays ([n_param_sets, d], the same values the caller already needs for spectra_tile_bytes); read during the
  * call only.  They let the host size shared-memory rings and pick the kernel variant without a device
- * round-trip.  With both NULL, or a GQA group above 4, or scale_group != 64, a slower CUDA-core kernel runs.
+ * round-trip.  With both NULL, or scale_group != 64, or width profiles outside the built variants, a slower
+ * CUDA-core kernel runs.  A GQA group of 5 to 8 query heads is taken in two passes over the tiles.
  * softmax_scale 0 means 1/sqrt(d).
  * out: device [batch, n_q_heads, d], out_dtype.  lse: device fp32 [batch, n_q_heads] or NULL.
  * workspace: device, >= spectra_attention_workspace_bytes(...), 16-byte aligned; scratch only, nothing is
@@ -216,6 +217,27 @@ int spectra_decode_attention(const spectra_config* cfg, const void* q, int q_dty
                              void* stream);
 size_t spectra_attention_workspace_bytes(const spectra_config* cfg, int32_t batch, int32_t n_kv_heads,
                                          int32_t n_q_heads, int32_t max_seq_len);
+
+/* ------------------------------------------------------------------------------------------------
+ * spectra_decode_step -- one decode step of one layer: Sec. 3.3 (each new token's key and value are
+ * down-projected, quantised and appended to the coded cache) followed by the latent-space attention of
+ * spectra_decode_attention over the grown cache, with the append folded into the attention's first launch.
+ * Same results, bit for bit in the cache, as spectra_encode(K), spectra_encode(V) (one new token per unit at
+ * position seq_len[sequence] - 1) followed by spectra_decode_attention.
+ * new_k, new_v: device [batch * n_kv_heads, d] (one vector per unit, unit order as above), x_dtype SPECTRA_F32
+ * or SPECTRA_BF16.  seq_len: device int32 [batch], the lengths INCLUDING the appended token (>= 1).
+ * w_enc_k/v, mean_rot_k/v as in spectra_encode; every other argument as in spectra_decode_attention
+ * (mean_rot_k is required here).  cache_k / cache_v are written (the appended token) and read.
+ */
+int spectra_decode_step(const spectra_config* cfg, const void* q, int q_dtype, const void* new_k, const void* new_v,
+                        int x_dtype, int32_t batch, int32_t n_kv_heads, int32_t n_q_heads, const int32_t* seq_len,
+                        int32_t max_seq_len, uint8_t* cache_k, const int64_t* unit_offset_k, uint8_t* cache_v,
+                        const int64_t* unit_offset_v, int64_t n_param_sets, const float* w_enc_k,
+                        const float* w_dec_k, const float* mean_rot_k, const uint8_t* widths_k, const float* w_enc_v,
+                        const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
+                        const uint8_t* widths_k_host, const uint8_t* widths_v_host, float softmax_scale, void* out,
+                        int out_dtype, float* lse, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                        void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Helpers (host only, no device work).

@@ -20,10 +20,11 @@ GAIN_ROTATE, GAIN_SQRT, GAIN_WHITEN = 0, 1, 2
 HEAD_DIM = 128
 TILE_TOKENS = 128
 ATTENTION_LAUNCHES = 3   # kernels one spectra_decode_attention call enqueues
+STEP_LAUNCHES = 3        # kernels one spectra_decode_step call enqueues on the tensor-core path (the append rides in the first)
 
 EXPORTS = [
     "spectra_fit_basis", "spectra_fit_basis_static", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
-    "spectra_decode_attention", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
+    "spectra_decode_attention", "spectra_decode_step", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
     "spectra_total_bits", "spectra_status_string",
 ]
 
@@ -180,3 +181,27 @@ def decode_attention(cfg, q, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len,
         _ptr(mean_rot_v), _ptr(widths_v), wkh, wvh, C.c_float(softmax_scale), _ptr(out), C.c_int(_dtype_code(out)), _ptr(lse),
         _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()), _ptr(status_word), _stream())
     _check(rc, "spectra_decode_attention")
+
+
+def decode_step(cfg, q, new_k, new_v, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k,
+                cache_v, unit_offset_v, n_param_sets, w_enc_k, w_dec_k, mean_rot_k, widths_k, w_enc_v, w_dec_v,
+                mean_rot_v, widths_v, softmax_scale, out, lse, workspace, status_word=None, widths_k_host=None,
+                widths_v_host=None):
+    """One decode step of a layer: appends new_k / new_v ([batch * n_kv_heads, 128], one vector per unit) at
+    position seq_len - 1 and attends over seq_len tokens (seq_len already counts the new token)."""
+    wkh = wvh = C.c_void_p(0)
+    if widths_k_host is not None:
+        assert widths_k_host.dtype.name == "uint8" and widths_k_host.flags.c_contiguous
+        assert widths_v_host.dtype.name == "uint8" and widths_v_host.flags.c_contiguous
+        assert widths_k_host.size == n_param_sets * HEAD_DIM == widths_v_host.size
+        wkh = widths_k_host.ctypes.data_as(C.c_void_p)
+        wvh = widths_v_host.ctypes.data_as(C.c_void_p)
+    assert new_k.dtype == new_v.dtype and new_k.is_contiguous() and new_v.is_contiguous()
+    rc = lib().spectra_decode_step(
+        C.byref(cfg), _ptr(q), C.c_int(_dtype_code(q)), _ptr(new_k), _ptr(new_v), C.c_int(_dtype_code(new_k)),
+        C.c_int32(batch), C.c_int32(n_kv_heads), C.c_int32(n_q_heads), _ptr(seq_len), C.c_int32(max_seq_len),
+        _ptr(cache_k), _ptr(unit_offset_k), _ptr(cache_v), _ptr(unit_offset_v), C.c_int64(n_param_sets),
+        _ptr(w_enc_k), _ptr(w_dec_k), _ptr(mean_rot_k), _ptr(widths_k), _ptr(w_enc_v), _ptr(w_dec_v), _ptr(mean_rot_v),
+        _ptr(widths_v), wkh, wvh, C.c_float(softmax_scale), _ptr(out), C.c_int(_dtype_code(out)), _ptr(lse),
+        _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()), _ptr(status_word), _stream())
+    _check(rc, "spectra_decode_step")

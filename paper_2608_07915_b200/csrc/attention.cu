@@ -17,6 +17,12 @@ int generic_splits(int n_units, int max_seq_len) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Token positions of a fused step on the generic path: unit u appends at seq_len[u / n_kv] - 1.
+__global__ void step_positions_kernel(const int32_t* seq_len, int n_kv, int n_units, int32_t* pos) {
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u < n_units) pos[u] = seq_len[u / n_kv] - 1;
+}
+
 int sm_count() {
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
@@ -113,15 +119,22 @@ extern "C" size_t spectra_attention_workspace_bytes(const spectra_config* cfg, i
   return generic > fast ? generic : fast;
 }
 
-extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q, int q_dtype, int32_t batch,
-                                        int32_t n_kv_heads, int32_t n_q_heads, const int32_t* seq_len,
-                                        int32_t max_seq_len, const uint8_t* cache_k, const int64_t* unit_offset_k,
-                                        const uint8_t* cache_v, const int64_t* unit_offset_v, int64_t n_param_sets,
-                                        const float* w_dec_k, const float* mean_rot_k, const uint8_t* widths_k,
-                                        const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
-                                        const uint8_t* widths_k_host, const uint8_t* widths_v_host,
-                                        float softmax_scale, void* out, int out_dtype, float* lse, void* workspace,
-                                        size_t workspace_bytes, int32_t* status_word, void* stream) {
+namespace {
+
+// New key and value vectors of a fused decode step (NULL new_k: plain attention call).
+struct StepAppend {
+  const void* new_k; const void* new_v; int x_dtype;
+  const float* w_enc_k; const float* w_enc_v; uint8_t* cache_k; uint8_t* cache_v;
+};
+
+int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_t batch, int32_t n_kv_heads,
+                   int32_t n_q_heads, const int32_t* seq_len, int32_t max_seq_len, const uint8_t* cache_k,
+                   const int64_t* unit_offset_k, const uint8_t* cache_v, const int64_t* unit_offset_v,
+                   int64_t n_param_sets, const float* w_dec_k, const float* mean_rot_k, const uint8_t* widths_k,
+                   const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
+                   const uint8_t* widths_k_host, const uint8_t* widths_v_host, float softmax_scale, void* out,
+                   int out_dtype, float* lse, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                   void* stream, const StepAppend* app) {
   int rc = check_config(cfg);
   if (rc) return rc;
   if (batch < 0 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || max_seq_len < 0 || n_param_sets < 1)
@@ -182,7 +195,16 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
       f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = F.max_vstrips;
       f.n_units = (int)n_vunits; f.npass = npass; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
-      attention_prep_kernel<<<(unsigned)n_vunits + 1, kPrepThreads, sizeof(PrepSmem), st>>>(a, f);
+      if (app) {
+        AppendArgs ak{app->new_k, app->x_dtype, 0, SPECTRA_SIDE_K, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
+                      app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, status_word, seq_len, n_kv_heads};
+        AppendArgs av{app->new_v, app->x_dtype, 0, SPECTRA_SIDE_V, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
+                      app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, status_word, seq_len, n_kv_heads};
+        decode_step_front_kernel<<<(unsigned)(n_vunits + 1 + 2 * n_units), kPrepThreads, sizeof(PrepSmem), st>>>(
+            a, f, ak, av, (int)n_units);
+      } else {
+        attention_prep_kernel<<<(unsigned)n_vunits + 1, kPrepThreads, sizeof(PrepSmem), st>>>(a, f);
+      }
       if (launch_status()) return SPECTRA_CUDA_ERROR;
       const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64;
       const int grid = sms * ctas_per_sm;
@@ -199,7 +221,18 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
     }
   }
 
-  // ---- generic path
+  // ---- generic path (a fused step appends through the ordinary encode launches first)
+  if (app) {
+    // positions: lengths minus one, written into the head of the workspace (the partials come after the appends)
+    int32_t* pos = reinterpret_cast<int32_t*>(workspace);
+    step_positions_kernel<<<(unsigned)((n_units + 255) / 256), 256, 0, st>>>(seq_len, n_kv_heads, (int)n_units, pos);
+    rc = spectra_encode(cfg, SPECTRA_SIDE_K, app->new_k, app->x_dtype, 0, n_units, n_param_sets, pos, 1, kD, kD,
+                        app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, status_word, stream);
+    if (rc) return rc;
+    rc = spectra_encode(cfg, SPECTRA_SIDE_V, app->new_v, app->x_dtype, 0, n_units, n_param_sets, pos, 1, kD, kD,
+                        app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, status_word, stream);
+    if (rc) return rc;
+  }
   if (cudaFuncSetAttribute(attention_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)sizeof(GenericSmem)) != cudaSuccess)
     return SPECTRA_CUDA_ERROR;
@@ -208,6 +241,42 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
   if (launch_status()) return SPECTRA_CUDA_ERROR;
   attention_combine_kernel<<<(unsigned)n_units, 128, 0, st>>>(a);
   return launch_status();
+}
+
+}  // namespace
+
+extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q, int q_dtype, int32_t batch,
+                                        int32_t n_kv_heads, int32_t n_q_heads, const int32_t* seq_len,
+                                        int32_t max_seq_len, const uint8_t* cache_k, const int64_t* unit_offset_k,
+                                        const uint8_t* cache_v, const int64_t* unit_offset_v, int64_t n_param_sets,
+                                        const float* w_dec_k, const float* mean_rot_k, const uint8_t* widths_k,
+                                        const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
+                                        const uint8_t* widths_k_host, const uint8_t* widths_v_host,
+                                        float softmax_scale, void* out, int out_dtype, float* lse, void* workspace,
+                                        size_t workspace_bytes, int32_t* status_word, void* stream) {
+  return attention_impl(cfg, q, q_dtype, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k,
+                        cache_v, unit_offset_v, n_param_sets, w_dec_k, mean_rot_k, widths_k, w_dec_v, mean_rot_v,
+                        widths_v, widths_k_host, widths_v_host, softmax_scale, out, out_dtype, lse, workspace,
+                        workspace_bytes, status_word, stream, nullptr);
+}
+
+extern "C" int spectra_decode_step(const spectra_config* cfg, const void* q, int q_dtype, const void* new_k,
+                                   const void* new_v, int x_dtype, int32_t batch, int32_t n_kv_heads,
+                                   int32_t n_q_heads, const int32_t* seq_len, int32_t max_seq_len, uint8_t* cache_k,
+                                   const int64_t* unit_offset_k, uint8_t* cache_v, const int64_t* unit_offset_v,
+                                   int64_t n_param_sets, const float* w_enc_k, const float* w_dec_k,
+                                   const float* mean_rot_k, const uint8_t* widths_k, const float* w_enc_v,
+                                   const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
+                                   const uint8_t* widths_k_host, const uint8_t* widths_v_host, float softmax_scale,
+                                   void* out, int out_dtype, float* lse, void* workspace, size_t workspace_bytes,
+                                   int32_t* status_word, void* stream) {
+  if (!new_k || !new_v || !w_enc_k || !w_enc_v || !mean_rot_k || !mean_rot_v) return SPECTRA_INVALID_ARG;
+  if (x_dtype != SPECTRA_F32 && x_dtype != SPECTRA_BF16) return SPECTRA_INVALID_ARG;
+  const StepAppend app{new_k, new_v, x_dtype, w_enc_k, w_enc_v, cache_k, cache_v};
+  return attention_impl(cfg, q, q_dtype, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k,
+                        cache_v, unit_offset_v, n_param_sets, w_dec_k, mean_rot_k, widths_k, w_dec_v, mean_rot_v,
+                        widths_v, widths_k_host, widths_v_host, softmax_scale, out, out_dtype, lse, workspace,
+                        workspace_bytes, status_word, stream, &app);
 }
 
 extern "C" size_t spectra_tile_bytes(const spectra_config* cfg, const uint8_t* widths_host) {

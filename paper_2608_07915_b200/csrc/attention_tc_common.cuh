@@ -22,6 +22,7 @@
 // analytically (K: precomputed per head and group; V: an extra all-ones MMA row sum).
 #pragma once
 #include "attention_generic.cuh"
+#include "encode_append.cuh"
 
 namespace spectra {
 
@@ -155,12 +156,13 @@ __device__ inline int count_group0(const StripTable& T, int c, int lane) {
 
 constexpr int kPrepThreads = 512;
 
-__global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p, FastArgs f) {
+// The work of CTA `bid` of the prep grid (f.n_units unit CTAs, then one CTA for the prefix sums).
+__device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f, int bid) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   PrepSmem& S = *reinterpret_cast<PrepSmem*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int kWarps = kPrepThreads / 32;
-  if ((int)blockIdx.x == f.n_units) {
+  if (bid == f.n_units) {
     // ---- tile prefix sums over units and each worker warp's first unit
     const int n_units = f.n_units;
     const int per = (n_units + 127) / 128;
@@ -203,7 +205,7 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
     }
     return;
   }
-  const int vu = blockIdx.x;
+  const int vu = bid;
   const int u = vu / f.npass, h0 = kFastGqa * (vu - u * f.npass);   // cache unit, first query head of this pass
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
@@ -335,6 +337,22 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
     D.vchan[k] = (uint8_t)c;
     D.vcoef[k] = 16777216.f * (float)(1 << TV.shift[k]) / (float)((1 << TV.width[c]) - 1);
   }
+}
+
+__global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p, FastArgs f) {
+  attention_prep_body(p, f, blockIdx.x);
+}
+
+// First launch of a fused decode step: the prep grid, then one CTA per unit-side that appends the new token
+// (threads 0..127 of it; the K side first).  The main kernel that follows reads what both parts wrote.
+__global__ void __launch_bounds__(kPrepThreads) decode_step_front_kernel(AttnArgs p, FastArgs f, AppendArgs ak,
+                                                                         AppendArgs av, int n_cache_units) {
+  const int n_prep = f.n_units + 1;
+  if ((int)blockIdx.x < n_prep) { attention_prep_body(p, f, blockIdx.x); return; }
+  if (threadIdx.x >= 128) return;
+  const int i = blockIdx.x - n_prep;
+  if (i < n_cache_units) encode_append_body(ak, i);
+  else encode_append_body(av, i - n_cache_units);
 }
 
 }  // namespace spectra

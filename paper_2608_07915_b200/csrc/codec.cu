@@ -45,6 +45,8 @@ __device__ inline void tile_product(const float* __restrict__ a, const float* __
   }
 }
 
+__global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) { encode_append_body(p, blockIdx.x); }
+
 struct EncodeArgs {
   const void* x; int x_dtype; int flags; int side; int scale_group;
   int64_t n_param_sets; const int32_t* pos0; int32_t n_new; int64_t stride_unit, stride_token;
@@ -249,7 +251,7 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   if (n_new <= kAppendMaxTokens) {   // decode-step appends: one light CTA per unit-side
     AppendArgs ap{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
-                  w_enc, mean_rot, widths, cache, unit_offset, status_word};
+                  w_enc, mean_rot, widths, cache, unit_offset, status_word, nullptr, 1};
     encode_append_kernel<<<(unsigned)n_units, 128, 0, (cudaStream_t)stream>>>(ap);
     return launch_status();
   }

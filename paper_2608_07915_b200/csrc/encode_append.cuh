@@ -15,14 +15,15 @@ struct AppendArgs {
   int64_t n_param_sets; const int32_t* pos0; int32_t n_new; int64_t stride_unit, stride_token;
   const float* w_enc; const float* mean_rot; const uint8_t* widths;
   uint8_t* cache; const int64_t* unit_offset; int32_t* status;
+  const int32_t* seq_len; int n_kv;      // with pos0 == NULL: the token goes to position seq_len[u / n_kv] - 1
 };
 
-__global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
+// The work of one CTA (threads 0..127 of it) for unit-side u.
+__device__ inline void encode_append_body(const AppendArgs& p, int u) {
   __shared__ float xs[kAppendMaxTokens][kD];
   __shared__ float red_lo[4], red_hi[4];
   __shared__ int cls_cnt[4][4];          // [class][warp]: strips of the class owned by the warp's channels
   __shared__ int grp_act[kMaxGroups];
-  const int u = blockIdx.x;
   const int ps = (int)(u % p.n_param_sets);
   const int j = threadIdx.x, lane = j & 31, warp = j >> 5;
   const int gs = p.scale_group, n_groups = kD / gs;
@@ -60,7 +61,7 @@ __global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
   const int tile_bytes = payload + 512 * n_act;
 
   // ---- stage the new tokens
-  const int pos_first = p.pos0[u];
+  const int pos_first = p.pos0 ? p.pos0[u] : p.seq_len[u / p.n_kv] - 1;
   for (int idx = j; idx < p.n_new * kD; idx += 128) {
     const int t = idx / kD, i = idx - t * kD;
     xs[t][i] = load_as_float(p.x, p.x_dtype, (int64_t)u * p.stride_unit + (int64_t)t * p.stride_token + i);

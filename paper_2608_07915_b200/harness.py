@@ -123,15 +123,27 @@ class CodedModelCache:
                             v.m_rot, v.widths, 0.0, out, lse, self.workspace, self.status,
                             k.widths_host if self.tensor_path else None, v.widths_host if self.tensor_path else None)
 
-    def decode_step(self, q_all, new_k_all, new_v_all, out_all, on_attend=None):
+    def step_layer(self, layer, q, new_k, new_v, out, lse=None):
+        """The fused call: append one token per unit at seq_len - 1 (seq_len already advanced) and attend."""
+        k, v = self.side[layer]
+        sp.decode_step(self.cfg, q, new_k, new_v, self.batch, self.H, self.Hq, self.seq_len, self.cap_tokens, k.cache,
+                       k.unit_offset, v.cache, v.unit_offset, self.H, k.w_enc, k.w_dec, k.m_rot, k.widths, v.w_enc,
+                       v.w_dec, v.m_rot, v.widths, 0.0, out, lse, self.workspace, self.status,
+                       k.widths_host if self.tensor_path else None, v.widths_host if self.tensor_path else None)
+
+    def decode_step(self, q_all, new_k_all, new_v_all, out_all, on_attend=None, fused=True):
         """q_all [layers, batch, Hq, d]; new_*_all [layers, n_units, d]; out_all like q_all.  Appends one token
-        per sequence in every layer, then attends over the grown cache; advances the lengths at the end."""
+        per sequence in every layer, then attends over the grown cache; advances the lengths at the end.  With
+        fused=True a layer is one spectra_decode_step call, else spectra_encode (K, V) + spectra_decode_attention."""
         self.seq_len += 1
         for layer in range(self.layers):
-            self.append(layer, new_k_all[layer], new_v_all[layer])
             if on_attend:
                 on_attend(layer, 0)
-            self.attend(layer, q_all[layer], out_all[layer])
+            if fused:
+                self.step_layer(layer, q_all[layer], new_k_all[layer], new_v_all[layer], out_all[layer])
+            else:
+                self.append(layer, new_k_all[layer], new_v_all[layer])
+                self.attend(layer, q_all[layer], out_all[layer])
             if on_attend:
                 on_attend(layer, 1)
         self.pos0 += 1

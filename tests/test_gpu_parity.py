@@ -468,3 +468,37 @@ def test_tiny_whole_pipeline_on_gpu_agrees_with_whole_oracle(sp):
     err_ref = np.linalg.norm(ref[0] - dense) / np.linalg.norm(dense)
     assert err_gpu <= 1.5 * err_ref + 1e-3                     # same quality as the oracle's codec at 4x
     assert H.rel_err_per_vector(got, ref[0]) <= 0.05           # and close to it (bases differ in degenerate tails)
+
+
+@pytest.mark.parametrize("name,tensor_path", [("tiny", True), ("tiny", False)])
+def test_fused_decode_step_equals_separate_calls(sp, name, tensor_path):
+    """spectra_decode_step = spectra_encode (K), spectra_encode (V), spectra_decode_attention: same cache bytes, same
+    outputs (the separate calls are the ones the other tests compare with the oracle)."""
+    import dataclasses
+    from paper_2608_07915_b200 import harness
+    wl = dataclasses.replace(si.WORKLOADS[name], batch=2)
+    models = []
+    for fused in (True, False):
+        m = harness.CodedModelCache(wl, layers=1, batch=2, extra_tokens=256)
+        m.tensor_path = tensor_path
+        m.build()
+        models.append(m)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    outs = []
+    dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
+    steps = [(torch.randn((1, 2, wl.q_heads, 128), generator=gen, device="cuda").to(dt),
+              torch.randn((1, 2 * wl.kv_heads, 128), generator=gen, device="cuda").to(dt),
+              torch.randn((1, 2 * wl.kv_heads, 128), generator=gen, device="cuda").to(dt)) for _ in range(130)]
+    for m, fused in zip(models, (True, False)):
+        out = torch.zeros((1, 2, wl.q_heads, 128), dtype=torch.float32, device="cuda")
+        for q, nk, nv in steps:                      # crosses a tile boundary (130 appended tokens)
+            m.decode_step(q, nk, nv, out, fused=fused)
+        torch.cuda.synchronize()
+        assert int(m.status.item()) == 0
+        outs.append(out.clone())
+    for side in (0, 1):
+        assert torch.equal(models[0].side[0][side].cache, models[1].side[0][side].cache)
+    if tensor_path:
+        assert torch.equal(outs[0], outs[1])
+    else:   # the CUDA-core kernel sums with shared-memory float atomics: equal up to summation order
+        assert torch.allclose(outs[0], outs[1], rtol=1e-5, atol=1e-6)
