@@ -287,21 +287,26 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
     }
   }
   __syncthreads();
-  // B fragments.  Each class is walked as two runs, one per scale group: run 0 = strips [0, n_g0), run 1 = strips
-  // [n_g0 rounded down to a pair, n); a chunk is 16 consecutive strips of a run and contributes to that run's
-  // scale group only (rows of the other group, or past the end, are zero).  Column n = head (n >> 1), hi
-  // (n & 1 == 0) or lo half of the fp16 split.  Variant u carries the factor 2^-p_eff(u) of the unpacking.
-  int chunk0 = 0;
+  // B fragments.  A class is walked in chunks of 16 consecutive strips; the strips of scale group 0 come first, so
+  // at most one chunk per class holds strips of both groups: it gets two entries, one per group.  An entry
+  // contributes to its scale group only (rows of the other group, or past the end, are zero).  Entries are stored
+  // chunk-major, group-minor: the order the main kernel walks them.  Column n = head (n >> 1), hi (n & 1 == 0) or
+  // lo half of the fp16 split.  Variant u carries the factor 2^-p_eff(u) of the unpacking.
+  int entry0 = 0;
   for (int c = 0; c < 4; c++) {
     const int first = TK.class_first[c], n = TK.class_first[c + 1] - first;
     const int n_g0 = S.ng0[0][c];
-    const int s1 = n_g0 & ~1;
-    const int nch0 = (n_g0 + 15) / 16, nch1 = n > n_g0 ? (n - s1 + 15) / 16 : 0;
+    const int nch = (n + 15) / 16;
+    const int b0 = n_g0 / 16;                                      // first chunk that holds a strip of group 1
+    const bool both = n > n_g0 && (n_g0 & 15) != 0;                // chunk b0 holds strips of both groups
+    const int n_entries = nch + (both ? 1 : 0);
     const int w = 8 >> c;
-    for (int idx = tid; idx < (nch0 + nch1) * 4 * 32; idx += kPrepThreads) {
-      const int ch = idx >> 7, u4 = (idx >> 5) & 3, ln = idx & 31;
-      const int run = ch >= nch0 ? 1 : 0;
-      const int start = run ? s1 + 16 * (ch - nch0) : 16 * ch;
+    for (int idx = tid; idx < n_entries * 4 * 32; idx += kPrepThreads) {
+      const int en = idx >> 7, u4 = (idx >> 5) & 3, ln = idx & 31;
+      int ch, run;                                                 // chunk and scale group of entry en
+      if (both) { ch = en <= b0 ? en : en - 1; run = en <= b0 ? 0 : 1; }
+      else { ch = en; run = 16 * en < n_g0 ? 0 : 1; }
+      const int start = 16 * ch;
       const int gid = ln >> 2, tg = ln & 3, h = gid >> 1, part = gid & 1;
       const int pe = w == 8 ? 0 : (w == 4 ? 4 * (u4 & 1) : (w == 2 ? 2 * u4 : u4));
       const __half scale = __ushort_as_half((unsigned short)((15 - pe) << 10));
@@ -313,15 +318,15 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
         for (int e = 0; e < 2; e++) {
           const int strip = start + 2 * tg + 8 * half + e;
           uint16_t bits = 0;
-          if (strip < n && h < G && (TK.chan[first + strip] >= 64 ? 1 : 0) == run)
+          if (strip < n && h < G && (strip >= n_g0 ? 1 : 0) == run)
             bits = __half_as_ushort(__hmul(part ? S.blo[h][first + strip] : S.bhi[h][first + strip], scale));
           v |= (uint32_t)bits << (16 * e);
         }
         r[half] = v;
       }
-      if (chunk0 + ch < kKcMax) D.kB[chunk0 + ch][u4][ln] = make_uint2(r[0], r[1]);
+      if (entry0 + en < kKcMax) D.kB[entry0 + en][u4][ln] = make_uint2(r[0], r[1]);
     }
-    chunk0 += nch0 + nch1;
+    entry0 += n_entries;
   }
   if (tid >= 64 && tid < 68) D.kcls[tid - 64] = pack_cls(TK, tid - 64, S.ng0[0][tid - 64]);
   if (tid >= 96 && tid < 100) D.vcls[tid - 96] = pack_cls(TV, tid - 96, S.ng0[1][tid - 96]);

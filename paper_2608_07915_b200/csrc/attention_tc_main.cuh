@@ -84,13 +84,13 @@ __device__ __forceinline__ void ld_halfwords(const unsigned char* p, uint32_t (&
 }
 
 // Four MMAs of one chunk into one scale group's accumulators: MMA u takes tokens u (row gid) and u + 4 (row
-// gid + 8) of the pass, pair slots tig and tig + 4 as its k columns, and B variant u (scaled by 2^-p_eff(u)).
+// gid + 8) of the pass, pair slots tig and tig + 4 as its k columns, and B variant u (scaled by 2^-p_eff(u); rows
+// of strips that belong to the other scale group, or lie past the end of the class, are zero).
 template <int W>
-__device__ __forceinline__ void k_chunk(uint32_t (&wa)[Unpack<W>::NW], uint32_t (&wb)[Unpack<W>::NW], int hp,
+__device__ __forceinline__ void k_chunk(const uint32_t (&wa)[Unpack<W>::NW], const uint32_t (&wb)[Unpack<W>::NW],
                                         const uint2* __restrict__ kb, float (&acc)[4][4]) {
   using U = Unpack<W>;
   constexpr int NW = U::NW;
-  if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
   uint32_t was[NW], wbs[NW];
   U::shifted(wa, was);
   U::shifted(wb, wbs);
@@ -101,27 +101,32 @@ __device__ __forceinline__ void k_chunk(uint32_t (&wa)[Unpack<W>::NW], uint32_t 
   }
 }
 
-// One run of a class of the K tile for one half tile: strips [start, end) of the class (start even), all of one
-// scale group.  Chunks of 16 strips = 8 interleaved pairs; `n` = strips in the class (an odd n means that the last
-// strip is stored alone).
+// One class of the K tile for one half tile.  Chunks of 16 strips = 8 interleaved pairs, in storage order; the
+// strips of scale group 0 come first (n_g0 of them), so at most one chunk per class holds strips of both groups: it
+// is multiplied twice, once per group, each time with the other group's rows zeroed in B.  The B table is walked in
+// the same order (chunk-major, group-minor).  An odd last strip of the class is stored alone (half-words in order).
 template <int W>
-__device__ __forceinline__ void k_run(const unsigned char* cbase, int n, int start, int end, const uint2* __restrict__& kb,
-                                      int hp, int gid, int tig, float (&acc)[4][4]) {
+__device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls, const uint2* __restrict__& kb,
+                                        int hp, int gid, int tig, float (&acc)[2][4][4]) {
   using U = Unpack<W>;
   constexpr int NW = U::NW;
+  const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
+  if (n == 0) return;
+  const unsigned char* cbase = ktile + (cls >> 16) * 16;
   const int thr = 4 * W * gid + (W == 1 ? 0 : 4 * NW * hp);    // this thread's token block inside a pair
-  const unsigned char* pa = cbase + 16 * W * start + 32 * W * tig + thr;
-  int s = start;
+  const unsigned char* pa = cbase + 32 * W * tig + thr;
+  int s = 0;
 #pragma unroll 1
-  for (; s + 16 <= end && s + 16 <= (n & ~1); s += 16, pa += 256 * W, kb += 4 * 32) {   // complete chunks
+  for (; s + 16 <= (n & ~1); s += 16, pa += 256 * W) {          // complete chunks
     uint32_t wa[NW], wb[NW];
     ld_words<NW>(pa, wa);
     ld_words<NW>(pa + 128 * W, wb);
-    k_chunk<W>(wa, wb, hp, kb, acc);
+    if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
+    if (s < n_g0) { k_chunk<W>(wa, wb, kb, acc[0]); kb += 4 * 32; }
+    if (s + 16 > n_g0) { k_chunk<W>(wa, wb, kb, acc[1]); kb += 4 * 32; }
   }
-#pragma unroll 1
-  for (; s < end; s += 16, kb += 4 * 32) {                     // the tail of the run
-    const int avail = min(16, n - s);                          // strips stored from s on (B rows past `end` are zero)
+  if (s < n) {                                                  // the last, incomplete chunk of the class
+    const int avail = n - s;                                    // strips stored from s on (B rows past them are zero)
     const unsigned char* cb = cbase + 16 * W * s;
     uint32_t wa[NW], wb[NW];
     if (!(avail & 1)) {
@@ -142,20 +147,10 @@ __device__ __forceinline__ void k_run(const unsigned char* cbase, int n, int sta
         else if (2 * ps < avail) ld_halfwords<NW>(cb + 32 * W * ps + thr_h, wd);
       }
     }
-    k_chunk<W>(wa, wb, hp, kb, acc);
+    if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
+    if (s < n_g0) { k_chunk<W>(wa, wb, kb, acc[0]); kb += 4 * 32; }
+    if (n > n_g0) { k_chunk<W>(wa, wb, kb, acc[1]); kb += 4 * 32; }
   }
-}
-
-// One class of the K tile for one half tile: run 0 = the strips of scale group 0, run 1 = those of group 1
-// (starting at the pair that holds its first strip).
-template <int W>
-__device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls, const uint2* __restrict__& kb,
-                                        int hp, int gid, int tig, float (&acc)[2][4][4]) {
-  const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
-  if (n == 0) return;
-  const unsigned char* cbase = ktile + (cls >> 16) * 16;
-  if (n_g0 > 0) k_run<W>(cbase, n, 0, n_g0, kb, hp, gid, tig, acc[0]);
-  if (n > n_g0) k_run<W>(cbase, n, n_g0 & ~1, n, kb, hp, gid, tig, acc[1]);
 }
 
 // One class of the V tile for one half tile, at most Q blocks of 16 strips, accumulators acc_o[OFF .. OFF + Q).
