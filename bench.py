@@ -305,6 +305,23 @@ def run_ours(args, wl):
     ms_e2e = _max_over_ranks(e0.elapsed_time(e1) / steps, world)
     status = int(model.status.item())
 
+    # ---- reconstruction (spectra_decode) of one layer's K side, outside the timed decode steps: reported beside
+    # the prefill encode as a phase figure
+    ls0 = model.side[0][0]
+    n_tok = torch.full((U,), wl.n_tokens, dtype=torch.int32, device="cuda")
+    recon = torch.empty((U, wl.n_tokens, d), dtype=torch.bfloat16, device="cuda")
+    rec_ms = []
+    for _ in range(3):
+        r0, r1 = ev(), ev()
+        r0.record()
+        sp.decode(model.cfg, 0, ls0.cache, ls0.unit_offset, U, H, n_tok, wl.n_tokens, ls0.w_dec, ls0.m_rot,
+                  ls0.widths, recon, None, wl.n_tokens * d, d)
+        r1.record()
+        torch.cuda.synchronize()
+        rec_ms.append(r0.elapsed_time(r1))
+    del recon
+    reconstruct_ms = min(rec_ms[1:])
+
     bytes_call = model.attention_bytes(layer=0)
     achieved = bytes_call / (attn_ms_avg * 1e-3) / 1e9
     h2d = sum(t[0].numel() * t.element_size() for t in (q_host, nk_host, nv_host))
@@ -330,7 +347,9 @@ def run_ours(args, wl):
         "phases": {"setup_s": setup_s, "fit_alloc_ms_total": model.timings["fit_alloc_ms"],
                    "prefill_encode_ms_total": model.timings["prefill_encode_ms"],
                    "prefill_encode_tokens_per_s": L * 2 * U * wl.n_tokens / max(model.timings["prefill_encode_ms"],
-                                                                               1e-9) * 1e3 / 2},
+                                                                               1e-9) * 1e3 / 2,
+                   "reconstruct_ms_per_layer_side": reconstruct_ms,
+                   "reconstruct_unit_tokens_per_s": U * wl.n_tokens / max(reconstruct_ms, 1e-9) * 1e3},
         "status_word": status,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

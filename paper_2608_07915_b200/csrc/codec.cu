@@ -229,6 +229,151 @@ __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
   }
 }
 
+// ---- decode with the inverse rotation on the tensor cores
+// xhat = (yhat + m') W_dec with both operands as two-way bf16 splits (a = a1 + a2, W = W1 + W2) and the three
+// products a1 W1 + a1 W2 + a2 W1 in fp32 accumulators: relative error about 2^-16, far inside the 2e-3 bound of the
+// reconstruction.  One CTA of 256 threads walks several tiles of one unit-side and converts W_dec once.
+constexpr int kDecTiles = 4;
+
+struct DecodeTcSmem {
+  StripTable tab;
+  alignas(16) __nv_bfloat16 w[2][kD * kLdB16];     // the two parts of W_dec, [k][n]
+  alignas(16) __nv_bfloat16 a[2][kTile * kLdB16];  // the two parts of yhat + m', [token][k]
+  alignas(16) uint8_t codes[kTile * kLdC];
+  float bias[kD];
+};
+
+__global__ void __launch_bounds__(kTcThreads, 1) decode_tc_kernel(DecodeArgs p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  DecodeTcSmem& S = *reinterpret_cast<DecodeTcSmem*>(smem_raw);
+  const int u = blockIdx.y;
+  const int ps = (int)(u % p.n_param_sets);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+  const int wm = warp & 3, wn = warp >> 2;
+  const int n = p.n_tokens[u];
+  const int tile_first = blockIdx.x * kDecTiles;
+  if (tile_first * kTile >= n) return;
+
+  build_strip_table(S.tab, p.widths + (int64_t)ps * kD, p.scale_group);
+  const StripTable& T = S.tab;
+  const float* wsrc = p.w_dec + (int64_t)ps * kD * kD;
+  for (int idx = tid; idx < kD * kD; idx += kTcThreads) {
+    const int k = idx / kD, nn = idx - k * kD;
+    const float v = wsrc[idx];
+    const __nv_bfloat16 w1 = __float2bfloat16_rn(v);
+    S.w[0][k * kLdB16 + nn] = w1;
+    S.w[1][k * kLdB16 + nn] = __float2bfloat16_rn(v - __bfloat162float(w1));
+  }
+  if (tid < kD) S.bias[tid] = p.mean_rot[(int64_t)ps * kD + tid];
+
+  for (int tt = 0; tt < kDecTiles; tt++) {
+    const int tile = tile_first + tt;
+    const int tile_pos = tile * kTile;
+    if (tile_pos >= n) break;
+    const int n_here = min(n - tile_pos, kTile);
+    const uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
+    __syncthreads();                                   // the previous tile's MMAs have read S.a
+    // unpack: thread t < 128 gathers the fields of token slot t (the upper half of the CTA takes the upper strips)
+    const int t = tid & (kTile - 1), part = tid >> 7;
+    if (part == 0)
+      for (int j = 0; j < kD; j += 4) *reinterpret_cast<uint32_t*>(&S.codes[t * kLdC + j]) = 0u;
+    __syncthreads();
+    {
+      const int k0 = part ? T.n_strips / 2 : 0, k1 = part ? T.n_strips : T.n_strips / 2;
+      for (int k = k0; k < k1; k++) {
+        int bo, bit;
+        locate_field(T, p.side, k, t, bo, bit);
+        const int w = 8 >> strip_class(T, k);
+        const unsigned hw = *reinterpret_cast<const uint16_t*>(tile_ptr + bo);
+        const unsigned field = (hw >> bit) & ((1u << w) - 1u);
+        if (field) atomicOr(reinterpret_cast<unsigned*>(&S.codes[(t * kLdC + T.chan[k]) & ~3]),
+                            (field << T.shift[k]) << (8 * ((t * kLdC + T.chan[k]) & 3)));
+      }
+    }
+    __syncthreads();
+    // dequantise (same operation order as the CUDA-core kernel), add the rotated mean, split into two bf16 parts
+    {
+      const int64_t obase = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + t) * p.stride_token;
+      const int g0 = part * (T.n_groups / 2), g1 = part ? T.n_groups : max(T.n_groups / 2, 1);
+      for (int g = (T.n_groups == 1 ? 0 : g0); g < (T.n_groups == 1 ? (part ? 0 : 1) : g1); g++) {
+        float lo_f = 0.f, R_f = 0.f;
+        if (T.meta_off[g] >= 0) {
+          const uint16_t* m = reinterpret_cast<const uint16_t*>(tile_ptr + T.meta_off[g]) + t;
+          lo_f = __half2float(__ushort_as_half(m[0]));
+          R_f = __half2float(__ushort_as_half(m[kTile]));
+        }
+        for (int j = g * p.scale_group; j < (g + 1) * p.scale_group; j++) {
+          const int b = T.width[j];
+          float v = 0.f;
+          if (b) {
+            v = lo_f;
+            if (R_f != 0.f) {
+              const float step = __fdiv_rn(R_f, (float)((1 << b) - 1));
+              v = __fadd_rn(__fmul_rn((float)S.codes[t * kLdC + j], step), lo_f);
+            }
+          }
+          if (p.yhat_out && t < n_here) p.yhat_out[obase + j] = v;
+          const float a = t < n_here ? v + S.bias[j] : 0.f;
+          const __nv_bfloat16 a1 = __float2bfloat16_rn(a);
+          S.a[0][t * kLdB16 + j] = a1;
+          S.a[1][t * kLdB16 + j] = __float2bfloat16_rn(a - __bfloat162float(a1));
+        }
+      }
+    }
+    __syncthreads();
+    if (!p.out) continue;
+    // ---- xhat = a W_dec on the tensor cores: warp (wm, wn) owns tokens [32 wm, +32) and channels [64 wn, +64)
+    float acc[2][8][4];
+#pragma unroll
+    for (int mb = 0; mb < 2; mb++)
+#pragma unroll
+      for (int nb = 0; nb < 8; nb++)
+#pragma unroll
+        for (int e = 0; e < 4; e++) acc[mb][nb][e] = 0.f;
+#pragma unroll 1
+    for (int ks = 0; ks < kD / 16; ks++) {
+      uint32_t a1[2][4], a2[2][4];
+#pragma unroll
+      for (int mb = 0; mb < 2; mb++) {
+        const int off = (32 * wm + 16 * mb + (lane & 7) + ((lane >> 3) & 1) * 8) * kLdB16 + 16 * ks + (lane >> 4) * 8;
+        ldmatrix_x4(a1[mb], &S.a[0][off]);
+        ldmatrix_x4(a2[mb], &S.a[1][off]);
+      }
+#pragma unroll
+      for (int np = 0; np < 4; np++) {                 // two 8-channel blocks per ldmatrix
+        const int off = (16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8) * kLdB16 + 64 * wn + 16 * np + (lane >> 4) * 8;
+        uint32_t b1[4], b2[4];
+        ldmatrix_x4_trans(b1, &S.w[0][off]);
+        ldmatrix_x4_trans(b2, &S.w[1][off]);
+#pragma unroll
+        for (int mb = 0; mb < 2; mb++) {
+          mma_bf16(acc[mb][2 * np], a1[mb], b1[0], b1[1]);
+          mma_bf16(acc[mb][2 * np + 1], a1[mb], b1[2], b1[3]);
+          mma_bf16(acc[mb][2 * np], a1[mb], b2[0], b2[1]);
+          mma_bf16(acc[mb][2 * np + 1], a1[mb], b2[2], b2[3]);
+          mma_bf16(acc[mb][2 * np], a2[mb], b1[0], b1[1]);
+          mma_bf16(acc[mb][2 * np + 1], a2[mb], b1[2], b1[3]);
+        }
+      }
+    }
+    // ---- store: a thread holds channel pairs (2 tig, 2 tig + 1) of rows gid and gid + 8 of each 16-token block
+#pragma unroll
+    for (int mb = 0; mb < 2; mb++)
+#pragma unroll
+      for (int half = 0; half < 2; half++) {
+        const int tok = 32 * wm + 16 * mb + gid + 8 * half;
+        if (tok >= n_here) continue;
+        const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + tok) * p.stride_token + 64 * wn + 2 * tig;
+#pragma unroll
+        for (int nb = 0; nb < 8; nb++) {
+          store_from_float(p.out, p.out_dtype, o + 8 * nb, acc[mb][nb][2 * half]);
+          store_from_float(p.out, p.out_dtype, o + 8 * nb + 1, acc[mb][nb][2 * half + 1]);
+        }
+      }
+  }
+}
+
 }  // namespace spectra
 
 using namespace spectra;
@@ -295,6 +440,15 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
                out_dtype, yhat_out, stride_unit, stride_token};
+  if (out) {   // reconstruction: inverse rotation on the tensor cores
+    if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)sizeof(DecodeTcSmem)) != cudaSuccess)
+      return SPECTRA_CUDA_ERROR;
+    const unsigned tiles = (unsigned)((max_tokens + kTile - 1) / kTile);
+    dim3 grid_tc((tiles + kDecTiles - 1) / kDecTiles, (unsigned)n_units);
+    decode_tc_kernel<<<grid_tc, kTcThreads, sizeof(DecodeTcSmem), (cudaStream_t)stream>>>(a);
+    return launch_status();
+  }
   if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CodecSmem)) !=
       cudaSuccess)
     return SPECTRA_CUDA_ERROR;
