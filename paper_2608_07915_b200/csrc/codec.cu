@@ -136,6 +136,8 @@ __global__ void __launch_bounds__(128, 1) encode_kernel(EncodeArgs p) {
   // pack: one half-word of the payload at a time, in storage order
   uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
   const int payload = T.class_off[4];
+  if (slot_lo == 0 && slot_hi == kTile) pack_full_tile(T, p.side, S.codes, kLdC, tile_ptr, tid, blockDim.x);
+  else
   for (int off = 2 * tid; off < payload; off += 2 * blockDim.x) {
     int w, first;
     const int k = halfword_owner(T, p.side, off, w, first);

@@ -153,6 +153,50 @@ __device__ inline int halfword_owner(const StripTable& T, int side, int off, int
   return T.class_first[c] + cnt - 1;
 }
 
+// Packs the payload of a completely written tile (all 128 slots) from a shared-memory code array
+// (codes[t * ld + channel], one byte each), one 32-bit word per step, with shifts only.  Called by all `nthreads`
+// threads of the CTA that owns the tile; stores are coalesced 4-byte words in storage order.
+__device__ inline void pack_full_tile(const StripTable& T, int side, const uint8_t* __restrict__ codes, int ld,
+                                      uint8_t* __restrict__ tile_ptr, int tid, int nthreads) {
+#pragma unroll
+  for (int c = 0; c < 4; c++) {
+    const int w = 8 >> c, lw = 3 - c;                       // field width and its log2
+    const int per = 16 >> lw;                               // tokens per half-word
+    const int first = T.class_first[c], n = T.class_first[c + 1] - first;
+    if (n == 0) continue;
+    uint32_t* dst = reinterpret_cast<uint32_t*>(tile_ptr + T.class_off[c]);
+    const unsigned fmask = (1u << w) - 1u;
+    const int words = 4 * w * n;                            // 32-bit words of the class region
+    for (int W = tid; W < words; W += nthreads) {
+      int k_lo, k_hi, t_lo, t_hi;                           // strip and first token of the low / high half-word
+      if (side == SPECTRA_SIDE_V) {
+        const int i_in = W >> (2 + lw), q = W & (4 * w - 1);
+        const int a = q >> lw, m = q & (w - 1);
+        k_lo = k_hi = first + i_in;
+        t_lo = 32 * a + m * per; t_hi = t_lo + 16;
+      } else {
+        const int paired_words = 8 * w * (n >> 1);          // words of the interleaved pairs
+        if (W < paired_words) {
+          const int p = W >> (3 + lw), nn = W & (8 * w - 1);
+          k_lo = first + 2 * p; k_hi = k_lo + 1;
+          t_lo = t_hi = nn * per;
+        } else {                                            // the odd last strip: half-words in order
+          const int j = W - paired_words;
+          k_lo = k_hi = first + n - 1;
+          t_lo = 2 * j * per; t_hi = t_lo + per;
+        }
+      }
+      const int c_lo = T.chan[k_lo], s_lo = T.shift[k_lo], c_hi = T.chan[k_hi], s_hi = T.shift[k_hi];
+      unsigned word = 0;
+      for (int e = 0; e < per; e++) {
+        word |= (((unsigned)codes[(t_lo + e) * ld + c_lo] >> s_lo) & fmask) << (e * w);
+        word |= (((unsigned)codes[(t_hi + e) * ld + c_hi] >> s_hi) & fmask) << (16 + e * w);
+      }
+      dst[W] = word;
+    }
+  }
+}
+
 __device__ inline float load_as_float(const void* p, int dtype, int64_t idx) {
   if (dtype == SPECTRA_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx]);
   return reinterpret_cast<const float*>(p)[idx];
