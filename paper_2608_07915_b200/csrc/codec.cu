@@ -236,6 +236,7 @@ __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
 // products a1 W1 + a1 W2 + a2 W1 in fp32 accumulators: relative error about 2^-16, far inside the 2e-3 bound of the
 // reconstruction.  One CTA of 256 threads walks several tiles of one unit-side and converts W_dec once.
 constexpr int kDecTiles = 4;
+constexpr int kDecThreads = 256;
 
 struct DecodeTcSmem {
   StripTable tab;
@@ -245,7 +246,7 @@ struct DecodeTcSmem {
   float bias[kD];
 };
 
-__global__ void __launch_bounds__(kTcThreads, 1) decode_tc_kernel(DecodeArgs p) {
+__global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   DecodeTcSmem& S = *reinterpret_cast<DecodeTcSmem*>(smem_raw);
   const int u = blockIdx.y;
@@ -260,7 +261,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) decode_tc_kernel(DecodeArgs p) 
   build_strip_table(S.tab, p.widths + (int64_t)ps * kD, p.scale_group);
   const StripTable& T = S.tab;
   const float* wsrc = p.w_dec + (int64_t)ps * kD * kD;
-  for (int idx = tid; idx < kD * kD; idx += kTcThreads) {
+  for (int idx = tid; idx < kD * kD; idx += kDecThreads) {
     const int k = idx / kD, nn = idx - k * kD;
     const float v = wsrc[idx];
     const __nv_bfloat16 w1 = __float2bfloat16_rn(v);
@@ -448,7 +449,7 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
       return SPECTRA_CUDA_ERROR;
     const unsigned tiles = (unsigned)((max_tokens + kTile - 1) / kTile);
     dim3 grid_tc((tiles + kDecTiles - 1) / kDecTiles, (unsigned)n_units);
-    decode_tc_kernel<<<grid_tc, kTcThreads, sizeof(DecodeTcSmem), (cudaStream_t)stream>>>(a);
+    decode_tc_kernel<<<grid_tc, kDecThreads, sizeof(DecodeTcSmem), (cudaStream_t)stream>>>(a);
     return launch_status();
   }
   if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CodecSmem)) !=
