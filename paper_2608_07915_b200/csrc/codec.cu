@@ -277,24 +277,11 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p)
     const int n_here = min(n - tile_pos, kTile);
     const uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
     __syncthreads();                                   // the previous tile's MMAs have read S.a
-    // unpack: thread t < 128 gathers the fields of token slot t (the upper half of the CTA takes the upper strips)
+    // unpack: word by word into the code array
     const int t = tid & (kTile - 1), part = tid >> 7;
-    if (part == 0)
-      for (int j = 0; j < kD; j += 4) *reinterpret_cast<uint32_t*>(&S.codes[t * kLdC + j]) = 0u;
+    for (int i = tid; i < kTile * kLdC / 4; i += kDecThreads) reinterpret_cast<uint32_t*>(S.codes)[i] = 0u;
     __syncthreads();
-    {
-      const int k0 = part ? T.n_strips / 2 : 0, k1 = part ? T.n_strips : T.n_strips / 2;
-      for (int k = k0; k < k1; k++) {
-        int bo, bit;
-        locate_field(T, p.side, k, t, bo, bit);
-        const int w = 8 >> strip_class(T, k);
-        const unsigned hw = *reinterpret_cast<const uint16_t*>(tile_ptr + bo);
-        const unsigned field = (hw >> bit) & ((1u << w) - 1u);
-        if (field) atomicOr(reinterpret_cast<unsigned*>(&S.codes[(t * kLdC + T.chan[k]) & ~3]),
-                            (field << T.shift[k]) << (8 * ((t * kLdC + T.chan[k]) & 3)));
-      }
-    }
-    __syncthreads();
+    unpack_tile(T, p.side, tile_ptr, S.codes, kLdC, tid, kDecThreads);
     // dequantise (same operation order as the CUDA-core kernel), add the rotated mean, split into two bf16 parts
     {
       const int64_t obase = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + t) * p.stride_token;

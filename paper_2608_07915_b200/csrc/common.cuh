@@ -197,6 +197,51 @@ __device__ inline void pack_full_tile(const StripTable& T, int side, const uint8
   }
 }
 
+// Inverse of pack_full_tile: scatters the fields of a tile's payload into a shared-memory code array
+// (codes[t * ld + channel], zeroed by the caller), one 32-bit word per step and one class after the other, so that
+// a code byte is touched by one thread at a time.  Called by all `nthreads` threads; ends with a barrier.
+__device__ inline void unpack_tile(const StripTable& T, int side, const uint8_t* __restrict__ tile_ptr,
+                                   uint8_t* __restrict__ codes, int ld, int tid, int nthreads) {
+#pragma unroll
+  for (int c = 0; c < 4; c++) {
+    const int w = 8 >> c, lw = 3 - c;
+    const int per = 16 >> lw;
+    const int first = T.class_first[c], n = T.class_first[c + 1] - first;
+    if (n) {
+      const uint32_t* src = reinterpret_cast<const uint32_t*>(tile_ptr + T.class_off[c]);
+      const unsigned fmask = (1u << w) - 1u;
+      const int words = 4 * w * n;
+      for (int W = tid; W < words; W += nthreads) {
+        int k_lo, k_hi, t_lo, t_hi;
+        if (side == SPECTRA_SIDE_V) {
+          const int i_in = W >> (2 + lw), q = W & (4 * w - 1);
+          const int a = q >> lw, m = q & (w - 1);
+          k_lo = k_hi = first + i_in;
+          t_lo = 32 * a + m * per; t_hi = t_lo + 16;
+        } else {
+          const int paired_words = 8 * w * (n >> 1);
+          if (W < paired_words) {
+            const int p = W >> (3 + lw), nn = W & (8 * w - 1);
+            k_lo = first + 2 * p; k_hi = k_lo + 1;
+            t_lo = t_hi = nn * per;
+          } else {
+            const int j = W - paired_words;
+            k_lo = k_hi = first + n - 1;
+            t_lo = 2 * j * per; t_hi = t_lo + per;
+          }
+        }
+        const int c_lo = T.chan[k_lo], s_lo = T.shift[k_lo], c_hi = T.chan[k_hi], s_hi = T.shift[k_hi];
+        const unsigned word = src[W];
+        for (int e = 0; e < per; e++) {
+          codes[(t_lo + e) * ld + c_lo] |= (uint8_t)(((word >> (e * w)) & fmask) << s_lo);
+          codes[(t_hi + e) * ld + c_hi] |= (uint8_t)(((word >> (16 + e * w)) & fmask) << s_hi);
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+
 __device__ inline float load_as_float(const void* p, int dtype, int64_t idx) {
   if (dtype == SPECTRA_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx]);
   return reinterpret_cast<const float*>(p)[idx];
