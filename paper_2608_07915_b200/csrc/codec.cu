@@ -234,9 +234,9 @@ __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
 // ---- decode with the inverse rotation on the tensor cores
 // xhat = (yhat + m') W_dec with both operands as two-way bf16 splits (a = a1 + a2, W = W1 + W2) and the three
 // products a1 W1 + a1 W2 + a2 W1 in fp32 accumulators: relative error about 2^-16, far inside the 2e-3 bound of the
-// reconstruction.  One CTA of 256 threads walks several tiles of one unit-side and converts W_dec once.
+// reconstruction.  One CTA of 512 threads walks several tiles of one unit-side and converts W_dec once.
 constexpr int kDecTiles = 4;
-constexpr int kDecThreads = 256;
+constexpr int kDecThreads = 512;
 
 struct DecodeTcSmem {
   StripTable tab;
@@ -278,50 +278,54 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p)
     const uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
     __syncthreads();                                   // the previous tile's MMAs have read S.a
     // unpack: word by word into the code array
-    const int t = tid & (kTile - 1), part = tid >> 7;
+    const int t = tid & (kTile - 1);
     for (int i = tid; i < kTile * kLdC / 4; i += kDecThreads) reinterpret_cast<uint32_t*>(S.codes)[i] = 0u;
     __syncthreads();
     unpack_tile(T, p.side, tile_ptr, S.codes, kLdC, tid, kDecThreads);
-    // dequantise (same operation order as the CUDA-core kernel), add the rotated mean, split into two bf16 parts
+    // dequantise (same operation order as the CUDA-core kernel), add the rotated mean, split into two bf16 parts:
+    // thread (token t, quarter qd) takes channels [32 qd, 32 qd + 32)
     {
+      const int qd = tid >> 7;
       const int64_t obase = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + t) * p.stride_token;
-      const int g0 = part * (T.n_groups / 2), g1 = part ? T.n_groups : max(T.n_groups / 2, 1);
-      for (int g = (T.n_groups == 1 ? 0 : g0); g < (T.n_groups == 1 ? (part ? 0 : 1) : g1); g++) {
-        float lo_f = 0.f, R_f = 0.f;
-        if (T.meta_off[g] >= 0) {
-          const uint16_t* m = reinterpret_cast<const uint16_t*>(tile_ptr + T.meta_off[g]) + t;
-          lo_f = __half2float(__ushort_as_half(m[0]));
-          R_f = __half2float(__ushort_as_half(m[kTile]));
-        }
-        for (int j = g * p.scale_group; j < (g + 1) * p.scale_group; j++) {
-          const int b = T.width[j];
-          float v = 0.f;
-          if (b) {
-            v = lo_f;
-            if (R_f != 0.f) {
-              const float step = __fdiv_rn(R_f, (float)((1 << b) - 1));
-              v = __fadd_rn(__fmul_rn((float)S.codes[t * kLdC + j], step), lo_f);
-            }
+      float lo_f = 0.f, R_f = 0.f;
+      int g_cur = -1;
+      for (int j = 32 * qd; j < 32 * qd + 32; j++) {
+        const int g = j / p.scale_group;
+        if (g != g_cur) {
+          g_cur = g; lo_f = 0.f; R_f = 0.f;
+          if (T.meta_off[g] >= 0) {
+            const uint16_t* m = reinterpret_cast<const uint16_t*>(tile_ptr + T.meta_off[g]) + t;
+            lo_f = __half2float(__ushort_as_half(m[0]));
+            R_f = __half2float(__ushort_as_half(m[kTile]));
           }
-          if (p.yhat_out && t < n_here) p.yhat_out[obase + j] = v;
-          const float a = t < n_here ? v + S.bias[j] : 0.f;
-          const __nv_bfloat16 a1 = __float2bfloat16_rn(a);
-          S.a[0][t * kLdB16 + j] = a1;
-          S.a[1][t * kLdB16 + j] = __float2bfloat16_rn(a - __bfloat162float(a1));
         }
+        const int b = T.width[j];
+        float v = 0.f;
+        if (b) {
+          v = lo_f;
+          if (R_f != 0.f) {
+            const float step = __fdiv_rn(R_f, (float)((1 << b) - 1));
+            v = __fadd_rn(__fmul_rn((float)S.codes[t * kLdC + j], step), lo_f);
+          }
+        }
+        if (p.yhat_out && t < n_here) p.yhat_out[obase + j] = v;
+        const float a = t < n_here ? v + S.bias[j] : 0.f;
+        const __nv_bfloat16 a1 = __float2bfloat16_rn(a);
+        S.a[0][t * kLdB16 + j] = a1;
+        S.a[1][t * kLdB16 + j] = __float2bfloat16_rn(a - __bfloat162float(a1));
       }
     }
     __syncthreads();
     if (!p.out) continue;
-    // ---- xhat = a W_dec on the tensor cores: warp (wm, wn) owns tokens [32 wm, +32) and channels [64 wn, +64)
-    float acc[2][8][4];
+    // ---- xhat = a W_dec on the tensor cores: warp (wm, wn) owns tokens [32 wm, +32) and channels [32 wn, +32)
+    float acc[2][4][4];
 #pragma unroll
     for (int mb = 0; mb < 2; mb++)
 #pragma unroll
-      for (int nb = 0; nb < 8; nb++)
+      for (int nb = 0; nb < 4; nb++)
 #pragma unroll
         for (int e = 0; e < 4; e++) acc[mb][nb][e] = 0.f;
-#pragma unroll 1
+#pragma unroll 2
     for (int ks = 0; ks < kD / 16; ks++) {
       uint32_t a1[2][4], a2[2][4];
 #pragma unroll
@@ -331,8 +335,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p)
         ldmatrix_x4(a2[mb], &S.a[1][off]);
       }
 #pragma unroll
-      for (int np = 0; np < 4; np++) {                 // two 8-channel blocks per ldmatrix
-        const int off = (16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8) * kLdB16 + 64 * wn + 16 * np + (lane >> 4) * 8;
+      for (int np = 0; np < 2; np++) {                 // two 8-channel blocks per ldmatrix
+        const int off = (16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8) * kLdB16 + 32 * wn + 16 * np + (lane >> 4) * 8;
         uint32_t b1[4], b2[4];
         ldmatrix_x4_trans(b1, &S.w[0][off]);
         ldmatrix_x4_trans(b2, &S.w[1][off]);
@@ -347,18 +351,25 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p)
         }
       }
     }
-    // ---- store: a thread holds channel pairs (2 tig, 2 tig + 1) of rows gid and gid + 8 of each 16-token block
+    // ---- store: a thread holds the channel pair (2 tig, 2 tig + 1) of rows gid and gid + 8 of each 16-token block
 #pragma unroll
     for (int mb = 0; mb < 2; mb++)
 #pragma unroll
       for (int half = 0; half < 2; half++) {
         const int tok = 32 * wm + 16 * mb + gid + 8 * half;
         if (tok >= n_here) continue;
-        const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + tok) * p.stride_token + 64 * wn + 2 * tig;
+        const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + tok) * p.stride_token + 32 * wn + 2 * tig;
+        // the pair goes out as one 4-byte (bf16) or 8-byte (fp32) store when its address allows it
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out) + (uintptr_t)o * (p.out_dtype == SPECTRA_BF16 ? 2 : 4);
+        const bool pair_ok = (addr & (p.out_dtype == SPECTRA_BF16 ? 3 : 7)) == 0;
 #pragma unroll
-        for (int nb = 0; nb < 8; nb++) {
-          store_from_float(p.out, p.out_dtype, o + 8 * nb, acc[mb][nb][2 * half]);
-          store_from_float(p.out, p.out_dtype, o + 8 * nb + 1, acc[mb][nb][2 * half + 1]);
+        for (int nb = 0; nb < 4; nb++) {
+          const float v0 = acc[mb][nb][2 * half], v1 = acc[mb][nb][2 * half + 1];
+          if (pair_ok && p.out_dtype == SPECTRA_BF16)
+            *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(p.out) + o + 8 * nb) = __floats2bfloat162_rn(v0, v1);
+          else if (pair_ok)
+            *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.out) + o + 8 * nb) = make_float2(v0, v1);
+          else { store_from_float(p.out, p.out_dtype, o + 8 * nb, v0); store_from_float(p.out, p.out_dtype, o + 8 * nb + 1, v1); }
         }
       }
   }
