@@ -278,41 +278,36 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p)
     const uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
     __syncthreads();                                   // the previous tile's MMAs have read S.a
     // unpack: word by word into the code array
-    const int t = tid & (kTile - 1);
     for (int i = tid; i < kTile * kLdC / 4; i += kDecThreads) reinterpret_cast<uint32_t*>(S.codes)[i] = 0u;
     __syncthreads();
     unpack_tile(T, p.side, tile_ptr, S.codes, kLdC, tid, kDecThreads);
     // dequantise (same operation order as the CUDA-core kernel), add the rotated mean, split into two bf16 parts:
-    // thread (token t, quarter qd) takes channels [32 qd, 32 qd + 32)
+    // thread (channel j, token quarter tq) walks tokens [32 tq, 32 tq + 32); the lanes of a warp share the token, so
+    // its metadata is one broadcast load and the stores of a step are contiguous
     {
-      const int qd = tid >> 7;
-      const int64_t obase = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + t) * p.stride_token;
-      float lo_f = 0.f, R_f = 0.f;
-      int g_cur = -1;
-      for (int j = 32 * qd; j < 32 * qd + 32; j++) {
-        const int g = j / p.scale_group;
-        if (g != g_cur) {
-          g_cur = g; lo_f = 0.f; R_f = 0.f;
-          if (T.meta_off[g] >= 0) {
-            const uint16_t* m = reinterpret_cast<const uint16_t*>(tile_ptr + T.meta_off[g]) + t;
-            lo_f = __half2float(__ushort_as_half(m[0]));
-            R_f = __half2float(__ushort_as_half(m[kTile]));
-          }
+      const int j = tid & (kD - 1), tq = tid >> 7;
+      const int b = T.width[j];
+      const int mo = T.meta_off[j / p.scale_group];
+      const float L = (float)((1 << b) - 1), bias = S.bias[j];
+      for (int tk = 32 * tq; tk < 32 * tq + 32; tk++) {
+        float lo_f = 0.f, R_f = 0.f;
+        if (mo >= 0) {
+          const uint16_t* m = reinterpret_cast<const uint16_t*>(tile_ptr + mo) + tk;
+          lo_f = __half2float(__ushort_as_half(m[0]));
+          R_f = __half2float(__ushort_as_half(m[kTile]));
         }
-        const int b = T.width[j];
         float v = 0.f;
         if (b) {
           v = lo_f;
-          if (R_f != 0.f) {
-            const float step = __fdiv_rn(R_f, (float)((1 << b) - 1));
-            v = __fadd_rn(__fmul_rn((float)S.codes[t * kLdC + j], step), lo_f);
-          }
+          if (R_f != 0.f) v = __fadd_rn(__fmul_rn((float)S.codes[tk * kLdC + j], __fdiv_rn(R_f, L)), lo_f);
         }
-        if (p.yhat_out && t < n_here) p.yhat_out[obase + j] = v;
-        const float a = t < n_here ? v + S.bias[j] : 0.f;
+        const bool live = tk < n_here;
+        if (p.yhat_out && live)
+          p.yhat_out[(int64_t)u * p.stride_unit + (int64_t)(tile_pos + tk) * p.stride_token + j] = v;
+        const float a = live ? v + bias : 0.f;
         const __nv_bfloat16 a1 = __float2bfloat16_rn(a);
-        S.a[0][t * kLdB16 + j] = a1;
-        S.a[1][t * kLdB16 + j] = __float2bfloat16_rn(a - __bfloat162float(a1));
+        S.a[0][tk * kLdB16 + j] = a1;
+        S.a[1][tk * kLdB16 + j] = __float2bfloat16_rn(a - __bfloat162float(a1));
       }
     }
     __syncthreads();
