@@ -101,6 +101,25 @@ __device__ __forceinline__ void k_chunk(const uint32_t (&wa)[Unpack<W>::NW], con
   }
 }
 
+// The chunk that holds strips of both scale groups: the A fragments are unpacked once and multiplied with both
+// groups' B entries (consecutive in the table).
+template <int W>
+__device__ __forceinline__ void k_chunk_both(const uint32_t (&wa)[Unpack<W>::NW], const uint32_t (&wb)[Unpack<W>::NW],
+                                             const uint2* __restrict__ kb, float (&acc)[2][4][4]) {
+  using U = Unpack<W>;
+  constexpr int NW = U::NW;
+  uint32_t was[NW], wbs[NW];
+  U::shifted(wa, was);
+  U::shifted(wb, wbs);
+#pragma unroll
+  for (int u = 0; u < 4; u++) {
+    const uint2 b0 = __ldg(kb + u * 32), b1 = __ldg(kb + (4 + u) * 32);
+    const uint32_t a0 = U::get(wa, was, u), a1 = U::get(wa, was, u + 4), a2 = U::get(wb, wbs, u), a3 = U::get(wb, wbs, u + 4);
+    mma16816(acc[0][u], a0, a1, a2, a3, b0.x, b0.y);
+    mma16816(acc[1][u], a0, a1, a2, a3, b1.x, b1.y);
+  }
+}
+
 // One class of the K tile for one half tile.  Chunks of 16 strips = 8 interleaved pairs, in storage order; the
 // strips of scale group 0 come first (n_g0 of them), so at most one chunk per class holds strips of both groups: it
 // is multiplied twice, once per group, each time with the other group's rows zeroed in B.  The B table is walked in
@@ -122,8 +141,9 @@ __device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls
     ld_words<NW>(pa, wa);
     ld_words<NW>(pa + 128 * W, wb);
     if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-    if (s < n_g0) { k_chunk<W>(wa, wb, kb, acc[0]); kb += 4 * 32; }
-    if (s + 16 > n_g0) { k_chunk<W>(wa, wb, kb, acc[1]); kb += 4 * 32; }
+    if (s + 16 <= n_g0) { k_chunk<W>(wa, wb, kb, acc[0]); kb += 4 * 32; }
+    else if (s >= n_g0) { k_chunk<W>(wa, wb, kb, acc[1]); kb += 4 * 32; }
+    else { k_chunk_both<W>(wa, wb, kb, acc); kb += 8 * 32; }
   }
   if (s < n) {                                                  // the last, incomplete chunk of the class
     const int avail = n - s;                                    // strips stored from s on (B rows past them are zero)
@@ -148,8 +168,9 @@ __device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls
       }
     }
     if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-    if (s < n_g0) { k_chunk<W>(wa, wb, kb, acc[0]); kb += 4 * 32; }
-    if (n > n_g0) { k_chunk<W>(wa, wb, kb, acc[1]); kb += 4 * 32; }
+    if (n <= n_g0) { k_chunk<W>(wa, wb, kb, acc[0]); kb += 4 * 32; }
+    else if (s >= n_g0) { k_chunk<W>(wa, wb, kb, acc[1]); kb += 4 * 32; }
+    else { k_chunk_both<W>(wa, wb, kb, acc); kb += 8 * 32; }
   }
 }
 
