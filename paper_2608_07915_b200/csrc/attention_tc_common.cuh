@@ -1,9 +1,11 @@
-// Fused coded-cache decode attention for GQA groups of up to 4 query heads and scale_group 64.
+// Fused coded-cache decode attention on the tensor cores (mma.sync), scale_group 64; a unit of this path is a
+// (sequence, kv-head, pass) triple, a pass being up to 4 query heads of the GQA group.
 //
 // Three kernels per call:
 //   prep    (one CTA per unit)  folds W_dec,K and the softmax scale into the query (q'), turns it into
 //           tensor-core B fragments per 16-strip chunk of the K tile, and lays out the per-unit descriptor;
-//           one extra CTA builds the tile prefix sums and each warp's starting unit.
+//           one extra CTA builds the tile prefix sums and each warp's starting unit.  In a fused decode step the
+//           same launch also carries one CTA per unit-side that appends the new token.
 //   main    persistent, one warp = one worker.  The (unit, tile) space is flattened and cut into equal
 //           contiguous ranges, one per warp.  A warp streams its K and V tiles into its own shared-memory
 //           ring with 1-D bulk copies (cp.async.bulk + mbarrier), and per 64-token half tile
@@ -14,12 +16,11 @@
 //             - unpacks V codes into A fragments (rows = strips, k = tokens) and accumulates the output in the
 //               rotated value space in registers.
 //           At the end of a unit the warp writes one partial record (max, sum, accumulators per V strip).
-//   combine (one CTA per unit)  merges the records (log-sum-exp), folds strips back into channels, adds the
-//           rotated mean and lifts the result once with W_dec,V.
+//   combine (one CTA per unit and head)  merges the records (log-sum-exp), folds strips back into channels, adds
+//           the rotated mean and lifts the result once with W_dec,V.
 //
-// Codes enter the MMA as fp16 numbers 2^w + code, built with one shift and one logic op per pair: the field is
-// moved to the top of the fp16 mantissa and OR-ed with the exponent of 2^w.  The constant 2^w is removed
-// analytically (K: precomputed per head and group; V: an extra all-ones MMA row sum).
+// Codes enter the MMA as fp16 subnormals: a field masked in place inside its 16-bit half is code * 2^(p - 24)
+// (p = its bit position), which the tensor core multiplies exactly; the power of two is folded into the B operand.
 #pragma once
 #include "attention_generic.cuh"
 #include "encode_append.cuh"
@@ -27,7 +28,7 @@
 namespace spectra {
 
 constexpr int kFastGqa = 4;
-constexpr int kKcMax = 32;       // upper bound of 16-strip chunks in a K tile (two runs per class)
+constexpr int kKcMax = 32;       // upper bound of B-table entries of a K tile (chunks of 16 strips, one doubled per class)
 constexpr int kFastWarps = 4;    // warps per CTA of the main kernel
 constexpr int kRecHead = 4;      // floats of a record's per-head header: m, l, plo0, plo1
 constexpr float kLog2e = 1.4426950408889634f;
@@ -39,7 +40,6 @@ struct alignas(16) UnitDesc {
   uint32_t vfirst[4];           // index of the first V strip of each class
   int32_t n_vstrips, pad0;
   float kscale[4];              // 2^-e_h
-  float kcorr[4][2];            // sum_k 2^w_k (B_hi + B_lo) per head and scale group
   float qlo[4][2];              // sum of q' over the active channels of a scale group
   float qconst[4];              // q' . m'_K (natural-log units)
   uint8_t vchan[kMaxStrips];    // channel of V strip k
@@ -258,16 +258,12 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
     if (mx > 0.f && isfinite(mx)) { int ex; frexpf(mx, &ex); e = 10 - ex; }
     e = max(-100, min(100, e));
     if (lane == 0) { S.escale[h] = e; D.kscale[h] = ldexpf(1.f, 24 - e); }
-    float corr0 = 0.f, corr1 = 0.f;
     for (int k = lane; k < nk; k += 32) {
       const int c = TK.chan[k];
       const float v = ldexpf(S.qrot[h][c] * (float)(1 << TK.shift[k]) / (float)((1 << TK.width[c]) - 1), e);
       const __half hi = __float2half_rn(v);
       const __half lo = __float2half_rn(v - __half2float(hi));
       S.bhi[h][k] = hi; S.blo[h][k] = lo;
-      const float off = (float)(1 << (8 >> strip_class(TK, k)));    // 2^w
-      const float t = off * (__half2float(hi) + __half2float(lo));
-      if (c < 64) corr0 += t; else corr1 += t;
     }
     float q0 = 0.f, q1 = 0.f, qc = 0.f;
     for (int j = lane; j < kD; j += 32) {
@@ -277,12 +273,11 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
     }
 #pragma unroll
     for (int s = 16; s; s >>= 1) {
-      corr0 += __shfl_xor_sync(0xffffffffu, corr0, s); corr1 += __shfl_xor_sync(0xffffffffu, corr1, s);
       q0 += __shfl_xor_sync(0xffffffffu, q0, s); q1 += __shfl_xor_sync(0xffffffffu, q1, s);
       qc += __shfl_xor_sync(0xffffffffu, qc, s);
     }
     if (lane == 0) {
-      D.kcorr[h][0] = corr0; D.kcorr[h][1] = corr1; D.qlo[h][0] = q0; D.qlo[h][1] = q1;
+      D.qlo[h][0] = q0; D.qlo[h][1] = q1;
       D.qconst[h] = qc / kLog2e;
     }
   }
