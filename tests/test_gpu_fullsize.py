@@ -5,7 +5,9 @@ Both sides get the same transforms and widths (fitted by the oracle from the sam
 every unit of the layer, appends one token per sequence and attends; the oracle does the same for the sampled
 (sequence, kv-head) units from the raw vectors alone.  Checked: code mismatches of the encode (rare +-1 ties
 only), and the attention output of the decode step on the same codes (the sampled units attend over the oracle's
-bytes; 2e-3, max |diff| / max |oracle| per vector).
+bytes; 2e-3, max |diff| / max |oracle| per vector).  A second step then goes through the fused call the benchmark
+times (spectra_decode_step): the token it appended is compared code by code with the oracle's encode, and its
+output with the oracle's attention over the very bytes the GPU holds after the step.
 """
 import dataclasses
 
@@ -113,3 +115,39 @@ def test_full_context_decode_step_matches_oracle(case):
                                     pk.widths, pv.w_dec, pv.m_rot, pv.widths, 64, 1.0 / np.sqrt(128.0))
         # bf16 queries on the GPU side are exactly the fp32 values the oracle used
         assert H.rel_err_per_vector(got[s, h], ref[0]) <= TOL, (case, s, h)
+    # ---- a second step through the fused call (the one bench.py times)
+    q2 = torch.randn((batch, wl.q_heads, d), generator=gen, device="cuda").to(torch.bfloat16)
+    nk2 = torch.randn((batch * Hk, d), generator=gen, device="cuda").to(torch.bfloat16)
+    nv2 = torch.randn((batch * Hk, d), generator=gen, device="cuda").to(torch.bfloat16)
+    out2 = torch.zeros((batch, wl.q_heads, d), dtype=torch.float32, device="cuda")
+    model.pos0 += 1
+    model.seq_len += 1
+    model.step_layer(0, q2, nk2, nv2, out2)
+    torch.cuda.synchronize()
+    assert int(model.status.item()) == 0
+    got2 = out2.cpu().numpy().reshape(batch, Hk, G, d)
+    qh2 = q2.float().cpu().numpy().reshape(batch, Hk, G, d).astype(np.float64)
+    new2 = {si.SIDE_K: nk2.float().cpu().numpy(), si.SIDE_V: nv2.float().cpu().numpy()}
+    n2 = N + 2
+    n_tiles2 = (n2 + 127) // 128
+    for (s, h) in sampled:
+        u = s * Hk + h
+        held = {}
+        for side in (si.SIDE_K, si.SIDE_V):
+            pr, tb, _ = oracle_caches[(s, h)][side]
+            ls = model.side[0][side]
+            a = int(ls.unit_offset_host[u])
+            g = ls.cache[a:a + n_tiles2 * tb].cpu().numpy()
+            # the appended token (position N + 1): the oracle encodes the same vector; ties differ by one level at most
+            one = np.zeros(tb, np.uint8)
+            slot = (N + 1) % 128
+            assert H.oracle_encode(pr, side, new2[side][u][None, None], [slot], one, np.zeros(1, np.int64)) == 0
+            cr, lr, rr = oc.unpack_token(one, pr.widths[0], 64, side, slot)
+            tile = (N + 1) // 128
+            cg, lg, rg = oc.unpack_token(g[tile * tb:(tile + 1) * tb], pr.widths[0], 64, side, slot)
+            assert np.abs(cr.astype(np.int64) - cg.astype(np.int64)).max() <= 1
+            held[side] = (pr, tb, g)
+        (pk, tbk, ck), (pv, tbv, cv) = held[si.SIDE_K], held[si.SIDE_V]
+        ref, _ = oc.attention_units("B", qh2[s, h][None], [n2], ck, [0], [tbk], cv, [0], [tbv], pk.w_dec, pk.m_rot,
+                                    pk.widths, pv.w_dec, pv.m_rot, pv.widths, 64, 1.0 / np.sqrt(128.0))
+        assert H.rel_err_per_vector(got2[s, h], ref[0]) <= TOL, (case, "fused", s, h)
