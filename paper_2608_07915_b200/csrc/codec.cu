@@ -4,6 +4,7 @@
 #include "common.cuh"
 #include "encode_append.cuh"
 #include "encode_tc.cuh"
+#include "encode_umma.cuh"
 
 namespace spectra {
 
@@ -401,12 +402,14 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
     // bf16 bulk encode: rotation on the tensor cores
     EncodeTcArgs ta{reinterpret_cast<const __nv_bfloat16*>(x), side, n_param_sets, pos0, n_new, stride_unit,
                     stride_token, w_enc, mean_rot, widths, cache, unit_offset, status_word};
-    if (cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)sizeof(EncodeTcSmem)) != cudaSuccess)
+    // rotation on the 5th-generation tensor cores (accumulator tile in tensor memory)
+    const size_t um_smem = sizeof(EncodeUmmaSmem) + 128;
+    if (cudaFuncSetAttribute(encode_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)um_smem) !=
+        cudaSuccess)
       return SPECTRA_CUDA_ERROR;
     const unsigned tiles = (unsigned)((n_new + 2 * kTile - 2) / kTile);
-    dim3 grid((tiles + kTcTilesPerCta - 1) / kTcTilesPerCta, (unsigned)n_units);
-    encode_tc_kernel<<<grid, kTcThreads, sizeof(EncodeTcSmem), (cudaStream_t)stream>>>(ta);
+    dim3 grid((tiles + kUmTilesPerCta - 1) / kUmTilesPerCta, (unsigned)n_units);
+    encode_umma_kernel<<<grid, kUmThreads, um_smem, (cudaStream_t)stream>>>(ta);
     return launch_status();
   }
   EncodeArgs a{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
