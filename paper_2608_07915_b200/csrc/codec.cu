@@ -232,29 +232,32 @@ __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
   }
 }
 
-// ---- decode with the inverse rotation on the tensor cores
+// ---- decode with the inverse rotation on the 5th-generation tensor cores (tcgen05)
 // xhat = (yhat + m') W_dec with both operands as two-way bf16 splits (a = a1 + a2, W = W1 + W2) and the three
-// products a1 W1 + a1 W2 + a2 W1 in fp32 accumulators: relative error about 2^-16, far inside the 2e-3 bound of the
-// reconstruction.  One CTA of 512 threads walks several tiles of one unit-side and converts W_dec once.
+// products a1 W1 + a1 W2 + a2 W1 accumulated in fp32 in tensor memory: relative error about 2^-16, far inside the
+// 2e-3 bound of the reconstruction.  One CTA of 512 threads walks several tiles of one unit-side and converts W_dec
+// once.  Operand layouts in shared memory as in encode_umma.cuh (a: K-major, W: MN-major core matrices).
 constexpr int kDecTiles = 4;
 constexpr int kDecThreads = 512;
 
 struct DecodeTcSmem {
   StripTable tab;
-  alignas(16) __nv_bfloat16 w[2][kD * kLdB16];     // the two parts of W_dec, [k][n]
-  alignas(16) __nv_bfloat16 a[2][kTile * kLdB16];  // the two parts of yhat + m', [token][k]
+  alignas(128) uint8_t w[2][kD * kD * 2];          // the two bf16 parts of W_dec, MN-major core layout
+  alignas(128) uint8_t a[2][kTile * kD * 2];       // the two bf16 parts of yhat + m', K-major core layout
   alignas(16) uint8_t codes[kTile * kLdC];
   float bias[kD];
+  alignas(8) uint64_t mma_done;
+  uint32_t tmem_base;
 };
 
 __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  DecodeTcSmem& S = *reinterpret_cast<DecodeTcSmem*>(smem_raw);
+  unsigned char* smem_al = smem_raw + ((128u - (um_smem_u32(smem_raw) & 127u)) & 127u);
+  DecodeTcSmem& S = *reinterpret_cast<DecodeTcSmem*>(smem_al);
   const int u = blockIdx.y;
   const int ps = (int)(u % p.n_param_sets);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int gid = lane >> 2, tig = lane & 3;
-  const int wm = warp & 3, wn = warp >> 2;
+  const int q4 = warp & 3, cb = warp >> 2;           // tensor-memory lane quarter, 32-channel block of this warp
   const int n = p.n_tokens[u];
   const int tile_first = blockIdx.x * kDecTiles;
   if (tile_first * kTile >= n) return;
@@ -266,30 +269,47 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p)
     const int k = idx / kD, nn = idx - k * kD;
     const float v = wsrc[idx];
     const __nv_bfloat16 w1 = __float2bfloat16_rn(v);
-    S.w[0][k * kLdB16 + nn] = w1;
-    S.w[1][k * kLdB16 + nn] = __float2bfloat16_rn(v - __bfloat162float(w1));
+    const int off = (nn >> 3) * 2048 + (k >> 3) * 128 + (k & 7) * 16 + (nn & 7) * 2;
+    *reinterpret_cast<__nv_bfloat16*>(&S.w[0][off]) = w1;
+    *reinterpret_cast<__nv_bfloat16*>(&S.w[1][off]) = __float2bfloat16_rn(v - __bfloat162float(w1));
   }
   if (tid < kD) S.bias[tid] = p.mean_rot[(int64_t)ps * kD + tid];
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(um_smem_u32(&S.mma_done)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid < 32) {                                    // warp 0 owns the tensor-memory allocation (128 columns)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(um_smem_u32(&S.tmem_base)), "r"(128u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tb = S.tmem_base;
+  uint32_t phase = 0;
+  bool ok = true;
 
-  for (int tt = 0; tt < kDecTiles; tt++) {
+  for (int tt = 0; tt < kDecTiles && ok; tt++) {
     const int tile = tile_first + tt;
     const int tile_pos = tile * kTile;
     if (tile_pos >= n) break;
     const int n_here = min(n - tile_pos, kTile);
     const uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
-    __syncthreads();                                   // the previous tile's MMAs have read S.a
+    __syncthreads();                                   // the previous tile's epilogue has read the accumulators
     // unpack: word by word into the code array
     for (int i = tid; i < kTile * kLdC / 4; i += kDecThreads) reinterpret_cast<uint32_t*>(S.codes)[i] = 0u;
     __syncthreads();
     unpack_tile(T, p.side, tile_ptr, S.codes, kLdC, tid, kDecThreads);
     // dequantise (same operation order as the CUDA-core kernel), add the rotated mean, split into two bf16 parts:
     // thread (channel j, token quarter tq) walks tokens [32 tq, 32 tq + 32); the lanes of a warp share the token, so
-    // its metadata is one broadcast load and the stores of a step are contiguous
+    // its metadata is one broadcast load
     {
       const int j = tid & (kD - 1), tq = tid >> 7;
       const int b = T.width[j];
       const int mo = T.meta_off[j / p.scale_group];
       const float L = (float)((1 << b) - 1), bias = S.bias[j];
+      const int joff = (j >> 3) * 2048 + (j & 7) * 2;   // K-major cores: k block j / 8, element j % 8
       for (int tk = 32 * tq; tk < 32 * tq + 32; tk++) {
         float lo_f = 0.f, R_f = 0.f;
         if (mo >= 0) {
@@ -307,68 +327,74 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p)
           p.yhat_out[(int64_t)u * p.stride_unit + (int64_t)(tile_pos + tk) * p.stride_token + j] = v;
         const float a = live ? v + bias : 0.f;
         const __nv_bfloat16 a1 = __float2bfloat16_rn(a);
-        S.a[0][tk * kLdB16 + j] = a1;
-        S.a[1][tk * kLdB16 + j] = __float2bfloat16_rn(a - __bfloat162float(a1));
+        const int off = joff + (tk >> 3) * 128 + (tk & 7) * 16;
+        *reinterpret_cast<__nv_bfloat16*>(&S.a[0][off]) = a1;
+        *reinterpret_cast<__nv_bfloat16*>(&S.a[1][off]) = __float2bfloat16_rn(a - __bfloat162float(a1));
       }
     }
+    if (!p.out) continue;                              // (the host launches this kernel with an output only)
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (!p.out) continue;
-    // ---- xhat = a W_dec on the tensor cores: warp (wm, wn) owns tokens [32 wm, +32) and channels [32 wn, +32)
-    float acc[2][4][4];
-#pragma unroll
-    for (int mb = 0; mb < 2; mb++)
-#pragma unroll
-      for (int nb = 0; nb < 4; nb++)
-#pragma unroll
-        for (int e = 0; e < 4; e++) acc[mb][nb][e] = 0.f;
-#pragma unroll 2
-    for (int ks = 0; ks < kD / 16; ks++) {
-      uint32_t a1[2][4], a2[2][4];
-#pragma unroll
-      for (int mb = 0; mb < 2; mb++) {
-        const int off = (32 * wm + 16 * mb + (lane & 7) + ((lane >> 3) & 1) * 8) * kLdB16 + 16 * ks + (lane >> 4) * 8;
-        ldmatrix_x4(a1[mb], &S.a[0][off]);
-        ldmatrix_x4(a2[mb], &S.a[1][off]);
+    // ---- xhat = a W_dec: 24 MMAs of 128 x 128 x 16 issued by one thread, accumulator tile in tensor memory
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t a0 = um_smem_u32(S.a[0]), a1 = um_smem_u32(S.a[1]);
+      const uint32_t w0 = um_smem_u32(S.w[0]), w1 = um_smem_u32(S.w[1]);
+#pragma unroll 1
+      for (int pr = 0; pr < 3; pr++) {                 // a1 W1, a1 W2, a2 W1
+        const uint32_t aa = pr == 2 ? a1 : a0, ww = pr == 1 ? w1 : w0;
+#pragma unroll 1
+        for (int ks = 0; ks < kD / 16; ks++)
+          um_mma_ss(tb, um_desc(aa + 4096 * ks, 2048, 128), um_desc(ww + 256 * ks, 128, 2048), kUmIdesc, (pr | ks) != 0);
       }
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(um_smem_u32(&S.mma_done)) : "memory");
+    }
+    {   // bounded wait for the accumulator tile
+      const uint32_t bar = um_smem_u32(&S.mma_done);
+      uint32_t done = 0;
+      for (int it = 0; it < (1 << 22) && !done; ++it)
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(done) : "r"(bar), "r"(phase) : "memory");
+      if (!done) ok = false;
+      phase ^= 1u;
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (ok) {
+      // ---- store: thread = token row 32 q4 + lane, channels [32 cb, 32 cb + 32)
+      float y[32];
+      const uint32_t src = tb + ((uint32_t)(q4 * 32) << 16) + 32u * cb;
+      um_ld16(src, y); um_ld16(src + 16, y + 16);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      const int tok = 32 * q4 + lane;
+      if (tok < n_here) {
+        const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + tok) * p.stride_token + 32 * cb;
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out) + (uintptr_t)o * (p.out_dtype == SPECTRA_BF16 ? 2 : 4);
+        if ((addr & 15) == 0 && p.out_dtype == SPECTRA_BF16) {
+          uint4* dst = reinterpret_cast<uint4*>(addr);
 #pragma unroll
-      for (int np = 0; np < 2; np++) {                 // two 8-channel blocks per ldmatrix
-        const int off = (16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8) * kLdB16 + 32 * wn + 16 * np + (lane >> 4) * 8;
-        uint32_t b1[4], b2[4];
-        ldmatrix_x4_trans(b1, &S.w[0][off]);
-        ldmatrix_x4_trans(b2, &S.w[1][off]);
+          for (int c = 0; c < 4; c++) {
+            __nv_bfloat162 h[4];
 #pragma unroll
-        for (int mb = 0; mb < 2; mb++) {
-          mma_bf16(acc[mb][2 * np], a1[mb], b1[0], b1[1]);
-          mma_bf16(acc[mb][2 * np + 1], a1[mb], b1[2], b1[3]);
-          mma_bf16(acc[mb][2 * np], a1[mb], b2[0], b2[1]);
-          mma_bf16(acc[mb][2 * np + 1], a1[mb], b2[2], b2[3]);
-          mma_bf16(acc[mb][2 * np], a2[mb], b1[0], b1[1]);
-          mma_bf16(acc[mb][2 * np + 1], a2[mb], b1[2], b1[3]);
+            for (int e = 0; e < 4; e++) h[e] = __floats2bfloat162_rn(y[8 * c + 2 * e], y[8 * c + 2 * e + 1]);
+            dst[c] = *reinterpret_cast<const uint4*>(h);
+          }
+        } else if ((addr & 15) == 0) {
+          float4* dst = reinterpret_cast<float4*>(addr);
+#pragma unroll
+          for (int c = 0; c < 8; c++) dst[c] = make_float4(y[4 * c], y[4 * c + 1], y[4 * c + 2], y[4 * c + 3]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; c++) store_from_float(p.out, p.out_dtype, o + c, y[c]);
         }
       }
     }
-    // ---- store: a thread holds the channel pair (2 tig, 2 tig + 1) of rows gid and gid + 8 of each 16-token block
-#pragma unroll
-    for (int mb = 0; mb < 2; mb++)
-#pragma unroll
-      for (int half = 0; half < 2; half++) {
-        const int tok = 32 * wm + 16 * mb + gid + 8 * half;
-        if (tok >= n_here) continue;
-        const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + tok) * p.stride_token + 32 * wn + 2 * tig;
-        // the pair goes out as one 4-byte (bf16) or 8-byte (fp32) store when its address allows it
-        const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out) + (uintptr_t)o * (p.out_dtype == SPECTRA_BF16 ? 2 : 4);
-        const bool pair_ok = (addr & (p.out_dtype == SPECTRA_BF16 ? 3 : 7)) == 0;
-#pragma unroll
-        for (int nb = 0; nb < 4; nb++) {
-          const float v0 = acc[mb][nb][2 * half], v1 = acc[mb][nb][2 * half + 1];
-          if (pair_ok && p.out_dtype == SPECTRA_BF16)
-            *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(p.out) + o + 8 * nb) = __floats2bfloat162_rn(v0, v1);
-          else if (pair_ok)
-            *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.out) + o + 8 * nb) = make_float2(v0, v1);
-          else { store_from_float(p.out, p.out_dtype, o + 8 * nb, v0); store_from_float(p.out, p.out_dtype, o + 8 * nb + 1, v1); }
-        }
-      }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
+  // ---- the warp that allocated the tensor memory frees it
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tb), "r"(128u) : "memory");
 }
 
 }  // namespace spectra
@@ -439,13 +465,14 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
                out_dtype, yhat_out, stride_unit, stride_token};
-  if (out) {   // reconstruction: inverse rotation on the tensor cores
-    if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)sizeof(DecodeTcSmem)) != cudaSuccess)
+  if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05)
+    const size_t dec_smem = sizeof(DecodeTcSmem) + 128;
+    if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem) !=
+        cudaSuccess)
       return SPECTRA_CUDA_ERROR;
     const unsigned tiles = (unsigned)((max_tokens + kTile - 1) / kTile);
     dim3 grid_tc((tiles + kDecTiles - 1) / kDecTiles, (unsigned)n_units);
-    decode_tc_kernel<<<grid_tc, kDecThreads, sizeof(DecodeTcSmem), (cudaStream_t)stream>>>(a);
+    decode_tc_kernel<<<grid_tc, kDecThreads, dec_smem, (cudaStream_t)stream>>>(a);
     return launch_status();
   }
   if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CodecSmem)) !=
