@@ -162,6 +162,49 @@ def test_encode_per_unit_positions_and_status_bits(sp):
     assert st == (sp.STATUS_NONFINITE | sp.STATUS_F16_RANGE)
 
 
+def test_bulk_bf16_encode_with_ragged_starts_keeps_earlier_tokens(sp):
+    """The bulk bf16 path (rotation on tcgen05) on ranges that start and end inside tiles, different per unit, on
+    top of tokens written before: earlier tokens stay byte for byte, the new ones match the oracle's encode of the
+    same bf16 vectors up to rare rounding ties, slots behind the range are cleared."""
+    wl = si.WORKLOADS["tiny"]
+    cfg = sp.default_config()
+    n_units, cap = 2, 640
+    X = [si.to_bf16_f32(si.draw_unit(wl, 0, u, si.SIDE_K, 0)[:cap]) for u in range(n_units)]
+    params = H.fit_params(X, 8.0)
+    dp = H.dev_params(params)
+    off, total = H.cache_layout(params, n_units, cap)
+    first = np.array([70, 129], np.int64)            # tokens [0, first) are written beforehand, one by one path aside
+    n_new = 300                                      # ends at 370 and 429: inside tiles
+    for side in (sp.SIDE_K, sp.SIDE_V):
+        ref = np.zeros(total, np.uint8)
+        cache = torch.zeros(total, dtype=torch.uint8, device="cuda")
+        for u in range(n_units):                     # the earlier tokens, by the oracle on both sides
+            H.oracle_encode(H.Params(params.w_enc[[u]], params.w_dec[[u]], params.m_rot[[u]], params.widths[[u]], 64),
+                            side, X[u][None, :first[u]], [0], ref[off[u]:], np.zeros(1, np.int64))
+        cache.copy_(torch.from_numpy(ref))
+        before = ref.copy()
+        xs = np.stack([X[u][first[u]:first[u] + n_new] for u in range(n_units)])
+        assert H.oracle_encode(params, side, xs, first, ref, off) == 0
+        st = _gpu_encode(sp, cfg, params, dp, side, H.to_dev(xs).to(torch.bfloat16),
+                         H.to_dev(first.astype(np.int32)), cache, H.to_dev(off))
+        assert st == 0
+        got = cache.cpu().numpy()
+        for u in range(n_units):
+            end = int(first[u]) + n_new
+            c_ref, m_ref = H.unpack_codes(params, side, ref, off, u, end)
+            c_got, m_got = H.unpack_codes(params, side, got, off, u, end)
+            c_old, m_old = H.unpack_codes(params, side, before, off, u, int(first[u]))
+            assert np.array_equal(c_got[:first[u]], c_old) and np.array_equal(m_got[:first[u]], m_old)
+            same_meta = (m_got == m_ref).all(axis=1)
+            diff = np.abs(c_got.astype(np.int64) - c_ref.astype(np.int64))
+            assert diff[same_meta].max() <= 1
+            assert (diff[same_meta] != 0).sum() <= 3 and (~same_meta).sum() <= 3
+            # slots of the last touched tile behind the range hold zeros
+            tail_tile_end = (end + 127) // 128 * 128
+            c_tail, m_tail = H.unpack_codes(params, side, got, off, u, tail_tile_end)
+            assert not c_tail[end:].any() and not m_tail[end:].any()
+
+
 # ----------------------------------------------------------------------------- config 0 end to end
 
 def _tiny_setup(sp, ratio=4.0, gain_mode=ofit.GAIN_SQRT, n=1024, gs=64):
