@@ -225,7 +225,8 @@ size_t spectra_attention_workspace_bytes(const spectra_config* cfg, int32_t batc
  * Same results, bit for bit in the cache, as spectra_encode(K), spectra_encode(V) (one new token per unit at
  * position seq_len[sequence] - 1) followed by spectra_decode_attention.
  * new_k, new_v: device [batch * n_kv_heads, d] (one vector per unit, unit order as above), x_dtype SPECTRA_F32
- * or SPECTRA_BF16.  seq_len: device int32 [batch], the lengths INCLUDING the appended token (>= 1).
+ * or SPECTRA_BF16.  seq_len: device int32 [batch], the lengths INCLUDING the appended token (a sequence with
+ * length 0 gets no append and a zero output row).
  * w_enc_k/v, mean_rot_k/v as in spectra_encode; every other argument as in spectra_decode_attention
  * (mean_rot_k is required here).  cache_k / cache_v are written (the appended token) and read.
  */

@@ -62,6 +62,7 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
 
   // ---- stage the new tokens
   const int pos_first = p.pos0 ? p.pos0[u] : p.seq_len[u / p.n_kv] - 1;
+  if (pos_first < 0) return;                 // fused step on an empty sequence: nothing to append (CTA-uniform)
   for (int idx = j; idx < p.n_new * kD; idx += 128) {
     const int t = idx / kD, i = idx - t * kD;
     xs[t][i] = load_as_float(p.x, p.x_dtype, (int64_t)u * p.stride_unit + (int64_t)t * p.stride_token + i);

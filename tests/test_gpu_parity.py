@@ -545,3 +545,31 @@ def test_fused_decode_step_equals_separate_calls(sp, name, tensor_path):
         assert torch.equal(outs[0], outs[1])
     else:   # the CUDA-core kernel sums with shared-memory float atomics: equal up to summation order
         assert torch.allclose(outs[0], outs[1], rtol=1e-5, atol=1e-6)
+
+
+def test_fused_decode_step_skips_empty_sequences(sp):
+    """A sequence of length 0 in a fused step gets no append (its cache stays as it was) and a zero output row."""
+    import dataclasses
+    from paper_2608_07915_b200 import harness
+    wl = dataclasses.replace(si.WORKLOADS["tiny"], batch=2)
+    m = harness.CodedModelCache(wl, layers=1, batch=2, extra_tokens=128)
+    m.build()
+    before = [m.side[0][s].cache.clone() for s in (0, 1)]
+    gen = torch.Generator(device="cuda").manual_seed(6)
+    q = torch.randn((2, wl.q_heads, 128), generator=gen, device="cuda")
+    nk = torch.randn((2 * wl.kv_heads, 128), generator=gen, device="cuda")
+    nv = torch.randn((2 * wl.kv_heads, 128), generator=gen, device="cuda")
+    out = torch.full((2, wl.q_heads, 128), 3.0, dtype=torch.float32, device="cuda")
+    m.seq_len += 1
+    m.seq_len[1] = 0
+    m.step_layer(0, q, nk, nv, out)
+    torch.cuda.synchronize()
+    assert int(m.status.item()) == 0
+    assert (out[1] == 0).all() and torch.isfinite(out[0]).all() and (out[0] != 3.0).any()
+    for s in (0, 1):
+        ls = m.side[0][s]
+        for u in range(wl.kv_heads, 2 * wl.kv_heads):            # units of the empty sequence
+            a = int(ls.unit_offset_host[u])
+            e = int(ls.unit_offset_host[u + 1]) if u + 1 < 2 * wl.kv_heads else ls.cache.numel()
+            assert torch.equal(ls.cache[a:e], before[s][a:e])
+        assert not torch.equal(ls.cache, before[s])               # the other sequence did get its token
