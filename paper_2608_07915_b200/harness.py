@@ -59,46 +59,62 @@ class CodedModelCache:
         cfg, H, d, N = self.cfg, self.H, self.d, self.n_tokens
         n_fit = min(self.wl.n_fit, N)
         f32 = dict(dtype=torch.float32, device=self.device)
-        fit_ws = torch.zeros(sp.fit_workspace_bytes(cfg, H), dtype=torch.uint8, device=self.device)
         ev = lambda: torch.cuda.Event(enable_timing=True)
         t_fit = t_enc = 0.0
-        for layer in range(self.layers):
-            for side in (si.SIDE_K, si.SIDE_V):
+        sides = [(layer, side) for layer in range(self.layers) for side in (si.SIDE_K, si.SIDE_V)]
+        n_ls = len(sides)
+        w_enc_all, w_dec_all = (torch.zeros((n_ls * H, d, d), **f32) for _ in range(2))
+        m_rot_all, var_all = (torch.zeros((n_ls * H, d), **f32) for _ in range(2))
+        widths_all = torch.zeros((n_ls * H, d), dtype=torch.uint8, device=self.device)
+        if any((params_override or {}).get(ls_key) is None for ls_key in sides):
+            # calibration of the whole model in one call: the fit tokens (sequence 0 of every layer, head and side)
+            # are gathered first, so that the per-matrix eigensolver CTAs fill the GPU
+            dt = torch.bfloat16 if self.wl.dtype == "bf16" else torch.float32
+            fit_x = torch.empty((n_ls * H, n_fit, d), dtype=dt, device=self.device)
+            for i, (layer, side) in enumerate(sides):
                 x = self.draw_layer_side(layer, side)
-                ls = LayerSide()
-                ls.w_enc, ls.w_dec = (torch.zeros((H, d, d), **f32) for _ in range(2))
-                ls.m_rot, ls.var = (torch.zeros((H, d), **f32) for _ in range(2))
-                ls.widths = torch.zeros((H, d), dtype=torch.uint8, device=self.device)
-                e0, e1, e2 = ev(), ev(), ev()
-                e0.record()
-                ov = (params_override or {}).get((layer, side))
-                if ov is not None:
-                    ls.w_enc.copy_(torch.from_numpy(np.ascontiguousarray(ov["w_enc"], np.float32)))
-                    ls.w_dec.copy_(torch.from_numpy(np.ascontiguousarray(ov["w_dec"], np.float32)))
-                    ls.m_rot.copy_(torch.from_numpy(np.ascontiguousarray(ov["m_rot"], np.float32)))
-                    ls.widths.copy_(torch.from_numpy(np.ascontiguousarray(ov["widths"], np.uint8)))
-                else:
-                    sp.fit_basis(cfg, x, H, n_fit, N * d, d, ls.w_enc, ls.w_dec, ls.m_rot, ls.var, None, None, fit_ws)
-                    sp.alloc_bits(cfg, ls.var, H, self.wl.ratio, ls.widths)
-                e1.record()
-                ls.widths_host = ls.widths.cpu().numpy()
-                ls.tile_bytes = np.array([sp.tile_bytes(cfg, w) for w in ls.widths_host], np.int64)
-                sizes = np.array([ls.tile_bytes[u % H] * self.cap_tiles for u in range(self.n_units)], np.int64)
-                ls.unit_offset_host = np.concatenate([[0], np.cumsum(sizes)[:-1]]).astype(np.int64)
-                ls.unit_offset = torch.from_numpy(ls.unit_offset_host).to(self.device)
-                ls.cache = torch.empty(int(sizes.sum()), dtype=torch.uint8, device=self.device)
-                self.pos0.zero_()
-                e1.record()
-                sp.encode(cfg, side, x, 0, self.n_units, H, self.pos0, N, N * d, d, ls.w_enc, ls.m_rot, ls.widths,
-                          ls.cache, ls.unit_offset, self.status)
-                e2.record()
-                torch.cuda.synchronize()
-                t_fit += e0.elapsed_time(e1) if time_phases else 0.0
-                t_enc += e1.elapsed_time(e2)
-                for u in self.keep_raw_units.get((layer, side), []):
-                    self.raw[(layer, side, u)] = x[u // H, u % H].float().cpu().numpy()
-                self.side[layer][side] = ls
+                fit_x[i * H:(i + 1) * H] = x[0, :, :n_fit]
                 del x
+            fit_ws = torch.zeros(sp.fit_workspace_bytes(cfg, n_ls * H), dtype=torch.uint8, device=self.device)
+            e0, e1 = ev(), ev()
+            e0.record()
+            sp.fit_basis(cfg, fit_x, n_ls * H, n_fit, n_fit * d, d, w_enc_all, w_dec_all, m_rot_all, var_all, None, None,
+                         fit_ws)
+            sp.alloc_bits(cfg, var_all, n_ls * H, self.wl.ratio, widths_all)
+            e1.record()
+            torch.cuda.synchronize()
+            t_fit = e0.elapsed_time(e1)
+            del fit_x, fit_ws
+        for i, (layer, side) in enumerate(sides):
+            x = self.draw_layer_side(layer, side)
+            ls = LayerSide()
+            ls.w_enc, ls.w_dec = w_enc_all[i * H:(i + 1) * H], w_dec_all[i * H:(i + 1) * H]
+            ls.m_rot, ls.var = m_rot_all[i * H:(i + 1) * H], var_all[i * H:(i + 1) * H]
+            ls.widths = widths_all[i * H:(i + 1) * H]
+            e1, e2 = ev(), ev()
+            ov = (params_override or {}).get((layer, side))
+            if ov is not None:
+                ls.w_enc.copy_(torch.from_numpy(np.ascontiguousarray(ov["w_enc"], np.float32)))
+                ls.w_dec.copy_(torch.from_numpy(np.ascontiguousarray(ov["w_dec"], np.float32)))
+                ls.m_rot.copy_(torch.from_numpy(np.ascontiguousarray(ov["m_rot"], np.float32)))
+                ls.widths.copy_(torch.from_numpy(np.ascontiguousarray(ov["widths"], np.uint8)))
+            ls.widths_host = ls.widths.cpu().numpy()
+            ls.tile_bytes = np.array([sp.tile_bytes(cfg, w) for w in ls.widths_host], np.int64)
+            sizes = np.array([ls.tile_bytes[u % H] * self.cap_tiles for u in range(self.n_units)], np.int64)
+            ls.unit_offset_host = np.concatenate([[0], np.cumsum(sizes)[:-1]]).astype(np.int64)
+            ls.unit_offset = torch.from_numpy(ls.unit_offset_host).to(self.device)
+            ls.cache = torch.empty(int(sizes.sum()), dtype=torch.uint8, device=self.device)
+            self.pos0.zero_()
+            e1.record()
+            sp.encode(cfg, side, x, 0, self.n_units, H, self.pos0, N, N * d, d, ls.w_enc, ls.m_rot, ls.widths,
+                      ls.cache, ls.unit_offset, self.status)
+            e2.record()
+            torch.cuda.synchronize()
+            t_enc += e1.elapsed_time(e2)
+            for u in self.keep_raw_units.get((layer, side), []):
+                self.raw[(layer, side, u)] = x[u // H, u % H].float().cpu().numpy()
+            self.side[layer][side] = ls
+            del x
         self.seq_len.fill_(N)
         self.pos0.fill_(N)
         self.timings = dict(fit_alloc_ms=t_fit, prefill_encode_ms=t_enc)
