@@ -21,6 +21,15 @@ __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, 
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
   const UnitDesc& D = f.desc[vu];
+  {  // the tail of this CTA's dependent chain reads W_dec,V, the rotated mean and the strip tables: ask for them now
+    const float* wv = p.w_dec_v + (int64_t)ps * kD * kD;
+#pragma unroll
+    for (int i = 0; i < 4; i++) prefetch_l2(wv + (tid * 4 + i) * 32);
+    if (tid < 4) prefetch_l2(p.mean_rot_v + (int64_t)ps * kD + tid * 32);
+    if (tid >= 32 && tid < 32 + kMaxStrips * 4 / 128) prefetch_l2(D.vcoef + (tid - 32) * 32);
+    if (tid >= 64 && tid < 64 + kMaxStrips / 128) prefetch_l2(D.vchan + (tid - 64) * 128);
+    if (tid == 96) prefetch_l2(p.widths_v + (int64_t)ps * kD);
+  }
   const long long total = f.tile_prefix[f.n_units];
   const long long ta = f.tile_prefix[vu], tb = f.tile_prefix[vu + 1];
   const int64_t hidx = (int64_t)b * p.n_q + hk * p.gqa + h0 + h;         // query head in the caller's order

@@ -210,15 +210,17 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
   const int G = min(kFastGqa, p.gqa - h0);                          // query heads of this pass
-  build_strip_tables(S.tk, p.widths_k + (int64_t)ps * kD, S.tv, p.widths_v + (int64_t)ps * kD, 64);
-  const StripTable& TK = S.tk;
-  const StripTable& TV = S.tv;
-  UnitDesc& D = f.desc[vu];
+  // The CTA's work is a chain of dependent phases; what the later phases read is asked for now (one line per thread).
+  prefetch_l2(p.w_dec_k + (int64_t)ps * kD * kD + tid * 32);
+  if (tid < 4 && p.mean_rot_k) prefetch_l2(p.mean_rot_k + (int64_t)ps * kD + tid * 32);
   for (int idx = tid; idx < kFastGqa * kD; idx += kPrepThreads) {
     const int h = idx / kD, i = idx - h * kD;
     S.qraw[h][i] = h < G ? load_as_float(p.q, p.q_dtype, ((int64_t)b * p.n_q + hk * p.gqa + h0 + h) * kD + i) : 0.f;
   }
-  __syncthreads();
+  build_strip_tables(S.tk, p.widths_k + (int64_t)ps * kD, S.tv, p.widths_v + (int64_t)ps * kD, 64);
+  const StripTable& TK = S.tk;
+  const StripTable& TV = S.tv;
+  UnitDesc& D = f.desc[vu];
   const float* wk = p.w_dec_k + (int64_t)ps * kD * kD;
   {
     float4 wrow[kD / kWarps];
@@ -345,14 +347,18 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
 
 // First launch of a fused decode step: the prep grid, then one CTA per unit-side that appends the new token
 // (threads 0..127 of it; the K side first).  The main kernel that follows reads what both parts wrote.
-__global__ void __launch_bounds__(kPrepThreads) decode_step_front_kernel(AttnArgs p, FastArgs f, AppendArgs ak,
+__global__ void __launch_bounds__(kPrepThreads, 2) decode_step_front_kernel(AttnArgs p, FastArgs f, AppendArgs ak,
                                                                          AppendArgs av, int n_cache_units) {
   const int n_prep = f.n_units + 1;
   if ((int)blockIdx.x < n_prep) { attention_prep_body(p, f, blockIdx.x); return; }
-  if (threadIdx.x >= 128) return;
   const int i = blockIdx.x - n_prep;
-  if (i < n_cache_units) encode_append_body(ak, i);
-  else encode_append_body(av, i - n_cache_units);
+  const AppendArgs& a = i < n_cache_units ? ak : av;
+  const int u = i < n_cache_units ? i : i - n_cache_units;
+  // all 512 threads ask the L2 for the unit's W_enc (one line each) before the 128 workers start their chain
+  if (!(a.flags & SPECTRA_ROTATED_INPUT))
+    prefetch_l2(a.w_enc + (int64_t)(u % a.n_param_sets) * kD * kD + threadIdx.x * 32);
+  if (threadIdx.x >= 128) return;
+  encode_append_body(a, u);
 }
 
 }  // namespace spectra

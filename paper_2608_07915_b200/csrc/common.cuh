@@ -242,6 +242,9 @@ __device__ inline void unpack_tile(const StripTable& T, int side, const uint8_t*
   }
 }
 
+// Asks the L2 for the 128-byte line that holds p; a later load then pays the L2's latency instead of the DRAM's.
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 __device__ inline float load_as_float(const void* p, int dtype, int64_t idx) {
   if (dtype == SPECTRA_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx]);
   return reinterpret_cast<const float*>(p)[idx];

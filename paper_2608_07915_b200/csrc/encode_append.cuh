@@ -29,6 +29,12 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
   const int gs = p.scale_group, n_groups = kD / gs;
   const int b = p.widths[(int64_t)ps * kD + j];
   const bool rotated = (p.flags & SPECTRA_ROTATED_INPUT) != 0;
+  // ---- stage the new tokens (these loads, the width and the position are in flight together)
+  const int pos_first = p.pos0 ? p.pos0[u] : p.seq_len[u / p.n_kv] - 1;
+  for (int idx = j; idx < p.n_new * kD; idx += 128) {
+    const int t = idx / kD, i = idx - t * kD;
+    xs[t][i] = load_as_float(p.x, p.x_dtype, (int64_t)u * p.stride_unit + (int64_t)t * p.stride_token + i);
+  }
 
   // ---- where this channel's strips live: rank inside each class, class offsets, tile size
   if (j < kMaxGroups) grp_act[j] = 0;
@@ -60,14 +66,7 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
   }
   const int tile_bytes = payload + 512 * n_act;
 
-  // ---- stage the new tokens
-  const int pos_first = p.pos0 ? p.pos0[u] : p.seq_len[u / p.n_kv] - 1;
   if (pos_first < 0) return;                 // fused step on an empty sequence: nothing to append (CTA-uniform)
-  for (int idx = j; idx < p.n_new * kD; idx += 128) {
-    const int t = idx / kD, i = idx - t * kD;
-    xs[t][i] = load_as_float(p.x, p.x_dtype, (int64_t)u * p.stride_unit + (int64_t)t * p.stride_token + i);
-  }
-  __syncthreads();
   const float* w = p.w_enc + (int64_t)ps * kD * kD;
   const float mr = rotated ? 0.f : p.mean_rot[(int64_t)ps * kD + j];
   uint8_t* base = p.cache + p.unit_offset[u];
