@@ -171,7 +171,10 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
   // heads is taken in passes of 4 (each pass is a unit of its own that reads the same tiles)
   const int npass = (gqa + kFastGqa - 1) / kFastGqa;
   const int64_t n_vunits = n_units * npass;
-  if (widths_k_host && cfg->scale_group == 64 && n_vunits <= 65534) {
+  // (its kernels fetch whole parameter matrices with bulk copies, which need 16-byte aligned sources)
+  const bool aligned = (((uintptr_t)w_dec_k | (uintptr_t)w_dec_v | (uintptr_t)(app ? app->w_enc_k : nullptr) |
+                         (uintptr_t)(app ? app->w_enc_v : nullptr)) & 15) == 0;
+  if (widths_k_host && cfg->scale_group == 64 && n_vunits <= 65534 && aligned) {
     const WidthFacts F = width_facts(widths_k_host, widths_v_host, n_param_sets);
     if (!F.ok) return SPECTRA_INVALID_ARG;
     const int sms = sm_count();
@@ -185,7 +188,8 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
     if (depth > 4) depth = 4;
     const int quota = pick_quota(F.vb);
     if (depth >= 1 && quota >= 0) {
-      FastLayout L = fast_layout(n_vunits, sms * ctas_per_sm * kFastWarps, F.max_vstrips);
+      const int vs_max = (F.max_vstrips + 3) & ~3;     // records are fetched with bulk copies: 16-byte multiples
+      FastLayout L = fast_layout(n_vunits, sms * ctas_per_sm * kFastWarps, vs_max);
       if (L.total > workspace_bytes) return SPECTRA_WORKSPACE_TOO_SMALL;
       char* ws = reinterpret_cast<char*>(workspace);
       FastArgs f{};
@@ -193,7 +197,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       f.tile_prefix = reinterpret_cast<int32_t*>(ws + L.prefix_off);
       f.warp_unit = reinterpret_cast<int32_t*>(ws + L.warp_off);
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
-      f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = F.max_vstrips;
+      f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = vs_max;
       f.n_units = (int)n_vunits; f.npass = npass; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
       if (app) {
         AppendArgs ak{app->new_k, app->x_dtype, 0, SPECTRA_SIDE_K, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
@@ -216,7 +220,10 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
         default: rc = launch_fast_main<0, 7, 3, 4>(a, f, grid, smem, st); break;
       }
       if (rc) return rc;
-      attention_mma_combine_kernel<<<(unsigned)(n_vunits * kFastGqa), 128, 0, st>>>(a, f);
+      if (cudaFuncSetAttribute(attention_mma_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kCombineDynSmem) != cudaSuccess)
+        return SPECTRA_CUDA_ERROR;
+      attention_mma_combine_kernel<<<(unsigned)(n_vunits * kFastGqa), 128, kCombineDynSmem, st>>>(a, f);
       return launch_status();
     }
   }

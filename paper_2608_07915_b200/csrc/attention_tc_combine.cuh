@@ -7,36 +7,60 @@
 
 namespace spectra {
 
-constexpr int kMaxRecSmem = 2048;   // record headers kept in shared memory; longer lists are re-read from global
+constexpr int kCombineBatch = 32;   // records merged per round (one per lane)
+constexpr int kCombineDynSmem = kD * kD * 4 + 16;   // W_dec,V and the barrier of its copy
 
+// A worker without tiles writes no record (only when there are fewer tiles than workers).
+__device__ __noinline__ bool worker_has_tiles(long long gw, long long total, int W) {
+  return (gw + 1) * total / W > gw * total / W;
+}
+
+// The CTA's work is a chain of dependent global reads, each costing a full memory latency, and it starts on a cold
+// instruction cache (straight-line code costs far more per instruction than a loop that is fetched once).  So the
+// reads are grouped into two rounds and rare cases are kept out of the main path: (1) everything whose address is
+// known at launch - W_dec,V (one bulk copy into shared memory), the tile prefix, the descriptor fields, the rotated
+// mean; (2) the unit's partial records, up to 32 at a time, headers and accumulators together, before any of them
+// is used.  Records are merged with a running maximum; every warp computes the weights of a batch redundantly
+// (lane i = record i), so the merge needs no cross-warp exchange.
 __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, FastArgs f) {
-  __shared__ float s_e[kMaxRecSmem];       // exp2(m_r - M), 0 for workers that wrote nothing
-  __shared__ float s_red[4][4];
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_w = reinterpret_cast<float*>(smem_raw);                    // W_dec,V [j][channel]
+  const uint32_t wbar = smem_u32(smem_raw + kD * kD * 4);
   __shared__ float s_o[kD];
-  __shared__ float s_part[4][kMaxStrips];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int vu = blockIdx.x / kFastGqa, h = blockIdx.x - vu * kFastGqa;   // unit of the tensor path, head slot of its pass
   const int u = vu / f.npass, h0 = kFastGqa * (vu - u * f.npass);
   if (h0 + h >= p.gqa) return;
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
   const UnitDesc& D = f.desc[vu];
-  {  // the tail of this CTA's dependent chain reads W_dec,V, the rotated mean and the strip tables: ask for them now
-    const float* wv = p.w_dec_v + (int64_t)ps * kD * kD;
-#pragma unroll
-    for (int i = 0; i < 4; i++) prefetch_l2(wv + (tid * 4 + i) * 32);
-    if (tid < 4) prefetch_l2(p.mean_rot_v + (int64_t)ps * kD + tid * 32);
-    if (tid >= 32 && tid < 32 + kMaxStrips * 4 / 128) prefetch_l2(D.vcoef + (tid - 32) * 32);
-    if (tid >= 64 && tid < 64 + kMaxStrips / 128) prefetch_l2(D.vchan + (tid - 64) * 128);
-    if (tid == 96) prefetch_l2(p.widths_v + (int64_t)ps * kD);
+  // ---- round 1
+  if (tid == 0) {
+    mbar_init(wbar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_expect_tx(wbar, kD * kD * 4);
+    bulk_load(smem_u32(s_w), p.w_dec_v + (int64_t)ps * kD * kD, kD * kD * 4, wbar);
   }
   const long long total = f.tile_prefix[f.n_units];
   const long long ta = f.tile_prefix[vu], tb = f.tile_prefix[vu + 1];
+  const int ns = D.n_vstrips;
+  const int vf1 = (int)D.vfirst[1], vf2 = (int)D.vfirst[2], vf3 = (int)D.vfirst[3];
+  constexpr int kPerThread = kMaxStrips / 128;      // strips tid, tid + 128, tid + 256
+  int chan[kPerThread];
+  float coef[kPerThread];
+#pragma unroll
+  for (int q = 0; q < kPerThread; q++) { chan[q] = D.vchan[tid + 128 * q]; coef[q] = D.vcoef[tid + 128 * q]; }
+  const bool has_width = p.widths_v[(int64_t)ps * kD + tid] != 0;
+  const float mean_rot = p.mean_rot_v[(int64_t)ps * kD + tid];
+  const float qconst = D.qconst[h];
   const int64_t hidx = (int64_t)b * p.n_q + hk * p.gqa + h0 + h;         // query head in the caller's order
   const int64_t oidx = hidx * kD + tid;
+  s_o[tid] = 0.f;
+  __syncthreads();                                           // the barrier's initialisation is visible to all
   if (tb <= ta) {                                            // empty sequence
     store_from_float(p.out, p.out_dtype, oidx, 0.f);
     if (p.lse && tid == 0) p.lse[hidx] = -INFINITY;
+    mbar_wait(wbar, 0);                                      // the copy must land before the shared memory is released
     return;
   }
   // workers whose tile ranges intersect this unit: the largest gw with floor(gw * total / W) <= tile
@@ -44,95 +68,113 @@ __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, 
   const int gw_first = (int)(((ta + 1) * W + total - 1) / total) - 1;
   const int gw_last = (int)((tb * W + total - 1) / total) - 1;
   const int nrec = gw_last - gw_first + 1;
-  const int64_t hoff = (int64_t)h * (kRecHead + f.vs_max);
-  auto rec_ptr = [&](int r) { return f.records + (int64_t)(gw_first + r + vu) * f.rec_stride + hoff; };
-  auto nonempty = [&](int r) {
-    const long long gw = gw_first + r;
-    return (gw + 1) * total / W > gw * total / W;
-  };
-  // ---- running maximum over the records
-  float m = -INFINITY;
-  for (int r = tid; r < nrec; r += 128)
-    if (nonempty(r)) m = fmaxf(m, rec_ptr(r)[0]);
+  const float* rec0 = f.records + (int64_t)(gw_first + vu) * f.rec_stride + (int64_t)h * (kRecHead + f.vs_max);
+  // ---- round 2
+  float M = -INFINITY, L = 0.f, P0 = 0.f, P1 = 0.f;
+  float acc[kPerThread];
 #pragma unroll
-  for (int s = 16; s; s >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, s));
-  if (lane == 0) s_red[0][warp] = m;
-  __syncthreads();
-  const float M = fmaxf(fmaxf(s_red[0][0], s_red[0][1]), fmaxf(s_red[0][2], s_red[0][3]));
-  __syncthreads();
-  // ---- weights of the records, softmax denominator, offset sums
-  float L = 0.f, P0 = 0.f, P1 = 0.f;
-  for (int r = tid; r < nrec; r += 128) {
-    float e = 0.f;
-    if (nonempty(r)) {
-      const float* rec = rec_ptr(r);
+  for (int q = 0; q < kPerThread; q++) acc[q] = 0.f;
+  if (total >= W) {
+    // every worker has tiles, so every record exists
+#pragma unroll 1
+    for (int r0 = 0; r0 < nrec; r0 += kCombineBatch) {
+      const int nb = min(kCombineBatch, nrec - r0);
+      const float* rb = rec0 + (int64_t)r0 * f.rec_stride;
+      float hd[4] = {-INFINITY, 0.f, 0.f, 0.f};
+      if (lane < nb) {
+#pragma unroll
+        for (int i = 0; i < 4; i++) hd[i] = rb[(int64_t)lane * f.rec_stride + i];
+      }
+      float v[kCombineBatch][2];
+#pragma unroll
+      for (int i = 0; i < kCombineBatch; i++) {
+        const float* rv = rb + (int64_t)i * f.rec_stride + kRecHead + tid;
+        v[i][0] = (i < nb && tid < ns) ? rv[0] : 0.f;
+        v[i][1] = (i < nb && tid + 128 < ns) ? rv[128] : 0.f;
+      }
+      float mb = hd[0];
+#pragma unroll
+      for (int s = 16; s; s >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, s));
+      const float Mn = fmaxf(M, mb);
+      const float alpha = M == -INFINITY ? 0.f : exp2f(M - Mn);
+      const float e = hd[0] == -INFINITY ? 0.f : exp2f(hd[0] - Mn);
+      float dl = e * hd[1], d0 = e * hd[2], d1 = e * hd[3];
+#pragma unroll
+      for (int s = 16; s; s >>= 1) {
+        dl += __shfl_xor_sync(0xffffffffu, dl, s);
+        d0 += __shfl_xor_sync(0xffffffffu, d0, s);
+        d1 += __shfl_xor_sync(0xffffffffu, d1, s);
+      }
+      L = fmaf(L, alpha, dl); P0 = fmaf(P0, alpha, d0); P1 = fmaf(P1, alpha, d1);
+#pragma unroll
+      for (int q = 0; q < kPerThread; q++) acc[q] *= alpha;
+#pragma unroll
+      for (int i = 0; i < kCombineBatch; i++) {
+        const float ei = __shfl_sync(0xffffffffu, e, i);
+        acc[0] = fmaf(ei, v[i][0], acc[0]);
+        acc[1] = fmaf(ei, v[i][1], acc[1]);
+      }
+      if (ns > 256) {                                        // third strip of a thread: widths rarely ask for it
+#pragma unroll 1
+        for (int i = 0; i < nb; i++) {
+          const float ei = __shfl_sync(0xffffffffu, e, i);
+          if (tid + 256 < ns) acc[2] = fmaf(ei, rb[(int64_t)i * f.rec_stride + kRecHead + tid + 256], acc[2]);
+        }
+      }
+      M = Mn;
+    }
+  } else {
+    // fewer tiles than workers (tiny calls): some workers wrote nothing; one record at a time
+#pragma unroll 1
+    for (int r = 0; r < nrec; r++) {
+      if (!worker_has_tiles(gw_first + r, total, W)) continue;
+      const float* rec = rec0 + (int64_t)r * f.rec_stride;
       const float mr = rec[0];
-      e = mr == -INFINITY ? 0.f : exp2f(mr - M);
-      L += e * rec[1]; P0 += e * rec[2]; P1 += e * rec[3];
-    }
-    if (r < kMaxRecSmem) s_e[r] = e;
-  }
+      if (mr == -INFINITY) continue;
+      const float Mn = fmaxf(M, mr);
+      const float alpha = M == -INFINITY ? 0.f : exp2f(M - Mn);
+      const float e = exp2f(mr - Mn);
+      L = fmaf(L, alpha, e * rec[1]); P0 = fmaf(P0, alpha, e * rec[2]); P1 = fmaf(P1, alpha, e * rec[3]);
 #pragma unroll
-  for (int s = 16; s; s >>= 1) {
-    L += __shfl_xor_sync(0xffffffffu, L, s);
-    P0 += __shfl_xor_sync(0xffffffffu, P0, s);
-    P1 += __shfl_xor_sync(0xffffffffu, P1, s);
-  }
-  if (lane == 0) { s_red[1][warp] = L; s_red[2][warp] = P0; s_red[3][warp] = P1; }
-  s_o[tid] = 0.f;
-  __syncthreads();
-  L = s_red[1][0] + s_red[1][1] + s_red[1][2] + s_red[1][3];
-  P0 = s_red[2][0] + s_red[2][1] + s_red[2][2] + s_red[2][3];
-  P1 = s_red[3][0] + s_red[3][1] + s_red[3][2] + s_red[3][3];
-  // ---- per-strip sums: warp w takes records w, w + 4, ..; lanes take strips lane, lane + 32, ..
-  const int ns = D.n_vstrips;
-  constexpr int kPerLane = kMaxStrips / 32;
-  float acc[kPerLane];
-#pragma unroll
-  for (int i = 0; i < kPerLane; i++) acc[i] = 0.f;
-  for (int r = warp; r < nrec; r += 4) {
-    float e;
-    if (r < kMaxRecSmem) e = s_e[r];
-    else { e = 0.f; if (nonempty(r)) { const float mr = rec_ptr(r)[0]; e = mr == -INFINITY ? 0.f : exp2f(mr - M); } }
-    if (e == 0.f) continue;
-    const float* rec = rec_ptr(r) + kRecHead;
-#pragma unroll
-    for (int i = 0; i < kPerLane; i++) {
-      const int k = lane + 32 * i;
-      if (k < ns) acc[i] = fmaf(e, rec[k], acc[i]);
+      for (int q = 0; q < kPerThread; q++)
+        acc[q] = fmaf(acc[q], alpha, tid + 128 * q < ns ? e * rec[kRecHead + tid + 128 * q] : 0.f);
+      M = Mn;
     }
   }
+  // strips of one class belong to distinct channels: adding class by class needs no atomics and has a fixed order
+#pragma unroll 1
+  for (int c = 0; c < 4; c++) {
 #pragma unroll
-  for (int i = 0; i < kPerLane; i++) s_part[warp][lane + 32 * i] = acc[i];
-  __syncthreads();
-  for (int k = tid; k < ns; k += 128) {
-    const float v = s_part[0][k] + s_part[1][k] + s_part[2][k] + s_part[3][k];
-    atomicAdd(&s_o[D.vchan[k]], v * D.vcoef[k]);
+    for (int q = 0; q < kPerThread; q++) {
+      const int k = tid + 128 * q;
+      if (k < ns && (k >= vf1) + (k >= vf2) + (k >= vf3) == c) s_o[chan[q]] += acc[q] * coef[q];
+    }
+    __syncthreads();
   }
-  __syncthreads();
   // ---- normalise, add the group offsets and the rotated mean, lift
   const bool live = L > 0.f;
-  float v = 0.f;
+  float val = 0.f;
   if (live) {
-    v = s_o[tid];
-    if (p.widths_v[(int64_t)ps * kD + tid]) v += tid < 64 ? P0 : P1;
-    v = v / L + p.mean_rot_v[(int64_t)ps * kD + tid];
+    val = s_o[tid];
+    if (has_width) val += tid < 64 ? P0 : P1;
+    val = val / L + mean_rot;
   }
   __syncthreads();
-  s_o[tid] = v;
+  s_o[tid] = val;
   __syncthreads();
-  const float* wv = p.w_dec_v + (int64_t)ps * kD * kD;
+  const bool ok = mbar_wait(wbar, 0);
+  if (!ok && tid == 0 && p.status) atomicOr(p.status, SPECTRA_STATUS_WAIT_TIMEOUT);
   float o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
-#pragma unroll 8
+#pragma unroll 4
   for (int j = 0; j < kD; j += 4) {
-    o0 = fmaf(s_o[j], wv[j * kD + tid], o0);
-    o1 = fmaf(s_o[j + 1], wv[(j + 1) * kD + tid], o1);
-    o2 = fmaf(s_o[j + 2], wv[(j + 2) * kD + tid], o2);
-    o3 = fmaf(s_o[j + 3], wv[(j + 3) * kD + tid], o3);
+    o0 = fmaf(s_o[j], s_w[j * kD + tid], o0);
+    o1 = fmaf(s_o[j + 1], s_w[(j + 1) * kD + tid], o1);
+    o2 = fmaf(s_o[j + 2], s_w[(j + 2) * kD + tid], o2);
+    o3 = fmaf(s_o[j + 3], s_w[(j + 3) * kD + tid], o3);
   }
-  store_from_float(p.out, p.out_dtype, oidx, live ? (o0 + o1) + (o2 + o3) : 0.f);
+  store_from_float(p.out, p.out_dtype, oidx, live && ok ? (o0 + o1) + (o2 + o3) : 0.f);
   if (p.lse && tid == 0)
-    p.lse[hidx] = live ? (M + log2f(L)) / kLog2e + D.qconst[h] : -INFINITY;
+    p.lse[hidx] = live ? (M + log2f(L)) / kLog2e + qconst : -INFINITY;
 }
 
 }  // namespace spectra

@@ -63,6 +63,19 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// L2 policy for data that is read once (the coded tiles): first in line for eviction, so that the stream does not
+// push out what the other kernels of the step re-read (parameters, descriptors, partial records).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)
@@ -346,7 +359,7 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
 }
 
 // First launch of a fused decode step: the prep grid, then one CTA per unit-side that appends the new token
-// (threads 0..127 of it; the K side first).  The main kernel that follows reads what both parts wrote.
+// (the K side first).  The main kernel that follows reads what both parts wrote.
 __global__ void __launch_bounds__(kPrepThreads, 2) decode_step_front_kernel(AttnArgs p, FastArgs f, AppendArgs ak,
                                                                          AppendArgs av, int n_cache_units) {
   const int n_prep = f.n_units + 1;
@@ -354,11 +367,7 @@ __global__ void __launch_bounds__(kPrepThreads, 2) decode_step_front_kernel(Attn
   const int i = blockIdx.x - n_prep;
   const AppendArgs& a = i < n_cache_units ? ak : av;
   const int u = i < n_cache_units ? i : i - n_cache_units;
-  // all 512 threads ask the L2 for the unit's W_enc (one line each) before the 128 workers start their chain
-  if (!(a.flags & SPECTRA_ROTATED_INPUT))
-    prefetch_l2(a.w_enc + (int64_t)(u % a.n_param_sets) * kD * kD + threadIdx.x * 32);
-  if (threadIdx.x >= 128) return;
-  encode_append_body(a, u);
+  encode_append_body<kPrepThreads / 128>(a, u);
 }
 
 }  // namespace spectra

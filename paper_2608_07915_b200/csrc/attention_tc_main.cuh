@@ -284,14 +284,15 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
     const uint32_t tbk = d.tbk, tbv = d.tbv;
     mbar_expect_tx(bars + 8 * slot, tbk);
     bulk_load(smem_u32(ring_k + slot * f.slot_k), p.cache_k + p.off_k[prod.u / f.npass] + (int64_t)prod.t * tbk, tbk,
-              bars + 8 * slot);
+              bars + 8 * slot, l2_evict_first_policy());
     v_src = p.cache_v + p.off_v[prod.u / f.npass] + (int64_t)prod.t * tbv;
     v_bytes = tbv;
     prod.next(f);
   };
   auto start_v = [&](int slot) {
     mbar_expect_tx(bars + 8 * (4 + slot), v_bytes);
-    bulk_load(smem_u32(ring_v + slot * f.slot_v), v_src, v_bytes, bars + 8 * (4 + slot));
+    bulk_load(smem_u32(ring_v + slot * f.slot_v), v_src, v_bytes, bars + 8 * (4 + slot),
+              l2_evict_first_policy());
   };
   if (lane == 0)
     for (int j = 0; j < min(D, count); j++) { start_k(j); start_v(j); }

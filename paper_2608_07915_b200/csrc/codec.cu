@@ -46,7 +46,7 @@ __device__ inline void tile_product(const float* __restrict__ a, const float* __
   }
 }
 
-__global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) { encode_append_body(p, blockIdx.x); }
+__global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) { encode_append_body<1>(p, blockIdx.x); }
 
 struct EncodeArgs {
   const void* x; int x_dtype; int flags; int side; int scale_group;

@@ -18,77 +18,98 @@ struct AppendArgs {
   const int32_t* seq_len; int n_kv;      // with pos0 == NULL: the token goes to position seq_len[u / n_kv] - 1
 };
 
-// The work of one CTA (threads 0..127 of it) for unit-side u.
+// The work of one CTA of 128 * NQ threads for unit-side u.  Threads 0..127 (group 0) are the workers, thread j =
+// rotated channel j.  With NQ > 1 the other groups only help with the rotation: group q holds rows
+// [q * 128 / NQ, (q + 1) * 128 / NQ) of the thread's column of W_enc in registers (all loads of the CTA in flight at
+// once) and the FMA chain is handed from group to group through shared memory, so the sum keeps its order
+// (ascending i, one chain) whatever NQ is.
+template <int NQ>
 __device__ inline void encode_append_body(const AppendArgs& p, int u) {
+  constexpr int kRows = kD / NQ;
   __shared__ float xs[kAppendMaxTokens][kD];
+  __shared__ float part[kD];
   __shared__ float red_lo[4], red_hi[4];
   __shared__ int cls_cnt[4][4];          // [class][warp]: strips of the class owned by the warp's channels
   __shared__ int grp_act[kMaxGroups];
   const int ps = (int)(u % p.n_param_sets);
-  const int j = threadIdx.x, lane = j & 31, warp = j >> 5;
+  const int q = threadIdx.x >> 7, j = threadIdx.x & 127, lane = j & 31, warp = j >> 5;
   const int gs = p.scale_group, n_groups = kD / gs;
-  const int b = p.widths[(int64_t)ps * kD + j];
   const bool rotated = (p.flags & SPECTRA_ROTATED_INPUT) != 0;
-  // ---- stage the new tokens (these loads, the width and the position are in flight together)
+  auto worker_sync = [] {                 // barrier among the 128 workers only
+    if constexpr (NQ == 1) __syncthreads();
+    else asm volatile("bar.sync 1, 128;" ::: "memory");
+  };
+  // ---- everything the CTA reads before it writes is requested here: width, position, new tokens, W_enc
+  const int b = p.widths[(int64_t)ps * kD + j];
   const int pos_first = p.pos0 ? p.pos0[u] : p.seq_len[u / p.n_kv] - 1;
-  for (int idx = j; idx < p.n_new * kD; idx += 128) {
+  for (int idx = threadIdx.x; idx < p.n_new * kD; idx += 128 * NQ) {
     const int t = idx / kD, i = idx - t * kD;
     xs[t][i] = load_as_float(p.x, p.x_dtype, (int64_t)u * p.stride_unit + (int64_t)t * p.stride_token + i);
   }
-
-  // ---- where this channel's strips live: rank inside each class, class offsets, tile size
-  if (j < kMaxGroups) grp_act[j] = 0;
+  float wreg[kRows];
+  if (!rotated) {
+    const float* w = p.w_enc + (int64_t)ps * kD * kD + (int64_t)q * kRows * kD + j;
+#pragma unroll
+    for (int i = 0; i < kRows; i++) wreg[i] = __ldg(w + i * kD);
+  }
+  if (q == 0 && j < kMaxGroups) grp_act[j] = 0;
   __syncthreads();
-  int rank_in_warp[4];
-#pragma unroll
-  for (int c = 0; c < 4; c++) {
-    const unsigned m = __ballot_sync(0xffffffffu, (b & (8 >> c)) != 0);
-    rank_in_warp[c] = __popc(m & ((1u << lane) - 1u));
-    if (lane == 0) cls_cnt[c][warp] = __popc(m);
-  }
-  if (b) grp_act[j / gs] = 1;
-  __syncthreads();
-  int cls_n[4], cls_off[4], my_rank[4];
-  int off = 0;
-#pragma unroll
-  for (int c = 0; c < 4; c++) {
-    int before = 0, n = 0;
-#pragma unroll
-    for (int w = 0; w < 4; w++) { if (w < warp) before += cls_cnt[c][w]; n += cls_cnt[c][w]; }
-    cls_n[c] = n; cls_off[c] = off; my_rank[c] = before + rank_in_warp[c];
-    off += 16 * (8 >> c) * n;
-  }
-  const int payload = off;
-  int meta_off = -1, n_act = 0;
-  for (int g = 0; g < n_groups; g++) {
-    if (g == j / gs && grp_act[g]) meta_off = payload + 512 * n_act;
-    n_act += grp_act[g];
-  }
-  const int tile_bytes = payload + 512 * n_act;
-
   if (pos_first < 0) return;                 // fused step on an empty sequence: nothing to append (CTA-uniform)
-  const float* w = p.w_enc + (int64_t)ps * kD * kD;
-  const float mr = rotated ? 0.f : p.mean_rot[(int64_t)ps * kD + j];
-  uint8_t* base = p.cache + p.unit_offset[u];
+
+  // ---- where this channel's strips live: rank inside each class, class offsets, tile size (workers)
+  int cls_n[4], cls_off[4], my_rank[4];
+  int meta_off = -1, tile_bytes = 0;
+  if (q == 0) {
+    int rank_in_warp[4];
+#pragma unroll
+    for (int c = 0; c < 4; c++) {
+      const unsigned m = __ballot_sync(0xffffffffu, (b & (8 >> c)) != 0);
+      rank_in_warp[c] = __popc(m & ((1u << lane) - 1u));
+      if (lane == 0) cls_cnt[c][warp] = __popc(m);
+    }
+    if (b) grp_act[j / gs] = 1;
+    worker_sync();
+    int off = 0;
+#pragma unroll
+    for (int c = 0; c < 4; c++) {
+      int before = 0, n = 0;
+#pragma unroll
+      for (int w = 0; w < 4; w++) { if (w < warp) before += cls_cnt[c][w]; n += cls_cnt[c][w]; }
+      cls_n[c] = n; cls_off[c] = off; my_rank[c] = before + rank_in_warp[c];
+      off += 16 * (8 >> c) * n;
+    }
+    const int payload = off;
+    int n_act = 0;
+    for (int g = 0; g < n_groups; g++) {
+      if (g == j / gs && grp_act[g]) meta_off = payload + 512 * n_act;
+      n_act += grp_act[g];
+    }
+    tile_bytes = payload + 512 * n_act;
+  }
+  const float mr = (rotated || q) ? 0.f : p.mean_rot[(int64_t)ps * kD + j];
+  uint8_t* base = q ? nullptr : p.cache + p.unit_offset[u];
   int status = 0;
 
   for (int t = 0; t < p.n_new; t++) {
     // rotate + centre: y_j = sum_i x_i W_enc[i][j] - m'_j (fp32 FMA chain in ascending i)
-    float y;
+    float y = 0.f;
     if (rotated) y = xs[t][j];
     else {
-      // all 128 loads of the column are issued before the FMA chain consumes them (latency-bound otherwise)
-      float wcol[kD / 4];
-      float a0 = 0.f;
 #pragma unroll
-      for (int blk = 0; blk < 4; blk++) {
+      for (int qq = 0; qq < NQ; qq++) {
+        if (q == qq) {
+          float a = qq ? part[j] : 0.f;
 #pragma unroll
-        for (int i = 0; i < kD / 4; i++) wcol[i] = __ldg(w + (blk * (kD / 4) + i) * kD + j);
-#pragma unroll
-        for (int i = 0; i < kD / 4; i++) a0 = fmaf(xs[t][blk * (kD / 4) + i], wcol[i], a0);
+          for (int i = 0; i < kRows; i++) a = fmaf(xs[t][qq * kRows + i], wreg[i], a);
+          if constexpr (NQ > 1) part[j] = a;
+          else y = a;
+        }
+        if constexpr (NQ > 1) __syncthreads();
       }
-      y = __fsub_rn(a0, mr);
+      if constexpr (NQ > 1) y = part[j];
+      y = __fsub_rn(y, mr);
     }
+    if (q) continue;                         // helpers are done with this token
     if (b && !isfinite(y)) status |= SPECTRA_STATUS_NONFINITE;
     // per-group minimum and maximum over the channels with a non-zero width
     float lo = b ? y : INFINITY, hi = b ? y : -INFINITY;
@@ -97,9 +118,9 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
       lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, s));
       hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, s));
     }
-    __syncthreads();
+    worker_sync();
     if (lane == 0) { red_lo[warp] = lo; red_hi[warp] = hi; }
-    __syncthreads();
+    worker_sync();
     if (gs > 32) {
       const int w0 = (j / gs) * (gs / 32);
       lo = red_lo[w0]; hi = red_hi[w0];
@@ -133,7 +154,7 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
     uint8_t* tile = base + (int64_t)(pos / kTile) * tile_bytes;
     if (slot == 0) {                                          // first token of a tile: clear the tile
       for (int i = j; i < tile_bytes / 16; i += 128) reinterpret_cast<uint4*>(tile)[i] = make_uint4(0, 0, 0, 0);
-      __syncthreads();
+      worker_sync();
     }
 #pragma unroll
     for (int c = 0; c < 4; c++) {
@@ -163,7 +184,7 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
       m[0] = __half_as_ushort(lo16);
       m[kTile] = __half_as_ushort(r16);
     }
-    __syncthreads();
+    worker_sync();
   }
   if (status && p.status) atomicOr(p.status, status);
 }
