@@ -172,8 +172,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
   const int npass = (gqa + kFastGqa - 1) / kFastGqa;
   const int64_t n_vunits = n_units * npass;
   // (its kernels fetch whole parameter matrices with bulk copies, which need 16-byte aligned sources)
-  const bool aligned = (((uintptr_t)w_dec_k | (uintptr_t)w_dec_v | (uintptr_t)(app ? app->w_enc_k : nullptr) |
-                         (uintptr_t)(app ? app->w_enc_v : nullptr)) & 15) == 0;
+  const bool aligned = (((uintptr_t)w_dec_k | (uintptr_t)w_dec_v) & 15) == 0;
   if (widths_k_host && cfg->scale_group == 64 && n_vunits <= 65534 && aligned) {
     const WidthFacts F = width_facts(widths_k_host, widths_v_host, n_param_sets);
     if (!F.ok) return SPECTRA_INVALID_ARG;
@@ -199,15 +198,20 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
       f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = vs_max;
       f.n_units = (int)n_vunits; f.npass = npass; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
+      if (cudaFuncSetAttribute(decode_step_front_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepDynSmem) !=
+              cudaSuccess ||
+          cudaFuncSetAttribute(attention_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepDynSmem) !=
+              cudaSuccess)
+        return SPECTRA_CUDA_ERROR;
       if (app) {
         AppendArgs ak{app->new_k, app->x_dtype, 0, SPECTRA_SIDE_K, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
                       app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, status_word, seq_len, n_kv_heads};
         AppendArgs av{app->new_v, app->x_dtype, 0, SPECTRA_SIDE_V, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
                       app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, status_word, seq_len, n_kv_heads};
-        decode_step_front_kernel<<<(unsigned)(n_vunits + 1 + 2 * n_units), kPrepThreads, sizeof(PrepSmem), st>>>(
+        decode_step_front_kernel<<<(unsigned)(n_vunits + 1 + 2 * n_units), kPrepThreads, kPrepDynSmem, st>>>(
             a, f, ak, av, (int)n_units);
       } else {
-        attention_prep_kernel<<<(unsigned)n_vunits + 1, kPrepThreads, sizeof(PrepSmem), st>>>(a, f);
+        attention_prep_kernel<<<(unsigned)n_vunits + 1, kPrepThreads, kPrepDynSmem, st>>>(a, f);
       }
       if (launch_status()) return SPECTRA_CUDA_ERROR;
       const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64;

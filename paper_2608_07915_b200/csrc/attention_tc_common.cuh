@@ -141,17 +141,23 @@ __device__ __forceinline__ float2 h2f2(uint32_t x) {
 }
 
 // ------------------------------------------------------------------------------------------------ prep kernel
+// These CTAs run once per call, on a cold instruction cache and with every global read paying a full memory latency.
+// So: one round of reads (W_dec,K by a bulk copy into shared memory; query, widths, rotated mean by plain loads
+// issued together), rolled loops, all 512 threads in every phase.
 struct PrepSmem {
   StripTable tk, tv;
   alignas(16) float qraw[kFastGqa][kD];
   alignas(16) float qrot[kFastGqa][kD];
+  float mrot[kD];
+  float kcoef[kMaxStrips];        // 2^shift / (2^width - 1) of K strip k
   __half bhi[kFastGqa][kMaxStrips];
   __half blo[kFastGqa][kMaxStrips];
-  float red[kFastGqa][4];
-  int escale[kFastGqa];
+  float red[4][kFastGqa][4];      // [quantity: max, q0, q1, qc][head][warp of the head's 128 threads]
   int scan[128];
-  int ng0[2][4];      // strips of scale group 0 per class: [K, V][class]
+  int ng0[2][4];                  // strips of scale group 0 per class: [K, V][class]
+  alignas(8) unsigned long long wbar;
 };
+constexpr int kPrepDynSmem = kD * kD * 4 + (int)sizeof(PrepSmem);   // W_dec,K (or W_enc of an append CTA) first
 
 __device__ inline uint32_t pack_cls(const StripTable& T, int c, int n_g0) {
   const int first = T.class_first[c], n = T.class_first[c + 1] - first;
@@ -172,7 +178,8 @@ constexpr int kPrepThreads = 512;
 // The work of CTA `bid` of the prep grid (f.n_units unit CTAs, then one CTA for the prefix sums).
 __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f, int bid) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  PrepSmem& S = *reinterpret_cast<PrepSmem*>(smem_raw);
+  float* s_w = reinterpret_cast<float*>(smem_raw);
+  PrepSmem& S = *reinterpret_cast<PrepSmem*>(smem_raw + kD * kD * 4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int kWarps = kPrepThreads / 32;
   if (bid == f.n_units) {
@@ -223,134 +230,163 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
   const int G = min(kFastGqa, p.gqa - h0);                          // query heads of this pass
-  // The CTA's work is a chain of dependent phases; what the later phases read is asked for now (one line per thread).
-  prefetch_l2(p.w_dec_k + (int64_t)ps * kD * kD + tid * 32);
-  if (tid < 4 && p.mean_rot_k) prefetch_l2(p.mean_rot_k + (int64_t)ps * kD + tid * 32);
-  for (int idx = tid; idx < kFastGqa * kD; idx += kPrepThreads) {
-    const int h = idx / kD, i = idx - h * kD;
+  // ---- the one round of reads
+  const uint32_t wbar = smem_u32(&S.wbar);
+  if (tid == 0) {
+    mbar_init(wbar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_expect_tx(wbar, kD * kD * 4);
+    bulk_load(smem_u32(s_w), p.w_dec_k + (int64_t)ps * kD * kD, kD * kD * 4, wbar);
+  }
+  {
+    const int h = tid >> 7, i = tid & (kD - 1);                     // 512 threads = 4 heads x 128 channels
     S.qraw[h][i] = h < G ? load_as_float(p.q, p.q_dtype, ((int64_t)b * p.n_q + hk * p.gqa + h0 + h) * kD + i) : 0.f;
+    if (tid < kD) S.mrot[tid] = p.mean_rot_k ? p.mean_rot_k[(int64_t)ps * kD + tid] : 0.f;
   }
   build_strip_tables(S.tk, p.widths_k + (int64_t)ps * kD, S.tv, p.widths_v + (int64_t)ps * kD, 64);
   const StripTable& TK = S.tk;
   const StripTable& TV = S.tv;
   UnitDesc& D = f.desc[vu];
-  const float* wk = p.w_dec_k + (int64_t)ps * kD * kD;
-  {
-    float4 wrow[kD / kWarps];
-#pragma unroll
-    for (int r = 0; r < kD / kWarps; r++)          // all row loads of this warp in flight together
-      wrow[r] = *reinterpret_cast<const float4*>(wk + (warp + kWarps * r) * kD + lane * 4);
-#pragma unroll
-    for (int r = 0; r < kD / kWarps; r++) {
-#pragma unroll
-      for (int h = 0; h < kFastGqa; h++) {
-        const float4 qv = *reinterpret_cast<const float4*>(&S.qraw[h][lane * 4]);
-        float acc = wrow[r].x * qv.x + wrow[r].y * qv.y + wrow[r].z * qv.z + wrow[r].w * qv.w;
-#pragma unroll
-        for (int s = 16; s; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-        if (lane == 0) S.qrot[h][warp + kWarps * r] = acc * p.scale * kLog2e;   // scores live in the log2 domain
-      }
-    }
-  }
-  if (warp >= 8) {                                  // meanwhile: group-0 strip counts per class (warps 8..15)
+  const int nk = TK.n_strips;
+  // ---- what depends on the widths only: strip coefficients, group-0 counts, the V side of the descriptor
+  for (int k = tid; k < nk; k += kPrepThreads)
+    S.kcoef[k] = (float)(1 << TK.shift[k]) / (float)((1 << TK.width[TK.chan[k]]) - 1);
+  if (warp >= 8) {
     const int side = (warp - 8) >> 2, c = (warp - 8) & 3;
     const int cnt = count_group0(side ? TV : TK, c, lane);
     if (lane == 0) S.ng0[side][c] = cnt;
-  }
-  __syncthreads();
-  // per-head power-of-two normalisation so that the fp16 hi/lo split of q'' = q' 2^shift / L is well conditioned
-  const int nk = TK.n_strips;
-  if (warp < kFastGqa) {
-    const int h = warp;  // one warp per head
-    float mx = 0.f;
-    for (int k = lane; k < nk; k += 32) {
-      const int c = TK.chan[k];
-      mx = fmaxf(mx, fabsf(S.qrot[h][c] * (float)(1 << TK.shift[k]) / (float)((1 << TK.width[c]) - 1)));
-    }
-#pragma unroll
-    for (int s = 16; s; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
-    int e = 0;
-    if (mx > 0.f && isfinite(mx)) { int ex; frexpf(mx, &ex); e = 10 - ex; }
-    e = max(-100, min(100, e));
-    if (lane == 0) { S.escale[h] = e; D.kscale[h] = ldexpf(1.f, 24 - e); }
-    for (int k = lane; k < nk; k += 32) {
-      const int c = TK.chan[k];
-      const float v = ldexpf(S.qrot[h][c] * (float)(1 << TK.shift[k]) / (float)((1 << TK.width[c]) - 1), e);
-      const __half hi = __float2half_rn(v);
-      const __half lo = __float2half_rn(v - __half2float(hi));
-      S.bhi[h][k] = hi; S.blo[h][k] = lo;
-    }
-    float q0 = 0.f, q1 = 0.f, qc = 0.f;
-    for (int j = lane; j < kD; j += 32) {
-      const float v = S.qrot[h][j];
-      if (TK.width[j]) { if (j < 64) q0 += v; else q1 += v; }
-      if (p.mean_rot_k) qc += v * p.mean_rot_k[(int64_t)ps * kD + j];
-    }
-#pragma unroll
-    for (int s = 16; s; s >>= 1) {
-      q0 += __shfl_xor_sync(0xffffffffu, q0, s); q1 += __shfl_xor_sync(0xffffffffu, q1, s);
-      qc += __shfl_xor_sync(0xffffffffu, qc, s);
-    }
-    if (lane == 0) {
-      D.qlo[h][0] = q0; D.qlo[h][1] = q1;
-      D.qconst[h] = qc / kLog2e;
-    }
-  }
-  __syncthreads();
-  // B fragments.  A class is walked in chunks of 16 consecutive strips; the strips of scale group 0 come first, so
-  // at most one chunk per class holds strips of both groups: it gets two entries, one per group.  An entry
-  // contributes to its scale group only (rows of the other group, or past the end, are zero).  Entries are stored
-  // chunk-major, group-minor: the order the main kernel walks them.  Column n = head (n >> 1), hi (n & 1 == 0) or
-  // lo half of the fp16 split.  Variant u carries the factor 2^-p_eff(u) of the unpacking.
-  int entry0 = 0;
-  for (int c = 0; c < 4; c++) {
-    const int first = TK.class_first[c], n = TK.class_first[c + 1] - first;
-    const int n_g0 = S.ng0[0][c];
-    const int nch = (n + 15) / 16;
-    const int b0 = n_g0 / 16;                                      // first chunk that holds a strip of group 1
-    const bool both = n > n_g0 && (n_g0 & 15) != 0;                // chunk b0 holds strips of both groups
-    const int n_entries = nch + (both ? 1 : 0);
-    const int w = 8 >> c;
-    for (int idx = tid; idx < n_entries * 4 * 32; idx += kPrepThreads) {
-      const int en = idx >> 7, u4 = (idx >> 5) & 3, ln = idx & 31;
-      int ch, run;                                                 // chunk and scale group of entry en
-      if (both) { ch = en <= b0 ? en : en - 1; run = en <= b0 ? 0 : 1; }
-      else { ch = en; run = 16 * en < n_g0 ? 0 : 1; }
-      const int start = 16 * ch;
-      const int gid = ln >> 2, tg = ln & 3, h = gid >> 1, part = gid & 1;
-      const int pe = w == 8 ? 0 : (w == 4 ? 4 * (u4 & 1) : (w == 2 ? 2 * u4 : u4));
-      const __half scale = __ushort_as_half((unsigned short)((15 - pe) << 10));
-      uint32_t r[2];
-#pragma unroll
-      for (int half = 0; half < 2; half++) {
-        uint32_t v = 0;
-#pragma unroll
-        for (int e = 0; e < 2; e++) {
-          const int strip = start + 2 * tg + 8 * half + e;
-          uint16_t bits = 0;
-          if (strip < n && h < G && (strip >= n_g0 ? 1 : 0) == run)
-            bits = __half_as_ushort(__hmul(part ? S.blo[h][first + strip] : S.bhi[h][first + strip], scale));
-          v |= (uint32_t)bits << (16 * e);
-        }
-        r[half] = v;
-      }
-      if (entry0 + en < kKcMax) D.kB[entry0 + en][u4][ln] = make_uint2(r[0], r[1]);
-    }
-    entry0 += n_entries;
-  }
-  if (tid >= 64 && tid < 68) D.kcls[tid - 64] = pack_cls(TK, tid - 64, S.ng0[0][tid - 64]);
-  if (tid >= 96 && tid < 100) D.vcls[tid - 96] = pack_cls(TV, tid - 96, S.ng0[1][tid - 96]);
-  if (tid >= 128 && tid < 132) D.vfirst[tid - 128] = TV.class_first[tid - 128];
-  if (tid == 0) {
-    D.tbk = TK.tile_bytes; D.tbv = TV.tile_bytes;
-    D.kmeta[0] = TK.meta_off[0]; D.kmeta[1] = TK.meta_off[1];
-    D.vmeta[0] = TV.meta_off[0]; D.vmeta[1] = TV.meta_off[1];
-    D.n_vstrips = TV.n_strips; D.pad0 = 0;
   }
   for (int k = tid; k < TV.n_strips; k += kPrepThreads) {
     const int c = TV.chan[k];
     D.vchan[k] = (uint8_t)c;
     D.vcoef[k] = 16777216.f * (float)(1 << TV.shift[k]) / (float)((1 << TV.width[c]) - 1);
+  }
+  // ---- q' = W_dec,K q (times the softmax scale, in the log2 domain).  A warp takes rows warp, warp + 16, .., two at
+  // a time: each lane multiplies its four columns of the rows with the four heads, and a transposing butterfly leaves
+  // every (row, head) sum in one lane after 9 shuffles instead of 40.
+  const bool landed = mbar_wait(wbar, 0);
+  if (!landed && tid == 0 && p.status) atomicOr(p.status, SPECTRA_STATUS_WAIT_TIMEOUT);
+  {
+    float4 qv[kFastGqa];
+#pragma unroll
+    for (int h = 0; h < kFastGqa; h++) qv[h] = *reinterpret_cast<const float4*>(&S.qraw[h][lane * 4]);
+    const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0, up4 = (lane & 4) != 0;
+    const float out_scale = landed ? p.scale * kLog2e : 0.f;
+#pragma unroll 1
+    for (int row = warp; row < kD; row += 2 * kWarps) {
+      const float4 wa = *reinterpret_cast<const float4*>(s_w + row * kD + lane * 4);
+      const float4 wb = *reinterpret_cast<const float4*>(s_w + (row + kWarps) * kD + lane * 4);
+      float pa[kFastGqa], pb[kFastGqa];
+#pragma unroll
+      for (int h = 0; h < kFastGqa; h++) {
+        pa[h] = wa.x * qv[h].x + wa.y * qv[h].y + wa.z * qv[h].z + wa.w * qv[h].w;
+        pb[h] = wb.x * qv[h].x + wb.y * qv[h].y + wb.z * qv[h].z + wb.w * qv[h].w;
+      }
+      // step 16 keeps heads {2 up16, 2 up16 + 1} of both rows, step 8 one head, step 4 one row
+      const float a0 = (up16 ? pa[2] : pa[0]) + __shfl_xor_sync(0xffffffffu, up16 ? pa[0] : pa[2], 16);
+      const float a1 = (up16 ? pa[3] : pa[1]) + __shfl_xor_sync(0xffffffffu, up16 ? pa[1] : pa[3], 16);
+      const float b0 = (up16 ? pb[2] : pb[0]) + __shfl_xor_sync(0xffffffffu, up16 ? pb[0] : pb[2], 16);
+      const float b1 = (up16 ? pb[3] : pb[1]) + __shfl_xor_sync(0xffffffffu, up16 ? pb[1] : pb[3], 16);
+      const float ah = (up8 ? a1 : a0) + __shfl_xor_sync(0xffffffffu, up8 ? a0 : a1, 8);
+      const float bh = (up8 ? b1 : b0) + __shfl_xor_sync(0xffffffffu, up8 ? b0 : b1, 8);
+      float k = (up4 ? bh : ah) + __shfl_xor_sync(0xffffffffu, up4 ? ah : bh, 4);
+      k += __shfl_xor_sync(0xffffffffu, k, 2);
+      k += __shfl_xor_sync(0xffffffffu, k, 1);
+      if ((lane & 3) == 0) S.qrot[2 * (int)up16 + (int)up8][row + (up4 ? kWarps : 0)] = k * out_scale;
+    }
+  }
+  __syncthreads();
+  // ---- per-head reductions, thread = (head, channel): largest |q' coef| over the strips (for the power-of-two
+  // normalisation of the fp16 hi/lo split), sums of q' per scale group, q' . m'_K
+  const int hh = tid >> 7, jj = tid & (kD - 1), wq = (tid >> 5) & 3;
+  {
+    float mx = 0.f;
+    for (int k = jj; k < nk; k += kD) mx = fmaxf(mx, fabsf(S.qrot[hh][TK.chan[k]] * S.kcoef[k]));
+    const float v = S.qrot[hh][jj];
+    float q0 = (TK.width[jj] && jj < 64) ? v : 0.f, q1 = (TK.width[jj] && jj >= 64) ? v : 0.f, qc = v * S.mrot[jj];
+#pragma unroll
+    for (int s = 16; s; s >>= 1) {
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+      q0 += __shfl_xor_sync(0xffffffffu, q0, s); q1 += __shfl_xor_sync(0xffffffffu, q1, s);
+      qc += __shfl_xor_sync(0xffffffffu, qc, s);
+    }
+    if (lane == 0) { S.red[0][hh][wq] = mx; S.red[1][hh][wq] = q0; S.red[2][hh][wq] = q1; S.red[3][hh][wq] = qc; }
+  }
+  __syncthreads();
+  {
+    const float mx = fmaxf(fmaxf(S.red[0][hh][0], S.red[0][hh][1]), fmaxf(S.red[0][hh][2], S.red[0][hh][3]));
+    int e = 0;
+    if (mx > 0.f && mx <= 3.4028234e38f) e = 10 - ((int)((__float_as_uint(mx) >> 23) & 0xffu) - 126);   // mx = m 2^ex, m in [0.5, 1)
+    e = max(-100, min(100, e));
+    const float pow2e = __uint_as_float((uint32_t)(e + 127) << 23);
+    if (jj == 0) {
+      D.kscale[hh] = __uint_as_float((uint32_t)(24 - e + 127) << 23);
+      D.qlo[hh][0] = (S.red[1][hh][0] + S.red[1][hh][1]) + (S.red[1][hh][2] + S.red[1][hh][3]);
+      D.qlo[hh][1] = (S.red[2][hh][0] + S.red[2][hh][1]) + (S.red[2][hh][2] + S.red[2][hh][3]);
+      D.qconst[hh] = ((S.red[3][hh][0] + S.red[3][hh][1]) + (S.red[3][hh][2] + S.red[3][hh][3])) / kLog2e;
+    }
+    for (int k = jj; k < nk; k += kD) {
+      const float v = S.qrot[hh][TK.chan[k]] * S.kcoef[k] * pow2e;
+      const __half hi = __float2half_rn(v);
+      S.bhi[hh][k] = hi;
+      S.blo[hh][k] = __float2half_rn(v - __half2float(hi));
+    }
+  }
+  __syncthreads();
+  // ---- B fragments.  An entry contributes to its scale group only (rows of the other group, or past the end of the
+  // class, are zero).  Column n = head (n >> 1), hi (n & 1 == 0) or lo half of the fp16 split.  Variant u carries
+  // the factor 2^-p_eff(u) of the unpacking.
+  // Entries: a class is walked in chunks of 16 consecutive strips; the strips of scale group 0 come first, so at most
+  // one chunk per class holds strips of both groups: it gets two entries, one per group.  Entries are stored
+  // chunk-major, group-minor: the order the main kernel walks them.
+  int ent_base[5];
+  ent_base[0] = 0;
+#pragma unroll
+  for (int c = 0; c < 4; c++) {
+    const int n = TK.class_first[c + 1] - TK.class_first[c], n_g0 = S.ng0[0][c];
+    ent_base[c + 1] = ent_base[c] + (n + 15) / 16 + ((n > n_g0 && (n_g0 & 15) != 0) ? 1 : 0);
+  }
+  const int n_entries = min(ent_base[4], kKcMax);
+#pragma unroll 1
+  for (int idx = tid; idx < n_entries * 4 * 32; idx += kPrepThreads) {
+    const int en = idx >> 7, u4 = (idx >> 5) & 3, ln = idx & 31;
+    const int c = (en >= ent_base[1]) + (en >= ent_base[2]) + (en >= ent_base[3]);
+    const int first = TK.class_first[c], n = TK.class_first[c + 1] - first, n_g0 = S.ng0[0][c];
+    const int local = en - (c == 0 ? 0 : (c == 1 ? ent_base[1] : (c == 2 ? ent_base[2] : ent_base[3])));
+    const int b0 = n_g0 >> 4;                                        // first chunk that holds a strip of group 1
+    const bool both = n > n_g0 && (n_g0 & 15) != 0;                  // chunk b0 holds strips of both groups
+    const int ch = both && local > b0 ? local - 1 : local;
+    const int run = both ? (local <= b0 ? 0 : 1) : (16 * local < n_g0 ? 0 : 1);
+    const int start = 16 * ch;
+    const int gid = ln >> 2, tg = ln & 3, h = gid >> 1, part = gid & 1;
+    const int pe = c == 0 ? 0 : (c == 1 ? 4 * (u4 & 1) : (c == 2 ? 2 * u4 : u4));
+    const __half scale = __ushort_as_half((unsigned short)((15 - pe) << 10));
+    uint32_t r[2];
+#pragma unroll
+    for (int half = 0; half < 2; half++) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int e = 0; e < 2; e++) {
+        const int strip = start + 2 * tg + 8 * half + e;
+        uint16_t bits = 0;
+        if (strip < n && h < G && (strip >= n_g0 ? 1 : 0) == run)
+          bits = __half_as_ushort(__hmul(part ? S.blo[h][first + strip] : S.bhi[h][first + strip], scale));
+        v |= (uint32_t)bits << (16 * e);
+      }
+      r[half] = v;
+    }
+    D.kB[en][u4][ln] = make_uint2(r[0], r[1]);
+  }
+  if (tid < 4) {
+    D.kcls[tid] = pack_cls(TK, tid, S.ng0[0][tid]);
+    D.vcls[tid] = pack_cls(TV, tid, S.ng0[1][tid]);
+    D.vfirst[tid] = TV.class_first[tid];
+  }
+  if (tid == 32) {
+    D.tbk = TK.tile_bytes; D.tbv = TV.tile_bytes;
+    D.kmeta[0] = TK.meta_off[0]; D.kmeta[1] = TK.meta_off[1];
+    D.vmeta[0] = TV.meta_off[0]; D.vmeta[1] = TV.meta_off[1];
+    D.n_vstrips = TV.n_strips; D.pad0 = 0;
   }
 }
 
@@ -367,7 +403,8 @@ __global__ void __launch_bounds__(kPrepThreads, 2) decode_step_front_kernel(Attn
   const int i = blockIdx.x - n_prep;
   const AppendArgs& a = i < n_cache_units ? ak : av;
   const int u = i < n_cache_units ? i : i - n_cache_units;
-  encode_append_body<kPrepThreads / 128>(a, u);
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  encode_append_body(a, u, smem_raw);
 }
 
 }  // namespace spectra

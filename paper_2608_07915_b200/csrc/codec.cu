@@ -46,7 +46,10 @@ __device__ inline void tile_product(const float* __restrict__ a, const float* __
   }
 }
 
-__global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) { encode_append_body<1>(p, blockIdx.x); }
+__global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
+  extern __shared__ __align__(16) unsigned char append_smem[];
+  encode_append_body(p, blockIdx.x, append_smem);
+}
 
 struct EncodeArgs {
   const void* x; int x_dtype; int flags; int side; int scale_group;
@@ -420,7 +423,10 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
   if (n_new <= kAppendMaxTokens) {   // decode-step appends: one light CTA per unit-side
     AppendArgs ap{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
                   w_enc, mean_rot, widths, cache, unit_offset, status_word, nullptr, 1};
-    encode_append_kernel<<<(unsigned)n_units, 128, 0, (cudaStream_t)stream>>>(ap);
+    if (cudaFuncSetAttribute(encode_append_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAppendDynSmem) !=
+        cudaSuccess)
+      return SPECTRA_CUDA_ERROR;
+    encode_append_kernel<<<(unsigned)n_units, 128, kAppendDynSmem, (cudaStream_t)stream>>>(ap);
     return launch_status();
   }
   if (x_dtype == SPECTRA_BF16 && !(flags & SPECTRA_ROTATED_INPUT) && cfg->scale_group == 64 &&

@@ -92,15 +92,63 @@ __device__ inline void build_strip_table(StripTable& T, const uint8_t* __restric
   __syncthreads();
 }
 
-// Two tables at once (at least 256 threads): warp 0 scans the first, warp 1 the second.
+// Two tables at once, by the first eight warps of the CTA (at least 256 threads): warp (side, class) counts its class,
+// the counts are exchanged through shared memory, then every warp places the strips of its own class.  Same result as
+// strip_table_scan, a quarter of its dependent chain (for callers whose whole run is a few microseconds).
 __device__ inline void build_strip_tables(StripTable& A, const uint8_t* __restrict__ wa, StripTable& B,
                                           const uint8_t* __restrict__ wb, int scale_group) {
-  const int tid = threadIdx.x;
+  __shared__ int cnt[2][4];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid < kD) A.width[tid] = wa[tid];
   else if (tid < 2 * kD) B.width[tid - kD] = wb[tid - kD];
   __syncthreads();
-  if (tid < 32) strip_table_scan(A, scale_group, tid);
-  else if (tid < 64) strip_table_scan(B, scale_group, tid - 32);
+  const int side = warp >> 2, c = warp & 3, w = 8 >> c;
+  StripTable& T = side ? B : A;
+  unsigned m[kD / 32];
+  int bw[kD / 32];
+  if (warp < 8) {
+    int n = 0;
+#pragma unroll
+    for (int word = 0; word < kD / 32; word++) {
+      bw[word] = T.width[word * 32 + lane];
+      m[word] = __ballot_sync(0xffffffffu, (bw[word] & w) != 0);
+      n += __popc(m[word]);
+    }
+    if (lane == 0) cnt[side][c] = n;
+  }
+  __syncthreads();
+  if (warp < 8) {
+    int first = 0, off = 0;
+    for (int cc = 0; cc < c; cc++) { first += cnt[side][cc]; off += 16 * (8 >> cc) * cnt[side][cc]; }
+    if (lane == 0) { T.class_first[c] = first; T.class_off[c] = off; }
+    int k0 = first;
+#pragma unroll
+    for (int word = 0; word < kD / 32; word++) {
+      if ((bw[word] & w) != 0) {
+        const int k = k0 + __popc(m[word] & ((1u << lane) - 1u));
+        T.chan[k] = (uint8_t)(word * 32 + lane);
+        T.shift[k] = (uint8_t)(bw[word] & (w - 1));
+      }
+      k0 += __popc(m[word]);
+    }
+    if (c == 3) {                       // the last class also closes the table: totals and the metadata offsets
+      const int count = k0, payload = off + 16 * w * cnt[side][3];
+      const int n_groups = kD / scale_group;
+      int n_act = 0;
+      for (int g = 0; g < n_groups; g++) {
+        bool any = false;
+        for (int j = g * scale_group + lane; j < (g + 1) * scale_group; j += 32) any |= T.width[j] != 0;
+        const bool act = __any_sync(0xffffffffu, any);
+        if (lane == 0) T.meta_off[g] = act ? payload + 512 * n_act : -1;
+        n_act += act ? 1 : 0;
+      }
+      if (lane == 0) {
+        T.n_strips = count; T.class_first[4] = count; T.class_off[4] = payload;
+        T.n_groups = n_groups; T.n_act = n_act; T.tile_bytes = payload + 512 * n_act;
+        for (int g = n_groups; g < kMaxGroups; g++) T.meta_off[g] = -1;
+      }
+    }
+  }
   __syncthreads();
 }
 

@@ -18,48 +18,73 @@ struct AppendArgs {
   const int32_t* seq_len; int n_kv;      // with pos0 == NULL: the token goes to position seq_len[u / n_kv] - 1
 };
 
-// The work of one CTA of 128 * NQ threads for unit-side u.  Threads 0..127 (group 0) are the workers, thread j =
-// rotated channel j.  With NQ > 1 the other groups only help with the rotation: group q holds rows
-// [q * 128 / NQ, (q + 1) * 128 / NQ) of the thread's column of W_enc in registers (all loads of the CTA in flight at
-// once) and the FMA chain is handed from group to group through shared memory, so the sum keeps its order
-// (ascending i, one chain) whatever NQ is.
-template <int NQ>
-__device__ inline void encode_append_body(const AppendArgs& p, int u) {
-  constexpr int kRows = kD / NQ;
+// Bounded wait for phase 0 of an mbarrier (each poll blocks for a bounded hardware interval).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar) {
+  for (int it = 0; it < (1 << 20); ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+constexpr int kAppendDynSmem = kD * kD * 4 + 16;   // W_enc and the barrier of its copy
+
+// The work of one CTA (its first 128 threads; the others leave at once) for unit-side u, thread j = rotated
+// channel j.  `smem` is kAppendDynSmem bytes of 16-byte aligned shared memory.  The CTA runs on a cold instruction
+// cache and every global read costs a full memory latency, so everything it reads is requested up front: W_enc by
+// one bulk copy into shared memory (plain loads when the matrix is not 16-byte aligned), the width, the position,
+// the new tokens, the rotated mean and the unit's offset together; the half-words that the new fields are merged
+// into are read while the copy is in flight.
+__device__ inline void encode_append_body(const AppendArgs& p, int u, unsigned char* smem) {
   __shared__ float xs[kAppendMaxTokens][kD];
-  __shared__ float part[kD];
   __shared__ float red_lo[4], red_hi[4];
   __shared__ int cls_cnt[4][4];          // [class][warp]: strips of the class owned by the warp's channels
   __shared__ int grp_act[kMaxGroups];
+  if (threadIdx.x >= 128) return;
+  float* s_w = reinterpret_cast<float*>(smem);
+  const uint32_t wbar = (uint32_t)__cvta_generic_to_shared(smem + kD * kD * 4);
   const int ps = (int)(u % p.n_param_sets);
-  const int q = threadIdx.x >> 7, j = threadIdx.x & 127, lane = j & 31, warp = j >> 5;
+  const int j = threadIdx.x, lane = j & 31, warp = j >> 5;
   const int gs = p.scale_group, n_groups = kD / gs;
   const bool rotated = (p.flags & SPECTRA_ROTATED_INPUT) != 0;
-  auto worker_sync = [] {                 // barrier among the 128 workers only
-    if constexpr (NQ == 1) __syncthreads();
-    else asm volatile("bar.sync 1, 128;" ::: "memory");
-  };
-  // ---- everything the CTA reads before it writes is requested here: width, position, new tokens, W_enc
+  auto cta_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };   // the 128 workers only
+  const float* w = p.w_enc + (int64_t)ps * kD * kD;
+  const bool bulk = !rotated && (reinterpret_cast<uintptr_t>(w) & 15) == 0;
+  if (bulk && j == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(wbar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(wbar), "r"(kD * kD * 4) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     (uint32_t)__cvta_generic_to_shared(s_w)),
+                 "l"(w), "r"(kD * kD * 4), "r"(wbar)
+                 : "memory");
+  }
   const int b = p.widths[(int64_t)ps * kD + j];
   const int pos_first = p.pos0 ? p.pos0[u] : p.seq_len[u / p.n_kv] - 1;
-  for (int idx = threadIdx.x; idx < p.n_new * kD; idx += 128 * NQ) {
+  const float mr = rotated ? 0.f : p.mean_rot[(int64_t)ps * kD + j];
+  uint8_t* base = p.cache + p.unit_offset[u];
+  for (int idx = j; idx < p.n_new * kD; idx += 128) {
     const int t = idx / kD, i = idx - t * kD;
     xs[t][i] = load_as_float(p.x, p.x_dtype, (int64_t)u * p.stride_unit + (int64_t)t * p.stride_token + i);
   }
-  float wreg[kRows];
-  if (!rotated) {
-    const float* w = p.w_enc + (int64_t)ps * kD * kD + (int64_t)q * kRows * kD + j;
-#pragma unroll
-    for (int i = 0; i < kRows; i++) wreg[i] = __ldg(w + i * kD);
+  if (!rotated && !bulk)
+    for (int i = 0; i < kD; i++) s_w[i * kD + j] = w[i * kD + j];
+  if (j < kMaxGroups) grp_act[j] = 0;
+  cta_sync();
+  if (pos_first < 0) {                       // fused step on an empty sequence: nothing to append (CTA-uniform)
+    if (bulk) mbar_wait_bounded(wbar);       // the copy must land before the shared memory is released
+    return;
   }
-  if (q == 0 && j < kMaxGroups) grp_act[j] = 0;
-  __syncthreads();
-  if (pos_first < 0) return;                 // fused step on an empty sequence: nothing to append (CTA-uniform)
 
-  // ---- where this channel's strips live: rank inside each class, class offsets, tile size (workers)
+  // ---- where this channel's strips live: rank inside each class, class offsets, tile size
   int cls_n[4], cls_off[4], my_rank[4];
   int meta_off = -1, tile_bytes = 0;
-  if (q == 0) {
+  {
     int rank_in_warp[4];
 #pragma unroll
     for (int c = 0; c < 4; c++) {
@@ -68,13 +93,13 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
       if (lane == 0) cls_cnt[c][warp] = __popc(m);
     }
     if (b) grp_act[j / gs] = 1;
-    worker_sync();
+    cta_sync();
     int off = 0;
 #pragma unroll
     for (int c = 0; c < 4; c++) {
       int before = 0, n = 0;
 #pragma unroll
-      for (int w = 0; w < 4; w++) { if (w < warp) before += cls_cnt[c][w]; n += cls_cnt[c][w]; }
+      for (int wi = 0; wi < 4; wi++) { if (wi < warp) before += cls_cnt[c][wi]; n += cls_cnt[c][wi]; }
       cls_n[c] = n; cls_off[c] = off; my_rank[c] = before + rank_in_warp[c];
       off += 16 * (8 >> c) * n;
     }
@@ -86,30 +111,51 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
     }
     tile_bytes = payload + 512 * n_act;
   }
-  const float mr = (rotated || q) ? 0.f : p.mean_rot[(int64_t)ps * kD + j];
-  uint8_t* base = q ? nullptr : p.cache + p.unit_offset[u];
+  // Half-word and bit of this channel's field of class c for tile slot `slot`.
+  auto locate = [&](int c, int slot, int& bo, int& bit) {
+    const int wd = 8 >> c, k = my_rank[c], n = cls_n[c];
+    if (p.side == SPECTRA_SIDE_V) {
+      const int a = slot >> 5, h = (slot >> 4) & 1, i = slot & 15;
+      bo = cls_off[c] + 16 * wd * k + 4 * (a * wd + ((i * wd) >> 4)) + 2 * h;
+      bit = (i * wd) & 15;
+    } else {
+      const int hw = (slot * wd) >> 4;
+      bit = (slot * wd) & 15;
+      if ((k | 1) < n) bo = cls_off[c] + 32 * wd * (k >> 1) + 4 * hw + 2 * (k & 1);
+      else bo = cls_off[c] + 16 * wd * k + 2 * hw;
+    }
+  };
   int status = 0;
+  bool w_ready = rotated || !bulk;
 
   for (int t = 0; t < p.n_new; t++) {
+    const int pos = pos_first + t;
+    const int slot = pos & (kTile - 1);
+    uint8_t* tile = base + (int64_t)(pos / kTile) * tile_bytes;
+    // the half-words the new fields go into (a tile's first token finds them cleared)
+    unsigned old[4] = {0u, 0u, 0u, 0u};
+    if (slot != 0) {
+#pragma unroll
+      for (int c = 0; c < 4; c++)
+        if (b & (8 >> c)) {
+          int bo, bit;
+          locate(c, slot, bo, bit);
+          old[c] = *reinterpret_cast<const uint16_t*>(tile + bo);
+        }
+    }
+    if (!w_ready) {
+      if (!mbar_wait_bounded(wbar)) status |= SPECTRA_STATUS_WAIT_TIMEOUT;
+      w_ready = true;
+    }
     // rotate + centre: y_j = sum_i x_i W_enc[i][j] - m'_j (fp32 FMA chain in ascending i)
-    float y = 0.f;
+    float y;
     if (rotated) y = xs[t][j];
     else {
-#pragma unroll
-      for (int qq = 0; qq < NQ; qq++) {
-        if (q == qq) {
-          float a = qq ? part[j] : 0.f;
-#pragma unroll
-          for (int i = 0; i < kRows; i++) a = fmaf(xs[t][qq * kRows + i], wreg[i], a);
-          if constexpr (NQ > 1) part[j] = a;
-          else y = a;
-        }
-        if constexpr (NQ > 1) __syncthreads();
-      }
-      if constexpr (NQ > 1) y = part[j];
-      y = __fsub_rn(y, mr);
+      float a0 = 0.f;
+#pragma unroll 8
+      for (int i = 0; i < kD; i++) a0 = fmaf(xs[t][i], s_w[i * kD + j], a0);
+      y = __fsub_rn(a0, mr);
     }
-    if (q) continue;                         // helpers are done with this token
     if (b && !isfinite(y)) status |= SPECTRA_STATUS_NONFINITE;
     // per-group minimum and maximum over the channels with a non-zero width
     float lo = b ? y : INFINITY, hi = b ? y : -INFINITY;
@@ -118,9 +164,9 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
       lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, s));
       hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, s));
     }
-    worker_sync();
+    cta_sync();
     if (lane == 0) { red_lo[warp] = lo; red_hi[warp] = hi; }
-    worker_sync();
+    cta_sync();
     if (gs > 32) {
       const int w0 = (j / gs) * (gs / 32);
       lo = red_lo[w0]; hi = red_hi[w0];
@@ -149,34 +195,19 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
       }
     }
     // ---- write into the tail tile
-    const int pos = pos_first + t;
-    const int slot = pos & (kTile - 1);
-    uint8_t* tile = base + (int64_t)(pos / kTile) * tile_bytes;
     if (slot == 0) {                                          // first token of a tile: clear the tile
       for (int i = j; i < tile_bytes / 16; i += 128) reinterpret_cast<uint4*>(tile)[i] = make_uint4(0, 0, 0, 0);
-      worker_sync();
+      cta_sync();
     }
 #pragma unroll
     for (int c = 0; c < 4; c++) {
       const int wd = 8 >> c;
       if (b & wd) {
-        const int shift = b & (wd - 1);
-        const unsigned field = ((unsigned)code >> shift) & ((1u << wd) - 1u);
-        const int k = my_rank[c], n = cls_n[c];
+        const unsigned field = ((unsigned)code >> (b & (wd - 1))) & ((1u << wd) - 1u);
         int bo, bit;
-        if (p.side == SPECTRA_SIDE_V) {
-          const int a = slot >> 5, h = (slot >> 4) & 1, i = slot & 15;
-          bo = cls_off[c] + 16 * wd * k + 4 * (a * wd + ((i * wd) >> 4)) + 2 * h;
-          bit = (i * wd) & 15;
-        } else {
-          const int hw = (slot * wd) >> 4;
-          bit = (slot * wd) & 15;
-          if ((k | 1) < n) bo = cls_off[c] + 32 * wd * (k >> 1) + 4 * hw + 2 * (k & 1);
-          else bo = cls_off[c] + 16 * wd * k + 2 * hw;
-        }
-        uint16_t* dst = reinterpret_cast<uint16_t*>(tile + bo);
+        locate(c, slot, bo, bit);
         const unsigned below = (1u << bit) - 1u;              // earlier tokens of the half-word are kept
-        *dst = (uint16_t)(((unsigned)(*dst) & below) | (field << bit));
+        *reinterpret_cast<uint16_t*>(tile + bo) = (uint16_t)((old[c] & below) | (field << bit));
       }
     }
     if (meta_off >= 0 && (j % gs) == 0) {                     // one writer per scale group
@@ -184,7 +215,7 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u) {
       m[0] = __half_as_ushort(lo16);
       m[kTile] = __half_as_ushort(r16);
     }
-    worker_sync();
+    cta_sync();
   }
   if (status && p.status) atomicOr(p.status, status);
 }
