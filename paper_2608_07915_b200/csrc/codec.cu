@@ -404,6 +404,37 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p)
 
 using namespace spectra;
 
+namespace {
+
+// Tensor map over the bf16 input of a bulk encode: dimensions (channel, token, unit), box 8 channels x 128 tokens, no
+// swizzle, zeros outside.  The driver's encoder is looked up through the runtime (no link against the driver library).
+bool make_token_map(CUtensorMap* map, const void* x, int64_t n_tokens, int64_t n_units, int64_t stride_token,
+                    int64_t stride_unit) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym ||
+        q != cudaDriverEntryPointSuccess)
+      return false;
+    fn = reinterpret_cast<EncodeFn>(sym);
+  }
+  if (n_tokens < 1 || n_units < 1) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)n_tokens, (cuuint64_t)n_units};
+  // a single unit or token leaves its stride unused; the encoder still wants a legal value
+  const cuuint64_t strides[2] = {(cuuint64_t)(stride_token > 0 ? stride_token : kD) * 2,
+                                 (cuuint64_t)(stride_unit > 0 ? stride_unit : n_tokens * kD) * 2};
+  const cuuint32_t box[3] = {8, (cuuint32_t)kTile, 1}, estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dtype, int flags,
                               int64_t n_units, int64_t n_param_sets, const int32_t* pos0, int32_t n_new,
                               int64_t stride_unit, int64_t stride_token, const float* w_enc, const float* mean_rot,
@@ -434,15 +465,19 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
     // bf16 bulk encode: rotation on the tensor cores
     EncodeTcArgs ta{reinterpret_cast<const __nv_bfloat16*>(x), side, n_param_sets, pos0, n_new, stride_unit,
                     stride_token, w_enc, mean_rot, widths, cache, unit_offset, status_word};
-    // rotation on the 5th-generation tensor cores (accumulator tile in tensor memory)
-    const size_t um_smem = sizeof(EncodeUmmaSmem) + 128;
-    if (cudaFuncSetAttribute(encode_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)um_smem) !=
-        cudaSuccess)
-      return SPECTRA_CUDA_ERROR;
-    const unsigned tiles = (unsigned)((n_new + 2 * kTile - 2) / kTile);
-    dim3 grid((tiles + kUmTilesPerCta - 1) / kUmTilesPerCta, (unsigned)n_units);
-    encode_umma_kernel<<<grid, kUmThreads, um_smem, (cudaStream_t)stream>>>(ta);
-    return launch_status();
+    // rotation on the 5th-generation tensor cores (accumulator tiles in tensor memory); the token tiles arrive by
+    // TMA: a 3-D map over x [unit][token][channel] whose box is 8 channels x 128 tokens
+    CUtensorMap xmap;
+    if (make_token_map(&xmap, x, n_new, n_units, stride_token, stride_unit)) {
+      const size_t um_smem = sizeof(EncodeUmmaSmem) + 128;
+      if (cudaFuncSetAttribute(encode_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)um_smem) !=
+          cudaSuccess)
+        return SPECTRA_CUDA_ERROR;
+      const unsigned tiles = (unsigned)((n_new + 2 * kTile - 2) / kTile);
+      dim3 grid((tiles + kUmTilesPerCta - 1) / kUmTilesPerCta, (unsigned)n_units);
+      encode_umma_kernel<<<grid, kUmThreads, um_smem, (cudaStream_t)stream>>>(ta, xmap);
+      return launch_status();
+    }
   }
   EncodeArgs a{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
                w_enc, mean_rot, widths, cache, unit_offset, status_word};
