@@ -23,13 +23,6 @@ __global__ void step_positions_kernel(const int32_t* seq_len, int n_kv, int n_un
   if (u < n_units) pos[u] = seq_len[u / n_kv] - 1;
 }
 
-int sm_count() {
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-  return sms;
-}
-
 // Workspace carve-up of the tensor-core path.
 struct FastLayout {
   size_t desc_off, prefix_off, warp_off, rec_off, total;

@@ -474,8 +474,12 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
           cudaSuccess)
         return SPECTRA_CUDA_ERROR;
       const unsigned tiles = (unsigned)((n_new + 2 * kTile - 2) / kTile);
-      dim3 grid((tiles + kUmTilesPerCta - 1) / kUmTilesPerCta, (unsigned)n_units);
-      encode_umma_kernel<<<grid, kUmThreads, um_smem, (cudaStream_t)stream>>>(ta, xmap);
+      const int n_groups = (int)tiles;                   // tile slots per unit
+      const long long n_items = (long long)n_groups * n_units;
+      const int sms = sm_count();
+      if (sms <= 0 || n_items > 0x7fffffffLL) return SPECTRA_CUDA_ERROR;
+      const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
+      encode_umma_kernel<<<grid, kUmThreads, um_smem, (cudaStream_t)stream>>>(ta, xmap, n_groups, (int)n_items);
       return launch_status();
     }
   }

@@ -26,6 +26,14 @@ inline int check_config(const spectra_config* c) {
   return SPECTRA_OK;
 }
 
+// SMs of the current device (0 if the query fails).
+inline int sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return sms;
+}
+
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? SPECTRA_OK : SPECTRA_CUDA_ERROR; }
 
 // Description of one unit-side's tile, built in shared memory from the 128 widths.
