@@ -5,6 +5,7 @@
 #include "encode_append.cuh"
 #include "encode_tc.cuh"
 #include "encode_umma.cuh"
+#include "decode_umma.cuh"
 
 namespace spectra {
 
@@ -166,12 +167,6 @@ __global__ void __launch_bounds__(128, 1) encode_kernel(EncodeArgs p) {
   }
 }
 
-struct DecodeArgs {
-  const uint8_t* cache; const int64_t* unit_offset; int side; int scale_group; int64_t n_param_sets;
-  const int32_t* n_tokens; const float* w_dec; const float* mean_rot; const uint8_t* widths;
-  void* out; int out_dtype; float* yhat_out; int64_t stride_unit, stride_token;
-};
-
 __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   CodecSmem& S = *reinterpret_cast<CodecSmem*>(smem_raw);
@@ -233,171 +228,6 @@ __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
     store_from_float(p.out, p.out_dtype, (int64_t)u * p.stride_unit + (int64_t)(tile_pos + tt) * p.stride_token + i,
                      S.y[tt * kLdY + i]);
   }
-}
-
-// ---- decode with the inverse rotation on the 5th-generation tensor cores (tcgen05)
-// xhat = (yhat + m') W_dec with both operands as two-way bf16 splits (a = a1 + a2, W = W1 + W2) and the three
-// products a1 W1 + a1 W2 + a2 W1 accumulated in fp32 in tensor memory: relative error about 2^-16, far inside the
-// 2e-3 bound of the reconstruction.  One CTA of 512 threads walks several tiles of one unit-side and converts W_dec
-// once.  Operand layouts in shared memory as in encode_umma.cuh (a: K-major, W: MN-major core matrices).
-constexpr int kDecTiles = 4;
-constexpr int kDecThreads = 512;
-
-struct DecodeTcSmem {
-  StripTable tab;
-  alignas(128) uint8_t w[2][kD * kD * 2];          // the two bf16 parts of W_dec, MN-major core layout
-  alignas(128) uint8_t a[2][kTile * kD * 2];       // the two bf16 parts of yhat + m', K-major core layout
-  alignas(16) uint8_t codes[kTile * kLdC];
-  float bias[kD];
-  alignas(8) uint64_t mma_done;
-  uint32_t tmem_base;
-};
-
-__global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  unsigned char* smem_al = smem_raw + ((128u - (um_smem_u32(smem_raw) & 127u)) & 127u);
-  DecodeTcSmem& S = *reinterpret_cast<DecodeTcSmem*>(smem_al);
-  const int u = blockIdx.y;
-  const int ps = (int)(u % p.n_param_sets);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int q4 = warp & 3, cb = warp >> 2;           // tensor-memory lane quarter, 32-channel block of this warp
-  const int n = p.n_tokens[u];
-  const int tile_first = blockIdx.x * kDecTiles;
-  if (tile_first * kTile >= n) return;
-
-  build_strip_table(S.tab, p.widths + (int64_t)ps * kD, p.scale_group);
-  const StripTable& T = S.tab;
-  const float* wsrc = p.w_dec + (int64_t)ps * kD * kD;
-  for (int idx = tid; idx < kD * kD; idx += kDecThreads) {
-    const int k = idx / kD, nn = idx - k * kD;
-    const float v = wsrc[idx];
-    const __nv_bfloat16 w1 = __float2bfloat16_rn(v);
-    const int off = (nn >> 3) * 2048 + (k >> 3) * 128 + (k & 7) * 16 + (nn & 7) * 2;
-    *reinterpret_cast<__nv_bfloat16*>(&S.w[0][off]) = w1;
-    *reinterpret_cast<__nv_bfloat16*>(&S.w[1][off]) = __float2bfloat16_rn(v - __bfloat162float(w1));
-  }
-  if (tid < kD) S.bias[tid] = p.mean_rot[(int64_t)ps * kD + tid];
-  if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(um_smem_u32(&S.mma_done)) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (tid < 32) {                                    // warp 0 owns the tensor-memory allocation (128 columns)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(um_smem_u32(&S.tmem_base)), "r"(128u) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tb = S.tmem_base;
-  uint32_t phase = 0;
-  bool ok = true;
-
-  for (int tt = 0; tt < kDecTiles && ok; tt++) {
-    const int tile = tile_first + tt;
-    const int tile_pos = tile * kTile;
-    if (tile_pos >= n) break;
-    const int n_here = min(n - tile_pos, kTile);
-    const uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
-    __syncthreads();                                   // the previous tile's epilogue has read the accumulators
-    // unpack: word by word into the code array
-    for (int i = tid; i < kTile * kLdC / 4; i += kDecThreads) reinterpret_cast<uint32_t*>(S.codes)[i] = 0u;
-    __syncthreads();
-    unpack_tile(T, p.side, tile_ptr, S.codes, kLdC, tid, kDecThreads);
-    // dequantise (same operation order as the CUDA-core kernel), add the rotated mean, split into two bf16 parts:
-    // thread (channel j, token quarter tq) walks tokens [32 tq, 32 tq + 32); the lanes of a warp share the token, so
-    // its metadata is one broadcast load
-    {
-      const int j = tid & (kD - 1), tq = tid >> 7;
-      const int b = T.width[j];
-      const int mo = T.meta_off[j / p.scale_group];
-      const float L = (float)((1 << b) - 1), bias = S.bias[j];
-      const int joff = (j >> 3) * 2048 + (j & 7) * 2;   // K-major cores: k block j / 8, element j % 8
-      for (int tk = 32 * tq; tk < 32 * tq + 32; tk++) {
-        float lo_f = 0.f, R_f = 0.f;
-        if (mo >= 0) {
-          const uint16_t* m = reinterpret_cast<const uint16_t*>(tile_ptr + mo) + tk;
-          lo_f = __half2float(__ushort_as_half(m[0]));
-          R_f = __half2float(__ushort_as_half(m[kTile]));
-        }
-        float v = 0.f;
-        if (b) {
-          v = lo_f;
-          if (R_f != 0.f) v = __fadd_rn(__fmul_rn((float)S.codes[tk * kLdC + j], __fdiv_rn(R_f, L)), lo_f);
-        }
-        const bool live = tk < n_here;
-        if (p.yhat_out && live)
-          p.yhat_out[(int64_t)u * p.stride_unit + (int64_t)(tile_pos + tk) * p.stride_token + j] = v;
-        const float a = live ? v + bias : 0.f;
-        const __nv_bfloat16 a1 = __float2bfloat16_rn(a);
-        const int off = joff + (tk >> 3) * 128 + (tk & 7) * 16;
-        *reinterpret_cast<__nv_bfloat16*>(&S.a[0][off]) = a1;
-        *reinterpret_cast<__nv_bfloat16*>(&S.a[1][off]) = __float2bfloat16_rn(a - __bfloat162float(a1));
-      }
-    }
-    if (!p.out) continue;                              // (the host launches this kernel with an output only)
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    // ---- xhat = a W_dec: 24 MMAs of 128 x 128 x 16 issued by one thread, accumulator tile in tensor memory
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t a0 = um_smem_u32(S.a[0]), a1 = um_smem_u32(S.a[1]);
-      const uint32_t w0 = um_smem_u32(S.w[0]), w1 = um_smem_u32(S.w[1]);
-#pragma unroll 1
-      for (int pr = 0; pr < 3; pr++) {                 // a1 W1, a1 W2, a2 W1
-        const uint32_t aa = pr == 2 ? a1 : a0, ww = pr == 1 ? w1 : w0;
-#pragma unroll 1
-        for (int ks = 0; ks < kD / 16; ks++)
-          um_mma_ss(tb, um_desc(aa + 4096 * ks, 2048, 128), um_desc(ww + 256 * ks, 128, 2048), kUmIdesc, (pr | ks) != 0);
-      }
-      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(um_smem_u32(&S.mma_done)) : "memory");
-    }
-    {   // bounded wait for the accumulator tile
-      const uint32_t bar = um_smem_u32(&S.mma_done);
-      uint32_t done = 0;
-      for (int it = 0; it < (1 << 22) && !done; ++it)
-        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                     : "=r"(done) : "r"(bar), "r"(phase) : "memory");
-      if (!done) ok = false;
-      phase ^= 1u;
-    }
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ok) {
-      // ---- store: thread = token row 32 q4 + lane, channels [32 cb, 32 cb + 32)
-      float y[32];
-      const uint32_t src = tb + ((uint32_t)(q4 * 32) << 16) + 32u * cb;
-      um_ld16(src, y); um_ld16(src + 16, y + 16);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      const int tok = 32 * q4 + lane;
-      if (tok < n_here) {
-        const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + tok) * p.stride_token + 32 * cb;
-        const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out) + (uintptr_t)o * (p.out_dtype == SPECTRA_BF16 ? 2 : 4);
-        if ((addr & 15) == 0 && p.out_dtype == SPECTRA_BF16) {
-          uint4* dst = reinterpret_cast<uint4*>(addr);
-#pragma unroll
-          for (int c = 0; c < 4; c++) {
-            __nv_bfloat162 h[4];
-#pragma unroll
-            for (int e = 0; e < 4; e++) h[e] = __floats2bfloat162_rn(y[8 * c + 2 * e], y[8 * c + 2 * e + 1]);
-            dst[c] = *reinterpret_cast<const uint4*>(h);
-          }
-        } else if ((addr & 15) == 0) {
-          float4* dst = reinterpret_cast<float4*>(addr);
-#pragma unroll
-          for (int c = 0; c < 8; c++) dst[c] = make_float4(y[4 * c], y[4 * c + 1], y[4 * c + 2], y[4 * c + 3]);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 32; c++) store_from_float(p.out, p.out_dtype, o + c, y[c]);
-        }
-      }
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  }
-  // ---- the warp that allocated the tensor memory frees it
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tb), "r"(128u) : "memory");
 }
 
 }  // namespace spectra
@@ -509,15 +339,18 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
   if (out && !w_dec) return SPECTRA_INVALID_ARG;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
-               out_dtype, yhat_out, stride_unit, stride_token};
-  if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05)
+               out_dtype, yhat_out, stride_unit, stride_token, nullptr};
+  if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05), persistent grid
     const size_t dec_smem = sizeof(DecodeTcSmem) + 128;
     if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem) !=
         cudaSuccess)
       return SPECTRA_CUDA_ERROR;
-    const unsigned tiles = (unsigned)((max_tokens + kTile - 1) / kTile);
-    dim3 grid_tc((tiles + kDecTiles - 1) / kDecTiles, (unsigned)n_units);
-    decode_tc_kernel<<<grid_tc, kDecThreads, dec_smem, (cudaStream_t)stream>>>(a);
+    const int tiles = (int)((max_tokens + kTile - 1) / kTile);
+    const long long n_slots = (long long)tiles * n_units;
+    const int sms = sm_count();
+    if (sms <= 0 || n_slots > 0x7fffffffLL) return SPECTRA_CUDA_ERROR;
+    const unsigned grid_tc = (unsigned)(n_slots < sms ? n_slots : sms);
+    decode_tc_kernel<<<grid_tc, kDecThreads, dec_smem, (cudaStream_t)stream>>>(a, tiles, (int)n_slots);
     return launch_status();
   }
   if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CodecSmem)) !=

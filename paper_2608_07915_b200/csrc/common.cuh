@@ -48,7 +48,7 @@ struct StripTable {
   int tile_bytes;
   uint8_t chan[kMaxStrips];
   uint8_t shift[kMaxStrips];
-  uint8_t width[kD];
+  alignas(16) uint8_t width[kD];   // read four and eight at a time
 };
 
 // The scan itself, run by one full warp after T.width has been filled.
