@@ -45,9 +45,10 @@ struct DecodeTcSmem {
     alignas(128) uint8_t a[2][kTile * kD * 2];     // the two bf16 parts of yhat + m', K-major core layout
     alignas(128) uint8_t raw[kDecRawMax];          // the packed tile
   } half[2];
-  alignas(16) float bias[kD];
-  alignas(16) float2 lrl[kD];                      // {L, RN(1 / L)}, L = 2^width - 1 ({0, 0} for width 0)
+  alignas(16) float4 chq[kD];                      // per channel {L, RN(1 / L), stored ? 1 : 0, m'}, L = 2^width - 1
+  uint32_t field1[kD];                             // the channel's first (widest) sub-field: see field_desc()
   uint16_t sbase[4][kD];                           // per class: byte offset of the channel's strip; bit 15: stored alone
+  uint8_t more[kD];                                // classes of the channel's further sub-fields (bit c), usually 0
   alignas(8) uint64_t raw_full[2], a_full[2], acc_full[2];
   uint32_t tmem_base;
 };
@@ -82,6 +83,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
   // the strip (paired strips of the K side and all strips of the V side; a strip stored alone uses half of it) and the
   // field's bit inside the half-word
   int tokoff[4], bitpos[4];
+  unsigned long long tokpack = 0;                        // both, 16 bits per class: offset (8 bits) | bit << 8
 #pragma unroll
   for (int c = 0; c < 4; c++) {
     const int w = 8 >> c;
@@ -93,6 +95,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
       tokoff[c] = 4 * ((t * w) >> 4);
       bitpos[c] = (t * w) & 15;
     }
+    tokpack |= (unsigned long long)(tokoff[c] | (bitpos[c] << 8)) << (16 * c);
   }
 
   for (int slot = (int)((long long)blockIdx.x * n_slots / gridDim.x); slot < slot_end;) {
@@ -115,12 +118,6 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
       *reinterpret_cast<__nv_bfloat16*>(&S.w[0][off]) = w1;
       *reinterpret_cast<__nv_bfloat16*>(&S.w[1][off]) = __float2bfloat16_rn(v - __bfloat162float(w1));
     }
-    if (threadIdx.x < kD) {
-      const int b = T.width[threadIdx.x];
-      const float L = (float)((1 << b) - 1);
-      S.bias[threadIdx.x] = p.mean_rot[(int64_t)ps * kD + threadIdx.x];
-      S.lrl[threadIdx.x] = b ? make_float2(L, __frcp_rn(L)) : make_float2(0.f, 0.f);
-    }
     for (int k = threadIdx.x; k < T.n_strips; k += kDecThreads) {
       const int c = strip_class(T, k);
       const int w = 8 >> c, i_in = k - T.class_first[c], cnt = T.class_first[c + 1] - T.class_first[c];
@@ -129,6 +126,24 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
       else if ((i_in | 1) < cnt) sb = T.class_off[c] + 32 * w * (i_in >> 1) + 2 * (i_in & 1);
       else sb = (T.class_off[c] + 16 * w * i_in) | 0x8000;
       S.sbase[c][T.chan[k]] = (uint16_t)sb;
+    }
+    __syncthreads();
+    if (threadIdx.x < kD) {
+      const int j = threadIdx.x, b = T.width[j];
+      const float L = (float)((1 << b) - 1);
+      S.chq[j] = b ? make_float4(L, __frcp_rn(L), 1.f, p.mean_rot[(int64_t)ps * kD + j])
+                   : make_float4(0.f, 0.f, 0.f, p.mean_rot[(int64_t)ps * kD + j]);
+      // first sub-field: strip offset (bits 0..15, bit 15 = stored alone), class (16..17), position of the field inside
+      // the code (18..20), field mask (24..31; 0: the channel stores nothing)
+      uint32_t d = 0, more = 0;
+      for (int c = 0; c < 4; c++) {
+        const int w = 8 >> c;
+        if (!(b & w)) continue;
+        if (!d) d = (uint32_t)S.sbase[c][j] | ((uint32_t)c << 16) | ((uint32_t)(b & (w - 1)) << 18) | (((1u << w) - 1u) << 24);
+        else more |= 1u << c;
+      }
+      S.field1[j] = d;
+      S.more[j] = (uint8_t)more;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // W parts: generic stores -> tensor-core reads
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -208,32 +223,40 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
               R_f = __half2float(__ushort_as_half(m[kTile]));
             }
           }
-          const uint2 w8 = *reinterpret_cast<const uint2*>(&T.width[j0]);
           float a[8];
 #pragma unroll
           for (int e = 0; e < 8; e++) {
             const int j = j0 + e;
-            const uint32_t b = ((e < 4 ? w8.x : w8.y) >> (8 * (e & 3))) & 0xffu;      // warp-uniform
-            uint32_t code = 0;
+            // the code: its first sub-field without a branch (all per-channel facts are warp-uniform), further ones
+            // (widths 3, 5, 6, 7) class by class
+            const uint32_t d = S.field1[j];
+            const uint32_t tk = (uint32_t)(tokpack >> ((d >> 12) & 0x30u)) & 0xfffu;     // this token in that class
+            const uint32_t off = (d & 0x7fffu) + ((d & 0x8000u) ? (tk & 0xffu) >> 1 : (tk & 0xffu));
+            const uint32_t hw = *reinterpret_cast<const uint16_t*>(src + off);
+            uint32_t code = ((hw >> (tk >> 8)) & (d >> 24)) << ((d >> 18) & 7u);
+            const uint32_t more = S.more[j];
+            if (more) {
+              const uint32_t b = T.width[j];
 #pragma unroll
-            for (int c = 0; c < 4; c++) {
-              const uint32_t w = 8u >> c;
-              if (b & w) {
-                const uint32_t sb = S.sbase[c][j];
-                const uint32_t off = (sb & 0x7fffu) + ((sb & 0x8000u) ? (uint32_t)tokoff[c] >> 1 : (uint32_t)tokoff[c]);
-                const uint32_t hw = *reinterpret_cast<const uint16_t*>(src + off);
-                code |= ((hw >> bitpos[c]) & ((1u << w) - 1u)) << (b & (w - 1u));
+              for (int c = 1; c < 4; c++) {
+                const uint32_t w = 8u >> c;
+                if (more & (1u << c)) {
+                  const uint32_t sb = S.sbase[c][j];
+                  const uint32_t o2 = (sb & 0x7fffu) + ((sb & 0x8000u) ? (uint32_t)tokoff[c] >> 1 : (uint32_t)tokoff[c]);
+                  const uint32_t h2 = *reinterpret_cast<const uint16_t*>(src + o2);
+                  code |= ((h2 >> bitpos[c]) & ((1u << w) - 1u)) << (b & (w - 1u));
+                }
               }
             }
-            const float2 lr = S.lrl[j];
-            const float q0 = __fmul_rn(R_f, lr.y);
-            const float q = __fmaf_rn(__fmaf_rn(-q0, lr.x, R_f), lr.y, q0);           // RN(R / L), see the header
+            // v = code * (R / L) + lo for a stored channel, 0 otherwise (R = 0 gives q = 0 and v = lo)
+            const float4 cq = S.chq[j];
+            const float q0 = __fmul_rn(R_f, cq.y);
+            const float q = __fmaf_rn(__fmaf_rn(-q0, cq.x, R_f), cq.y, q0);           // RN(R / L), see the header
             const float cf = __uint_as_float(0x4B000000u | code) - 8388608.f;         // (float)code
-            float v = 0.f;
-            if (b) v = R_f != 0.f ? __fadd_rn(__fmul_rn(cf, q), lo_f) : lo_f;
+            const float v = __fadd_rn(__fmul_rn(cf, q), __fmul_rn(lo_f, cq.z));
             if (p.yhat_out && live)
               p.yhat_out[(int64_t)u * p.stride_unit + (int64_t)(tile_pos + t) * p.stride_token + j] = v;
-            a[e] = live ? v + S.bias[j] : 0.f;
+            a[e] = live ? v + cq.w : 0.f;
           }
           uint32_t hi[4], lw[4];
 #pragma unroll
