@@ -247,8 +247,12 @@ def test_tiny_encode_end_to_end_mismatches_are_rare_ties(sp, gain_mode):
         assert (~same_meta).mean() <= 2e-3
 
 
-def test_tiny_decode_matches_oracle(sp):
-    wl, S = _tiny_setup(sp, 4.0)
+@pytest.mark.parametrize("ratio,shift", [(4.0, 0), (2.0, 0), (8.0, 2)],
+                         ids=["staged", "tile_larger_than_the_staging_buffer", "cache_not_16_byte_aligned"])
+def test_tiny_decode_matches_oracle(sp, ratio, shift):
+    """The reconstruction kernel stages packed tiles in shared memory with bulk copies when they fit and the cache
+    is 16-byte aligned, and reads them in place otherwise: all three ways give the oracle's numbers."""
+    wl, S = _tiny_setup(sp, ratio)
     cfg = sp.default_config()
     for side, name in ((sp.SIDE_K, "k"), (sp.SIDE_V, "v")):
         s = S[name]
@@ -262,7 +266,9 @@ def test_tiny_decode_matches_oracle(sp):
         for dt in (torch.float32, torch.bfloat16):
             out = torch.full((1, 1024, 128), 7.0, dtype=dt, device="cuda")
             yhat = torch.zeros((1, 1024, 128), dtype=torch.float32, device="cuda")
-            sp.decode(cfg, side, H.to_dev(ref), H.to_dev(s["off"]), 1, 1,
+            cache_dev = torch.zeros(ref.size + 16, dtype=torch.uint8, device="cuda")
+            cache_dev[shift:shift + ref.size] = H.to_dev(ref)
+            sp.decode(cfg, side, cache_dev[shift:], H.to_dev(s["off"]), 1, 1,
                       torch.tensor([n], dtype=torch.int32, device="cuda"), n, dp["w_dec"], dp["m_rot"], dp["widths"],
                       out, yhat, 1024 * 128, 128)
             torch.cuda.synchronize()
