@@ -205,7 +205,8 @@ int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, co
  * round-trip.  With both NULL, or scale_group != 64, or width profiles outside the built variants, a slower
  * CUDA-core kernel runs; so it does when w_dec_k or w_dec_v is not 16-byte aligned (the tensor-core path fetches
  * whole parameter matrices with bulk copies).  A GQA group of 5 to 8 query heads is taken in two passes over the
- * tiles.  Partial sums of a sequence are merged in a fixed order: results are bit-reproducible from run to run.
+ * tiles.  On the tensor-core path the partial sums of a sequence are merged in a fixed order (results are
+ * bit-reproducible from run to run); the CUDA-core kernel accumulates with shared-memory atomics (they are not).
  * softmax_scale 0 means 1/sqrt(d).
  * out: device [batch, n_q_heads, d], out_dtype.  lse: device fp32 [batch, n_q_heads] or NULL.
  * workspace: device, >= spectra_attention_workspace_bytes(...), 16-byte aligned; scratch only, nothing is
