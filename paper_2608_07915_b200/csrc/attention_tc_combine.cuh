@@ -7,7 +7,7 @@
 
 namespace spectra {
 
-constexpr int kCombineBatch = 32;   // records merged per round (one per lane)
+constexpr int kCombineBatch = 32;   // records merged per batch (one per lane)
 constexpr int kCombineDynSmem = kD * kD * 4 + 16;   // W_dec,V and the barrier of its copy
 
 // A worker without tiles writes no record (only when there are fewer tiles than workers).
@@ -17,7 +17,7 @@ __device__ __noinline__ bool worker_has_tiles(long long gw, long long total, int
 
 // The CTA's work is a chain of dependent global reads, each costing a full memory latency, and it starts on a cold
 // instruction cache (straight-line code costs far more per instruction than a loop that is fetched once).  So the
-// reads are grouped into two rounds and rare cases are kept out of the main path: (1) everything whose address is
+// reads are issued in two groups and rare cases are kept out of the main path: (1) everything whose address is
 // known at launch - W_dec,V (one bulk copy into shared memory), the tile prefix, the descriptor fields, the rotated
 // mean; (2) the unit's partial records, up to 32 at a time, headers and accumulators together, before any of them
 // is used.  Records are merged with a running maximum; every warp computes the weights of a batch redundantly
@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, 
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
   const UnitDesc& D = f.desc[vu];
-  // ---- round 1
+  // ---- first group of reads
   if (tid == 0) {
     mbar_init(wbar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, 
   const int gw_last = (int)((tb * W + total - 1) / total) - 1;
   const int nrec = gw_last - gw_first + 1;
   const float* rec0 = f.records + (int64_t)(gw_first + vu) * f.rec_stride + (int64_t)h * (kRecHead + f.vs_max);
-  // ---- round 2
+  // ---- second group of reads
   float M = -INFINITY, L = 0.f, P0 = 0.f, P1 = 0.f;
   float acc[kPerThread];
 #pragma unroll

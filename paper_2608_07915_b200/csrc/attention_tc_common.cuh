@@ -142,7 +142,7 @@ __device__ __forceinline__ float2 h2f2(uint32_t x) {
 
 // ------------------------------------------------------------------------------------------------ prep kernel
 // These CTAs run once per call, on a cold instruction cache and with every global read paying a full memory latency.
-// So: one round of reads (W_dec,K by a bulk copy into shared memory; query, widths, rotated mean by plain loads
+// So: one group of reads issued together (W_dec,K by a bulk copy into shared memory; query, widths, rotated mean by plain loads
 // issued together), rolled loops, all 512 threads in every phase.
 struct PrepSmem {
   StripTable tk, tv;
@@ -230,7 +230,7 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
   const int G = min(kFastGqa, p.gqa - h0);                          // query heads of this pass
-  // ---- the one round of reads
+  // ---- all reads, issued together
   const uint32_t wbar = smem_u32(&S.wbar);
   if (tid == 0) {
     mbar_init(wbar, 1);
