@@ -220,7 +220,18 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       if (cudaFuncSetAttribute(attention_mma_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kCombineDynSmem) != cudaSuccess)
         return SPECTRA_CUDA_ERROR;
-      attention_mma_combine_kernel<<<(unsigned)(n_vunits * kFastGqa), 128, kCombineDynSmem, st>>>(a, f);
+      {
+        // the combine kernel may start while the main kernel drains: its first group of reads does not depend on the
+        // main kernel, and it waits (griddepcontrol.wait) before it touches the partial records
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3((unsigned)(n_vunits * kFastGqa)); lc.blockDim = dim3(128);
+        lc.dynamicSmemBytes = kCombineDynSmem; lc.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at; lc.numAttrs = 1;
+        if (cudaLaunchKernelEx(&lc, attention_mma_combine_kernel, a, f) != cudaSuccess) return SPECTRA_CUDA_ERROR;
+      }
       return launch_status();
     }
   }

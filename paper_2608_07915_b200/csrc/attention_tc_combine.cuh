@@ -56,6 +56,7 @@ __global__ void __launch_bounds__(128) attention_mma_combine_kernel(AttnArgs p, 
   const int64_t hidx = (int64_t)b * p.n_q + hk * p.gqa + h0 + h;         // query head in the caller's order
   const int64_t oidx = hidx * kD + tid;
   s_o[tid] = 0.f;
+  asm volatile("griddepcontrol.wait;" ::: "memory");         // from here on the main kernel's records are read
   __syncthreads();                                           // the barrier's initialisation is visible to all
   if (tb <= ta) {                                            // empty sequence
     store_from_float(p.out, p.out_dtype, oidx, 0.f);

@@ -266,6 +266,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncwarp();
 
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel may be scheduled as SMs free up
   const long long total = f.tile_prefix[f.n_units];
   const long long g0 = (long long)gw * total / f.total_warps;
   const long long g1 = (long long)(gw + 1) * total / f.total_warps;
