@@ -165,7 +165,8 @@ int spectra_alloc_bits(const spectra_config* cfg, const float* var_alloc, int64_
  * widths: device uint8 [n_param_sets, d].  cache: device; unit_offset: device int64 [n_units], byte offset
  * of the unit-side's first tile, multiple of 16.  status_word: device int32, OR-ed with SPECTRA_STATUS_* bits,
  * may be NULL.
- * The caller guarantees capacity: every touched tile lies inside its buffer.
+ * The caller guarantees capacity: every touched tile lies inside its buffer.  cache must be 16-byte aligned
+ * (SPECTRA_INVALID_ARG otherwise).
  * Speed, not results, depends on alignment: bf16 input with a 16-byte aligned x and strides that are multiples of 8
  * elements (and scale_group 64, more than 16 tokens) takes the tensor-core path; anything else a CUDA-core kernel.
  */
@@ -179,8 +180,9 @@ int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dty
  * of every unit-side; fp32 accumulation.  out: device, out_dtype SPECTRA_F32 or SPECTRA_BF16, element
  * (u, t, i) at out[u*stride_unit + t*stride_token + i].  n_tokens: device int32 [n_units];
  * max_tokens (host value) bounds it.  yhat_out (device fp32, same strides, may be NULL) receives the
- * dequantised rotated coordinates.  Packed tiles are fetched with bulk copies when cache + unit_offset[u] is 16-byte
- * aligned (and a tile is at most 10 KB), else read in place: same results, lower speed.
+ * dequantised rotated coordinates.  cache must be 2-byte aligned (SPECTRA_INVALID_ARG otherwise).  Packed tiles are
+ * fetched with bulk copies when cache + unit_offset[u] is 16-byte aligned (and a tile is at most 10 KB), else read in
+ * place: same results, lower speed.
  */
 int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
                    int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
@@ -203,9 +205,9 @@ int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, co
  * arrays ([n_param_sets, d], the same values the caller already needs for spectra_tile_bytes); read during the
  * call only.  They let the host size shared-memory rings and pick the kernel variant without a device
  * round-trip.  With both NULL, or scale_group != 64, or width profiles outside the built variants, a slower
- * CUDA-core kernel runs; so it does when w_dec_k or w_dec_v is not 16-byte aligned (the tensor-core path fetches
- * whole parameter matrices with bulk copies).  A GQA group of 5 to 8 query heads is taken in two passes over the
- * tiles.  On the tensor-core path the partial sums of a sequence are merged in a fixed order (results are
+ * CUDA-core kernel runs.  w_dec_k, w_dec_v, cache_k, cache_v and workspace must be 16-byte aligned
+ * (SPECTRA_INVALID_ARG otherwise: the kernels use 16-byte accesses and bulk copies).  A GQA group of 5 to 8 query
+ * heads is taken in two passes over the tiles.  On the tensor-core path the partial sums of a sequence are merged in a fixed order (results are
  * bit-reproducible from run to run); the CUDA-core kernel accumulates with shared-memory atomics (they are not).
  * softmax_scale 0 means 1/sqrt(d).
  * out: device [batch, n_q_heads, d], out_dtype.  lse: device fp32 [batch, n_q_heads] or NULL.

@@ -142,6 +142,9 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
     return SPECTRA_INVALID_ARG;
   if (lse && !mean_rot_k) return SPECTRA_INVALID_ARG;
   if ((widths_k_host == nullptr) != (widths_v_host == nullptr)) return SPECTRA_INVALID_ARG;
+  // the kernels read the parameter matrices, the caches and the workspace with 16-byte accesses and bulk copies
+  if ((((uintptr_t)w_dec_k | (uintptr_t)w_dec_v | (uintptr_t)cache_k | (uintptr_t)cache_v | (uintptr_t)workspace) & 15) != 0)
+    return SPECTRA_INVALID_ARG;
   const int64_t n_units = (int64_t)batch * n_kv_heads;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   if (workspace_bytes < spectra_attention_workspace_bytes(cfg, batch, n_kv_heads, n_q_heads, max_seq_len))
@@ -164,9 +167,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
   // heads is taken in passes of 4 (each pass is a unit of its own that reads the same tiles)
   const int npass = (gqa + kFastGqa - 1) / kFastGqa;
   const int64_t n_vunits = n_units * npass;
-  // (its kernels fetch whole parameter matrices with bulk copies, which need 16-byte aligned sources)
-  const bool aligned = (((uintptr_t)w_dec_k | (uintptr_t)w_dec_v) & 15) == 0;
-  if (widths_k_host && cfg->scale_group == 64 && n_vunits <= 65534 && aligned) {
+  if (widths_k_host && cfg->scale_group == 64 && n_vunits <= 65534) {
     const WidthFacts F = width_facts(widths_k_host, widths_v_host, n_param_sets);
     if (!F.ok) return SPECTRA_INVALID_ARG;
     const int sms = sm_count();

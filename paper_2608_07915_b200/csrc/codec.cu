@@ -279,6 +279,7 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
   if ((flags & SPECTRA_ROTATED_INPUT) && x_dtype != SPECTRA_F32) return SPECTRA_INVALID_ARG;
   if (n_units == 0 || n_new == 0) return SPECTRA_OK;
   if (!x || !pos0 || !widths || !cache || !unit_offset) return SPECTRA_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(cache) & 15) return SPECTRA_INVALID_ARG;      // tiles are cleared and packed with 16- and 4-byte stores
   if (!(flags & SPECTRA_ROTATED_INPUT) && (!w_enc || !mean_rot)) return SPECTRA_INVALID_ARG;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   if (n_new <= kAppendMaxTokens) {   // decode-step appends: one light CTA per unit-side
@@ -335,6 +336,7 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
   if (out_dtype != SPECTRA_F32 && out_dtype != SPECTRA_BF16) return SPECTRA_INVALID_ARG;
   if (n_units == 0 || max_tokens == 0) return SPECTRA_OK;
   if (!cache || !unit_offset || !n_tokens || !widths || !mean_rot) return SPECTRA_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(cache) & 1) return SPECTRA_INVALID_ARG;       // the packed fields are read as half-words
   if (!out && !yhat_out) return SPECTRA_INVALID_ARG;
   if (out && !w_dec) return SPECTRA_INVALID_ARG;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;

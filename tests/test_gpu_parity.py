@@ -326,6 +326,31 @@ def test_tiny_attention_matches_oracle(sp, ratio, n, host_widths):
     assert np.abs(lse[0] - lse_b[0]).max() <= 2e-3
 
 
+def test_attention_rejects_parameters_that_are_not_16_byte_aligned(sp):
+    """The attention kernels read W_dec with 16-byte accesses and bulk copies: a matrix at an odd float offset is
+    refused on the host (no launch), as the header says."""
+    wl, S = _tiny_setup(sp, 8.0)
+    cfg = sp.default_config()
+    n = 256
+    pk, pv = S["k"]["params"], S["v"]["params"]
+    dk, dv = H.dev_params(pk), H.dev_params(pv)
+
+    def shifted(t):                                        # the same values, one float further on
+        buf = torch.zeros(t.numel() + 1, dtype=t.dtype, device="cuda")
+        buf[1:] = t.reshape(-1)
+        return buf[1:].view(t.shape)
+    out = torch.zeros((1, 4, 128), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(sp.attention_workspace_bytes(cfg, 1, 1, 4, n), dtype=torch.uint8, device="cuda")
+    cache = torch.zeros(int(S["k"]["total"]), dtype=torch.uint8, device="cuda")
+    q = torch.zeros((1, 4, 128), dtype=torch.float32, device="cuda")
+    for wk, wv in ((shifted(dk["w_dec"]), dv["w_dec"]), (dk["w_dec"], shifted(dv["w_dec"]))):
+        with pytest.raises(sp.SpectraError):
+            sp.decode_attention(cfg, q, 1, 1, 4, H.to_dev(np.asarray([n], np.int32)), n, cache, H.to_dev(S["k"]["off"]),
+                                cache, H.to_dev(S["v"]["off"]), 1, wk, dk["m_rot"], dk["widths"], wv, dv["m_rot"],
+                                dv["widths"], 0.0, out, None, ws, None, pk.widths, pv.widths)
+    torch.cuda.synchronize()
+
+
 def _multi_unit_setup(wl, n_seq, n_tokens, ratio, gs=64, seq_lens=None):
     """One layer of a (possibly GQA-7) workload: per-head parameter sets shared by the sequences of the batch."""
     S = {}
