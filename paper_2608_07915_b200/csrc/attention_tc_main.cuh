@@ -372,11 +372,16 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
           const float a1 = acc[1][u][cb] + acc[1][u][cb + 1];
           float v = kscale * ((e ? r0.y : r0.x) * a0 + (e ? r1.y : r1.x) * a1) + (e ? lo0.y : lo0.x) * qlo0 +
                     (e ? lo1.y : lo1.x) * qlo1;
-          if (tok0 + ii >= n_seq) v = -INFINITY;
           s[ii] = v;
-          mx = fmaxf(mx, v);
         }
       }
+      if ((cons.t + 1) * kTile > n_seq) {                      // only the unit's last tile has slots past the end
+#pragma unroll
+        for (int ii = 0; ii < 8; ii++)
+          if (tok0 + ii >= n_seq) s[ii] = -INFINITY;
+      }
+#pragma unroll
+      for (int ii = 0; ii < 8; ii++) mx = fmaxf(mx, s[ii]);
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
