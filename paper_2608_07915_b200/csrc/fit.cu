@@ -11,7 +11,7 @@ constexpr int kMomChunk = 256;
 
 struct FitWorkspace {   // per unit, all fp64
   double S[kD * kD];
-  double VT[kD * kD];   // rows are eigenvectors (transposed so that plane rotations touch contiguous rows)
+  double VT[kD * kD];   // unused (the eigenvectors are accumulated in shared memory); kept for the workspace size
   double s[kD];
 };
 
@@ -57,25 +57,40 @@ __global__ void __launch_bounds__(256) moments_kernel(const void* x, int x_dtype
 }
 
 // ------------------------------------------------------------------------------------------------
-// Eigensolver: cyclic two-sided Jacobi in fp64, round-robin ordering (127 rounds of 64 disjoint
-// plane rotations per sweep), one CTA of 512 threads per matrix, matrix in shared memory.
-constexpr int kLdJ = kD + 1;
+// Eigensolver: cyclic two-sided Jacobi in fp64, round-robin ordering (127 rounds of 64 disjoint plane rotations per
+// sweep), one CTA of 512 threads per matrix.  Everything a round touches is in shared memory: the symmetric matrix
+// as its packed upper triangle (66 KB) and the accumulated eigenvectors (rows, 132 KB).  A round is one barrier
+// pair: 64 threads derive the rotations from the 2 x 2 diagonal blocks; then every 2 x 2 block (pair i, pair j),
+// i <= j, of the matrix is transformed by one thread as J_i^T B J_j (a matrix entry belongs to exactly one block, so
+// the rows-then-columns order of the textbook update needs no barrier in between), and the eigenvector rows of each
+// pair are rotated by eight threads.
+constexpr int kLdV = kD + 1;                       // row stride of the eigenvector array (bank spread)
+constexpr int kTri = kD * (kD + 1) / 2;            // entries of the packed upper triangle
+constexpr int kPairs = kD / 2;                     // rotations per round
+constexpr int kBlocks = kPairs * (kPairs - 1) / 2; // off-diagonal 2 x 2 blocks per round
 constexpr int kMaxSweeps = 30;
 
 struct EigSmem {
-  double A[kD * kLdJ];
-  double c[64], s[64];
-  int pp[64], qq[64];
+  double A[kTri];                                  // entry (r, c), r <= c, at tri(r, c)
+  double VT[kD * kLdV];                            // rows are eigenvectors
+  double c[kPairs], s[kPairs];
+  int pp[kPairs], qq[kPairs];
   double red[16];
-  double lam[kD];
+  double lam[kD], lam_sorted[kD];
   int order[kD];
   double mu[kD], m[kD], gam[kD];
+  unsigned short blk[kBlocks];                     // (i << 8) | j of the off-diagonal blocks, i < j
 };
 
 struct FitOut {
   float* w_enc; float* w_dec; float* mean_rot; float* var_alloc; float* eigval; float* basis_u;
   int gain_mode; int64_t n_tokens;
 };
+
+__device__ __forceinline__ int tri(int r, int c) {              // r <= c
+  return r * kD - ((r * (r - 1)) >> 1) + (c - r);
+}
+__device__ __forceinline__ int sym(int r, int c) { return r <= c ? tri(r, c) : tri(c, r); }
 
 __device__ inline double block_sum_512(double v, double* red) {
 #pragma unroll
@@ -97,32 +112,37 @@ __global__ void __launch_bounds__(512, 1) eigen_kernel(FitWorkspace* ws, FitOut 
   for (int idx = tid; idx < kD * kD; idx += 512) {
     const int r = idx / kD, c = idx - r * kD;
     // symmetrise: the two triangles were accumulated by different threads in the same order, but keep it exact
-    E.A[r * kLdJ + c] = 0.5 * (W.S[r * kD + c] + W.S[c * kD + r]) * inv_n;
-    W.VT[idx] = r == c ? 1.0 : 0.0;
+    if (r <= c) E.A[tri(r, c)] = 0.5 * (W.S[r * kD + c] + W.S[c * kD + r]) * inv_n;
+    E.VT[r * kLdV + c] = r == c ? 1.0 : 0.0;
+  }
+  for (int b = tid; b < kBlocks; b += 512) {                    // enumerate i < j once
+    int i = 0, rem = b;
+    while (rem >= kPairs - 1 - i) { rem -= kPairs - 1 - i; i++; }
+    E.blk[b] = (unsigned short)((i << 8) | (i + 1 + rem));
   }
   if (tid < kD) E.mu[tid] = W.s[tid] * inv_n;
   __syncthreads();
   double fro = 0.0;
-  for (int idx = tid; idx < kD * kD; idx += 512) { const double v = E.A[(idx / kD) * kLdJ + idx % kD]; fro += v * v; }
-  fro = block_sum_512(fro, E.red);
+  for (int idx = tid; idx < kTri; idx += 512) { const double v = E.A[idx]; fro += v * v; }
+  double diag2 = 0.0;
+  if (tid < kD) { const double v = E.A[tri(tid, tid)]; diag2 = v * v; }
+  fro = 2.0 * block_sum_512(fro, E.red) - block_sum_512(diag2, E.red);
   const double tol2 = 1e-28 * fro;   // (1e-14 ||C||_F)^2
 
   const int pair = tid >> 3, sub = tid & 7;
   for (int sweep = 0; sweep < kMaxSweeps; sweep++) {
-    double off = 0.0;
-    for (int idx = tid; idx < kD * kD; idx += 512) {
-      const int r = idx / kD, c = idx - r * kD;
-      if (r != c) { const double v = E.A[r * kLdJ + c]; off += v * v; }
-    }
-    off = block_sum_512(off, E.red);
+    double all2 = 0.0, dg2 = 0.0;
+    for (int idx = tid; idx < kTri; idx += 512) { const double v = E.A[idx]; all2 += v * v; }
+    if (tid < kD) { const double v = E.A[tri(tid, tid)]; dg2 = v * v; }
+    const double off = 2.0 * (block_sum_512(all2, E.red) - block_sum_512(dg2, E.red));
     if (off <= tol2) break;
     for (int round = 0; round < kD - 1; round++) {
-      if (tid < 64) {
+      if (tid < kPairs) {
         int p, q;
         if (tid == 0) { p = kD - 1; q = round; }
         else { p = (round + tid) % (kD - 1); q = (round - tid + (kD - 1)) % (kD - 1); }
         if (p > q) { const int t = p; p = q; q = t; }
-        const double app = E.A[p * kLdJ + p], aqq = E.A[q * kLdJ + q], apq = E.A[p * kLdJ + q];
+        const double app = E.A[tri(p, p)], aqq = E.A[tri(q, q)], apq = E.A[tri(p, q)];
         double c = 1.0, s = 0.0;
         if (apq != 0.0 && fabs(apq) > 1e-300) {
           const double tau = (aqq - app) / (2.0 * apq);
@@ -133,29 +153,46 @@ __global__ void __launch_bounds__(512, 1) eigen_kernel(FitWorkspace* ws, FitOut 
         E.c[tid] = c; E.s[tid] = s; E.pp[tid] = p; E.qq[tid] = q;
       }
       __syncthreads();
-      const int p = E.pp[pair], q = E.qq[pair];
-      const double c = E.c[pair], s = E.s[pair];
-      // rows: A <- J^T A ; eigenvector rows: VT <- J^T VT
-      for (int k = sub; k < kD; k += 8) {
-        const double ap = E.A[p * kLdJ + k], aq = E.A[q * kLdJ + k];
-        E.A[p * kLdJ + k] = c * ap - s * aq;
-        E.A[q * kLdJ + k] = s * ap + c * aq;
-        const double vp = W.VT[p * kD + k], vq = W.VT[q * kD + k];
-        W.VT[p * kD + k] = c * vp - s * vq;
-        W.VT[q * kD + k] = s * vp + c * vq;
+      // the matrix: A <- J^T A J, block by block.  With J^T = [[c, -s], [s, c]] on rows (p, q):
+      //   rows:    x_p' = c x_p - s x_q,  x_q' = s x_p + c x_q;  columns the same with the other pair's (c, s)
+      for (int b = tid; b < kBlocks + kPairs; b += 512) {
+        if (b < kBlocks) {
+          const int i = E.blk[b] >> 8, j = E.blk[b] & 0xff;
+          const int pi = E.pp[i], qi = E.qq[i], pj = E.pp[j], qj = E.qq[j];
+          const double ci = E.c[i], si = E.s[i], cj = E.c[j], sj = E.s[j];
+          const int i00 = sym(pi, pj), i01 = sym(pi, qj), i10 = sym(qi, pj), i11 = sym(qi, qj);
+          const double b00 = E.A[i00], b01 = E.A[i01], b10 = E.A[i10], b11 = E.A[i11];
+          const double r00 = ci * b00 - si * b10, r01 = ci * b01 - si * b11;      // rows by pair i
+          const double r10 = si * b00 + ci * b10, r11 = si * b01 + ci * b11;
+          E.A[i00] = cj * r00 - sj * r01; E.A[i01] = sj * r00 + cj * r01;        // columns by pair j
+          E.A[i10] = cj * r10 - sj * r11; E.A[i11] = sj * r10 + cj * r11;
+        } else {
+          const int i = b - kBlocks;
+          const int p = E.pp[i], q = E.qq[i];
+          const double c = E.c[i], s = E.s[i];
+          const double app = E.A[tri(p, p)], aqq = E.A[tri(q, q)], apq = E.A[tri(p, q)];
+          const double r00 = c * app - s * apq, r01 = c * apq - s * aqq;          // rows
+          const double r10 = s * app + c * apq, r11 = s * apq + c * aqq;
+          E.A[tri(p, p)] = c * r00 - s * r01;                                     // columns
+          E.A[tri(q, q)] = s * r10 + c * r11;
+          E.A[tri(p, q)] = s * r00 + c * r01;
+        }
       }
-      __syncthreads();
-      // columns: A <- A J
-      for (int k = sub; k < kD; k += 8) {
-        const double ap = E.A[k * kLdJ + p], aq = E.A[k * kLdJ + q];
-        E.A[k * kLdJ + p] = c * ap - s * aq;
-        E.A[k * kLdJ + q] = s * ap + c * aq;
+      // the eigenvector rows: VT <- J^T VT
+      {
+        const int p = E.pp[pair], q = E.qq[pair];
+        const double c = E.c[pair], s = E.s[pair];
+        for (int k = sub; k < kD; k += 8) {
+          const double vp = E.VT[p * kLdV + k], vq = E.VT[q * kLdV + k];
+          E.VT[p * kLdV + k] = c * vp - s * vq;
+          E.VT[q * kLdV + k] = s * vp + c * vq;
+        }
       }
       __syncthreads();
     }
   }
   // ---- order eigenvalues (descending, ties by index), fix signs, assemble the transform
-  if (tid < kD) E.lam[tid] = E.A[tid * kLdJ + tid];
+  if (tid < kD) E.lam[tid] = E.A[tri(tid, tid)];
   __syncthreads();
   if (tid < kD) {
     const double l = E.lam[tid];
@@ -167,7 +204,7 @@ __global__ void __launch_bounds__(512, 1) eigen_kernel(FitWorkspace* ws, FitOut 
   if (tid < kD) {
     // output column j = tid comes from Jacobi row order[j]
     const int src = E.order[tid];
-    const double* v = W.VT + src * kD;
+    const double* v = E.VT + src * kLdV;
     int kmax = 0; double amax = -1.0;
     for (int k = 0; k < kD; k++) { const double a = fabs(v[k]); if (a > amax) { amax = a; kmax = k; } }
     const double sign = v[kmax] < 0.0 ? -1.0 : 1.0;
@@ -177,12 +214,12 @@ __global__ void __launch_bounds__(512, 1) eigen_kernel(FitWorkspace* ws, FitOut 
     const double lam = fmax(E.lam[src], 0.0);
     E.m[tid] = m;
     E.gam[tid] = sign;            // stash the sign; replaced by the gain below
-    E.A[tid * kLdJ + tid] = lam;  // sorted eigenvalue j now on the diagonal slot j (diagonal no longer needed)
+    E.lam_sorted[tid] = lam;      // eigenvalue j in descending order
   }
   __syncthreads();
   if (tid < kD) {
-    const double lam = E.A[tid * kLdJ + tid];
-    const double lam1 = E.A[0];
+    const double lam = E.lam_sorted[tid];
+    const double lam1 = E.lam_sorted[0];
     const double m = E.m[tid];
     const double var = fmax(lam - m * m, 0.0);
     const double floor_v = 1e-12 * lam1;
@@ -194,7 +231,7 @@ __global__ void __launch_bounds__(512, 1) eigen_kernel(FitWorkspace* ws, FitOut 
     o.mean_rot[base + tid] = (float)(m * g);
     o.var_alloc[base + tid] = (float)(o.gain_mode == SPECTRA_GAIN_WHITEN ? var : var * g * g);
     if (o.eigval) o.eigval[base + tid] = (float)lam;
-    const double* v = W.VT + E.order[tid] * kD;
+    const double* v = E.VT + E.order[tid] * kLdV;
     const int64_t mb = (int64_t)u * kD * kD;
     for (int k = 0; k < kD; k++) {
       const double ukj = sign * v[k];                       // U[k][j], j = tid
