@@ -77,6 +77,26 @@ def test_bad_arguments_are_rejected_before_any_launch(lib):
     assert attn(2, 8) == sp.INVALID_ARG                                                      # null pointers
 
 
+def test_misaligned_buffers_are_refused_on_the_host(lib):
+    """The kernels use 16-byte (attention, encode) and 2-byte (decode) accesses on these buffers; the entry points
+    check the alignment before anything is launched (the pointers below are never dereferenced)."""
+    cfg = sp.default_config()
+    null = C.c_void_p(0)
+    p = lambda a: C.c_void_p(a)
+    ok = 0x10000
+    # spectra_encode: cache one byte off
+    assert lib.spectra_encode(C.byref(cfg), 0, p(ok), sp.F32, 0, C.c_int64(1), C.c_int64(1), p(ok), 1, C.c_int64(128),
+                              C.c_int64(128), p(ok), p(ok), p(ok), p(ok + 1), p(ok), null, null) == sp.INVALID_ARG
+    # spectra_decode: odd cache address
+    assert lib.spectra_decode(C.byref(cfg), 0, p(ok + 1), p(ok), C.c_int64(1), C.c_int64(1), p(ok), 128, p(ok), p(ok),
+                              p(ok), p(ok), sp.F32, null, C.c_int64(128 * 128), C.c_int64(128), null) == sp.INVALID_ARG
+    # spectra_decode_attention: W_dec,K four bytes off
+    big = C.c_size_t(1 << 30)
+    assert lib.spectra_decode_attention(C.byref(cfg), p(ok), sp.F32, 1, 1, 4, p(ok), 128, p(ok), p(ok), p(ok), p(ok),
+                                        C.c_int64(1), p(ok + 4), null, p(ok), p(ok), p(ok), p(ok), null, null,
+                                        C.c_float(0), p(ok), sp.F32, null, p(ok), big, null, null) == sp.INVALID_ARG
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(sp, "_lib", None)
     monkeypatch.setattr(sp, "_LIB_PATH", str(tmp_path / "nope.so"))
