@@ -82,9 +82,9 @@ int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem
 }
 
 // Quota tuples (V blocks of 16 strips per class 8, 4, 2, 1) the main kernel is built for, smallest first.
-// They cover the width profiles that reverse water-filling produces at 4x to 12x on decaying spectra; anything
-// else runs on the CUDA-core kernel.
-constexpr int kQuotas[][4] = {{0, 1, 8, 2}, {0, 1, 3, 6}, {0, 1, 6, 4}, {0, 8, 2, 2}, {0, 7, 3, 4}};
+// They cover the width profiles that reverse water-filling produces at 4x, 6x, 8x, 10x, 12x and 16x on decaying
+// spectra; anything else runs on the CUDA-core kernel.
+constexpr int kQuotas[][4] = {{0, 1, 8, 2}, {0, 1, 3, 6}, {0, 1, 6, 4}, {0, 8, 2, 2}, {0, 7, 3, 4}, {0, 1, 2, 7}, {0, 1, 8, 5}};
 constexpr int kNumQuotas = sizeof(kQuotas) / sizeof(kQuotas[0]);
 
 int pick_quota(const int (&vb)[4]) {
@@ -215,7 +215,9 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
         case 1: rc = launch_fast_main<0, 1, 3, 6>(a, f, grid, smem, st); break;
         case 2: rc = launch_fast_main<0, 1, 6, 4>(a, f, grid, smem, st); break;
         case 3: rc = launch_fast_main<0, 8, 2, 2>(a, f, grid, smem, st); break;
-        default: rc = launch_fast_main<0, 7, 3, 4>(a, f, grid, smem, st); break;
+        case 4: rc = launch_fast_main<0, 7, 3, 4>(a, f, grid, smem, st); break;
+        case 5: rc = launch_fast_main<0, 1, 2, 7>(a, f, grid, smem, st); break;
+        default: rc = launch_fast_main<0, 1, 8, 5>(a, f, grid, smem, st); break;
       }
       if (rc) return rc;
       if (cudaFuncSetAttribute(attention_mma_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -305,7 +305,7 @@ def _gpu_attention(sp, cfg, q_dev, batch, n_kv, n_q, seq_len, max_len, K, V, cac
 
 
 @pytest.mark.parametrize("host_widths", [True, False], ids=["tensor", "generic"])
-@pytest.mark.parametrize("ratio", [4.0, 8.0, 12.0])
+@pytest.mark.parametrize("ratio", [4.0, 6.0, 8.0, 12.0, 16.0])
 @pytest.mark.parametrize("n", [1024, 1000, 77])
 def test_tiny_attention_matches_oracle(sp, ratio, n, host_widths):
     wl, S = _tiny_setup(sp, ratio)
