@@ -208,7 +208,9 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
         attention_prep_kernel<<<(unsigned)n_vunits + 1, kPrepThreads, kPrepDynSmem, st>>>(a, f);
       }
       if (launch_status()) return SPECTRA_CUDA_ERROR;
-      const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64;
+      // the last chunk of a K run and the last block of a V class read up to 15 strips past the end of their class
+      // (zero rows of B, unused accumulator rows): the pad keeps those reads inside the CTA's shared memory
+      const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64 + 2048;
       const int grid = sms * ctas_per_sm;
       switch (quota) {
         case 0: rc = launch_fast_main<0, 1, 8, 2>(a, f, grid, smem, st); break;

@@ -28,7 +28,8 @@
 namespace spectra {
 
 constexpr int kFastGqa = 4;
-constexpr int kKcMax = 32;       // upper bound of B-table entries of a K tile (chunks of 16 strips, one doubled per class)
+constexpr int kKcMax = 40;       // upper bound of B-table entries of a K tile: 384 strips in 8 (class, group) runs, each
+                                 // run rounded up to whole chunks of 16 strips and a group-1 run starting on an even strip
 constexpr int kFastWarps = 4;    // warps per CTA of the main kernel
 constexpr int kRecHead = 4;      // floats of a record's per-head header: m, l, plo0, plo1
 constexpr float kLog2e = 1.4426950408889634f;
@@ -36,7 +37,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct alignas(16) UnitDesc {
   int32_t tbk, tbv;
   int32_t kmeta[2], vmeta[2];   // byte offset of lo16[128] of scale group g (R16 256 bytes later), -1 if inactive
-  uint32_t kcls[4], vcls[4];    // per class: strips | strips of scale group 0 << 8 | (byte offset / 16) << 16
+  uint32_t krun[2][4];          // K runs [scale group][class]: (byte offset of the first pair) / 16 | chunks << 16 |
+                                // slot of a strip stored alone in the last chunk << 24 | (there is one) << 27
+  uint32_t vcls[4];             // per V class: strips | strips of scale group 0 << 8 | (byte offset / 16) << 16
   uint32_t vfirst[4];           // index of the first V strip of each class
   int32_t n_vstrips, pad0;
   float kscale[4];              // 2^-e_h
@@ -44,7 +47,7 @@ struct alignas(16) UnitDesc {
   float qconst[4];              // q' . m'_K (natural-log units)
   uint8_t vchan[kMaxStrips];    // channel of V strip k
   float vcoef[kMaxStrips];      // 2^24 * 2^shift / (2^width - 1): turns the strip's accumulator into its share of yhat
-  uint2 kB[kKcMax][4][32];      // [chunk][MMA u of the chunk][lane] -> (b0, b1)
+  uint4 kB[kKcMax][2][32];      // [chunk in walk order][MMAs {0,1} or {2,3}][lane] -> (b0, b1) of the two MMAs
 };
 
 struct FastArgs {
@@ -333,35 +336,41 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
     }
   }
   __syncthreads();
-  // ---- B fragments.  An entry contributes to its scale group only (rows of the other group, or past the end of the
-  // class, are zero).  Column n = head (n >> 1), hi (n & 1 == 0) or lo half of the fp16 split.  Variant u carries
-  // the factor 2^-p_eff(u) of the unpacking.
-  // Entries: a class is walked in chunks of 16 consecutive strips; the strips of scale group 0 come first, so at most
-  // one chunk per class holds strips of both groups: it gets two entries, one per group.  Entries are stored
-  // chunk-major, group-minor: the order the main kernel walks them.
-  int ent_base[5];
+  // ---- B fragments.  The main kernel walks the K tile one scale group at a time and, inside a group, class by
+  // class: run (g, c) covers the group's strips of class c in chunks of 16 strips (8 stored pairs).  The strips of
+  // scale group 0 come first in a class, so its run starts at pair 0; the run of group 1 starts at the pair that
+  // holds the class's first group-1 strip.  An entry's rows outside the run's group, or past the end of the class,
+  // are zero.  Column n = head (n >> 1), hi (n & 1 == 0) or lo half of the fp16 split.  Variant u carries the factor
+  // 2^-p_eff(u) of the unpacking.  Entries are stored in walk order.
+  int ent_base[9], run_start[8];
   ent_base[0] = 0;
 #pragma unroll
-  for (int c = 0; c < 4; c++) {
+  for (int r = 0; r < 8; r++) {
+    const int g = r >> 2, c = r & 3;
     const int n = TK.class_first[c + 1] - TK.class_first[c], n_g0 = S.ng0[0][c];
-    ent_base[c + 1] = ent_base[c] + (n + 15) / 16 + ((n > n_g0 && (n_g0 & 15) != 0) ? 1 : 0);
+    const int sp = g ? (n_g0 >> 1) : 0;                                   // first pair of the run
+    const int pairs = g ? (n > n_g0 ? ((n + 1) >> 1) - sp : 0) : ((n_g0 + 1) >> 1);
+    run_start[r] = 2 * sp;
+    ent_base[r + 1] = ent_base[r] + ((pairs + 7) >> 3);
   }
-  const int n_entries = min(ent_base[4], kKcMax);
+  const int n_entries = min(ent_base[8], kKcMax);
 #pragma unroll 1
   for (int idx = tid; idx < n_entries * 4 * 32; idx += kPrepThreads) {
     const int en = idx >> 7, u4 = (idx >> 5) & 3, ln = idx & 31;
-    const int c = (en >= ent_base[1]) + (en >= ent_base[2]) + (en >= ent_base[3]);
+    int r = 0;
+#pragma unroll
+    for (int k = 1; k < 8; k++) r += en >= ent_base[k];
+    int eb = 0, start = 0;
+#pragma unroll
+    for (int k = 0; k < 8; k++) if (k == r) { eb = ent_base[k]; start = run_start[k]; }
+    const int g = r >> 2, c = r & 3;
     const int first = TK.class_first[c], n = TK.class_first[c + 1] - first, n_g0 = S.ng0[0][c];
-    const int local = en - (c == 0 ? 0 : (c == 1 ? ent_base[1] : (c == 2 ? ent_base[2] : ent_base[3])));
-    const int b0 = n_g0 >> 4;                                        // first chunk that holds a strip of group 1
-    const bool both = n > n_g0 && (n_g0 & 15) != 0;                  // chunk b0 holds strips of both groups
-    const int ch = both && local > b0 ? local - 1 : local;
-    const int run = both ? (local <= b0 ? 0 : 1) : (16 * local < n_g0 ? 0 : 1);
-    const int start = 16 * ch;
+    const int lo_s = g ? n_g0 : 0, hi_s = g ? n : n_g0;                   // strips of the class that belong to the run
+    start += 16 * (en - eb);
     const int gid = ln >> 2, tg = ln & 3, h = gid >> 1, part = gid & 1;
     const int pe = c == 0 ? 0 : (c == 1 ? 4 * (u4 & 1) : (c == 2 ? 2 * u4 : u4));
     const __half scale = __ushort_as_half((unsigned short)((15 - pe) << 10));
-    uint32_t r[2];
+    uint32_t rr[2];
 #pragma unroll
     for (int half = 0; half < 2; half++) {
       uint32_t v = 0;
@@ -369,20 +378,32 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
       for (int e = 0; e < 2; e++) {
         const int strip = start + 2 * tg + 8 * half + e;
         uint16_t bits = 0;
-        if (strip < n && h < G && (strip >= n_g0 ? 1 : 0) == run)
+        if (strip >= lo_s && strip < hi_s && h < G)
           bits = __half_as_ushort(__hmul(part ? S.blo[h][first + strip] : S.bhi[h][first + strip], scale));
         v |= (uint32_t)bits << (16 * e);
       }
-      r[half] = v;
+      rr[half] = v;
     }
-    D.kB[en][u4][ln] = make_uint2(r[0], r[1]);
+    reinterpret_cast<uint2*>(&D.kB[en][u4 >> 1][ln])[u4 & 1] = make_uint2(rr[0], rr[1]);
   }
-  if (tid < 4) {
-    D.kcls[tid] = pack_cls(TK, tid, S.ng0[0][tid]);
-    D.vcls[tid] = pack_cls(TV, tid, S.ng0[1][tid]);
-    D.vfirst[tid] = TV.class_first[tid];
+  if (tid < 8) {
+    const int g = tid >> 2, c = tid & 3, w = 8 >> c;
+    const int n = TK.class_first[c + 1] - TK.class_first[c], n_g0 = S.ng0[0][c];
+    const int sp = g ? (n_g0 >> 1) : 0;
+    const int pairs = g ? (n > n_g0 ? ((n + 1) >> 1) - sp : 0) : ((n_g0 + 1) >> 1);
+    const int nch = (pairs + 7) >> 3;
+    // a class with an odd number of strips stores its last strip alone; it belongs to the class's last run
+    const bool lone = (n & 1) && pairs > 0 && (g ? true : n == n_g0);
+    const int slot = lone ? (((n - 1) >> 1) - sp) & 7 : 0;
+    D.krun[g][c] = (uint32_t)((TK.class_off[c] + 32 * w * sp) / 16) | ((uint32_t)nch << 16) | ((uint32_t)slot << 24) |
+                   ((uint32_t)(lone ? 1 : 0) << 27);
   }
-  if (tid == 32) {
+  if (tid >= 32 && tid < 36) {
+    const int c = tid - 32;
+    D.vcls[c] = pack_cls(TV, c, S.ng0[1][c]);
+    D.vfirst[c] = TV.class_first[c];
+  }
+  if (tid == 64) {
     D.tbk = TK.tile_bytes; D.tbv = TV.tile_bytes;
     D.kmeta[0] = TK.meta_off[0]; D.kmeta[1] = TK.meta_off[1];
     D.vmeta[0] = TV.meta_off[0]; D.vmeta[1] = TV.meta_off[1];

@@ -7,6 +7,11 @@
 // position-dependent power of two is folded into the B operand (exact): on the K side the four MMAs of a chunk
 // take the tokens whose fields share a position, on the V side the probabilities get one scaled copy per class.
 //
+// A warp works on a whole 128-token tile at a time: a thread owns tokens 16 gid .. 16 gid + 15 (two half tiles of
+// eight), so one shared-memory load brings both half tiles' words of a strip pair and one B fragment serves both.
+// The K tile is walked one scale group at a time (all classes of group 0, then all classes of group 1): a single
+// set of score accumulators is live, and each (class, group) run is a short loop whose body is compile-time code.
+//
 // The V accumulators live in registers, one 16-strip block per accumulator.  Their number and their class must be
 // compile-time facts, so the kernel is instantiated for a few "quota" tuples (blocks per class 8, 4, 2, 1); the
 // host picks the smallest tuple that covers the widths of the call.
@@ -49,7 +54,7 @@ template <> struct Unpack<2> {   // 1 word, 8 tokens (bits 0, 2, .., 14)
   static __device__ __forceinline__ void shifted(const uint32_t (&w)[NW], uint32_t (&ws)[NW]) { ws[0] = w[0] >> 8; }
   static __host__ __device__ constexpr int peff(int u) { return 2 * (u & 3); }
 };
-template <> struct Unpack<1> {   // 1 word (already shifted right by 8 * pass), 8 tokens at bits 0..7
+template <> struct Unpack<1> {   // 1 word (already shifted right by 8 * half tile), 8 tokens at bits 0..7
   static constexpr int NW = 1;
   static __device__ __forceinline__ uint32_t get(const uint32_t (&w)[NW], const uint32_t (&ws)[NW], int ii) {
     return ((ii & 4) ? ws[0] : w[0]) & (0x00010001u << (ii & 3));
@@ -68,145 +73,133 @@ __device__ __forceinline__ uint32_t hmul2_pow2(uint32_t x, int neg_exp) {   // x
   return *reinterpret_cast<const uint32_t*>(&r);
 }
 
-// Plain loads of n words from shared memory (the compiler may schedule them freely between barrier waits).
-template <int NW>
-__device__ __forceinline__ void ld_words(const unsigned char* p, uint32_t (&w)[NW]) {
-  if constexpr (NW == 4) { const uint4 v = *reinterpret_cast<const uint4*>(p); w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w; }
-  else if constexpr (NW == 2) { const uint2 v = *reinterpret_cast<const uint2*>(p); w[0] = v.x; w[1] = v.y; }
-  else w[0] = *reinterpret_cast<const uint32_t*>(p);
-}
-// Same for a strip stored alone (half-words in order): each half-word becomes the low half of a word.
-template <int NW>
-__device__ __forceinline__ void ld_halfwords(const unsigned char* p, uint32_t (&w)[NW]) {
-  if constexpr (NW == 4) { const uint2 v = *reinterpret_cast<const uint2*>(p); w[0] = v.x & 0xffffu; w[1] = v.x >> 16; w[2] = v.y & 0xffffu; w[3] = v.y >> 16; }
-  else if constexpr (NW == 2) { const uint32_t v = *reinterpret_cast<const uint32_t*>(p); w[0] = v & 0xffffu; w[1] = v >> 16; }
-  else w[0] = *reinterpret_cast<const uint16_t*>(p);
-}
-
-// Four MMAs of one chunk into one scale group's accumulators: MMA u takes tokens u (row gid) and u + 4 (row
-// gid + 8) of the pass, pair slots tig and tig + 4 as its k columns, and B variant u (scaled by 2^-p_eff(u); rows
-// of strips that belong to the other scale group, or lie past the end of the class, are zero).
+// A thread's words of one strip pair (K) or strip (V) for the whole tile: W words of 32 bits, the first half of
+// them for half tile 0 and the rest for half tile 1 (W = 1: one word, half tile 1 in the upper byte of each half).
 template <int W>
-__device__ __forceinline__ void k_chunk(const uint32_t (&wa)[Unpack<W>::NW], const uint32_t (&wb)[Unpack<W>::NW],
-                                        const uint2* __restrict__ kb, float (&acc)[4][4]) {
-  using U = Unpack<W>;
-  constexpr int NW = U::NW;
-  uint32_t was[NW], wbs[NW];
-  U::shifted(wa, was);
-  U::shifted(wb, wbs);
+__device__ __forceinline__ void ld_tile_words(const unsigned char* p, uint32_t (&x)[W]) {
+  if constexpr (W == 8) {
+    const uint4 a = *reinterpret_cast<const uint4*>(p), b = *reinterpret_cast<const uint4*>(p + 16);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  } else if constexpr (W == 4) {
+    const uint4 a = *reinterpret_cast<const uint4*>(p);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+  } else if constexpr (W == 2) {
+    const uint2 a = *reinterpret_cast<const uint2*>(p);
+    x[0] = a.x; x[1] = a.y;
+  } else {
+    x[0] = *reinterpret_cast<const uint32_t*>(p);
+  }
+}
+// The same words of a K strip that is stored alone (half-words in order): each half-word becomes the low half of a
+// word, the partner strip's half is zero.  p points at the thread's first half-word (2 W gid bytes into the strip).
+template <int W>
+__device__ __forceinline__ void ld_lone_words(const unsigned char* p, uint32_t (&x)[W]) {
+  if constexpr (W == 1) {
+    x[0] = *reinterpret_cast<const uint16_t*>(p);
+  } else {
+    uint32_t h[W / 2];
+    ld_tile_words<W / 2>(p, h);
 #pragma unroll
-  for (int u = 0; u < 4; u++) {
-    const uint2 b = __ldg(kb + u * 32);
-    mma16816(acc[u], U::get(wa, was, u), U::get(wa, was, u + 4), U::get(wb, wbs, u), U::get(wb, wbs, u + 4), b.x, b.y);
+    for (int i = 0; i < W / 2; i++) { x[2 * i] = h[i] & 0xffffu; x[2 * i + 1] = h[i] >> 16; }
+  }
+}
+template <int W, int HP>
+__device__ __forceinline__ void half_tile_words(const uint32_t (&x)[W], uint32_t (&w)[Unpack<W>::NW]) {
+  if constexpr (W == 1) w[0] = HP ? x[0] >> 8 : x[0];
+  else {
+#pragma unroll
+    for (int i = 0; i < Unpack<W>::NW; i++) w[i] = x[Unpack<W>::NW * HP + i];
   }
 }
 
-// The chunk that holds strips of both scale groups: the A fragments are unpacked once and multiplied with both
-// groups' B entries (consecutive in the table).
-template <int W>
-__device__ __forceinline__ void k_chunk_both(const uint32_t (&wa)[Unpack<W>::NW], const uint32_t (&wb)[Unpack<W>::NW],
-                                             const uint2* __restrict__ kb, float (&acc)[2][4][4]) {
+// One chunk (8 strip pairs x 128 tokens) into the score accumulators: per half tile, MMA u takes tokens u (row
+// gid) and u + 4 (row gid + 8), pair slots tig and tig + 4 as its k columns, and B variant u (scaled by
+// 2^-p_eff(u); rows of strips outside the run's scale group, or past the end of the class, are zero).
+template <int W, int HP>
+__device__ __forceinline__ void k_chunk_half(const uint32_t (&xa)[W], const uint32_t (&xb)[W], const uint4& b01,
+                                             const uint4& b23, float (&acc)[4][4]) {
   using U = Unpack<W>;
   constexpr int NW = U::NW;
-  uint32_t was[NW], wbs[NW];
+  uint32_t wa[NW], wb[NW], was[NW], wbs[NW];
+  half_tile_words<W, HP>(xa, wa);
+  half_tile_words<W, HP>(xb, wb);
   U::shifted(wa, was);
   U::shifted(wb, wbs);
-#pragma unroll
-  for (int u = 0; u < 4; u++) {
-    const uint2 b0 = __ldg(kb + u * 32), b1 = __ldg(kb + (4 + u) * 32);
-    const uint32_t a0 = U::get(wa, was, u), a1 = U::get(wa, was, u + 4), a2 = U::get(wb, wbs, u), a3 = U::get(wb, wbs, u + 4);
-    mma16816(acc[0][u], a0, a1, a2, a3, b0.x, b0.y);
-    mma16816(acc[1][u], a0, a1, a2, a3, b1.x, b1.y);
-  }
+  mma16816(acc[0], U::get(wa, was, 0), U::get(wa, was, 4), U::get(wb, wbs, 0), U::get(wb, wbs, 4), b01.x, b01.y);
+  mma16816(acc[1], U::get(wa, was, 1), U::get(wa, was, 5), U::get(wb, wbs, 1), U::get(wb, wbs, 5), b01.z, b01.w);
+  mma16816(acc[2], U::get(wa, was, 2), U::get(wa, was, 6), U::get(wb, wbs, 2), U::get(wb, wbs, 6), b23.x, b23.y);
+  mma16816(acc[3], U::get(wa, was, 3), U::get(wa, was, 7), U::get(wb, wbs, 3), U::get(wb, wbs, 7), b23.z, b23.w);
 }
 
-// One class of the K tile for one half tile.  Chunks of 16 strips = 8 interleaved pairs, in storage order; the
-// strips of scale group 0 come first (n_g0 of them), so at most one chunk per class holds strips of both groups: it
-// is multiplied twice, once per group, each time with the other group's rows zeroed in B.  The B table is walked in
-// the same order (chunk-major, group-minor).  An odd last strip of the class is stored alone (half-words in order).
+// One (class, scale group) run of the K tile: `run` = byte offset / 16 of its first pair | chunks << 16 |
+// slot of a strip stored alone in the last chunk << 24 | (such a strip exists) << 27.  The B table is walked in the
+// same order; kb points at this lane's entry of the next chunk.
 template <int W>
-__device__ __forceinline__ void k_class(const unsigned char* ktile, uint32_t cls, const uint2* __restrict__& kb,
-                                        int hp, int gid, int tig, float (&acc)[2][4][4]) {
-  using U = Unpack<W>;
-  constexpr int NW = U::NW;
-  const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
-  if (n == 0) return;
-  const unsigned char* cbase = ktile + (cls >> 16) * 16;
-  const int thr = 4 * W * gid + (W == 1 ? 0 : 4 * NW * hp);    // this thread's token block inside a pair
-  const unsigned char* pa = cbase + 32 * W * tig + thr;
-  int s = 0;
+__device__ __forceinline__ void k_run(const unsigned char* ktile, uint32_t run, const uint4* __restrict__& kb,
+                                      int gid, int tig, float (&acc)[2][4][4]) {
+  const int nch = (int)(run >> 16) & 0xff;
+  if (nch == 0) return;
+  const unsigned char* pa = ktile + (run & 0xffffu) * 16 + 32 * W * tig + 4 * W * gid;
+  const int lone_i = (run >> 27) & 1u ? nch - 1 : -1;
 #pragma unroll 1
-  for (; s + 16 <= (n & ~1); s += 16, pa += 256 * W) {          // complete chunks
-    uint32_t wa[NW], wb[NW];
-    ld_words<NW>(pa, wa);
-    ld_words<NW>(pa + 128 * W, wb);
-    if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-    if (s + 16 <= n_g0) { k_chunk<W>(wa, wb, kb, acc[0]); kb += 4 * 32; }
-    else if (s >= n_g0) { k_chunk<W>(wa, wb, kb, acc[1]); kb += 4 * 32; }
-    else { k_chunk_both<W>(wa, wb, kb, acc); kb += 8 * 32; }
-  }
-  if (s < n) {                                                  // the last, incomplete chunk of the class
-    const int avail = n - s;                                    // strips stored from s on (B rows past them are zero)
-    const unsigned char* cb = cbase + 16 * W * s;
-    uint32_t wa[NW], wb[NW];
-    if (!(avail & 1)) {
-      // whole pairs only: slots past the end re-read the last pair
-      const int last = (avail >> 1) - 1;
-      ld_words<NW>(cb + 32 * W * min(tig, last) + thr, wa);
-      ld_words<NW>(cb + 32 * W * min(tig + 4, last) + thr, wb);
-    } else {
-      // the class has an odd number of strips: its last strip is stored alone, half-words in order
-#pragma unroll
-      for (int i = 0; i < NW; i++) { wa[i] = 0u; wb[i] = 0u; }
-      const int thr_h = 2 * W * gid + (W == 1 ? 0 : 2 * NW * hp);
-#pragma unroll
-      for (int half = 0; half < 2; half++) {
-        const int ps = tig + 4 * half;
-        uint32_t (&wd)[NW] = half ? wb : wa;
-        if (2 * ps + 1 < avail) ld_words<NW>(cb + 32 * W * ps + thr, wd);
-        else if (2 * ps < avail) ld_halfwords<NW>(cb + 32 * W * ps + thr_h, wd);
+  for (int i = 0; i < nch; i++, pa += 256 * W, kb += 64) {
+    uint32_t xa[W], xb[W];
+    ld_tile_words<W>(pa, xa);
+    ld_tile_words<W>(pa + 128 * W, xb);
+    const uint4 b01 = __ldg(kb), b23 = __ldg(kb + 32);
+    if (i == lone_i) {
+      const int slot = (int)(run >> 24) & 7;
+      if (tig == (slot & 3)) {
+        // the pair of this slot is one strip stored alone: re-read it as half-words
+        const unsigned char* pl = pa - 32 * W * tig - 4 * W * gid + 32 * W * slot + 2 * W * gid;
+        if (slot & 4) ld_lone_words<W>(pl, xb);
+        else ld_lone_words<W>(pl, xa);
       }
     }
-    if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-    if (n <= n_g0) { k_chunk<W>(wa, wb, kb, acc[0]); kb += 4 * 32; }
-    else if (s >= n_g0) { k_chunk<W>(wa, wb, kb, acc[1]); kb += 4 * 32; }
-    else { k_chunk_both<W>(wa, wb, kb, acc); kb += 8 * 32; }
+    k_chunk_half<W, 0>(xa, xb, b01, b23, acc[0]);
+    k_chunk_half<W, 1>(xa, xb, b01, b23, acc[1]);
   }
 }
 
-// One class of the V tile for one half tile, at most Q blocks of 16 strips, accumulators acc_o[OFF .. OFF + Q).
-// The probabilities first get the class's position scales; MMA u of a block contracts the token pairs of B
-// fragments u and u + 4.
+// One class of the V tile, at most Q blocks of 16 strips, accumulators acc_o[OFF .. OFF + Q).  The probabilities
+// first get the class's position scales; per half tile, MMA u of a block contracts the token pairs of B fragments
+// u and u + 4.  Rows past the end of the class read whatever follows in shared memory (finite after masking); their
+// accumulators are never stored.
+template <int W, int HP, int NACC>
+__device__ __forceinline__ void v_block_half(const uint32_t (&xa)[W], const uint32_t (&xb)[W], const uint32_t (&pw)[8],
+                                             float (&acc)[4]) {
+  using U = Unpack<W>;
+  constexpr int NW = U::NW;
+  uint32_t wa[NW], wb[NW], was[NW], wbs[NW];
+  half_tile_words<W, HP>(xa, wa);
+  half_tile_words<W, HP>(xb, wb);
+  U::shifted(wa, was);
+  U::shifted(wb, wbs);
+#pragma unroll
+  for (int u = 0; u < 4; u++)
+    mma16816(acc, U::get(wa, was, u), U::get(wb, wbs, u), U::get(wa, was, u + 4), U::get(wb, wbs, u + 4), pw[u], pw[u + 4]);
+}
 template <int W, int Q, int OFF, int NACC>
-__device__ __forceinline__ void v_class(const unsigned char* vtile, uint32_t cls, int hp, int gid, int tig,
-                                        const uint32_t (&pb)[8], float (&acc_o)[NACC][4]) {
+__device__ __forceinline__ void v_class(const unsigned char* vtile, uint32_t cls, int gid, int tig,
+                                        const uint32_t (&pb)[2][8], float (&acc_o)[NACC][4]) {
   if constexpr (Q > 0) {
     using U = Unpack<W>;
-    constexpr int NW = U::NW;
     const int n = cls & 0xff;
     if (n == 0) return;
-    uint32_t pw[8];
+    uint32_t pw[2][8];
 #pragma unroll
-    for (int ii = 0; ii < 8; ii++) pw[ii] = hmul2_pow2(pb[ii], U::peff(ii));
-    const unsigned char* cbase = vtile + (cls >> 16) * 16 + 4 * W * tig + (W == 1 ? 0 : 4 * NW * hp);
+    for (int hp = 0; hp < 2; hp++)
+#pragma unroll
+      for (int ii = 0; ii < 8; ii++) pw[hp][ii] = hmul2_pow2(pb[hp][ii], U::peff(ii));
+    const unsigned char* cbase = vtile + (cls >> 16) * 16 + 4 * W * tig + 16 * W * gid;
 #pragma unroll
     for (int bi = 0; bi < Q; bi++) {
       if (16 * bi < n) {
-        uint32_t wa[NW], wb[NW], was[NW], wbs[NW];
-        if (16 * bi + 16 <= n) {
-          ld_words<NW>(cbase + 16 * W * (16 * bi + gid), wa);
-          ld_words<NW>(cbase + 16 * W * (16 * bi + gid + 8), wb);
-        } else {                               // rows past the end repeat the last strip; their results are unused
-          ld_words<NW>(cbase + 16 * W * min(16 * bi + gid, n - 1), wa);
-          ld_words<NW>(cbase + 16 * W * min(16 * bi + gid + 8, n - 1), wb);
-        }
-        if constexpr (W == 1) { wa[0] >>= 8 * hp; wb[0] >>= 8 * hp; }
-        U::shifted(wa, was);
-        U::shifted(wb, wbs);
-#pragma unroll
-        for (int u = 0; u < 4; u++)
-          mma16816(acc_o[OFF + bi], U::get(wa, was, u), U::get(wb, wbs, u), U::get(wa, was, u + 4),
-                   U::get(wb, wbs, u + 4), pw[u], pw[u + 4]);
+        uint32_t xa[W], xb[W];
+        ld_tile_words<W>(cbase + 16 * W * (16 * bi), xa);
+        ld_tile_words<W>(cbase + 16 * W * (16 * bi + 8), xb);
+        v_block_half<W, 0, NACC>(xa, xb, pw[0], acc_o[OFF + bi]);
+        v_block_half<W, 1, NACC>(xa, xb, pw[1], acc_o[OFF + bi]);
       }
     }
   }
@@ -248,6 +241,27 @@ struct TileCursor {   // walks the flattened (unit, tile) space; all fields are 
     if (t >= nt) { u++; t = 0; seek_unit(f); }
   }
 };
+
+// Adds one scale group's share to the scores of this thread's 16 tokens, in units of 1 / kscale:
+// s'_t += R_t * (hi + lo partial sums) + lo_t * (sum of q' over the group's active channels / kscale).
+// meta points at lo16[16 gid] of the group; R16 follows 256 bytes later.
+__device__ __forceinline__ void fold_group(const unsigned char* meta, float qlo, const float (&acc)[2][4][4],
+                                           float (&s)[16], bool first) {
+  uint32_t lo[8], rg[8];
+  ld_tile_words<8>(meta, lo);
+  ld_tile_words<8>(meta + 256, rg);
+#pragma unroll
+  for (int r = 0; r < 8; r++) {
+    const float2 l2 = h2f2(lo[r]), r2 = h2f2(rg[r]);
+#pragma unroll
+    for (int e = 0; e < 2; e++) {
+      const int hp = r >> 2, ii = 2 * (r & 3) + e, u = ii & 3, cb = (ii >> 2) * 2;
+      const float a = acc[hp][u][cb] + acc[hp][u][cb + 1];            // hi + lo halves of q'
+      const float base = first ? (e ? l2.y : l2.x) * qlo : fmaf(e ? l2.y : l2.x, qlo, s[8 * hp + ii]);
+      s[8 * hp + ii] = fmaf(e ? r2.y : r2.x, a, base);
+    }
+  }
+}
 
 template <int Q8, int Q4, int Q2, int Q1>
 __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnArgs p, FastArgs f) {
@@ -301,10 +315,10 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
 
   float acc_o[NACC][4];
   float m_run = -INFINITY, l_run = 0.f, plo0 = 0.f, plo1 = 0.f;
-  uint32_t kcls[4], vcls[4];
+  uint32_t krun[2][4], vcls[4];
   int kmeta0 = -1, kmeta1 = -1, vmeta0 = -1, vmeta1 = -1;
   float kscale = 0.f, qlo0 = 0.f, qlo1 = 0.f;
-  const uint2* kB = nullptr;
+  const uint4* kB = nullptr;
   int n_seq = 0;
   bool fresh = true, ok = true;
   float boost = 0.f;          // power-of-two lift of the probabilities (see below); -1 = not chosen yet
@@ -317,9 +331,10 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
     if (fresh) {
       const UnitDesc& d = f.desc[cons.u];
 #pragma unroll
-      for (int c = 0; c < 4; c++) { kcls[c] = d.kcls[c]; vcls[c] = d.vcls[c]; }
+      for (int c = 0; c < 4; c++) { krun[0][c] = d.krun[0][c]; krun[1][c] = d.krun[1][c]; vcls[c] = d.vcls[c]; }
       kmeta0 = d.kmeta[0]; kmeta1 = d.kmeta[1]; vmeta0 = d.vmeta[0]; vmeta1 = d.vmeta[1];
-      kscale = d.kscale[tig]; qlo0 = d.qlo[tig][0]; qlo1 = d.qlo[tig][1];
+      kscale = d.kscale[tig];                                  // a power of two: the divisions are exact
+      qlo0 = d.qlo[tig][0] / kscale; qlo1 = d.qlo[tig][1] / kscale;
       kB = &d.kB[0][0][0];
       n_seq = p.seq_len[(cons.u / f.npass) / p.n_kv];
 #pragma unroll
@@ -331,83 +346,84 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
       boost = -1.f;
     }
 
-#pragma unroll 1
-    for (int hp = 0; hp < 2; hp++) {
-      // ------------------------------------------------------------ scores of 64 tokens
-      if (hp == 0) ok = mbar_wait(bars + 8 * slot, parity);
+    // ------------------------------------------------------------ scores of the tile's 128 tokens, in units of 1 / kscale
+    ok = mbar_wait(bars + 8 * slot, parity);
+    float s[16];
+    {
+      const uint4* kb = kB + lane;       // walks the B fragment table in run order
       float acc[2][4][4];
+      if (kmeta0 >= 0) {
 #pragma unroll
-      for (int g = 0; g < 2; g++)
+        for (int hp = 0; hp < 2; hp++)
 #pragma unroll
-        for (int u = 0; u < 4; u++)
+          for (int u = 0; u < 4; u++)
 #pragma unroll
-          for (int e = 0; e < 4; e++) acc[g][u][e] = 0.f;
-      const uint2* kb = kB + lane;       // walks the B fragment table in chunk order
-      k_class<8>(ktile, kcls[0], kb, hp, gid, tig, acc);
-      k_class<4>(ktile, kcls[1], kb, hp, gid, tig, acc);
-      k_class<2>(ktile, kcls[2], kb, hp, gid, tig, acc);
-      k_class<1>(ktile, kcls[3], kb, hp, gid, tig, acc);
-
-      // per-token group minimum and range of the K tile (fp16), this thread's 8 tokens: token ii is MMA u = ii & 3,
-      // row gid (ii < 4) or gid + 8; the fp16 pair r holds tokens 2r and 2r + 1
-      const int tok_off = 2 * (gid * 16 + 8 * hp);
-      uint32_t klo0[4] = {0, 0, 0, 0}, kr0[4] = {0, 0, 0, 0}, klo1[4] = {0, 0, 0, 0}, kr1[4] = {0, 0, 0, 0};
-      if (kmeta0 >= 0) { ld_words<4>(ktile + kmeta0 + tok_off, klo0); ld_words<4>(ktile + kmeta0 + 256 + tok_off, kr0); }
-      if (kmeta1 >= 0) { ld_words<4>(ktile + kmeta1 + tok_off, klo1); ld_words<4>(ktile + kmeta1 + 256 + tok_off, kr1); }
-      if (hp == 1 && issued_k < count) {     // the K slot is free: refill it with the tile D positions ahead
-        __syncwarp();
-        if (lane == 0) { fence_async_smem(); start_k(issued_k % D); }
-        issued_k++;
+            for (int e = 0; e < 4; e++) acc[hp][u][e] = 0.f;
+        k_run<8>(ktile, krun[0][0], kb, gid, tig, acc);
+        k_run<4>(ktile, krun[0][1], kb, gid, tig, acc);
+        k_run<2>(ktile, krun[0][2], kb, gid, tig, acc);
+        k_run<1>(ktile, krun[0][3], kb, gid, tig, acc);
+        fold_group(ktile + kmeta0 + 32 * gid, qlo0, acc, s, true);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; i++) s[i] = 0.f;
       }
-      float s[8];
-      float mx = -INFINITY;
-      const int tok0 = cons.t * kTile + gid * 16 + 8 * hp;
+      if (kmeta1 >= 0) {
 #pragma unroll
-      for (int r = 0; r < 4; r++) {
-        const float2 lo0 = h2f2(klo0[r]), r0 = h2f2(kr0[r]), lo1 = h2f2(klo1[r]), r1 = h2f2(kr1[r]);
+        for (int hp = 0; hp < 2; hp++)
 #pragma unroll
-        for (int e = 0; e < 2; e++) {
-          const int ii = 2 * r + e, u = ii & 3, cb = (ii >> 2) * 2;
-          const float a0 = acc[0][u][cb] + acc[0][u][cb + 1];   // hi + lo halves of q'
-          const float a1 = acc[1][u][cb] + acc[1][u][cb + 1];
-          float v = kscale * ((e ? r0.y : r0.x) * a0 + (e ? r1.y : r1.x) * a1) + (e ? lo0.y : lo0.x) * qlo0 +
-                    (e ? lo1.y : lo1.x) * qlo1;
-          s[ii] = v;
-        }
+          for (int u = 0; u < 4; u++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) acc[hp][u][e] = 0.f;
+        k_run<8>(ktile, krun[1][0], kb, gid, tig, acc);
+        k_run<4>(ktile, krun[1][1], kb, gid, tig, acc);
+        k_run<2>(ktile, krun[1][2], kb, gid, tig, acc);
+        k_run<1>(ktile, krun[1][3], kb, gid, tig, acc);
+        fold_group(ktile + kmeta1 + 32 * gid, qlo1, acc, s, false);
       }
-      if ((cons.t + 1) * kTile > n_seq) {                      // only the unit's last tile has slots past the end
+    }
+    if (issued_k < count) {     // the K slot is free: refill it with the tile D positions ahead
+      __syncwarp();
+      if (lane == 0) { fence_async_smem(); start_k(issued_k % D); }
+      issued_k++;
+    }
+    if ((cons.t + 1) * kTile > n_seq) {                      // only the unit's last tile has slots past the end
+      const int tok0 = cons.t * kTile + gid * 16;
 #pragma unroll
-        for (int ii = 0; ii < 8; ii++)
-          if (tok0 + ii >= n_seq) s[ii] = -INFINITY;
-      }
+      for (int i = 0; i < 16; i++)
+        if (tok0 + i >= n_seq) s[i] = -INFINITY;
+    }
+    float mx = s[0];
 #pragma unroll
-      for (int ii = 0; ii < 8; ii++) mx = fmaxf(mx, s[ii]);
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-      if (mx > m_run) {        // new running maximum for this thread's head: rescale what has been accumulated
-        const float alpha = fast_exp2(m_run - mx);   // exp2(-inf) = 0 on the first tile
-        m_run = mx;
-        l_run *= alpha; plo0 *= alpha; plo1 *= alpha;
+    for (int i = 1; i < 16; i++) mx = fmaxf(mx, s[i]);
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+    mx *= kscale;                                            // kscale is a positive power of two: exact
+    if (mx > m_run) {        // new running maximum for this thread's head: rescale what has been accumulated
+      const float alpha = fast_exp2(m_run - mx);   // exp2(-inf) = 0 on the first tile
+      m_run = mx;
+      l_run *= alpha; plo0 *= alpha; plo1 *= alpha;
 #pragma unroll
-        for (int mb = 0; mb < NACC; mb++)
+      for (int mb = 0; mb < NACC; mb++)
 #pragma unroll
-          for (int e = 0; e < 4; e++) acc_o[mb][e] *= alpha;
-      }
-      if (hp == 0) ok = ok && mbar_wait(bars + 8 * (4 + slot), parity);
-      uint32_t vlo0[4] = {0, 0, 0, 0}, vr0[4] = {0, 0, 0, 0}, vlo1[4] = {0, 0, 0, 0}, vr1[4] = {0, 0, 0, 0};
-      if (vmeta0 >= 0) { ld_words<4>(vtile + vmeta0 + tok_off, vlo0); ld_words<4>(vtile + vmeta0 + 256 + tok_off, vr0); }
-      if (vmeta1 >= 0) { ld_words<4>(vtile + vmeta1 + tok_off, vlo1); ld_words<4>(vtile + vmeta1 + 256 + tok_off, vr1); }
-      // probabilities times the V group ranges, as fp16 pairs (group 0, group 1), transposed into B fragments
-      uint32_t pb[8];
+        for (int e = 0; e < 4; e++) acc_o[mb][e] *= alpha;
+    }
+    ok = ok && mbar_wait(bars + 8 * (4 + slot), parity);
+    // probabilities times the V group ranges, as fp16 pairs (group 0, group 1), transposed into B fragments
+    uint32_t pb[2][8];
+    {
+      uint32_t vr0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, vr1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      if (vmeta0 >= 0) ld_tile_words<8>(vtile + vmeta0 + 256 + 32 * gid, vr0);
+      if (vmeta1 >= 0) ld_tile_words<8>(vtile + vmeta1 + 256 + 32 * gid, vr1);
       if (boost < 0.f) {
-        // First half tile of this warp's share of the unit.  Probabilities are exp2(s - max) <= 1 and enter the
+        // First tile of this warp's share of the unit.  Probabilities are exp2(s - max) <= 1 and enter the
         // tensor core as fp16 times the V group range; with tens of thousands of tokens the typical probability is
         // far below the fp16 normal range.  Lift everything by 2^boost (the record's maximum is lowered by the same
-        // amount, so the merge is unaffected), leaving room for group ranges 8x larger than in this half tile.
+        // amount, so the merge is unaffected), leaving room for group ranges 8x larger than in this tile.
         float rmax = 0.f;
 #pragma unroll
-        for (int r = 0; r < 4; r++) {
+        for (int r = 0; r < 8; r++) {
           const float2 a = h2f2(vr0[r]), b = h2f2(vr1[r]);
           rmax = fmaxf(rmax, fmaxf(fmaxf(a.x, a.y), fmaxf(b.x, b.y)));
         }
@@ -417,29 +433,32 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
         boost = (float)max(0, min(13, 13 - e));
       }
       const float m_use = (m_run == -INFINITY ? 0.f : m_run) - boost;
+      uint32_t vlo0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, vlo1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      if (vmeta0 >= 0) ld_tile_words<8>(vtile + vmeta0 + 32 * gid, vlo0);
+      if (vmeta1 >= 0) ld_tile_words<8>(vtile + vmeta1 + 32 * gid, vlo1);
 #pragma unroll
-      for (int r = 0; r < 4; r++) {
+      for (int r = 0; r < 8; r++) {
         const float2 lo0 = h2f2(vlo0[r]), r0 = h2f2(vr0[r]), lo1 = h2f2(vlo1[r]), r1 = h2f2(vr1[r]);
 #pragma unroll
         for (int e = 0; e < 2; e++) {
-          const int ii = 2 * r + e;
-          const float pr = fast_exp2(s[ii] - m_use);
+          const int hp = r >> 2, ii = 2 * (r & 3) + e;
+          const float pr = fast_exp2(fmaf(s[8 * hp + ii], kscale, -m_use));
           l_run += pr;
           plo0 = fmaf(pr, e ? lo0.y : lo0.x, plo0);
           plo1 = fmaf(pr, e ? lo1.y : lo1.x, plo1);
-          pb[ii] = movmatrix_trans(pack_half2_sat(pr * (e ? r0.y : r0.x), pr * (e ? r1.y : r1.x)));
+          pb[hp][ii] = movmatrix_trans(pack_half2_sat(pr * (e ? r0.y : r0.x), pr * (e ? r1.y : r1.x)));
         }
       }
-      // ------------------------------------------------------------ P~ x V codes
-      v_class<8, Q8, 0, NACC>(vtile, vcls[0], hp, gid, tig, pb, acc_o);
-      v_class<4, Q4, Q8, NACC>(vtile, vcls[1], hp, gid, tig, pb, acc_o);
-      v_class<2, Q2, Q8 + Q4, NACC>(vtile, vcls[2], hp, gid, tig, pb, acc_o);
-      v_class<1, Q1, Q8 + Q4 + Q2, NACC>(vtile, vcls[3], hp, gid, tig, pb, acc_o);
-      if (hp == 1 && issued_v < issued_k) {
-        __syncwarp();
-        if (lane == 0) { fence_async_smem(); start_v(issued_v % D); }
-        issued_v++;
-      }
+    }
+    // ------------------------------------------------------------ P~ x V codes
+    v_class<8, Q8, 0, NACC>(vtile, vcls[0], gid, tig, pb, acc_o);
+    v_class<4, Q4, Q8, NACC>(vtile, vcls[1], gid, tig, pb, acc_o);
+    v_class<2, Q2, Q8 + Q4, NACC>(vtile, vcls[2], gid, tig, pb, acc_o);
+    v_class<1, Q1, Q8 + Q4 + Q2, NACC>(vtile, vcls[3], gid, tig, pb, acc_o);
+    if (issued_v < issued_k) {
+      __syncwarp();
+      if (lane == 0) { fence_async_smem(); start_v(issued_v % D); }
+      issued_v++;
     }
     // ------------------------------------------------------------ end of this warp's share of the unit?
     const bool last_of_unit = (cons.t + 1 >= cons.nt) || (j + 1 >= count);
