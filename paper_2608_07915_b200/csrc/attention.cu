@@ -36,7 +36,7 @@ FastLayout fast_layout(int64_t n_units, int total_warps, int vs_max) {
   size_t off = 0;
   L.desc_off = off; off = align_up(off + sizeof(UnitDesc) * (size_t)n_units, 256);
   L.prefix_off = off; off = align_up(off + sizeof(int32_t) * (size_t)(n_units + 1), 256);
-  L.warp_off = off; off = align_up(off + sizeof(int32_t) * (size_t)total_warps, 256);
+  L.warp_off = off; off = align_up(off + sizeof(int4) * (size_t)total_warps, 256);
   L.rec_off = off; off = align_up(off + sizeof(float) * (size_t)L.rec_stride * (size_t)(total_warps + n_units), 256);
   L.total = off;
   return L;
@@ -108,7 +108,7 @@ extern "C" size_t spectra_attention_workspace_bytes(const spectra_config* cfg, i
   int sms = sm_count();
   if (sms <= 0) sms = 160;
   const int npass = (n_q_heads / n_kv_heads + kFastGqa - 1) / kFastGqa;
-  const size_t fast = fast_layout(n_units * npass, sms * 3 * kFastWarps, kMaxStrips).total;
+  const size_t fast = fast_layout(n_units * npass, sms * kFastCtasPerSm * kFastWarps, kMaxStrips).total;
   return generic > fast ? generic : fast;
 }
 
@@ -176,7 +176,8 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
     const int slot_v = (int)align_up((size_t)(F.max_tile_v > 16 ? F.max_tile_v : 16), 128);
     const size_t pair = (size_t)slot_k + slot_v;
     const size_t budget = 200 * 1024;
-    int ctas_per_sm = 3 * kFastWarps * pair <= budget ? 3 : (2 * kFastWarps * pair <= budget ? 2 : 1);
+    int ctas_per_sm = kFastCtasPerSm;
+    while (ctas_per_sm > 1 && (size_t)ctas_per_sm * (kFastWarps * pair + 2048 + kFastWarps * (64 + kWarpStateBytes)) > budget) ctas_per_sm--;
     int depth = (int)(budget / ((size_t)ctas_per_sm * kFastWarps * pair));
     if (depth > 4) depth = 4;
     const int quota = pick_quota(F.vb);
@@ -188,7 +189,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       FastArgs f{};
       f.desc = reinterpret_cast<UnitDesc*>(ws + L.desc_off);
       f.tile_prefix = reinterpret_cast<int32_t*>(ws + L.prefix_off);
-      f.warp_unit = reinterpret_cast<int32_t*>(ws + L.warp_off);
+      f.warp_start = reinterpret_cast<int4*>(ws + L.warp_off);
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
       f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = vs_max;
       f.n_units = (int)n_vunits; f.npass = npass; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
@@ -210,7 +211,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       if (launch_status()) return SPECTRA_CUDA_ERROR;
       // the last chunk of a K run and the last block of a V class read up to 15 strips past the end of their class
       // (zero rows of B, unused accumulator rows): the pad keeps those reads inside the CTA's shared memory
-      const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64 + 2048;
+      const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64 + kFastWarps * kWarpStateBytes + 2048;
       const int grid = sms * ctas_per_sm;
       switch (quota) {
         case 0: rc = launch_fast_main<0, 1, 8, 2>(a, f, grid, smem, st); break;

@@ -31,6 +31,7 @@ constexpr int kFastGqa = 4;
 constexpr int kKcMax = 40;       // upper bound of B-table entries of a K tile: 384 strips in 8 (class, group) runs, each
                                  // run rounded up to whole chunks of 16 strips and a group-1 run starting on an even strip
 constexpr int kFastWarps = 4;    // warps per CTA of the main kernel
+constexpr int kFastCtasPerSm = 3; // CTAs of the main kernel per SM its register budget is set for
 constexpr int kRecHead = 4;      // floats of a record's per-head header: m, l, plo0, plo1
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -51,7 +52,7 @@ struct alignas(16) UnitDesc {
 };
 
 struct FastArgs {
-  UnitDesc* desc; int32_t* tile_prefix; int32_t* warp_unit; float* records;
+  UnitDesc* desc; int32_t* tile_prefix; int4* warp_start; float* records;
   int total_warps; int rec_stride; int vs_max;
   int n_units;       // units of the tensor path: (sequence, kv-head, pass); a pass takes up to 4 query heads of the group
   int npass;
@@ -217,14 +218,17 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
     __syncthreads();
     const int* pre = in_smem ? sprefix : f.tile_prefix;
     const long long total = pre[n_units];
+    // each worker warp's share of the flattened tile space: first unit with a tile of the share, first tile inside
+    // that unit, tiles of that unit, tiles of the share
     for (int gw = tid; gw < f.total_warps; gw += kPrepThreads) {
-      const long long g0 = (long long)gw * total / f.total_warps;
+      const long long g0 = (long long)gw * total / f.total_warps, g1 = (long long)(gw + 1) * total / f.total_warps;
       int lo = 0, hi = n_units;             // first unit whose end is beyond g0
       while (lo < hi) {
         const int mid = (lo + hi) >> 1;
         if (pre[mid + 1] > g0) hi = mid; else lo = mid + 1;
       }
-      f.warp_unit[gw] = lo;
+      const int u0 = min(lo, n_units - 1);
+      f.warp_start[gw] = make_int4(lo, (int)(g0 - pre[u0]), pre[u0 + 1] - pre[u0], (int)(g1 - g0));
     }
     return;
   }

@@ -114,58 +114,84 @@ __device__ __forceinline__ void half_tile_words(const uint32_t (&x)[W], uint32_t
 
 // One chunk (8 strip pairs x 128 tokens) into the score accumulators: per half tile, MMA u takes tokens u (row
 // gid) and u + 4 (row gid + 8), pair slots tig and tig + 4 as its k columns, and B variant u (scaled by
-// 2^-p_eff(u); rows of strips outside the run's scale group, or past the end of the class, are zero).
-template <int W, int HP>
-__device__ __forceinline__ void k_chunk_half(const uint32_t (&xa)[W], const uint32_t (&xb)[W], const uint4& b01,
-                                             const uint4& b23, float (&acc)[4][4]) {
+// 2^-p_eff(u); rows of strips outside the run's scale group, or past the end of the class, are zero).  The MMAs
+// that use variants 0 and 1 come first; then b01 is reloaded with the next chunk's entry while the MMAs of variants
+// 2 and 3 run, and b23 after those: the B fragments are fetched half a chunk ahead without a second set of registers.
+template <int W>
+__device__ __forceinline__ void k_chunk(const uint32_t (&xa)[W], const uint32_t (&xb)[W], uint4& b01, uint4& b23,
+                                        const uint4* __restrict__ kb_next, float (&acc)[2][4][4]) {
   using U = Unpack<W>;
   constexpr int NW = U::NW;
-  uint32_t wa[NW], wb[NW], was[NW], wbs[NW];
-  half_tile_words<W, HP>(xa, wa);
-  half_tile_words<W, HP>(xb, wb);
-  U::shifted(wa, was);
-  U::shifted(wb, wbs);
-  mma16816(acc[0], U::get(wa, was, 0), U::get(wa, was, 4), U::get(wb, wbs, 0), U::get(wb, wbs, 4), b01.x, b01.y);
-  mma16816(acc[1], U::get(wa, was, 1), U::get(wa, was, 5), U::get(wb, wbs, 1), U::get(wb, wbs, 5), b01.z, b01.w);
-  mma16816(acc[2], U::get(wa, was, 2), U::get(wa, was, 6), U::get(wb, wbs, 2), U::get(wb, wbs, 6), b23.x, b23.y);
-  mma16816(acc[3], U::get(wa, was, 3), U::get(wa, was, 7), U::get(wb, wbs, 3), U::get(wb, wbs, 7), b23.z, b23.w);
+  uint32_t wa0[NW], wb0[NW], was0[NW], wbs0[NW], wa1[NW], wb1[NW], was1[NW], wbs1[NW];
+  half_tile_words<W, 0>(xa, wa0);
+  half_tile_words<W, 0>(xb, wb0);
+  half_tile_words<W, 1>(xa, wa1);
+  half_tile_words<W, 1>(xb, wb1);
+  U::shifted(wa0, was0);
+  U::shifted(wb0, wbs0);
+  U::shifted(wa1, was1);
+  U::shifted(wb1, wbs1);
+  mma16816(acc[0][0], U::get(wa0, was0, 0), U::get(wa0, was0, 4), U::get(wb0, wbs0, 0), U::get(wb0, wbs0, 4), b01.x, b01.y);
+  mma16816(acc[1][0], U::get(wa1, was1, 0), U::get(wa1, was1, 4), U::get(wb1, wbs1, 0), U::get(wb1, wbs1, 4), b01.x, b01.y);
+  mma16816(acc[0][1], U::get(wa0, was0, 1), U::get(wa0, was0, 5), U::get(wb0, wbs0, 1), U::get(wb0, wbs0, 5), b01.z, b01.w);
+  mma16816(acc[1][1], U::get(wa1, was1, 1), U::get(wa1, was1, 5), U::get(wb1, wbs1, 1), U::get(wb1, wbs1, 5), b01.z, b01.w);
+  b01 = __ldg(kb_next);
+  mma16816(acc[0][2], U::get(wa0, was0, 2), U::get(wa0, was0, 6), U::get(wb0, wbs0, 2), U::get(wb0, wbs0, 6), b23.x, b23.y);
+  mma16816(acc[1][2], U::get(wa1, was1, 2), U::get(wa1, was1, 6), U::get(wb1, wbs1, 2), U::get(wb1, wbs1, 6), b23.x, b23.y);
+  mma16816(acc[0][3], U::get(wa0, was0, 3), U::get(wa0, was0, 7), U::get(wb0, wbs0, 3), U::get(wb0, wbs0, 7), b23.z, b23.w);
+  mma16816(acc[1][3], U::get(wa1, was1, 3), U::get(wa1, was1, 7), U::get(wb1, wbs1, 3), U::get(wb1, wbs1, 7), b23.z, b23.w);
+  b23 = __ldg(kb_next + 32);
 }
 
 // One (class, scale group) run of the K tile: `run` = byte offset / 16 of its first pair | chunks << 16 |
-// slot of a strip stored alone in the last chunk << 24 | (such a strip exists) << 27.  The B table is walked in the
-// same order; kb points at this lane's entry of the next chunk.
-template <int W>
+// slot of a strip stored alone in the last chunk << 24 | (such a strip exists) << 27.  A run has at most MAXC chunks
+// (64 channels per scale group; a group-1 run may start in the middle of a chunk).  The loop is unrolled with an
+// early exit, so that offsets are immediates and the next chunk's words are loaded while the current chunk is
+// multiplied.  The B table is walked in the same order; on entry b01, b23 hold the run's first entry and kb points
+// at this lane's part of it; on exit they hold the entry after the run (the first of the next run; past the last
+// run a spare entry of the table, never used).
+template <int W, int MAXC>
 __device__ __forceinline__ void k_run(const unsigned char* ktile, uint32_t run, const uint4* __restrict__& kb,
-                                      int gid, int tig, float (&acc)[2][4][4]) {
+                                      uint4& b01, uint4& b23, int gid, int tig, float (&acc)[2][4][4]) {
   const int nch = (int)(run >> 16) & 0xff;
   if (nch == 0) return;
   const unsigned char* pa = ktile + (run & 0xffffu) * 16 + 32 * W * tig + 4 * W * gid;
   const int lone_i = (run >> 27) & 1u ? nch - 1 : -1;
-#pragma unroll 1
-  for (int i = 0; i < nch; i++, pa += 256 * W, kb += 64) {
-    uint32_t xa[W], xb[W];
-    ld_tile_words<W>(pa, xa);
-    ld_tile_words<W>(pa + 128 * W, xb);
-    const uint4 b01 = __ldg(kb), b23 = __ldg(kb + 32);
-    if (i == lone_i) {
-      const int slot = (int)(run >> 24) & 7;
-      if (tig == (slot & 3)) {
-        // the pair of this slot is one strip stored alone: re-read it as half-words
-        const unsigned char* pl = pa - 32 * W * tig - 4 * W * gid + 32 * W * slot + 2 * W * gid;
-        if (slot & 4) ld_lone_words<W>(pl, xb);
-        else ld_lone_words<W>(pl, xa);
-      }
+  uint32_t xa[W], xb[W];
+  ld_tile_words<W>(pa, xa);
+  ld_tile_words<W>(pa + 128 * W, xb);
+#pragma unroll
+  for (int i = 0; i < MAXC; i++) {
+    if (i >= nch) break;
+    uint32_t ya[W], yb[W];
+    if (i + 1 < MAXC) {                       // the next chunk's words (whatever follows the run if this is its last)
+      ld_tile_words<W>(pa + 256 * W * (i + 1), ya);
+      ld_tile_words<W>(pa + 256 * W * (i + 1) + 128 * W, yb);
     }
-    k_chunk_half<W, 0>(xa, xb, b01, b23, acc[0]);
-    k_chunk_half<W, 1>(xa, xb, b01, b23, acc[1]);
+    if (i == lone_i) {
+      // the pair in slot `slot` of this chunk is one strip stored alone: the threads of that slot re-read it as
+      // half-words (all threads load, a select keeps the result where it belongs)
+      const int slot = (int)(run >> 24) & 7;
+      uint32_t t[W];
+      ld_lone_words<W>(ktile + (run & 0xffffu) * 16 + 256 * W * i + 32 * W * slot + 2 * W * gid, t);
+      const bool mine_a = tig == slot, mine_b = tig + 4 == slot;
+#pragma unroll
+      for (int k = 0; k < W; k++) { xa[k] = mine_a ? t[k] : xa[k]; xb[k] = mine_b ? t[k] : xb[k]; }
+    }
+    k_chunk<W>(xa, xb, b01, b23, kb + 64 * (i + 1), acc);
+    if (i + 1 < MAXC) {
+#pragma unroll
+      for (int k = 0; k < W; k++) { xa[k] = ya[k]; xb[k] = yb[k]; }
+    }
   }
+  kb += 64 * nch;
 }
 
 // One class of the V tile, at most Q blocks of 16 strips, accumulators acc_o[OFF .. OFF + Q).  The probabilities
 // first get the class's position scales; per half tile, MMA u of a block contracts the token pairs of B fragments
 // u and u + 4.  Rows past the end of the class read whatever follows in shared memory (finite after masking); their
 // accumulators are never stored.
-template <int W, int HP, int NACC>
+template <int W, int HP>
 __device__ __forceinline__ void v_block_half(const uint32_t (&xa)[W], const uint32_t (&xb)[W], const uint32_t (&pw)[8],
                                              float (&acc)[4]) {
   using U = Unpack<W>;
@@ -192,14 +218,22 @@ __device__ __forceinline__ void v_class(const unsigned char* vtile, uint32_t cls
 #pragma unroll
       for (int ii = 0; ii < 8; ii++) pw[hp][ii] = hmul2_pow2(pb[hp][ii], U::peff(ii));
     const unsigned char* cbase = vtile + (cls >> 16) * 16 + 4 * W * tig + 16 * W * gid;
+    uint32_t xa[W], xb[W];
+    ld_tile_words<W>(cbase, xa);
+    ld_tile_words<W>(cbase + 16 * W * 8, xb);
 #pragma unroll
     for (int bi = 0; bi < Q; bi++) {
-      if (16 * bi < n) {
-        uint32_t xa[W], xb[W];
-        ld_tile_words<W>(cbase + 16 * W * (16 * bi), xa);
-        ld_tile_words<W>(cbase + 16 * W * (16 * bi + 8), xb);
-        v_block_half<W, 0, NACC>(xa, xb, pw[0], acc_o[OFF + bi]);
-        v_block_half<W, 1, NACC>(xa, xb, pw[1], acc_o[OFF + bi]);
+      if (16 * bi >= n) break;
+      uint32_t ya[W], yb[W];
+      if (bi + 1 < Q) {                       // the next block's words (whatever follows the class if this is its last)
+        ld_tile_words<W>(cbase + 16 * W * (16 * bi + 16), ya);
+        ld_tile_words<W>(cbase + 16 * W * (16 * bi + 24), yb);
+      }
+      v_block_half<W, 0>(xa, xb, pw[0], acc_o[OFF + bi]);
+      v_block_half<W, 1>(xa, xb, pw[1], acc_o[OFF + bi]);
+      if (bi + 1 < Q) {
+#pragma unroll
+        for (int k = 0; k < W; k++) { xa[k] = ya[k]; xb[k] = yb[k]; }
       }
     }
   }
@@ -227,44 +261,50 @@ __device__ __forceinline__ uint32_t pack_half2_sat(float a, float b) {
   return d;
 }
 
-struct TileCursor {   // walks the flattened (unit, tile) space; all fields are warp-uniform
-  int u, t, nt;
-  __device__ __forceinline__ void seek_unit(const FastArgs& f) {
-    while (u < f.n_units) {
-      nt = f.tile_prefix[u + 1] - f.tile_prefix[u];
-      if (t < nt) break;
-      u++; t = 0;
-    }
-  }
-  __device__ __forceinline__ void next(const FastArgs& f) {
-    t++;
-    if (t >= nt) { u++; t = 0; seek_unit(f); }
-  }
+// Per-warp state in shared memory: the head of the current unit's descriptor (read as broadcast loads where it is
+// used, instead of sitting in registers through the whole tile) and the two producer cursors, which only lane 0
+// touches: the next tile to copy is the previous one plus the tile size until the unit's tiles run out.
+struct TileProducer {
+  uint64_t addr;         // global address of the next tile to copy
+  uint32_t tb;           // tile bytes of the unit
+  int32_t rem;           // tiles of the unit not yet copied
+  int32_t unit, pad;
 };
+struct WarpState {
+  alignas(16) uint32_t head[20];   // UnitDesc words 0..5 (tbk, tbv, kmeta[2], vmeta[2]), two spare words, then words
+                                   // 6..17 (krun[2][4], vcls[4]) on 16-byte boundaries
+  TileProducer k, v;
+};
+static_assert(sizeof(WarpState) == 128, "WarpState layout");
+constexpr int kWarpStateBytes = 128;
 
 // Adds one scale group's share to the scores of this thread's 16 tokens, in units of 1 / kscale:
 // s'_t += R_t * (hi + lo partial sums) + lo_t * (sum of q' over the group's active channels / kscale).
 // meta points at lo16[16 gid] of the group; R16 follows 256 bytes later.
+template <bool FIRST>
 __device__ __forceinline__ void fold_group(const unsigned char* meta, float qlo, const float (&acc)[2][4][4],
-                                           float (&s)[16], bool first) {
-  uint32_t lo[8], rg[8];
-  ld_tile_words<8>(meta, lo);
-  ld_tile_words<8>(meta + 256, rg);
+                                           float (&s)[16]) {
 #pragma unroll
-  for (int r = 0; r < 8; r++) {
-    const float2 l2 = h2f2(lo[r]), r2 = h2f2(rg[r]);
+  for (int half = 0; half < 2; half++) {
+    uint32_t lo[4], rg[4];
+    ld_tile_words<4>(meta + 16 * half, lo);
+    ld_tile_words<4>(meta + 256 + 16 * half, rg);
 #pragma unroll
-    for (int e = 0; e < 2; e++) {
-      const int hp = r >> 2, ii = 2 * (r & 3) + e, u = ii & 3, cb = (ii >> 2) * 2;
-      const float a = acc[hp][u][cb] + acc[hp][u][cb + 1];            // hi + lo halves of q'
-      const float base = first ? (e ? l2.y : l2.x) * qlo : fmaf(e ? l2.y : l2.x, qlo, s[8 * hp + ii]);
-      s[8 * hp + ii] = fmaf(e ? r2.y : r2.x, a, base);
+    for (int r = 0; r < 4; r++) {
+      const float2 l2 = h2f2(lo[r]), r2 = h2f2(rg[r]);
+#pragma unroll
+      for (int e = 0; e < 2; e++) {
+        const int ii = 2 * r + e, u = ii & 3, cb = (ii >> 2) * 2;
+        const float a = acc[half][u][cb] + acc[half][u][cb + 1];            // hi + lo halves of q'
+        const float base = FIRST ? (e ? l2.y : l2.x) * qlo : fmaf(e ? l2.y : l2.x, qlo, s[8 * half + ii]);
+        s[8 * half + ii] = fmaf(e ? r2.y : r2.x, a, base);
+      }
     }
   }
 }
 
 template <int Q8, int Q4, int Q2, int Q1>
-__global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnArgs p, FastArgs f) {
+__global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma_kernel(AttnArgs p, FastArgs f) {
   constexpr int NACC = Q8 + Q4 + Q2 + Q1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -275,68 +315,82 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
   unsigned char* ring_k = smem_raw + warp * warp_bytes;
   unsigned char* ring_v = ring_k + D * f.slot_k;
   const uint32_t bars = smem_u32(smem_raw) + kFastWarps * warp_bytes + warp * (2 * 4 * 8);  // K slots 0..3, V slots 0..3
+  WarpState& ws = *reinterpret_cast<WarpState*>(smem_raw + kFastWarps * warp_bytes + kFastWarps * 64 + warp * kWarpStateBytes);
   if (lane == 0)
     for (int s = 0; s < 2 * 4; s++) mbar_init(bars + 8 * s, 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncwarp();
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel may be scheduled as SMs free up
-  const long long total = f.tile_prefix[f.n_units];
-  const long long g0 = (long long)gw * total / f.total_warps;
-  const long long g1 = (long long)(gw + 1) * total / f.total_warps;
-  const int count = (int)(g1 - g0);
+  const int4 start = f.warp_start[gw];                 // first unit, first tile in it, tiles of that unit, tiles of the share
+  const int count = start.w;
   if (count <= 0) return;
-
-  TileCursor cons, prod;
-  cons.u = f.warp_unit[gw]; cons.t = (int)(g0 - f.tile_prefix[cons.u]); cons.nt = 0; cons.seek_unit(f);
-  prod = cons;
-  // Copies are started by lane 0; every lane keeps the same counts of tiles whose K / V copy has been started.
-  int issued_k = 0, issued_v = 0;
-  const uint8_t* v_src = nullptr;   // V tile that goes with the most recently started K tile (lane 0)
-  uint32_t v_bytes = 0;
+  int cu = start.x, ct = start.y, cnt = start.z;       // consumer: unit, tile, tiles of the unit
+  // Copies are started by lane 0, whose cursors live in shared memory; every lane keeps the same counts of tiles
+  // whose K / V copy has been started.  A unit's tiles are contiguous: its next tile is one tile size further.
+  auto next_unit = [&](TileProducer& q, int side) {    // the unit's tiles are used up: move to the next unit with tiles
+    int u = q.unit + 1, n = 0;
+    while (u < f.n_units) {
+      n = f.tile_prefix[u + 1] - f.tile_prefix[u];
+      if (n > 0) break;
+      u++;
+    }
+    const UnitDesc& d = f.desc[min(u, f.n_units - 1)];
+    q.unit = u; q.rem = n;
+    q.tb = side ? d.tbv : d.tbk;
+    q.addr = (uint64_t)(side ? p.cache_v + p.off_v[u / f.npass] : p.cache_k + p.off_k[u / f.npass]);
+  };
   auto start_k = [&](int slot) {
-    const UnitDesc& d = f.desc[prod.u];
-    const uint32_t tbk = d.tbk, tbv = d.tbv;
-    mbar_expect_tx(bars + 8 * slot, tbk);
-    bulk_load(smem_u32(ring_k + slot * f.slot_k), p.cache_k + p.off_k[prod.u / f.npass] + (int64_t)prod.t * tbk, tbk,
-              bars + 8 * slot, l2_evict_first_policy());
-    v_src = p.cache_v + p.off_v[prod.u / f.npass] + (int64_t)prod.t * tbv;
-    v_bytes = tbv;
-    prod.next(f);
+    if (ws.k.rem == 0) next_unit(ws.k, 0);
+    const uint32_t tb = ws.k.tb;
+    const uint64_t a = ws.k.addr;
+    mbar_expect_tx(bars + 8 * slot, tb);
+    bulk_load(smem_u32(ring_k + slot * f.slot_k), (const void*)a, tb, bars + 8 * slot
+              , l2_evict_first_policy()
+              );
+    ws.k.addr = a + tb; ws.k.rem--;
   };
   auto start_v = [&](int slot) {
-    mbar_expect_tx(bars + 8 * (4 + slot), v_bytes);
-    bulk_load(smem_u32(ring_v + slot * f.slot_v), v_src, v_bytes, bars + 8 * (4 + slot),
-              l2_evict_first_policy());
+    if (ws.v.rem == 0) next_unit(ws.v, 1);
+    const uint32_t tb = ws.v.tb;
+    const uint64_t a = ws.v.addr;
+    mbar_expect_tx(bars + 8 * (4 + slot), tb);
+    bulk_load(smem_u32(ring_v + slot * f.slot_v), (const void*)a, tb, bars + 8 * (4 + slot)
+              , l2_evict_first_policy()
+              );
+    ws.v.addr = a + tb; ws.v.rem--;
   };
-  if (lane == 0)
-    for (int j = 0; j < min(D, count); j++) { start_k(j); start_v(j); }
-  issued_k = issued_v = min(D, count);
+  int issued_k = min(D, count), issued_v = issued_k;
+  int fill_k = issued_k % D, fill_v = fill_k;           // slots the next K / V copies go to
+  if (lane == 0) {
+    const UnitDesc& d = f.desc[cu];
+    const uint32_t tbk = d.tbk, tbv = d.tbv;
+    ws.k.unit = cu; ws.k.rem = cnt - ct; ws.k.tb = tbk;
+    ws.k.addr = (uint64_t)(p.cache_k + p.off_k[cu / f.npass] + (int64_t)ct * tbk);
+    ws.v.unit = cu; ws.v.rem = cnt - ct; ws.v.tb = tbv;
+    ws.v.addr = (uint64_t)(p.cache_v + p.off_v[cu / f.npass] + (int64_t)ct * tbv);
+    for (int j = 0; j < issued_k; j++) { start_k(j); start_v(j); }
+  }
 
   float acc_o[NACC][4];
   float m_run = -INFINITY, l_run = 0.f, plo0 = 0.f, plo1 = 0.f;
-  uint32_t krun[2][4], vcls[4];
-  int kmeta0 = -1, kmeta1 = -1, vmeta0 = -1, vmeta1 = -1;
   float kscale = 0.f, qlo0 = 0.f, qlo1 = 0.f;
-  const uint4* kB = nullptr;
   int n_seq = 0;
   bool fresh = true, ok = true;
   float boost = 0.f;          // power-of-two lift of the probabilities (see below); -1 = not chosen yet
+  int slot = 0;
+  uint32_t parity = 0;
 
   for (int j = 0; j < count && ok; j++) {
-    const int slot = j % D;
-    const uint32_t parity = (uint32_t)(j / D) & 1u;
     const unsigned char* ktile = ring_k + slot * f.slot_k;
     const unsigned char* vtile = ring_v + slot * f.slot_v;
     if (fresh) {
-      const UnitDesc& d = f.desc[cons.u];
-#pragma unroll
-      for (int c = 0; c < 4; c++) { krun[0][c] = d.krun[0][c]; krun[1][c] = d.krun[1][c]; vcls[c] = d.vcls[c]; }
-      kmeta0 = d.kmeta[0]; kmeta1 = d.kmeta[1]; vmeta0 = d.vmeta[0]; vmeta1 = d.vmeta[1];
+      const UnitDesc& d = f.desc[cu];
+      __syncwarp();
+      if (lane < 18) ws.head[lane < 6 ? lane : lane + 2] = reinterpret_cast<const uint32_t*>(&d)[lane];
       kscale = d.kscale[tig];                                  // a power of two: the divisions are exact
       qlo0 = d.qlo[tig][0] / kscale; qlo1 = d.qlo[tig][1] / kscale;
-      kB = &d.kB[0][0][0];
-      n_seq = p.seq_len[(cons.u / f.npass) / p.n_kv];
+      n_seq = p.seq_len[(cu / f.npass) / p.n_kv];
 #pragma unroll
       for (int mb = 0; mb < NACC; mb++)
 #pragma unroll
@@ -344,51 +398,57 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
       m_run = -INFINITY; l_run = 0.f; plo0 = 0.f; plo1 = 0.f;
       fresh = false;
       boost = -1.f;
+      __syncwarp();
     }
 
     // ------------------------------------------------------------ scores of the tile's 128 tokens, in units of 1 / kscale
     ok = mbar_wait(bars + 8 * slot, parity);
     float s[16];
     {
-      const uint4* kb = kB + lane;       // walks the B fragment table in run order
+      const uint4* kb = &f.desc[cu].kB[0][0][0] + lane;   // walks the B fragment table in run order, one entry ahead
+      uint4 b01 = __ldg(kb), b23 = __ldg(kb + 32);
+      const int kmeta0 = (int)ws.head[2], kmeta1 = (int)ws.head[3];
       float acc[2][4][4];
       if (kmeta0 >= 0) {
+        const uint4 runs = *reinterpret_cast<const uint4*>(&ws.head[8]);
 #pragma unroll
         for (int hp = 0; hp < 2; hp++)
 #pragma unroll
           for (int u = 0; u < 4; u++)
 #pragma unroll
             for (int e = 0; e < 4; e++) acc[hp][u][e] = 0.f;
-        k_run<8>(ktile, krun[0][0], kb, gid, tig, acc);
-        k_run<4>(ktile, krun[0][1], kb, gid, tig, acc);
-        k_run<2>(ktile, krun[0][2], kb, gid, tig, acc);
-        k_run<1>(ktile, krun[0][3], kb, gid, tig, acc);
-        fold_group(ktile + kmeta0 + 32 * gid, qlo0, acc, s, true);
+        k_run<8, 4>(ktile, runs.x, kb, b01, b23, gid, tig, acc);
+        k_run<4, 4>(ktile, runs.y, kb, b01, b23, gid, tig, acc);
+        k_run<2, 4>(ktile, runs.z, kb, b01, b23, gid, tig, acc);
+        k_run<1, 4>(ktile, runs.w, kb, b01, b23, gid, tig, acc);
+        fold_group<true>(ktile + kmeta0 + 32 * gid, qlo0, acc, s);
       } else {
 #pragma unroll
         for (int i = 0; i < 16; i++) s[i] = 0.f;
       }
       if (kmeta1 >= 0) {
+        const uint4 runs = *reinterpret_cast<const uint4*>(&ws.head[12]);
 #pragma unroll
         for (int hp = 0; hp < 2; hp++)
 #pragma unroll
           for (int u = 0; u < 4; u++)
 #pragma unroll
             for (int e = 0; e < 4; e++) acc[hp][u][e] = 0.f;
-        k_run<8>(ktile, krun[1][0], kb, gid, tig, acc);
-        k_run<4>(ktile, krun[1][1], kb, gid, tig, acc);
-        k_run<2>(ktile, krun[1][2], kb, gid, tig, acc);
-        k_run<1>(ktile, krun[1][3], kb, gid, tig, acc);
-        fold_group(ktile + kmeta1 + 32 * gid, qlo1, acc, s, false);
+        k_run<8, 5>(ktile, runs.x, kb, b01, b23, gid, tig, acc);
+        k_run<4, 5>(ktile, runs.y, kb, b01, b23, gid, tig, acc);
+        k_run<2, 5>(ktile, runs.z, kb, b01, b23, gid, tig, acc);
+        k_run<1, 5>(ktile, runs.w, kb, b01, b23, gid, tig, acc);
+        fold_group<false>(ktile + kmeta1 + 32 * gid, qlo1, acc, s);
       }
     }
     if (issued_k < count) {     // the K slot is free: refill it with the tile D positions ahead
       __syncwarp();
-      if (lane == 0) { fence_async_smem(); start_k(issued_k % D); }
+      if (lane == 0) { fence_async_smem(); start_k(fill_k); }
       issued_k++;
+      fill_k = fill_k + 1 == D ? 0 : fill_k + 1;
     }
-    if ((cons.t + 1) * kTile > n_seq) {                      // only the unit's last tile has slots past the end
-      const int tok0 = cons.t * kTile + gid * 16;
+    if ((ct + 1) * kTile > n_seq) {                      // only the unit's last tile has slots past the end
+      const int tok0 = ct * kTile + gid * 16;
 #pragma unroll
       for (int i = 0; i < 16; i++)
         if (tok0 + i >= n_seq) s[i] = -INFINITY;
@@ -413,14 +473,15 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
     // probabilities times the V group ranges, as fp16 pairs (group 0, group 1), transposed into B fragments
     uint32_t pb[2][8];
     {
-      uint32_t vr0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, vr1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-      if (vmeta0 >= 0) ld_tile_words<8>(vtile + vmeta0 + 256 + 32 * gid, vr0);
-      if (vmeta1 >= 0) ld_tile_words<8>(vtile + vmeta1 + 256 + 32 * gid, vr1);
+      const int vmeta0 = (int)ws.head[4], vmeta1 = (int)ws.head[5];
       if (boost < 0.f) {
         // First tile of this warp's share of the unit.  Probabilities are exp2(s - max) <= 1 and enter the
         // tensor core as fp16 times the V group range; with tens of thousands of tokens the typical probability is
         // far below the fp16 normal range.  Lift everything by 2^boost (the record's maximum is lowered by the same
         // amount, so the merge is unaffected), leaving room for group ranges 8x larger than in this tile.
+        uint32_t vr0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, vr1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        if (vmeta0 >= 0) ld_tile_words<8>(vtile + vmeta0 + 256 + 32 * gid, vr0);
+        if (vmeta1 >= 0) ld_tile_words<8>(vtile + vmeta1 + 256 + 32 * gid, vr1);
         float rmax = 0.f;
 #pragma unroll
         for (int r = 0; r < 8; r++) {
@@ -433,35 +494,48 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
         boost = (float)max(0, min(13, 13 - e));
       }
       const float m_use = (m_run == -INFINITY ? 0.f : m_run) - boost;
-      uint32_t vlo0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, vlo1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-      if (vmeta0 >= 0) ld_tile_words<8>(vtile + vmeta0 + 32 * gid, vlo0);
-      if (vmeta1 >= 0) ld_tile_words<8>(vtile + vmeta1 + 32 * gid, vlo1);
 #pragma unroll
-      for (int r = 0; r < 8; r++) {
-        const float2 lo0 = h2f2(vlo0[r]), r0 = h2f2(vr0[r]), lo1 = h2f2(vlo1[r]), r1 = h2f2(vr1[r]);
+      for (int half = 0; half < 2; half++) {
+        uint32_t vlo0[4] = {0, 0, 0, 0}, vlo1[4] = {0, 0, 0, 0}, vr0[4] = {0, 0, 0, 0}, vr1[4] = {0, 0, 0, 0};
+        if (vmeta0 >= 0) {
+          ld_tile_words<4>(vtile + vmeta0 + 32 * gid + 16 * half, vlo0);
+          ld_tile_words<4>(vtile + vmeta0 + 256 + 32 * gid + 16 * half, vr0);
+        }
+        if (vmeta1 >= 0) {
+          ld_tile_words<4>(vtile + vmeta1 + 32 * gid + 16 * half, vlo1);
+          ld_tile_words<4>(vtile + vmeta1 + 256 + 32 * gid + 16 * half, vr1);
+        }
 #pragma unroll
-        for (int e = 0; e < 2; e++) {
-          const int hp = r >> 2, ii = 2 * (r & 3) + e;
-          const float pr = fast_exp2(fmaf(s[8 * hp + ii], kscale, -m_use));
-          l_run += pr;
-          plo0 = fmaf(pr, e ? lo0.y : lo0.x, plo0);
-          plo1 = fmaf(pr, e ? lo1.y : lo1.x, plo1);
-          pb[hp][ii] = movmatrix_trans(pack_half2_sat(pr * (e ? r0.y : r0.x), pr * (e ? r1.y : r1.x)));
+        for (int r = 0; r < 4; r++) {
+          const float2 lo0 = h2f2(vlo0[r]), r0 = h2f2(vr0[r]), lo1 = h2f2(vlo1[r]), r1 = h2f2(vr1[r]);
+#pragma unroll
+          for (int e = 0; e < 2; e++) {
+            const int ii = 2 * r + e;
+            const float pr = fast_exp2(fmaf(s[8 * half + ii], kscale, -m_use));
+            l_run += pr;
+            plo0 = fmaf(pr, e ? lo0.y : lo0.x, plo0);
+            plo1 = fmaf(pr, e ? lo1.y : lo1.x, plo1);
+            pb[half][ii] = movmatrix_trans(pack_half2_sat(pr * (e ? r0.y : r0.x), pr * (e ? r1.y : r1.x)));
+          }
         }
       }
     }
     // ------------------------------------------------------------ P~ x V codes
-    v_class<8, Q8, 0, NACC>(vtile, vcls[0], gid, tig, pb, acc_o);
-    v_class<4, Q4, Q8, NACC>(vtile, vcls[1], gid, tig, pb, acc_o);
-    v_class<2, Q2, Q8 + Q4, NACC>(vtile, vcls[2], gid, tig, pb, acc_o);
-    v_class<1, Q1, Q8 + Q4 + Q2, NACC>(vtile, vcls[3], gid, tig, pb, acc_o);
+    {
+      const uint4 vc = *reinterpret_cast<const uint4*>(&ws.head[16]);
+      v_class<8, Q8, 0, NACC>(vtile, vc.x, gid, tig, pb, acc_o);
+      v_class<4, Q4, Q8, NACC>(vtile, vc.y, gid, tig, pb, acc_o);
+      v_class<2, Q2, Q8 + Q4, NACC>(vtile, vc.z, gid, tig, pb, acc_o);
+      v_class<1, Q1, Q8 + Q4 + Q2, NACC>(vtile, vc.w, gid, tig, pb, acc_o);
+    }
     if (issued_v < issued_k) {
       __syncwarp();
-      if (lane == 0) { fence_async_smem(); start_v(issued_v % D); }
+      if (lane == 0) { fence_async_smem(); start_v(fill_v); }
       issued_v++;
+      fill_v = fill_v + 1 == D ? 0 : fill_v + 1;
     }
     // ------------------------------------------------------------ end of this warp's share of the unit?
-    const bool last_of_unit = (cons.t + 1 >= cons.nt) || (j + 1 >= count);
+    const bool last_of_unit = (ct + 1 >= cnt) || (j + 1 >= count);
     if (last_of_unit) {
       float l = l_run, q0 = plo0, q1 = plo1;
 #pragma unroll
@@ -470,16 +544,26 @@ __global__ void __launch_bounds__(kFastWarps * 32, 3) attention_mma_kernel(AttnA
         q0 += __shfl_xor_sync(0xffffffffu, q0, sft);
         q1 += __shfl_xor_sync(0xffffffffu, q1, sft);
       }
-      float* rec = f.records + (int64_t)(gw + cons.u) * f.rec_stride + tig * (kRecHead + f.vs_max);
+      float* rec = f.records + (int64_t)(gw + cu) * f.rec_stride + tig * (kRecHead + f.vs_max);
       if (gid == 0) { rec[0] = m_run - boost; rec[1] = l; rec[2] = q0; rec[3] = q1; }
-      const UnitDesc& d = f.desc[cons.u];
-      store_class<Q8, 0, NACC>(rec, vcls[0], d.vfirst[0], gid, acc_o);
-      store_class<Q4, Q8, NACC>(rec, vcls[1], d.vfirst[1], gid, acc_o);
-      store_class<Q2, Q8 + Q4, NACC>(rec, vcls[2], d.vfirst[2], gid, acc_o);
-      store_class<Q1, Q8 + Q4 + Q2, NACC>(rec, vcls[3], d.vfirst[3], gid, acc_o);
+      const UnitDesc& d = f.desc[cu];
+      store_class<Q8, 0, NACC>(rec, ws.head[16], d.vfirst[0], gid, acc_o);
+      store_class<Q4, Q8, NACC>(rec, ws.head[17], d.vfirst[1], gid, acc_o);
+      store_class<Q2, Q8 + Q4, NACC>(rec, ws.head[18], d.vfirst[2], gid, acc_o);
+      store_class<Q1, Q8 + Q4 + Q2, NACC>(rec, ws.head[19], d.vfirst[3], gid, acc_o);
       fresh = true;
     }
-    cons.next(f);
+    // next tile of the flattened (unit, tile) space
+    ct++;
+    if (ct >= cnt) {
+      cu++; ct = 0;
+      while (cu < f.n_units) {
+        cnt = f.tile_prefix[cu + 1] - f.tile_prefix[cu];
+        if (cnt > 0) break;
+        cu++;
+      }
+    }
+    if (++slot == D) { slot = 0; parity ^= 1u; }
   }
   if (!ok) {
     if (lane == 0 && p.status) atomicOr(p.status, SPECTRA_STATUS_WAIT_TIMEOUT);
