@@ -2,6 +2,8 @@
 import itertools
 import os
 
+import math
+
 import numpy as np
 import pytest
 
@@ -215,20 +217,101 @@ def test_latent_attention_equals_reconstruct_then_attend(mode):
     assert np.abs(la - lb).max() <= 1e-10
 
 
-def test_attention_at_eight_bits_matches_dense_textbook_attention():
+def _handworked_case():
+    """Three tokens, d = 8, scale group 4, widths chosen so that every rotated coordinate lies exactly on its
+    quantiser grid (group minimum, range and step are exact binary fractions): yhat = y with no rounding anywhere.
+    Transforms are signed, scaled permutations (not involutions, so a transposed matrix changes the result) and
+    the rotated means are as large as the data.  Everything below the inputs was worked out by hand."""
+    d, gs = 8, 4
+    k = dict(
+        widths=np.array([2, 2, 2, 2, 1, 1, 0, 1], np.uint8),       # channel 6 is dropped: it reconstructs to its mean
+        # group 0 (3 levels above the minimum): steps 1, 1, 0.25; group 1 (one bit): ranges 2, 1 and a constant group
+        y=np.array([[-1.5, -0.5, 0.5, 1.5, 0, 2, 7.0, 2],
+                    [1, -2, 0, -1, -1, 0, 7.0, -1],
+                    [0.25, 1, 0.5, 0.75, 3, 3, 7.0, 3]], np.float32),
+        m=np.array([0.5, -1, 2, 0, 1, 0, 3, -0.5], np.float32),
+        perm=[2, 0, 3, 1, 6, 4, 7, 5], coef=[1, 2, -1, 0.5, 1, -2, 1, 4])
+    v = dict(
+        widths=np.array([2, 2, 0, 2, 1, 1, 1, 1], np.uint8),
+        y=np.array([[2, -1, 9.0, 1, -4, -4, -2, -4],
+                    [0, 0.75, 9.0, 0.25, 1, 1, 1, 1],
+                    [-3, 3, 9.0, 1, 0.5, 1.5, 1.5, 0.5]], np.float32),
+        m=np.array([-1, 0.5, 2, 1, 0, -2, 0.25, 4], np.float32),
+        perm=[1, 3, 0, 2, 5, 7, 4, 6], coef=[2, 1, -1, 4, 0.5, 1, -2, 1])
+    for side, c in ((codec.SIDE_K, k), (codec.SIDE_V, v)):
+        w = np.zeros((d, d), np.float32)                            # xhat_i = coef_i * (yhat + m')_{perm_i}
+        for i in range(d):
+            w[c["perm"][i], i] = c["coef"][i]
+        c["wd"] = w
+        c["tb"] = codec.tile_bytes(c["widths"], gs)
+        c["cache"] = np.zeros(c["tb"], np.uint8)
+        st, _ = codec.encode_unit(c["y"], w, c["m"], c["widths"], gs, side, 0, c["cache"], c["tb"], rotated_input=True)
+        assert st == 0
+    # By hand: z = yhat + m' (dropped channel: z = m'), then xhat_i = coef_i * z_{perm_i}
+    k_hat = np.array([[2.5, -2.0, -1.5, -0.75, 3.0, -2.0, 1.5, 8.0],
+                      [2.0, 3.0, 1.0, -1.5, 3.0, 0.0, -1.5, 0.0],
+                      [2.5, 1.5, -0.75, 0.0, 3.0, -8.0, 2.5, 12.0]])
+    v_hat = np.array([[-1.0, 2.0, -1.0, 8.0, -3.0, 0.0, 8.0, -1.75],
+                      [2.5, 1.25, 1.0, 8.0, -0.5, 5.0, -2.0, 1.25],
+                      [7.0, 2.0, 4.0, 8.0, -0.25, 4.5, -1.0, 1.75]])
+    return d, gs, k, v, k_hat, v_hat
+
+
+@pytest.mark.parametrize("mode", ["A", "B"])
+def test_attention_on_a_handworked_case(mode):
+    """Sec. 3.3 (Mode A: reconstruct, then attend) and the appendix "Latent-space attention and memory" (Mode B:
+    q' = q W_up^T, scores q' c^T, one lift of the output) on a case small enough to work by hand, with rotated
+    means m'_K, m'_V that matter, a dropped channel and a constant group.  Head 0 has q = 0: every score is equal,
+    the output is the plain mean of the three reconstructed values and lse = ln 3.  Head 1: the three scores
+    scale * q . k_hat_t are 0.125, -0.625 and -0.4375."""
+    d, gs, k, v, k_hat, v_hat = _handworked_case()
+    _, xk = codec.decode_unit(k["cache"], k["tb"], 3, k["wd"], k["m"], k["widths"], gs, codec.SIDE_K)
+    _, xv = codec.decode_unit(v["cache"], v["tb"], 3, v["wd"], v["m"], v["widths"], gs, codec.SIDE_V)
+    assert np.array_equal(xk, k_hat) and np.array_equal(xv, v_hat)
+    q = np.array([[0.0] * 8, [0.5, -0.25, 0, 1, 0, 0.125, 0, -0.0625]])
+    out, lse = codec.attention_units(mode, q[None], [3], k["cache"], [0], [k["tb"]], v["cache"], [0], [v["tb"]],
+                                     k["wd"][None], k["m"][None], k["widths"][None], v["wd"][None], v["m"][None],
+                                     v["widths"][None], gs, 0.5)
+    mean_v = [(-1.0 + 2.5 + 7.0) / 3, (2.0 + 1.25 + 2.0) / 3, (-1.0 + 1.0 + 4.0) / 3, 8.0, (-3.0 - 0.5 - 0.25) / 3,
+              (0.0 + 5.0 + 4.5) / 3, (8.0 - 2.0 - 1.0) / 3, (-1.75 + 1.25 + 1.75) / 3]
+    assert np.abs(out[0, 0] - mean_v).max() <= 1e-14
+    assert abs(lse[0, 0] - math.log(3.0)) <= 1e-14
+    e = [math.exp(0.125), math.exp(-0.625), math.exp(-0.4375)]
+    want = [(e[0] * v_hat[0][i] + e[1] * v_hat[1][i] + e[2] * v_hat[2][i]) / sum(e) for i in range(8)]
+    assert np.abs(out[0, 1] - want).max() <= 1e-14
+    assert abs(lse[0, 1] - math.log(sum(e))) <= 1e-14
+    # one token fewer is a different answer: the functions attend to exactly n tokens
+    out2, _ = codec.attention_units(mode, q[None], [2], k["cache"], [0], [k["tb"]], v["cache"], [0], [v["tb"]],
+                                    k["wd"][None], k["m"][None], k["widths"][None], v["wd"][None], v["m"][None],
+                                    v["widths"][None], gs, 0.5)
+    assert np.abs(out2[0, 0] - (v_hat[0] + v_hat[1]) / 2).max() <= 1e-14
+
+
+def test_attention_at_eight_bits_is_within_the_quantisation_bound_of_dense_attention():
+    """Mode A at 8 bits per channel against textbook softmax attention on the raw vectors.  The tolerance is the
+    bound the quantisation error itself gives: with delta = max_t |scale q.(k_hat_t - k_t)| the softmax weights
+    move by at most e^(2 delta) - 1 in total variation, so
+        |out - dense| <= max_t |v_hat_t - v_t|_inf + (e^(2 delta) - 1) max_t |v_t|_inf,   |lse - lse_dense| <= delta."""
     n = 256
     c = _coded_tiny(4.0, fit.GAIN_WHITEN, n, widths_override=8)
     q = si.draw_queries(si.WORKLOADS["tiny"], 0, 0).astype(np.float64)
     oa, la = _attend(c, q, "A", n)
     K, V = c["k"]["X"].astype(np.float64), c["v"]["X"].astype(np.float64)
-    s = q @ K.T / np.sqrt(128.0)
+    k, v = c["k"], c["v"]
+    _, k_hat = codec.decode_unit(k["cache"], k["tb"], n, k["wd"], k["mr"], k["widths"], 64, codec.SIDE_K)
+    _, v_hat = codec.decode_unit(v["cache"], v["tb"], n, v["wd"], v["mr"], v["widths"], 64, codec.SIDE_V)
+    scale = 1.0 / np.sqrt(128.0)
+    s = q @ K.T * scale
     p = np.exp(s - s.max(axis=1, keepdims=True))
     lse = np.log(p.sum(axis=1)) + s.max(axis=1)
     p /= p.sum(axis=1, keepdims=True)
     assert np.allclose(p.sum(axis=1), 1.0)
     dense = p @ V
-    assert np.abs(oa[0] - dense).max() <= 2e-2 * np.abs(dense).max()
-    assert np.abs(la[0] - lse).max() <= 5e-2
+    delta = np.abs(q @ (k_hat - K).T * scale).max(axis=1)                    # per head
+    bound = np.abs(v_hat - V).max() + (np.exp(2 * delta) - 1) * np.abs(V).max()
+    assert delta.max() < 0.02 and bound.max() < 0.03      # an order of magnitude below the tolerances this replaces
+    assert (np.abs(oa[0] - dense).max(axis=1) <= bound * (1 + 1e-9)).all()
+    assert (np.abs(la[0] - lse) <= delta * (1 + 1e-9)).all()
 
 
 def test_reconstruction_error_shrinks_with_rate_and_respects_step():
@@ -251,23 +334,3 @@ def test_importance_allocation_beats_uniform_at_low_rate():
     wf = _attend(_coded_tiny(8.0, fit.GAIN_WHITEN, n), q, "A", n)[0]
     un = _attend(_coded_tiny(8.0, fit.GAIN_WHITEN, n, widths_override=2), q, "A", n)[0]
     assert np.linalg.norm(wf - dense) < np.linalg.norm(un - dense)
-
-
-def test_split_merge_of_partial_softmax_equals_unsplit():
-    """The log-sum-exp merge of partial (max, sum, accumulator) triples over any partition of the sequence
-    gives the unsplit softmax-weighted sum (textbook identity used by the sequence split)."""
-    rng = np.random.default_rng(21)
-    s = rng.standard_normal(1000) * 4
-    v = rng.standard_normal((1000, 8))
-    p = np.exp(s - s.max())
-    whole = (p[:, None] * v).sum(0) / p.sum()
-    cuts = [0, 17, 300, 301, 640, 1000]
-    parts = []
-    for a, b in zip(cuts[:-1], cuts[1:]):
-        m = s[a:b].max()
-        e = np.exp(s[a:b] - m)
-        parts.append((m, e.sum(), (e[:, None] * v[a:b]).sum(0)))
-    M = max(m for m, _, _ in parts)
-    l = sum(np.exp(m - M) * li for m, li, _ in parts)
-    o = sum(np.exp(m - M) * oi for m, _, oi in parts)
-    assert np.abs(o / l - whole).max() <= 1e-12
