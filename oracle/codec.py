@@ -151,6 +151,20 @@ def unpack_token(tile, widths, gs, side, t):
     return codes, lo16, r16
 
 
+def unpack_unit(cache, tile_stride, n, widths, gs, side):
+    """Codes [n, d] and metadata lo16, R16 [n, d / gs] of tokens [0, n) of one unit-side (cache starts at its
+    first tile)."""
+    widths = _u8(widths)
+    d = widths.size
+    cache = _u8(cache)
+    codes = np.zeros((n, d), np.uint16)
+    lo16 = np.zeros((n, d // gs), np.uint16)
+    r16 = np.zeros((n, d // gs), np.uint16)
+    lib().spo_unpack_unit(_p(cache), C.c_int64(tile_stride), C.c_int64(n), _p(widths), C.c_int(d), C.c_int(gs),
+                          C.c_int(side), _p(codes), _p(lo16), _p(r16))
+    return codes, lo16, r16
+
+
 def rotate_token(x, w_enc, m_rot):
     x = _f32(x)
     w_enc = _f32(w_enc)

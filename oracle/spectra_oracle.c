@@ -304,6 +304,15 @@ void spo_unpack_token(const uint8_t* tile, const uint8_t* widths, int d, int gs,
   }
 }
 
+/* Tokens [0, n) of one unit-side, one spo_unpack_token per token: codes [n, d], lo16 and R16 [n, d / gs]. */
+void spo_unpack_unit(const uint8_t* cache, int64_t tile_stride, int64_t n, const uint8_t* widths, int d, int gs,
+                     int side, uint16_t* codes, uint16_t* lo16, uint16_t* R16) {
+  const int ng = d / gs;
+  for (int64_t t = 0; t < n; t++)
+    spo_unpack_token(cache + (t / SPO_TILE) * tile_stride, widths, d, gs, side, (int)(t % SPO_TILE), codes + t * d,
+                     lo16 + t * ng, R16 + t * ng);
+}
+
 /* ---------------------------------------------------------------- rotate / encode / decode */
 
 /* y_j = sum_i x_i W_enc[i][j] - m'_j, accumulated in fp64 in index order, rounded once to fp32. */

@@ -99,6 +99,18 @@ def draw_unit(wl, layer, head, side, seq, n_tokens=None, start=0):
     return to_bf16_f32(x) if wl.dtype == "bf16" else x
 
 
+def mean_offset(wl, layer, head, side, scale=1.0):
+    """A constant vector [d] fp32 to add to every cache vector of one (layer, head, side): +-scale standard
+    deviations of each channel (seeded signs).  The recipe above is zero-mean; with this offset the rotated means
+    the codec removes and restores are as large as the spread of the data."""
+    recipe = wl.k if side == SIDE_K else wl.v
+    a = mixing_matrix(wl.config_id, layer, head, side, recipe, wl.head_dim)
+    sigma = np.sqrt((a * a).sum(axis=0))
+    sign = _rng(wl.config_id, layer, head, side, 0x4D).choice([-1.0, 1.0], size=wl.head_dim)
+    c = (scale * sign * sigma).astype(np.float32)
+    return to_bf16_f32(c) if wl.dtype == "bf16" else c
+
+
 def draw_queries(wl, layer, seq, step=0):
     """Decode queries [q_heads, d] fp32 (bf16-representable for bf16 workloads)."""
     rng = _rng(wl.config_id, layer, 0xAB, seq, step)

@@ -97,3 +97,21 @@ def draw_units(wl, layer, side, n_seq, n_tokens):
         for h in range(wl.kv_heads):
             out[s * wl.kv_heads + h] = si.draw_unit(wl, layer, h, side, s, n_tokens=n_tokens)
     return out
+
+
+def f16_ordinal(h):
+    """Maps fp16 bit patterns to integers that are ordered like the values (adjacent values differ by one)."""
+    h = np.asarray(h, np.uint16).astype(np.int32)
+    return np.where(h & 0x8000, -(h & 0x7FFF), h & 0x7FFF)
+
+
+def compare_coded_units(ref_cache, got_cache, tb, n, widths, gs, side):
+    """Every token of one unit-side, the oracle's bytes against the library's: returns (entries that differ, active
+    entries, largest code difference, largest metadata difference in fp16 steps, tokens whose metadata differ).
+    Tokens whose metadata differ are not set apart: their entries count like all others."""
+    cr, lr, rr = oc.unpack_unit(ref_cache, tb, n, widths, gs, side)
+    cg, lg, rg = oc.unpack_unit(got_cache, tb, n, widths, gs, side)
+    diff = np.abs(cr.astype(np.int32) - cg.astype(np.int32))
+    active = int((np.asarray(widths) > 0).sum()) * n
+    meta = np.maximum(np.abs(f16_ordinal(lr) - f16_ordinal(lg)), np.abs(f16_ordinal(rr) - f16_ordinal(rg)))
+    return int((diff != 0).sum()), active, int(diff.max()), int(meta.max()), int((meta.max(axis=1) != 0).sum())
