@@ -27,7 +27,14 @@ METRIC = "coded_kv_decode_attention_kv_tokens_per_s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (one layer of the workload),
 # from the ncu capture summarised in profiles/attention_mma_kernel_llama32_2layer.md (same per-launch shape)
 NCU_TRAFFIC_BYTES = {"llama32": 173.1e6}
+# share of the dominant kernel (attention_mma_kernel) in the device time of a decode step, from the launch list of
+# this command summarised in profiles/decode_step_launch_list_llama32.md
+MAIN_KERNEL_SHARE = {"llama32": 0.827}
 UNIT = "KV tokens/s"
+MIN_TIMED_SECONDS = 0.5      # the --steps set is repeated until the timed region is at least this long
+# what the metric's path computes in: codes and probabilities enter mma.sync as fp16 (codes exactly, the query as
+# a hi + lo pair), sums are fp32
+ARITHMETIC = "f16xf16->f32"
 
 
 def _peaks():
@@ -170,18 +177,20 @@ class OracleSample:
         return dt, H * (self.n + 1), min(oc.num_threads(), H)
 
 
-def _oracle_rate(wl, seconds_budget, reps=1):
-    """Sizes a sample so that `reps` oracle steps take about seconds_budget; returns (times, token_heads, threads,
-    description)."""
-    probe = OracleSample(wl, 512)
-    dt, th, threads = probe.step()
-    per_th = dt / th
-    n = int(max(128, min(wl.n_tokens, (seconds_budget / reps / per_th / wl.kv_heads) // 128 * 128)))
+ORACLE_SAMPLE_TOKENS = 32768      # cached tokens per head of the oracle's sample, the same in both legs
+
+
+def _oracle_rate(wl, reps=1, warm=0):
+    """The oracle's fixed sample: all kv-heads of layer 0, sequence 0, min(context, 32768) cached tokens.  Runs
+    warm + reps decode steps on it; returns (times of the reps, token_heads per step, threads, description)."""
+    n = min(wl.n_tokens, ORACLE_SAMPLE_TOKENS)
     sample = OracleSample(wl, n)
     times = []
-    for _ in range(reps):
+    th = threads = 0
+    for i in range(warm + reps):
         dt, th, threads = sample.step()
-        times.append(dt)
+        if i >= warm:
+            times.append(dt)
     desc = (f"layer 0, sequence 0, {wl.kv_heads} kv-heads x {n} cached tokens, built and run by the oracle alone; "
             f"one step = append 1 token per unit + Mode B attention; token-heads/s divided by layers*kv_heads")
     return times, th, threads, desc
@@ -192,9 +201,8 @@ def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    reps = args.warmup + args.steps
-    times, th, threads, desc = _oracle_rate(wl, 90.0, reps)
-    t = float(np.mean(times[args.warmup:]))
+    times, th, threads, desc = _oracle_rate(wl, args.steps, args.warmup)
+    t = float(np.mean(times))
     value = th / t / (wl.layers * wl.kv_heads)          # same unit as the GPU arm: KV tokens/s of the full model
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
@@ -219,7 +227,8 @@ def run_ours(args, wl):
     dev = torch.device("cuda", local)
     steps, warmup = args.steps, max(args.warmup, 3)
     hbm_gbs, peak_kind = _peaks()
-    model = harness.CodedModelCache(wl, layers=args.layers or None, extra_tokens=3 * steps + warmup + 32)
+    model = harness.CodedModelCache(wl, layers=args.layers or None,
+                                    extra_tokens=(2 * args.max_repeats + 3) * steps + warmup + 64)
     t0 = time.perf_counter()
     model.build(time_phases=True)
     setup_s = time.perf_counter() - t0
@@ -272,19 +281,34 @@ def run_ours(args, wl):
             graphs.append(g)
         for k in range(n_in):
             graphs[k].replay()
+    # the --steps set is repeated so that the timed region lasts at least MIN_TIMED_SECONDS (one untimed set sizes it)
     _barrier(world)
-    sampler = ClockSampler(local)
-    sampler.start()
-    e_start, e_end = ev(), ev()
-    e_start.record()
+    p0, p1 = ev(), ev()
+    p0.record()
     for i in range(steps):
         if graphs:
             graphs[i % n_in].replay()
         else:
-            step_resident(i, timed=True)
-    e_end.record()
+            step_resident(i)
+    p1.record()
+    torch.cuda.synchronize()
+    repeats = int(max(1, min(args.max_repeats, np.ceil(MIN_TIMED_SECONDS * 1e3 / max(p0.elapsed_time(p1), 1e-3)))))
+    repeats = int(_max_over_ranks(float(repeats), world))
     _barrier(world)
-    ms_step = _max_over_ranks(e_start.elapsed_time(e_end) / steps, world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    marks = [ev() for _ in range(repeats + 1)]
+    marks[0].record()
+    for r in range(repeats):
+        for i in range(steps):
+            if graphs:
+                graphs[i % n_in].replay()
+            else:
+                step_resident(i, timed=True)
+        marks[r + 1].record()
+    _barrier(world)
+    ms_step = _max_over_ranks(marks[0].elapsed_time(marks[repeats]) / (steps * repeats), world)
+    ms_step_sets = [marks[r].elapsed_time(marks[r + 1]) / steps for r in range(repeats)]
     if graphs:
         # events cannot be recorded inside a replayed graph: time the attention calls of the same steps, launched
         # directly, right after the timed region (same buffers, same lengths + 1 per step)
@@ -310,11 +334,11 @@ def run_ours(args, wl):
     _barrier(world)
     e0, e1 = ev(), ev()
     e0.record()
-    for i in range(steps):
+    for i in range(steps * repeats):
         step_e2e(i)
     e1.record()
     _barrier(world)
-    ms_e2e = _max_over_ranks(e0.elapsed_time(e1) / steps, world)
+    ms_e2e = _max_over_ranks(e0.elapsed_time(e1) / (steps * repeats), world)
     status = int(model.status.item())
 
     # ---- reconstruction (spectra_decode) of one layer's K side, outside the timed decode steps: reported beside
@@ -339,13 +363,19 @@ def run_ours(args, wl):
     enc_bytes = L * 2 * U * wl.n_tokens * d * 2 + tile_bytes_all * (wl.n_tokens // 128)
     rec_bytes = U * wl.n_tokens * d * 2 + sum(int(ls0.tile_bytes[u % H]) for u in range(U)) * (wl.n_tokens // 128)
     bytes_call = model.attention_bytes(layer=0)
-    achieved = bytes_call / (attn_ms_avg * 1e-3) / 1e9
+    # duration of one launch of the dominant kernel inside the timed region: the step's device time per layer times
+    # the kernel's share of a step in the committed launch list; the directly launched layer call (front + main +
+    # combine between two events) is kept beside it
+    share = MAIN_KERNEL_SHARE.get(wl.name)
+    ms_launch = ms_step / L * share if share else attn_ms_avg
+    achieved = bytes_call / (ms_launch * 1e-3) / 1e9
     h2d = sum(t[0].numel() * t.element_size() for t in (q_host, nk_host, nv_host))
     d2h = out_host.numel() * out_host.element_size()
     line = {
         "metric": METRIC, "value": world * kv_tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
-        "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "steps": steps, "repeats": repeats, "warmup": warmup, "ms_per_step": ms_step,
+        "ms_per_step_median_of_sets": float(np.median(ms_step_sets)), "timed_region_s": ms_step * steps * repeats * 1e-3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": ARITHMETIC, "data": "synthetic",
         "config": {"workload": wl.name, "layers": L, "batch": B, "kv_heads": H, "q_heads": Hq, "head_dim": d,
                    "context": n_ctx, "ratio": wl.ratio, "cache_dtype_replaced": "bf16",
                    "coded_cache_gb": model.coded_bytes() / 1e9, "parallelism": f"replicas{world}",
@@ -354,12 +384,17 @@ def run_ours(args, wl):
                    else "WARNING: coded cache fits L2"},
         "e2e": {"value": world * kv_tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
-        "gpu_launches": steps * L * (sp.STEP_LAUNCHES if args.fused else 2 + sp.ATTENTION_LAUNCHES),
+        "gpu_launches": steps * repeats * L * (sp.STEP_LAUNCHES if args.fused else 2 + sp.ATTENTION_LAUNCHES),
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "spectra_decode_step (one layer call: append + attention)" if args.fused
-                     else "spectra_decode_attention (one layer call)", "achieved": achieved,
-                     "peak": hbm_gbs, "unit": "GB/s", "frac": achieved / hbm_gbs, "peak_kind": peak_kind,
-                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "bytes_per_launch": bytes_call, "ms_per_launch": attn_ms_avg},
+        "roofline": {"bound": "hbm", "kernel": "attention_mma_kernel (one launch = one layer of the step)",
+                     "achieved": achieved, "peak": hbm_gbs, "unit": "GB/s", "frac": achieved / hbm_gbs,
+                     "peak_kind": peak_kind, "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "bytes_per_launch": bytes_call,
+                     "ms_per_launch": ms_launch,
+                     "ms_per_launch_from": "ms_per_step / layers * main_kernel_share" if share else "direct layer call",
+                     "main_kernel_share": share,
+                     "layer_call_direct_ms": attn_ms_avg,
+                     "layer_call_direct_frac": bytes_call / (attn_ms_avg * 1e-3) / 1e9 / hbm_gbs,
+                     "whole_step_frac": bytes_call * L / (ms_step * 1e-3) / 1e9 / hbm_gbs},
         "phases": {"setup_s": setup_s, "fit_alloc_ms_total": model.timings["fit_alloc_ms"],
                    "prefill_encode_ms_total": model.timings["prefill_encode_ms"],
                    "prefill_encode_tokens_per_s": L * 2 * U * wl.n_tokens / max(model.timings["prefill_encode_ms"],
@@ -374,15 +409,60 @@ def run_ours(args, wl):
                    "reconstruct_frac_of_hbm": rec_bytes / max(reconstruct_ms, 1e-9) / 1e6 / hbm_gbs},
         "status_word": status,
     }
+    if rank == 0 and world == 1 and args.other_workloads and not args.layers:
+        del model, q_dev, nk_dev, nv_dev
+        torch.cuda.empty_cache()
+        line["other_workloads"] = _other_workloads(args, hbm_gbs)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        times, th, threads, desc = _oracle_rate(wl, 15.0, 1)
-        line["cpu_baseline"] = {"value": th / times[0] / (wl.layers * wl.kv_heads), "unit": UNIT, "cores": threads,
-                                "kind": "oracle", "sample": desc}
+        times, th, threads, desc = _oracle_rate(wl, 3, 1)
+        line["cpu_baseline"] = {"value": th / float(np.mean(times)) / (wl.layers * wl.kv_heads), "unit": UNIT,
+                                "cores": threads, "kind": "oracle", "sample": desc}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def _other_workloads(args, hbm_gbs):
+    """One layer of each other workload shape: the fused layer call (front + main + combine) launched directly and
+    timed with CUDA events, the L2 flushed before every timed call (one layer's coded cache can fit the L2)."""
+    import torch
+
+    import spectra_inputs as si
+    from paper_2608_07915_b200 import harness
+    out = {}
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for name in ("llama1", "qwen28", "long128k", "batch32"):
+        wl = si.WORKLOADS[name]
+        n_calls, n_warm = 10, 3
+        m = harness.CodedModelCache(wl, layers=1, extra_tokens=n_calls + n_warm + 8)
+        m.build()
+        L, B, Hq, d, U = 1, m.batch, m.Hq, m.d, m.n_units
+        gen = torch.Generator(device="cuda").manual_seed(4321)
+        q = torch.randn((1, B, Hq, d), generator=gen, device="cuda").to(torch.bfloat16)
+        nk = torch.randn((1, U, d), generator=gen, device="cuda").to(torch.bfloat16)
+        nv = torch.randn((1, U, d), generator=gen, device="cuda").to(torch.bfloat16)
+        o = torch.zeros((1, B, Hq, d), dtype=torch.bfloat16, device="cuda")
+        ms = []
+        for i in range(n_warm + n_calls):
+            flush.zero_()
+            e0, e1 = ev(), ev()
+            e0.record()
+            m.decode_step(q, nk, nv, o, fused=True)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= n_warm:
+                ms.append(e0.elapsed_time(e1))
+        b = m.attention_bytes(layer=0)
+        t = float(np.median(ms))
+        out[name] = {"layers_timed": 1, "batch": B, "context": int(m.seq_len.max().item()), "ratio": wl.ratio,
+                     "ms_per_layer_call": t, "bytes_per_layer_call": b, "frac_of_hbm": b / (t * 1e-3) / 1e9 / hbm_gbs,
+                     "status_word": int(m.status.item()), "l2": "flushed before every timed call"}
+        del m, q, nk, nv, o
+        torch.cuda.empty_cache()
+    return out
 
 
 def main():
@@ -394,6 +474,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers than the workload (invalid as a result)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", dest="other_workloads", action="store_false",
+                    help="skip the one-layer timings of the other workload shapes")
+    ap.add_argument("--max-repeats", type=int, default=64, help="upper bound of the repeats of the --steps set")
     ap.add_argument("--unfused", dest="fused", action="store_false",
                     help="per layer: spectra_encode (K, V) + spectra_decode_attention instead of spectra_decode_step")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
