@@ -2,12 +2,14 @@
  * libspectra -- SPECTRA KV-cache codec, data-parallel hot path, for NVIDIA B200 (sm_100a).
  *
  * C ABI.  Every pointer marked "device" is caller-owned device memory (any allocator);
- * pointers marked "host" are ordinary host memory.  The library allocates nothing and keeps
- * no state between calls.  All work is enqueued on `stream` (a cudaStream_t passed as void*,
+ * pointers marked "host" are ordinary host memory.  The library allocates nothing and carries
+ * no results from one call to the next (all it remembers is, per device, the address of the fixed
+ * scratch array of spectra_fit_basis_static).  All work is enqueued on `stream` (a cudaStream_t passed as void*,
  * NULL = the legacy default stream) and the calls return without synchronising.  Arguments
  * are validated on the host before anything is launched; a non-zero return value means that
  * nothing was enqueued.  Data-dependent anomalies (non-finite input, metadata beyond the
- * fp16 range) are OR-ed into a caller-supplied device status word, never trapped.
+ * fp16 range, a token position beyond the stated capacity, a unit whose layout does not match
+ * the host's copy of the widths) are OR-ed into a caller-supplied device status word, never trapped.
  *
  * Vocabulary (paper notation).  A unit is one (sequence, kv-head) of one layer; a side is its
  * keys (K) or values (V).  d = head_dim = 128.  Per unit-side the codec holds a decorrelating
@@ -83,6 +85,16 @@ extern "C" {
 #define SPECTRA_STATUS_NONFINITE 1 /* a non-finite coordinate reached the quantiser */
 #define SPECTRA_STATUS_F16_RANGE 2 /* a group minimum or range was saturated to the fp16 range */
 #define SPECTRA_STATUS_WAIT_TIMEOUT 4 /* a bounded wait on an on-chip copy gave up; the results are invalid */
+#define SPECTRA_STATUS_CAPACITY 8 /* a token position beyond the stated capacity: that token was not written (append) or
+                                     the sequence was attended as empty (attention) */
+#define SPECTRA_STATUS_BAD_LAYOUT 16 /* the tensor-core attention path found a unit whose device-side widths or offsets
+                                        do not match what the host copy of the widths promised (tile larger than its
+                                        shared-memory slot, more strips than the kernel variant holds, tile stream not
+                                        16-byte aligned): the unit's tiles were not read and its output is invalid */
+
+/* return values of spectra_attention_path */
+#define SPECTRA_PATH_CUDA_CORE 0
+#define SPECTRA_PATH_TENSOR_CORE 1
 
 #define SPECTRA_GAIN_ROTATE 0 /* gamma = 1: a pure rotation */
 #define SPECTRA_GAIN_SQRT 1   /* gamma_j = lambda_j^(-1/4): the paper's square-root split (Eq. 3) */
@@ -125,8 +137,8 @@ size_t spectra_fit_workspace_bytes(const spectra_config* cfg, int64_t n_units);
  * inside a host process with a fixed, pre-carved memory arena, or a component started after the process has
  * frozen its allocator (allocation there would synchronise the device or is simply forbidden).  It takes the
  * same inputs and writes the same outputs, but needs no workspace argument: the scratch (second-moment sums and
- * eigenvector rows, fp64) lives in a fixed array inside the library image, sized for at most
- * SPECTRA_FIT_STATIC_MAX_UNITS unit-sides per call (about 263 KB each, 2.1 MB in all, held by every device that
+ * means, fp64) lives in a fixed array inside the library image, sized for at most
+ * SPECTRA_FIT_STATIC_MAX_UNITS unit-sides per call (about 132 KB each, 1.1 MB in all, held by every device that
  * loads the library until the process exits).
  *   - n_units > SPECTRA_FIT_STATIC_MAX_UNITS returns SPECTRA_CAPACITY and enqueues nothing; fit larger sets in
  *     slices of that many unit-sides.
@@ -165,7 +177,9 @@ int spectra_alloc_bits(const spectra_config* cfg, const float* var_alloc, int64_
  * widths: device uint8 [n_param_sets, d].  cache: device; unit_offset: device int64 [n_units], byte offset
  * of the unit-side's first tile, multiple of 16.  status_word: device int32, OR-ed with SPECTRA_STATUS_* bits,
  * may be NULL.
- * The caller guarantees capacity: every touched tile lies inside its buffer.  cache must be 16-byte aligned
+ * capacity_tokens: tokens every unit-side's buffer holds (spectra_cache_bytes); a token whose position is at or
+ * beyond it is not written and SPECTRA_STATUS_CAPACITY is set in the status word.  0 switches the check off: the
+ * caller then guarantees that every touched tile lies inside its buffer.  cache must be 16-byte aligned
  * (SPECTRA_INVALID_ARG otherwise).
  * Speed, not results, depends on alignment: bf16 input with a 16-byte aligned x and strides that are multiples of 8
  * elements (and scale_group 64, more than 16 tokens) takes the tensor-core path; anything else a CUDA-core kernel.
@@ -173,7 +187,8 @@ int spectra_alloc_bits(const spectra_config* cfg, const float* var_alloc, int64_
 int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dtype, int flags, int64_t n_units,
                    int64_t n_param_sets, const int32_t* pos0, int32_t n_new, int64_t stride_unit,
                    int64_t stride_token, const float* w_enc, const float* mean_rot, const uint8_t* widths,
-                   uint8_t* cache, const int64_t* unit_offset, int32_t* status_word, void* stream);
+                   uint8_t* cache, const int64_t* unit_offset, int32_t capacity_tokens, int32_t* status_word,
+                   void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * spectra_decode -- Sec. 3.3 (Mode A reconstruction): xhat = (yhat + m') W_dec for tokens [0, n_tokens[u])
@@ -182,12 +197,13 @@ int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dty
  * max_tokens (host value) bounds it.  yhat_out (device fp32, same strides, may be NULL) receives the
  * dequantised rotated coordinates.  cache must be 2-byte aligned (SPECTRA_INVALID_ARG otherwise).  Packed tiles are
  * fetched with bulk copies when cache + unit_offset[u] is 16-byte aligned (and a tile is at most 10 KB), else read in
- * place: same results, lower speed.
+ * place: same results, lower speed.  status_word: device int32 or NULL; a bounded wait of the tensor-core kernel that
+ * gives up sets SPECTRA_STATUS_WAIT_TIMEOUT there (the reconstruction is then invalid).
  */
 int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
                    int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
                    const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out, int out_dtype,
-                   float* yhat_out, int64_t stride_unit, int64_t stride_token, void* stream);
+                   float* yhat_out, int64_t stride_unit, int64_t stride_token, int32_t* status_word, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * spectra_decode_attention -- appendix "Latent-space attention and memory" (Mode B): one decode query per
@@ -198,14 +214,18 @@ int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, co
  *     o' = sum_t softmax(s)_t yhat^V_t    (online softmax, rotated value space, sequence split across CTAs)
  *     out = (o' + m'_V) W_dec,V           (one lift per query head)
  * Units are ordered u = sequence * n_kv_heads + kv_head; query head hq belongs to kv-head hq / (n_q_heads /
- * n_kv_heads).  q: device [batch, n_q_heads, d], q_dtype.  seq_len: device int32 [batch] (tokens attended,
- * <= max_seq_len; 0 gives a zero output row and lse = -inf).  cache_k/v with unit_offset_k/v: as in
+ * n_kv_heads).  q: device [batch, n_q_heads, d], q_dtype.  seq_len: device int32 [batch] (tokens attended; 0 gives
+ * a zero output row and lse = -inf).  max_seq_len (host value) is the capacity of every sequence's buffers in tokens:
+ * a sequence whose seq_len exceeds it sets SPECTRA_STATUS_CAPACITY and is treated as empty, nothing past the end of a
+ * buffer is read.  cache_k/v with unit_offset_k/v: as in
  * spectra_encode.  Parameter arrays as in spectra_encode/decode ([n_param_sets, ...]); mean_rot_k is read
  * only when lse != NULL and may be NULL otherwise.  widths_k_host / widths_v_host: HOST copies of the two width
  * arrays ([n_param_sets, d], the same values the caller already needs for spectra_tile_bytes); read during the
  * call only.  They let the host size shared-memory rings and pick the kernel variant without a device
  * round-trip.  With both NULL, or scale_group != 64, or width profiles outside the built variants, a slower
- * CUDA-core kernel runs.  w_dec_k, w_dec_v, cache_k, cache_v and workspace must be 16-byte aligned
+ * CUDA-core kernel runs (spectra_attention_path tells which).  The tensor-core path checks every unit on the device
+ * against the widths the kernels read: a unit that does not match the host copy (see SPECTRA_STATUS_BAD_LAYOUT) is
+ * skipped, never copied from.  w_dec_k, w_dec_v, cache_k, cache_v and workspace must be 16-byte aligned
  * (SPECTRA_INVALID_ARG otherwise: the kernels use 16-byte accesses and bulk copies).  A GQA group of 5 to 8 query
  * heads is taken in two passes over the tiles.  On the tensor-core path the partial sums of a sequence are merged in a fixed order (results are
  * bit-reproducible from run to run); the CUDA-core kernel accumulates with shared-memory atomics (they are not).
@@ -236,7 +256,8 @@ size_t spectra_attention_workspace_bytes(const spectra_config* cfg, int32_t batc
  * or SPECTRA_BF16.  seq_len: device int32 [batch], the lengths INCLUDING the appended token (a sequence with
  * length 0 gets no append and a zero output row).
  * w_enc_k/v, mean_rot_k/v as in spectra_encode; every other argument as in spectra_decode_attention
- * (mean_rot_k is required here).  cache_k / cache_v are written (the appended token) and read.
+ * (mean_rot_k is required here).  cache_k / cache_v are written (the appended token) and read.  A sequence with
+ * seq_len > max_seq_len gets no append (SPECTRA_STATUS_CAPACITY) and is attended as empty.
  */
 int spectra_decode_step(const spectra_config* cfg, const void* q, int q_dtype, const void* new_k, const void* new_v,
                         int x_dtype, int32_t batch, int32_t n_kv_heads, int32_t n_q_heads, const int32_t* seq_len,
@@ -251,12 +272,19 @@ int spectra_decode_step(const spectra_config* cfg, const void* q, int q_dtype, c
 /* ------------------------------------------------------------------------------------------------
  * Helpers (host only, no device work).
  * spectra_tile_bytes: size of one packed tile for the given widths (host uint8 [d]); 0 on bad arguments.
+ * spectra_cache_bytes: bytes of one unit-side's buffer for capacity_tokens tokens (whole tiles); 0 on bad arguments.
+ * spectra_attention_path: which kernels spectra_decode_attention / spectra_decode_step will run for these host
+ *   widths ([n_param_sets, d] each, may be NULL): SPECTRA_PATH_TENSOR_CORE or SPECTRA_PATH_CUDA_CORE; -1 on bad
+ *   arguments.
  * spectra_config_default: fills cfg with head_dim 128, tile 128, scale_group 64, width_group 1, b_max 8,
  *   SPECTRA_GAIN_SQRT, layout 1.
  * spectra_total_bits: Btot = floor(16 d / ratio) clamped to b_max * d.
  * spectra_status_string: name of a return code.
  */
 size_t spectra_tile_bytes(const spectra_config* cfg, const uint8_t* widths_host);
+size_t spectra_cache_bytes(const spectra_config* cfg, const uint8_t* widths_host, int64_t capacity_tokens);
+int spectra_attention_path(const spectra_config* cfg, int32_t n_kv_heads, int32_t n_q_heads, int64_t n_param_sets,
+                           const uint8_t* widths_k_host, const uint8_t* widths_v_host);
 void spectra_config_default(spectra_config* cfg);
 int32_t spectra_total_bits(const spectra_config* cfg, double ratio);
 const char* spectra_status_string(int code);

@@ -15,7 +15,8 @@ OK, INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CAPACITY, CUDA_ERROR = range(
 F32, BF16 = 0, 1
 SIDE_K, SIDE_V = 0, 1
 ROTATED_INPUT = 1
-STATUS_NONFINITE, STATUS_F16_RANGE, STATUS_WAIT_TIMEOUT = 1, 2, 4
+STATUS_NONFINITE, STATUS_F16_RANGE, STATUS_WAIT_TIMEOUT, STATUS_CAPACITY, STATUS_BAD_LAYOUT = 1, 2, 4, 8, 16
+PATH_CUDA_CORE, PATH_TENSOR_CORE = 0, 1
 GAIN_ROTATE, GAIN_SQRT, GAIN_WHITEN = 0, 1, 2
 HEAD_DIM = 128
 TILE_TOKENS = 128
@@ -25,7 +26,7 @@ STEP_LAUNCHES = 3        # kernels one spectra_decode_step call enqueues on the 
 EXPORTS = [
     "spectra_fit_basis", "spectra_fit_basis_static", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
     "spectra_decode_attention", "spectra_decode_step", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
-    "spectra_total_bits", "spectra_status_string",
+    "spectra_total_bits", "spectra_status_string", "spectra_cache_bytes", "spectra_attention_path",
 ]
 
 
@@ -49,6 +50,7 @@ def lib():
         _lib.spectra_fit_workspace_bytes.restype = C.c_size_t
         _lib.spectra_attention_workspace_bytes.restype = C.c_size_t
         _lib.spectra_tile_bytes.restype = C.c_size_t
+        _lib.spectra_cache_bytes.restype = C.c_size_t
         _lib.spectra_total_bits.restype = C.c_int32
         _lib.spectra_status_string.restype = C.c_char_p
         _lib.spectra_config_default.restype = None
@@ -88,6 +90,28 @@ def _dtype_code(t):
     if t.dtype == torch.bfloat16:
         return BF16
     raise SpectraError(f"unsupported tensor dtype {t.dtype}")
+
+
+def cache_bytes(cfg, widths_host, capacity_tokens):
+    """Bytes of one unit-side's buffer that holds capacity_tokens tokens (whole tiles)."""
+    arr = (C.c_uint8 * HEAD_DIM)(*[int(w) for w in widths_host])
+    return int(lib().spectra_cache_bytes(C.byref(cfg), arr, C.c_int64(capacity_tokens)))
+
+
+def attention_path(cfg, n_kv_heads, n_q_heads, n_param_sets, widths_k_host, widths_v_host):
+    """PATH_TENSOR_CORE or PATH_CUDA_CORE: the kernels decode_attention / decode_step will run for these host widths
+    (numpy uint8 [n_param_sets, 128] each, or None)."""
+    wk = wv = C.c_void_p(0)
+    if widths_k_host is not None and widths_v_host is not None:
+        assert widths_k_host.dtype.name == "uint8" and widths_k_host.flags.c_contiguous
+        assert widths_v_host.dtype.name == "uint8" and widths_v_host.flags.c_contiguous
+        wk = widths_k_host.ctypes.data_as(C.c_void_p)
+        wv = widths_v_host.ctypes.data_as(C.c_void_p)
+    rc = int(lib().spectra_attention_path(C.byref(cfg), C.c_int32(n_kv_heads), C.c_int32(n_q_heads),
+                                          C.c_int64(n_param_sets), wk, wv))
+    if rc < 0:
+        raise SpectraError("spectra_attention_path: invalid arguments")
+    return rc
 
 
 def tile_bytes(cfg, widths_host):
@@ -144,21 +168,23 @@ def alloc_bits(cfg, var_alloc, n_units, ratio, widths):
 
 
 def encode(cfg, side, x, flags, n_units, n_param_sets, pos0, n_new, stride_unit, stride_token, w_enc, mean_rot,
-           widths, cache, unit_offset, status_word=None):
+           widths, cache, unit_offset, status_word=None, capacity_tokens=0):
+    """capacity_tokens: tokens each unit-side's buffer holds (0: not checked)."""
     rc = lib().spectra_encode(C.byref(cfg), C.c_int(side), _ptr(x), C.c_int(_dtype_code(x)), C.c_int(flags),
                               C.c_int64(n_units), C.c_int64(n_param_sets), _ptr(pos0), C.c_int32(n_new),
                               C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(w_enc), _ptr(mean_rot),
-                              _ptr(widths), _ptr(cache), _ptr(unit_offset), _ptr(status_word), _stream())
+                              _ptr(widths), _ptr(cache), _ptr(unit_offset), C.c_int32(capacity_tokens),
+                              _ptr(status_word), _stream())
     _check(rc, "spectra_encode")
 
 
 def decode(cfg, side, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec, mean_rot, widths, out,
-           yhat_out, stride_unit, stride_token):
+           yhat_out, stride_unit, stride_token, status_word=None):
     out_code = _dtype_code(out) if out is not None else F32
     rc = lib().spectra_decode(C.byref(cfg), C.c_int(side), _ptr(cache), _ptr(unit_offset), C.c_int64(n_units),
                               C.c_int64(n_param_sets), _ptr(n_tokens), C.c_int32(max_tokens), _ptr(w_dec),
                               _ptr(mean_rot), _ptr(widths), _ptr(out), C.c_int(out_code), _ptr(yhat_out),
-                              C.c_int64(stride_unit), C.c_int64(stride_token), _stream())
+                              C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(status_word), _stream())
     _check(rc, "spectra_decode")
 
 

@@ -87,6 +87,28 @@ int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem
 constexpr int kQuotas[][4] = {{0, 1, 8, 2}, {0, 1, 3, 6}, {0, 1, 6, 4}, {0, 8, 2, 2}, {0, 7, 3, 4}, {0, 1, 2, 7}, {0, 1, 8, 5}};
 constexpr int kNumQuotas = sizeof(kQuotas) / sizeof(kQuotas[0]);
 
+int pick_quota(const int (&vb)[4]);
+
+// Launch shape of the tensor-core path for a set of widths: shared-memory slot sizes, CTAs per SM, ring depth and
+// the kernel variant (quota < 0 or depth < 1: the widths fall outside the built variants).
+struct FastPlan { int slot_k, slot_v, ctas_per_sm, depth, quota; };
+
+FastPlan plan_fast(const WidthFacts& F) {
+  FastPlan P{};
+  P.slot_k = (int)align_up((size_t)(F.max_tile_k > 16 ? F.max_tile_k : 16), 128);
+  P.slot_v = (int)align_up((size_t)(F.max_tile_v > 16 ? F.max_tile_v : 16), 128);
+  const size_t pair = (size_t)P.slot_k + P.slot_v;
+  const size_t budget = 200 * 1024;
+  P.ctas_per_sm = kFastCtasPerSm;
+  while (P.ctas_per_sm > 1 &&
+         (size_t)P.ctas_per_sm * (kFastWarps * pair + 2048 + kFastWarps * (64 + kWarpStateBytes)) > budget)
+    P.ctas_per_sm--;
+  P.depth = (int)(budget / ((size_t)P.ctas_per_sm * kFastWarps * pair));
+  if (P.depth > 4) P.depth = 4;
+  P.quota = pick_quota(F.vb);
+  return P;
+}
+
 int pick_quota(const int (&vb)[4]) {
   for (int i = 0; i < kNumQuotas; i++) {
     bool fits = true;
@@ -161,6 +183,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
   a.partials = reinterpret_cast<float*>(workspace);
   a.n_splits = generic_splits((int)n_units, max_seq_len);
   a.status = status_word;
+  a.max_seq_len = max_seq_len;
   cudaStream_t st = (cudaStream_t)stream;
 
   // ---- tensor-core path: scale group 64, host copy of the widths available; a GQA group of more than 4 query
@@ -172,15 +195,9 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
     if (!F.ok) return SPECTRA_INVALID_ARG;
     const int sms = sm_count();
     if (sms <= 0) return SPECTRA_CUDA_ERROR;
-    const int slot_k = (int)align_up((size_t)(F.max_tile_k > 16 ? F.max_tile_k : 16), 128);
-    const int slot_v = (int)align_up((size_t)(F.max_tile_v > 16 ? F.max_tile_v : 16), 128);
+    const FastPlan P = plan_fast(F);
+    const int slot_k = P.slot_k, slot_v = P.slot_v, ctas_per_sm = P.ctas_per_sm, depth = P.depth, quota = P.quota;
     const size_t pair = (size_t)slot_k + slot_v;
-    const size_t budget = 200 * 1024;
-    int ctas_per_sm = kFastCtasPerSm;
-    while (ctas_per_sm > 1 && (size_t)ctas_per_sm * (kFastWarps * pair + 2048 + kFastWarps * (64 + kWarpStateBytes)) > budget) ctas_per_sm--;
-    int depth = (int)(budget / ((size_t)ctas_per_sm * kFastWarps * pair));
-    if (depth > 4) depth = 4;
-    const int quota = pick_quota(F.vb);
     if (depth >= 1 && quota >= 0) {
       const int vs_max = (F.max_vstrips + 3) & ~3;     // records are fetched with bulk copies: 16-byte multiples
       FastLayout L = fast_layout(n_vunits, sms * ctas_per_sm * kFastWarps, vs_max);
@@ -193,6 +210,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
       f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = vs_max;
       f.n_units = (int)n_vunits; f.npass = npass; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
+      for (int c = 0; c < 4; c++) f.vq[c] = kQuotas[quota][c];
       if (cudaFuncSetAttribute(decode_step_front_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepDynSmem) !=
               cudaSuccess ||
           cudaFuncSetAttribute(attention_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepDynSmem) !=
@@ -200,9 +218,11 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
         return SPECTRA_CUDA_ERROR;
       if (app) {
         AppendArgs ak{app->new_k, app->x_dtype, 0, SPECTRA_SIDE_K, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
-                      app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, status_word, seq_len, n_kv_heads};
+                      app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, status_word, seq_len, n_kv_heads,
+                      max_seq_len};
         AppendArgs av{app->new_v, app->x_dtype, 0, SPECTRA_SIDE_V, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
-                      app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, status_word, seq_len, n_kv_heads};
+                      app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, status_word, seq_len, n_kv_heads,
+                      max_seq_len};
         decode_step_front_kernel<<<(unsigned)(n_vunits + 1 + 2 * n_units), kPrepThreads, kPrepDynSmem, st>>>(
             a, f, ak, av, (int)n_units);
       } else {
@@ -248,10 +268,10 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
     int32_t* pos = reinterpret_cast<int32_t*>(workspace);
     step_positions_kernel<<<(unsigned)((n_units + 255) / 256), 256, 0, st>>>(seq_len, n_kv_heads, (int)n_units, pos);
     rc = spectra_encode(cfg, SPECTRA_SIDE_K, app->new_k, app->x_dtype, 0, n_units, n_param_sets, pos, 1, kD, kD,
-                        app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, status_word, stream);
+                        app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, max_seq_len, status_word, stream);
     if (rc) return rc;
     rc = spectra_encode(cfg, SPECTRA_SIDE_V, app->new_v, app->x_dtype, 0, n_units, n_param_sets, pos, 1, kD, kD,
-                        app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, status_word, stream);
+                        app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, max_seq_len, status_word, stream);
     if (rc) return rc;
   }
   if (cudaFuncSetAttribute(attention_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -298,6 +318,24 @@ extern "C" int spectra_decode_step(const spectra_config* cfg, const void* q, int
                         cache_v, unit_offset_v, n_param_sets, w_dec_k, mean_rot_k, widths_k, w_dec_v, mean_rot_v,
                         widths_v, widths_k_host, widths_v_host, softmax_scale, out, out_dtype, lse, workspace,
                         workspace_bytes, status_word, stream, &app);
+}
+
+extern "C" int spectra_attention_path(const spectra_config* cfg, int32_t n_kv_heads, int32_t n_q_heads,
+                                      int64_t n_param_sets, const uint8_t* widths_k_host,
+                                      const uint8_t* widths_v_host) {
+  if (check_config(cfg) || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || n_param_sets < 1) return -1;
+  if (n_q_heads / n_kv_heads > kMaxGqa) return -1;
+  if (!widths_k_host || !widths_v_host || cfg->scale_group != 64) return SPECTRA_PATH_CUDA_CORE;
+  const WidthFacts F = width_facts(widths_k_host, widths_v_host, n_param_sets);
+  if (!F.ok) return -1;
+  const FastPlan P = plan_fast(F);
+  return P.depth >= 1 && P.quota >= 0 ? SPECTRA_PATH_TENSOR_CORE : SPECTRA_PATH_CUDA_CORE;
+}
+
+extern "C" size_t spectra_cache_bytes(const spectra_config* cfg, const uint8_t* widths_host, int64_t capacity_tokens) {
+  const size_t tb = spectra_tile_bytes(cfg, widths_host);
+  if (tb == 0 || capacity_tokens < 0) return 0;
+  return tb * (size_t)((capacity_tokens + kTile - 1) / kTile);
 }
 
 extern "C" size_t spectra_tile_bytes(const spectra_config* cfg, const uint8_t* widths_host) {

@@ -17,7 +17,15 @@ struct AttnArgs {
   const float* w_dec_k; const float* mean_rot_k; const uint8_t* widths_k;
   const float* w_dec_v; const float* mean_rot_v; const uint8_t* widths_v;
   float scale; void* out; int out_dtype; float* lse; float* partials; int n_splits; int32_t* status;
+  int max_seq_len;   // capacity of every sequence's buffers in tokens: a longer seq_len is reported and attends to nothing
 };
+
+// Tokens sequence b attends to: its length, or 0 when the length exceeds what the buffers hold (the caller learns
+// of it through SPECTRA_STATUS_CAPACITY; nothing past a buffer's end is ever read or written).
+__device__ __forceinline__ int attended_tokens(const AttnArgs& p, int b) {
+  const int n = p.seq_len[b];
+  return n > p.max_seq_len ? 0 : n;
+}
 
 struct GenericSmem {
   StripTable tk, tv;
@@ -42,7 +50,8 @@ __global__ void __launch_bounds__(128) attention_generic_kernel(AttnArgs p) {
   const int b = u / p.n_kv, hk = u - b * p.n_kv;
   const int ps = (int)(u % p.n_param_sets);
   const int G = p.gqa, gs = p.scale_group;
-  const int n = p.seq_len[b];
+  const int n = attended_tokens(p, b);
+  if (split == 0 && hk == 0 && tid == 0 && p.seq_len[b] > p.max_seq_len && p.status) atomicOr(p.status, SPECTRA_STATUS_CAPACITY);
   const int n_tiles = (n + kTile - 1) / kTile;
   const int per = (n_tiles + p.n_splits - 1) / p.n_splits;
   const int tile_begin = split * per, tile_end = min(tile_begin + per, n_tiles);

@@ -36,13 +36,14 @@ constexpr int kRecHead = 4;      // floats of a record's per-head header: m, l, 
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct alignas(16) UnitDesc {
-  int32_t tbk, tbv;
+  int32_t tbk, tbv;             // tile bytes (16 for a unit whose layout was refused: its copies stay harmless)
   int32_t kmeta[2], vmeta[2];   // byte offset of lo16[128] of scale group g (R16 256 bytes later), -1 if inactive
   uint32_t krun[2][4];          // K runs [scale group][class]: (byte offset of the first pair) / 16 | chunks << 16 |
                                 // slot of a strip stored alone in the last chunk << 24 | (there is one) << 27
   uint32_t vcls[4];             // per V class: strips | strips of scale group 0 << 8 | (byte offset / 16) << 16
   uint32_t vfirst[4];           // index of the first V strip of each class
   int32_t n_vstrips, pad0;
+  int64_t src_k, src_v;         // byte offset of the unit's first K / V tile from the cache base (0 if refused)
   float kscale[4];              // 2^-e_h
   float qlo[4][2];              // sum of q' over the active channels of a scale group
   float qconst[4];              // q' . m'_K (natural-log units)
@@ -57,7 +58,20 @@ struct FastArgs {
   int n_units;       // units of the tensor path: (sequence, kv-head, pass); a pass takes up to 4 query heads of the group
   int npass;
   int depth; int slot_k, slot_v;
+  int vq[4];         // V blocks per class the launched main kernel is built for
 };
+
+// What the main kernel relies on for one unit, checked on the device against the widths the kernels actually read
+// (the host sized the shared-memory slots and picked the kernel variant from its own copy of the widths): tiles fit
+// their slots, every V class fits its quota of 16-strip blocks, the B table fits, and both tile streams start on a
+// 16-byte boundary (bulk copies).
+__host__ __device__ inline bool fast_layout_ok(int tile_bytes_k, int tile_bytes_v, const int (&vblocks)[4],
+                                               int k_entries, unsigned long long addr_k, unsigned long long addr_v,
+                                               int slot_k, int slot_v, const int (&vq)[4]) {
+  bool ok = tile_bytes_k <= slot_k && tile_bytes_v <= slot_v && k_entries <= kKcMax;
+  for (int c = 0; c < 4; c++) ok = ok && vblocks[c] <= vq[c];
+  return ok && (addr_k & 15ull) == 0 && (addr_v & 15ull) == 0;
+}
 
 // ------------------------------------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -189,10 +203,12 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
   if (bid == f.n_units) {
     // ---- tile prefix sums over units and each worker warp's first unit
     const int n_units = f.n_units;
+    for (int b = tid; b < p.batch; b += kPrepThreads)
+      if (p.seq_len[b] > p.max_seq_len && p.status) atomicOr(p.status, SPECTRA_STATUS_CAPACITY);
     const int per = (n_units + 127) / 128;
     int local = 0;
     if (tid < 128) {
-      for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (p.seq_len[(i / f.npass) / p.n_kv] + kTile - 1) / kTile;
+      for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (attended_tokens(p, (i / f.npass) / p.n_kv) + kTile - 1) / kTile;
       S.scan[tid] = local;
     }
     __syncthreads();
@@ -206,7 +222,7 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
       int run = S.scan[tid];
       for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) {
         f.tile_prefix[i] = run;
-        run += (p.seq_len[(i / f.npass) / p.n_kv] + kTile - 1) / kTile;
+        run += (attended_tokens(p, (i / f.npass) / p.n_kv) + kTile - 1) / kTile;
       }
     }
     __syncthreads();
@@ -407,11 +423,24 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
     D.vcls[c] = pack_cls(TV, c, S.ng0[1][c]);
     D.vfirst[c] = TV.class_first[c];
   }
+  // ---- the unit's layout against what the host assumed; a refused unit gets harmless copies and no work
+  int vblocks[4];
+#pragma unroll
+  for (int c = 0; c < 4; c++) vblocks[c] = (TV.class_first[c + 1] - TV.class_first[c] + 15) >> 4;
+  const unsigned long long addr_k = (unsigned long long)(p.cache_k + p.off_k[u]), addr_v = (unsigned long long)(p.cache_v + p.off_v[u]);
+  const bool ok = fast_layout_ok(TK.tile_bytes, TV.tile_bytes, vblocks, ent_base[8], addr_k, addr_v, f.slot_k, f.slot_v, f.vq);
   if (tid == 64) {
-    D.tbk = TK.tile_bytes; D.tbv = TV.tile_bytes;
-    D.kmeta[0] = TK.meta_off[0]; D.kmeta[1] = TK.meta_off[1];
-    D.vmeta[0] = TV.meta_off[0]; D.vmeta[1] = TV.meta_off[1];
-    D.n_vstrips = TV.n_strips; D.pad0 = 0;
+    D.tbk = ok ? TK.tile_bytes : 16; D.tbv = ok ? TV.tile_bytes : 16;
+    D.kmeta[0] = ok ? TK.meta_off[0] : -1; D.kmeta[1] = ok ? TK.meta_off[1] : -1;
+    D.vmeta[0] = ok ? TV.meta_off[0] : -1; D.vmeta[1] = ok ? TV.meta_off[1] : -1;
+    D.n_vstrips = ok ? TV.n_strips : 0; D.pad0 = 0;
+    D.src_k = ok ? p.off_k[u] : 0; D.src_v = ok ? p.off_v[u] : 0;
+    if (!ok && p.status) atomicOr(p.status, SPECTRA_STATUS_BAD_LAYOUT);
+  }
+  if (!ok) {
+    __syncthreads();
+    if (tid < 8) D.krun[tid >> 2][tid & 3] = 0;
+    if (tid >= 32 && tid < 36) D.vcls[tid - 32] = 0;
   }
 }
 

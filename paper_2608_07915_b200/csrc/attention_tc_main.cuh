@@ -338,7 +338,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
     const UnitDesc& d = f.desc[min(u, f.n_units - 1)];
     q.unit = u; q.rem = n;
     q.tb = side ? d.tbv : d.tbk;
-    q.addr = (uint64_t)(side ? p.cache_v + p.off_v[u / f.npass] : p.cache_k + p.off_k[u / f.npass]);
+    q.addr = (uint64_t)(side ? p.cache_v + d.src_v : p.cache_k + d.src_k);
   };
   auto start_k = [&](int slot) {
     if (ws.k.rem == 0) next_unit(ws.k, 0);
@@ -366,9 +366,9 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
     const UnitDesc& d = f.desc[cu];
     const uint32_t tbk = d.tbk, tbv = d.tbv;
     ws.k.unit = cu; ws.k.rem = cnt - ct; ws.k.tb = tbk;
-    ws.k.addr = (uint64_t)(p.cache_k + p.off_k[cu / f.npass] + (int64_t)ct * tbk);
+    ws.k.addr = (uint64_t)(p.cache_k + d.src_k + (int64_t)ct * tbk);
     ws.v.unit = cu; ws.v.rem = cnt - ct; ws.v.tb = tbv;
-    ws.v.addr = (uint64_t)(p.cache_v + p.off_v[cu / f.npass] + (int64_t)ct * tbv);
+    ws.v.addr = (uint64_t)(p.cache_v + d.src_v + (int64_t)ct * tbv);
     for (int j = 0; j < issued_k; j++) { start_k(j); start_v(j); }
   }
 
@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
       if (lane < 18) ws.head[lane < 6 ? lane : lane + 2] = reinterpret_cast<const uint32_t*>(&d)[lane];
       kscale = d.kscale[tig];                                  // a power of two: the divisions are exact
       qlo0 = d.qlo[tig][0] / kscale; qlo1 = d.qlo[tig][1] / kscale;
-      n_seq = p.seq_len[(cu / f.npass) / p.n_kv];
+      n_seq = attended_tokens(p, (cu / f.npass) / p.n_kv);
 #pragma unroll
       for (int mb = 0; mb < NACC; mb++)
 #pragma unroll

@@ -3,7 +3,6 @@
 // read-modify-write of a partly filled tail tile needs no atomics.
 #include "common.cuh"
 #include "encode_append.cuh"
-#include "encode_tc.cuh"
 #include "encode_umma.cuh"
 #include "decode_umma.cuh"
 
@@ -54,7 +53,7 @@ __global__ void __launch_bounds__(128) encode_append_kernel(AppendArgs p) {
 
 struct EncodeArgs {
   const void* x; int x_dtype; int flags; int side; int scale_group;
-  int64_t n_param_sets; const int32_t* pos0; int32_t n_new; int64_t stride_unit, stride_token;
+  int64_t n_param_sets; const int32_t* pos0; int32_t n_new; int32_t capacity; int64_t stride_unit, stride_token;
   const float* w_enc; const float* mean_rot; const uint8_t* widths;
   uint8_t* cache; const int64_t* unit_offset; int32_t* status;
 };
@@ -66,7 +65,11 @@ __global__ void __launch_bounds__(128, 1) encode_kernel(EncodeArgs p) {
   const int ps = (int)(u % p.n_param_sets);
   const int tid = threadIdx.x;
   const int pos_first = p.pos0[u];
-  const int pos_end = pos_first + p.n_new;
+  int pos_end = pos_first + p.n_new;
+  if (p.capacity > 0 && pos_end > p.capacity) {          // tokens past the capacity are not written; reported once
+    pos_end = max(p.capacity, pos_first);
+    if (blockIdx.x == 0 && tid == 0 && p.status) atomicOr(p.status, SPECTRA_STATUS_CAPACITY);
+  }
   const int tile = pos_first / kTile + blockIdx.x;
   const int tile_pos = tile * kTile;
   if (tile_pos >= pos_end) return;
@@ -269,10 +272,11 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
                               int64_t n_units, int64_t n_param_sets, const int32_t* pos0, int32_t n_new,
                               int64_t stride_unit, int64_t stride_token, const float* w_enc, const float* mean_rot,
                               const uint8_t* widths, uint8_t* cache, const int64_t* unit_offset,
-                              int32_t* status_word, void* stream) {
+                              int32_t capacity_tokens, int32_t* status_word, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
-  if ((side != SPECTRA_SIDE_K && side != SPECTRA_SIDE_V) || n_units < 0 || n_new < 0 || n_param_sets < 1)
+  if ((side != SPECTRA_SIDE_K && side != SPECTRA_SIDE_V) || n_units < 0 || n_new < 0 || n_param_sets < 1 ||
+      capacity_tokens < 0)
     return SPECTRA_INVALID_ARG;
   if (x_dtype != SPECTRA_F32 && x_dtype != SPECTRA_BF16) return SPECTRA_INVALID_ARG;
   if (flags & ~SPECTRA_ROTATED_INPUT) return SPECTRA_INVALID_ARG;
@@ -284,7 +288,7 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   if (n_new <= kAppendMaxTokens) {   // decode-step appends: one light CTA per unit-side
     AppendArgs ap{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
-                  w_enc, mean_rot, widths, cache, unit_offset, status_word, nullptr, 1};
+                  w_enc, mean_rot, widths, cache, unit_offset, status_word, nullptr, 1, capacity_tokens};
     if (cudaFuncSetAttribute(encode_append_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAppendDynSmem) !=
         cudaSuccess)
       return SPECTRA_CUDA_ERROR;
@@ -294,7 +298,7 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
   if (x_dtype == SPECTRA_BF16 && !(flags & SPECTRA_ROTATED_INPUT) && cfg->scale_group == 64 &&
       stride_token % 8 == 0 && stride_unit % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
     // bf16 bulk encode: rotation on the tensor cores
-    EncodeTcArgs ta{reinterpret_cast<const __nv_bfloat16*>(x), side, n_param_sets, pos0, n_new, stride_unit,
+    EncodeTcArgs ta{reinterpret_cast<const __nv_bfloat16*>(x), side, n_param_sets, pos0, n_new, capacity_tokens, stride_unit,
                     stride_token, w_enc, mean_rot, widths, cache, unit_offset, status_word};
     // rotation on the 5th-generation tensor cores (accumulator tiles in tensor memory); the token tiles arrive by
     // TMA: a 3-D map over x [unit][token][channel] whose box is 8 channels x 128 tokens
@@ -314,7 +318,7 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
       return launch_status();
     }
   }
-  EncodeArgs a{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
+  EncodeArgs a{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, capacity_tokens, stride_unit, stride_token,
                w_enc, mean_rot, widths, cache, unit_offset, status_word};
   if (cudaFuncSetAttribute(encode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CodecSmem)) !=
       cudaSuccess)
@@ -328,7 +332,7 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
                               int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
                               const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out,
                               int out_dtype, float* yhat_out, int64_t stride_unit, int64_t stride_token,
-                              void* stream) {
+                              int32_t* status_word, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   if ((side != SPECTRA_SIDE_K && side != SPECTRA_SIDE_V) || n_units < 0 || max_tokens < 0 || n_param_sets < 1)
@@ -341,7 +345,7 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
   if (out && !w_dec) return SPECTRA_INVALID_ARG;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
-               out_dtype, yhat_out, stride_unit, stride_token, nullptr};
+               out_dtype, yhat_out, stride_unit, stride_token, status_word};
   if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05), persistent grid
     const size_t dec_smem = sizeof(DecodeTcSmem) + 128;
     if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem) !=

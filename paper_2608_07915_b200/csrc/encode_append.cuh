@@ -16,6 +16,7 @@ struct AppendArgs {
   const float* w_enc; const float* mean_rot; const uint8_t* widths;
   uint8_t* cache; const int64_t* unit_offset; int32_t* status;
   const int32_t* seq_len; int n_kv;      // with pos0 == NULL: the token goes to position seq_len[u / n_kv] - 1
+  int32_t capacity;                      // tokens a unit-side's buffer holds (0: not checked)
 };
 
 // Bounded wait for phase 0 of an mbarrier (each poll blocks for a bounded hardware interval).
@@ -65,7 +66,13 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u, unsigned c
                  : "memory");
   }
   const int b = p.widths[(int64_t)ps * kD + j];
-  const int pos_first = p.pos0 ? p.pos0[u] : p.seq_len[u / p.n_kv] - 1;
+  int pos_first = p.pos0 ? p.pos0[u] : p.seq_len[u / p.n_kv] - 1;
+  int n_new = p.n_new;
+  if (p.capacity > 0 && pos_first + n_new > p.capacity) {   // tokens past the capacity are not written; reported once
+    if (j == 0 && p.status) atomicOr(p.status, SPECTRA_STATUS_CAPACITY);
+    n_new = max(0, p.capacity - pos_first);
+    if (n_new == 0) pos_first = -1;
+  }
   const float mr = rotated ? 0.f : p.mean_rot[(int64_t)ps * kD + j];
   uint8_t* base = p.cache + p.unit_offset[u];
   for (int idx = j; idx < p.n_new * kD; idx += 128) {
@@ -128,7 +135,7 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u, unsigned c
   int status = 0;
   bool w_ready = rotated || !bulk;
 
-  for (int t = 0; t < p.n_new; t++) {
+  for (int t = 0; t < n_new; t++) {
     const int pos = pos_first + t;
     const int slot = pos & (kTile - 1);
     uint8_t* tile = base + (int64_t)(pos / kTile) * tile_bytes;

@@ -11,7 +11,6 @@ constexpr int kMomChunk = 256;
 
 struct FitWorkspace {   // per unit, all fp64
   double S[kD * kD];
-  double VT[kD * kD];   // unused (the eigenvectors are accumulated in shared memory); kept for the workspace size
   double s[kD];
 };
 

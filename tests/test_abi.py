@@ -43,7 +43,7 @@ def test_config_default_and_host_helpers(lib):
     assert sp.tile_bytes(cfg, [2] * 64 + [0] * 64) == 16 * 128 + 512
     assert sp.tile_bytes(cfg, [0] * 128) == 0
     assert sp.status_string(0) == "SPECTRA_OK" and sp.status_string(3) == "SPECTRA_WORKSPACE_TOO_SMALL"
-    assert sp.fit_workspace_bytes(cfg, 2) > 2 * 2 * 128 * 128 * 8
+    assert sp.fit_workspace_bytes(cfg, 2) >= 2 * (128 * 128 + 128) * 8
     assert sp.attention_workspace_bytes(cfg, 8, 8, 32, 32768) > 0
 
 
@@ -60,13 +60,16 @@ def test_bad_arguments_are_rejected_before_any_launch(lib):
     assert lib.spectra_fit_workspace_bytes(C.byref(bad), C.c_int64(1)) == 0
     bad = sp.default_config(b_max=9)
     assert lib.spectra_encode(C.byref(bad), 0, null, 0, 0, C.c_int64(1), C.c_int64(1), null, 1, C.c_int64(0),
-                              C.c_int64(0), null, null, null, null, null, null, null) == sp.INVALID_ARG
+                              C.c_int64(0), null, null, null, null, null, 0, null, null) == sp.INVALID_ARG
     # rotated input must be fp32; unknown flags; bad side
-    args = (C.c_int64(1), C.c_int64(1), null, 1, C.c_int64(0), C.c_int64(0), null, null, null, null, null, null, null)
+    args = (C.c_int64(1), C.c_int64(1), null, 1, C.c_int64(0), C.c_int64(0), null, null, null, null, null, 0, null,
+            null)
     assert lib.spectra_encode(C.byref(cfg), 0, null, sp.BF16, sp.ROTATED_INPUT, *args) == sp.INVALID_ARG
     assert lib.spectra_encode(C.byref(cfg), 0, null, sp.F32, 8, *args) == sp.INVALID_ARG
     assert lib.spectra_encode(C.byref(cfg), 2, null, sp.F32, 0, *args) == sp.INVALID_ARG
     assert lib.spectra_encode(C.byref(cfg), 0, null, sp.F32, 0, *args) == sp.INVALID_ARG     # null pointers
+    neg = (C.c_int64(1), C.c_int64(1), null, 1, C.c_int64(0), C.c_int64(0), null, null, null, null, null, -5, null, null)
+    assert lib.spectra_encode(C.byref(cfg), 0, null, sp.F32, 0, *neg) == sp.INVALID_ARG      # negative capacity
     # attention: query heads must be a multiple of kv heads; group size above 8 unsupported
     def attn(n_kv, n_q):
         return lib.spectra_decode_attention(C.byref(cfg), null, 0, 1, n_kv, n_q, null, 128, null, null, null, null,
@@ -86,15 +89,45 @@ def test_misaligned_buffers_are_refused_on_the_host(lib):
     ok = 0x10000
     # spectra_encode: cache one byte off
     assert lib.spectra_encode(C.byref(cfg), 0, p(ok), sp.F32, 0, C.c_int64(1), C.c_int64(1), p(ok), 1, C.c_int64(128),
-                              C.c_int64(128), p(ok), p(ok), p(ok), p(ok + 1), p(ok), null, null) == sp.INVALID_ARG
+                              C.c_int64(128), p(ok), p(ok), p(ok), p(ok + 1), p(ok), 0, null, null) == sp.INVALID_ARG
     # spectra_decode: odd cache address
     assert lib.spectra_decode(C.byref(cfg), 0, p(ok + 1), p(ok), C.c_int64(1), C.c_int64(1), p(ok), 128, p(ok), p(ok),
-                              p(ok), p(ok), sp.F32, null, C.c_int64(128 * 128), C.c_int64(128), null) == sp.INVALID_ARG
+                              p(ok), p(ok), sp.F32, null, C.c_int64(128 * 128), C.c_int64(128), null,
+                              null) == sp.INVALID_ARG
     # spectra_decode_attention: W_dec,K four bytes off
     big = C.c_size_t(1 << 30)
     assert lib.spectra_decode_attention(C.byref(cfg), p(ok), sp.F32, 1, 1, 4, p(ok), 128, p(ok), p(ok), p(ok), p(ok),
                                         C.c_int64(1), p(ok + 4), null, p(ok), p(ok), p(ok), p(ok), null, null,
                                         C.c_float(0), p(ok), sp.F32, null, p(ok), big, null, null) == sp.INVALID_ARG
+
+
+def test_cache_bytes_and_attention_path(lib):
+    """Host helpers: a unit-side's buffer size for a capacity in tokens, and which kernels an attention call will
+    run for a set of widths (the tensor-core kernel is built for a few tuples of V blocks per class; scale groups
+    other than 64, missing host widths and profiles outside the tuples take the CUDA-core kernel)."""
+    import numpy as np
+    cfg = sp.default_config()
+    w4 = [4] * 128
+    assert sp.cache_bytes(cfg, w4, 0) == 0
+    assert sp.cache_bytes(cfg, w4, 1) == sp.tile_bytes(cfg, w4)
+    assert sp.cache_bytes(cfg, w4, 128) == sp.tile_bytes(cfg, w4)
+    assert sp.cache_bytes(cfg, w4, 129) == 2 * sp.tile_bytes(cfg, w4)
+    assert sp.cache_bytes(cfg, w4, 32768 + 64) == 257 * 9216
+    assert sp.cache_bytes(cfg, [9] * 128, 128) == 0                                   # bad widths
+    two = np.full((1, 128), 2, np.uint8)                                             # 8 blocks of 2-bit strips
+    assert sp.attention_path(cfg, 8, 32, 1, two, two) == sp.PATH_TENSOR_CORE
+    assert sp.attention_path(cfg, 4, 28, 1, two, two) == sp.PATH_TENSOR_CORE        # groups of 7 heads: two passes
+    assert sp.attention_path(cfg, 8, 32, 1, None, None) == sp.PATH_CUDA_CORE        # no host widths
+    assert sp.attention_path(sp.default_config(scale_group=32), 8, 32, 1, two, two) == sp.PATH_CUDA_CORE
+    eight = np.full((1, 128), 8, np.uint8)                                           # an 8-bit V class: no variant
+    assert sp.attention_path(cfg, 8, 32, 1, two, eight) == sp.PATH_CUDA_CORE
+    assert sp.attention_path(cfg, 8, 32, 1, eight, two) == sp.PATH_TENSOR_CORE      # the K side has no such limit
+    three = np.full((1, 128), 3, np.uint8)                                           # 8 + 8 blocks: beyond every tuple
+    assert sp.attention_path(cfg, 8, 32, 1, two, three) == sp.PATH_CUDA_CORE
+    with pytest.raises(sp.SpectraError):
+        sp.attention_path(cfg, 3, 8, 1, two, two)
+    with pytest.raises(sp.SpectraError):
+        sp.attention_path(cfg, 8, 32, 1, two, np.full((1, 128), 9, np.uint8))
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

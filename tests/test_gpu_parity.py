@@ -671,3 +671,115 @@ def test_inputs_with_a_large_mean_reconstruction_attention_and_fused_step(sp, te
     ref2, lse2 = _oracle_attention(4, q2[None].astype(np.float64), [n + 1], S["k"], S["v"], held["k"], held["v"])
     assert H.rel_err_per_vector(out.cpu().numpy()[0], ref2[0]) <= TOL
     assert np.abs(lse_d.cpu().numpy()[0] - lse2[0]).max() <= 2e-3
+
+
+def test_appends_beyond_the_capacity_are_reported_not_written(sp):
+    """spectra_encode with a capacity: tokens at positions >= capacity_tokens are not written and the status word gets
+    SPECTRA_STATUS_CAPACITY, on the append kernel (a few tokens), the CUDA-core bulk kernel (fp32) and the
+    tensor-core bulk kernel (bf16).  The buffer is followed by a guard region that must stay untouched."""
+    wl = si.WORKLOADS["tiny"]
+    cfg = sp.default_config()
+    X = si.draw_unit(wl, 0, 0, si.SIDE_K, 0, n_tokens=512)
+    params = H.fit_params([X], 8.0)
+    dp = H.dev_params(params)
+    tb = int(params.tile_bytes[0])
+    cap = 256                                              # two tiles
+    assert sp.cache_bytes(cfg, params.widths[0], cap) == 2 * tb
+    for dt, first, n_new in ((torch.float32, 250, 10), (torch.float32, 100, 300), (torch.bfloat16, 100, 300),
+                             (torch.float32, 256, 4)):
+        ref = np.zeros(2 * tb, np.uint8)
+        n_fit = max(0, min(cap - first, n_new))
+        xs = si.to_bf16_f32(X[first:first + n_new]) if dt == torch.bfloat16 else X[first:first + n_new]
+        if n_fit:
+            assert H.oracle_encode(params, si.SIDE_K, xs[None, :n_fit], [first], ref, np.zeros(1, np.int64)) == 0
+        buf = torch.full((2 * tb + 4096,), 0x5C, dtype=torch.uint8, device="cuda")
+        buf[:2 * tb] = 0
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        sp.encode(cfg, si.SIDE_K, H.to_dev(xs[None]).to(dt), 0, 1, 1, torch.tensor([first], dtype=torch.int32, device="cuda"),
+                  n_new, n_new * 128, 128, dp["w_enc"], dp["m_rot"], dp["widths"], buf,
+                  torch.zeros(1, dtype=torch.int64, device="cuda"), status, capacity_tokens=cap)
+        torch.cuda.synchronize()
+        assert int(status.item()) == sp.STATUS_CAPACITY
+        got = buf.cpu().numpy()
+        assert (got[2 * tb:] == 0x5C).all()                # nothing past the buffer
+        if n_fit:
+            bad, tot, dmax, mmax, _ = H.compare_coded_units(ref, got[:2 * tb], tb, cap, params.widths[0], 64, si.SIDE_K)
+            assert dmax <= 1 and mmax <= 1 and bad <= 3
+        else:
+            assert not got[:2 * tb].any()
+    # within the capacity: no bit
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    buf = torch.zeros(2 * tb, dtype=torch.uint8, device="cuda")
+    sp.encode(cfg, si.SIDE_K, H.to_dev(X[None, :256]), 0, 1, 1, torch.zeros(1, dtype=torch.int32, device="cuda"), 256,
+              256 * 128, 128, dp["w_enc"], dp["m_rot"], dp["widths"], buf, torch.zeros(1, dtype=torch.int64, device="cuda"),
+              status, capacity_tokens=cap)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+
+@pytest.mark.parametrize("tensor_path", [True, False], ids=["tensor", "generic"])
+def test_sequence_longer_than_max_seq_len_is_reported_and_skipped(sp, tensor_path):
+    """Attention and the fused step treat max_seq_len as the capacity: a sequence whose seq_len exceeds it sets
+    SPECTRA_STATUS_CAPACITY, gets no append and a zero output row; the other sequence is unaffected."""
+    import dataclasses
+    from paper_2608_07915_b200 import harness
+    wl = dataclasses.replace(si.WORKLOADS["tiny"], batch=2)
+    m = harness.CodedModelCache(wl, layers=1, batch=2, extra_tokens=128)
+    m.tensor_path = tensor_path
+    m.build()
+    before = [m.side[0][s].cache.clone() for s in (0, 1)]
+    gen = torch.Generator(device="cuda").manual_seed(8)
+    q = torch.randn((2, wl.q_heads, 128), generator=gen, device="cuda")
+    nk = torch.randn((2 * wl.kv_heads, 128), generator=gen, device="cuda")
+    nv = torch.randn((2 * wl.kv_heads, 128), generator=gen, device="cuda")
+    ref = torch.zeros((2, wl.q_heads, 128), dtype=torch.float32, device="cuda")
+    m.seq_len += 1
+    m.step_layer(0, q, nk, nv, ref)                       # both sequences in range
+    torch.cuda.synchronize()
+    assert int(m.status.item()) == 0
+    for s in (0, 1):
+        m.side[0][s].cache.copy_(before[s])
+    m.seq_len[1] = m.cap_tokens + 1                        # beyond what the buffers hold
+    out = torch.full((2, wl.q_heads, 128), 3.0, dtype=torch.float32, device="cuda")
+    m.step_layer(0, q, nk, nv, out)
+    torch.cuda.synchronize()
+    assert int(m.status.item()) == sp.STATUS_CAPACITY
+    assert (out[1] == 0).all()
+    if tensor_path:
+        assert torch.equal(out[0], ref[0])
+    else:
+        assert torch.allclose(out[0], ref[0], rtol=1e-5, atol=1e-6)
+    for s in (0, 1):
+        ls = m.side[0][s]
+        a = int(ls.unit_offset_host[wl.kv_heads])
+        assert torch.equal(ls.cache[a:], before[s][a:])   # the units of the out-of-range sequence were not touched
+
+
+def test_tensor_core_path_refuses_units_whose_widths_differ_from_the_host_copy(sp):
+    """The host sizes the shared-memory tile slots from its copy of the widths.  If the widths on the device ask for
+    larger tiles (a caller's mistake), the kernels must not copy them: the unit is skipped, SPECTRA_STATUS_BAD_LAYOUT
+    is set, and the call completes with finite outputs."""
+    wl, S = _tiny_setup(sp, 4.0)
+    cfg = sp.default_config()
+    n = 512
+    caches = {}
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        c = np.zeros(S[name]["total"], np.uint8)
+        H.oracle_encode(S[name]["params"], side, S[name]["X"][None, :n], [0], c, S[name]["off"])
+        caches[name] = c
+    pk, pv = S["k"]["params"], S["v"]["params"]
+    dk, dv = H.dev_params(pk), H.dev_params(pv)
+    host_k = np.minimum(pk.widths, 2).astype(np.uint8)      # the host believes in narrower channels: smaller tiles
+    host_v = np.minimum(pv.widths, 2).astype(np.uint8)
+    assert sp.attention_path(cfg, 1, 4, 1, host_k, host_v) == sp.PATH_TENSOR_CORE
+    q = H.to_dev(si.draw_queries(wl, 0, 0)[None])
+    out = torch.full((1, 4, 128), 3.0, dtype=torch.float32, device="cuda")
+    ws = torch.zeros(sp.attention_workspace_bytes(cfg, 1, 1, 4, n), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sp.decode_attention(cfg, q, 1, 1, 4, H.to_dev(np.asarray([n], np.int32)), n, H.to_dev(caches["k"]),
+                        H.to_dev(S["k"]["off"]), H.to_dev(caches["v"]), H.to_dev(S["v"]["off"]), 1, dk["w_dec"],
+                        dk["m_rot"], dk["widths"], dv["w_dec"], dv["m_rot"], dv["widths"], 0.0, out, None, ws, status,
+                        host_k, host_v)
+    torch.cuda.synchronize()
+    assert int(status.item()) == sp.STATUS_BAD_LAYOUT
+    assert torch.isfinite(out).all()
