@@ -373,11 +373,10 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
   }
 
   float acc_o[NACC][4];
-  float m_run = -INFINITY, l_run = 0.f, plo0 = 0.f, plo1 = 0.f;
+  float m_ref = -INFINITY, l_run = 0.f, plo0 = 0.f, plo1 = 0.f;
   float kscale = 0.f, qlo0 = 0.f, qlo1 = 0.f;
   int n_seq = 0;
   bool fresh = true, ok = true;
-  float boost = 0.f;          // power-of-two lift of the probabilities (see below); -1 = not chosen yet
   int slot = 0;
   uint32_t parity = 0;
 
@@ -395,9 +394,8 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
       for (int mb = 0; mb < NACC; mb++)
 #pragma unroll
         for (int e = 0; e < 4; e++) acc_o[mb][e] = 0.f;
-      m_run = -INFINITY; l_run = 0.f; plo0 = 0.f; plo1 = 0.f;
+      m_ref = -INFINITY; l_run = 0.f; plo0 = 0.f; plo1 = 0.f;
       fresh = false;
-      boost = -1.f;
       __syncwarp();
     }
 
@@ -453,69 +451,58 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
       for (int i = 0; i < 16; i++)
         if (tok0 + i >= n_seq) s[i] = -INFINITY;
     }
-    float mx = s[0];
-#pragma unroll
-    for (int i = 1; i < 16; i++) mx = fmaxf(mx, s[i]);
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-    mx *= kscale;                                            // kscale is a positive power of two: exact
-    if (mx > m_run) {        // new running maximum for this thread's head: rescale what has been accumulated
-      const float alpha = fast_exp2(m_run - mx);   // exp2(-inf) = 0 on the first tile
-      m_run = mx;
-      l_run *= alpha; plo0 *= alpha; plo1 *= alpha;
-#pragma unroll
-      for (int mb = 0; mb < NACC; mb++)
-#pragma unroll
-        for (int e = 0; e < 4; e++) acc_o[mb][e] *= alpha;
-    }
     ok = ok && mbar_wait(bars + 8 * (4 + slot), parity);
-    // probabilities times the V group ranges, as fp16 pairs (group 0, group 1), transposed into B fragments
+    // Probabilities enter the tensor core as fp16, multiplied by the V group range of their token: p~ = 2^(s - m_ref) R.
+    // The reference exponent m_ref of this warp's share of the unit is kept 13 binades below the largest s + log2 R
+    // seen so far (per head), so that no p~ exceeds 2^13 (fp16 holds 65504) while the bulk of them, far smaller with
+    // tens of thousands of tokens, stays in fp16's normal range.  Whenever a tile raises it, everything accumulated
+    // so far is rescaled: a new maximum score and a token with an unusually large value range are the same event.
+    // The record carries m_ref, so the merge of the splits is unaffected.
     uint32_t pb[2][8];
     {
       const int vmeta0 = (int)ws.head[4], vmeta1 = (int)ws.head[5];
-      if (boost < 0.f) {
-        // First tile of this warp's share of the unit.  Probabilities are exp2(s - max) <= 1 and enter the
-        // tensor core as fp16 times the V group range; with tens of thousands of tokens the typical probability is
-        // far below the fp16 normal range.  Lift everything by 2^boost (the record's maximum is lowered by the same
-        // amount, so the merge is unaffected), leaving room for group ranges 8x larger than in this tile.
-        uint32_t vr0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, vr1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        if (vmeta0 >= 0) ld_tile_words<8>(vtile + vmeta0 + 256 + 32 * gid, vr0);
-        if (vmeta1 >= 0) ld_tile_words<8>(vtile + vmeta1 + 256 + 32 * gid, vr1);
-        float rmax = 0.f;
+      uint32_t vr0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, vr1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      if (vmeta0 >= 0) ld_tile_words<8>(vtile + vmeta0 + 256 + 32 * gid, vr0);
+      if (vmeta1 >= 0) ld_tile_words<8>(vtile + vmeta1 + 256 + 32 * gid, vr1);
+      float mx = s[0];
 #pragma unroll
-        for (int r = 0; r < 8; r++) {
-          const float2 a = h2f2(vr0[r]), b = h2f2(vr1[r]);
-          rmax = fmaxf(rmax, fmaxf(fmaxf(a.x, a.y), fmaxf(b.x, b.y)));
-        }
+      for (int i = 1; i < 16; i++) mx = fmaxf(mx, s[i]);
+      __half2 rm = __hmax2(*reinterpret_cast<const __half2*>(&vr0[0]), *reinterpret_cast<const __half2*>(&vr1[0]));
 #pragma unroll
-        for (int sft = 1; sft <= 16; sft <<= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, sft));
-        const int e = (int)((__float_as_uint(rmax) >> 23) & 0xff) - 126;     // rmax < 2^e
-        boost = (float)max(0, min(13, 13 - e));
+      for (int r = 1; r < 8; r++)
+        rm = __hmax2(rm, __hmax2(*reinterpret_cast<const __half2*>(&vr0[r]), *reinterpret_cast<const __half2*>(&vr1[r])));
+      const float rmax = fmaxf(__low2float(rm), __high2float(rm));          // ranges are non-negative
+      const int e = (int)((__float_as_uint(rmax) >> 23) & 0xff) - 126;      // rmax < 2^e
+      float need = fmaf(mx, kscale, (float)(e - 13));                       // kscale is a positive power of two
+      need = fmaxf(need, __shfl_xor_sync(0xffffffffu, need, 4));
+      need = fmaxf(need, __shfl_xor_sync(0xffffffffu, need, 8));
+      need = fmaxf(need, __shfl_xor_sync(0xffffffffu, need, 16));
+      if (need > m_ref) {      // rescale what has been accumulated (exp2(-inf) = 0 on the first tile)
+        const float alpha = fast_exp2(m_ref - need);
+        m_ref = need;
+        l_run *= alpha; plo0 *= alpha; plo1 *= alpha;
+#pragma unroll
+        for (int mb = 0; mb < NACC; mb++)
+#pragma unroll
+          for (int e2 = 0; e2 < 4; e2++) acc_o[mb][e2] *= alpha;
       }
-      const float m_use = (m_run == -INFINITY ? 0.f : m_run) - boost;
+      const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
 #pragma unroll
       for (int half = 0; half < 2; half++) {
-        uint32_t vlo0[4] = {0, 0, 0, 0}, vlo1[4] = {0, 0, 0, 0}, vr0[4] = {0, 0, 0, 0}, vr1[4] = {0, 0, 0, 0};
-        if (vmeta0 >= 0) {
-          ld_tile_words<4>(vtile + vmeta0 + 32 * gid + 16 * half, vlo0);
-          ld_tile_words<4>(vtile + vmeta0 + 256 + 32 * gid + 16 * half, vr0);
-        }
-        if (vmeta1 >= 0) {
-          ld_tile_words<4>(vtile + vmeta1 + 32 * gid + 16 * half, vlo1);
-          ld_tile_words<4>(vtile + vmeta1 + 256 + 32 * gid + 16 * half, vr1);
-        }
+        uint32_t vlo0[4] = {0, 0, 0, 0}, vlo1[4] = {0, 0, 0, 0};
+        if (vmeta0 >= 0) ld_tile_words<4>(vtile + vmeta0 + 32 * gid + 16 * half, vlo0);
+        if (vmeta1 >= 0) ld_tile_words<4>(vtile + vmeta1 + 32 * gid + 16 * half, vlo1);
 #pragma unroll
         for (int r = 0; r < 4; r++) {
-          const float2 lo0 = h2f2(vlo0[r]), r0 = h2f2(vr0[r]), lo1 = h2f2(vlo1[r]), r1 = h2f2(vr1[r]);
+          const float2 lo0 = h2f2(vlo0[r]), r0 = h2f2(vr0[4 * half + r]), lo1 = h2f2(vlo1[r]), r1 = h2f2(vr1[4 * half + r]);
 #pragma unroll
-          for (int e = 0; e < 2; e++) {
-            const int ii = 2 * r + e;
+          for (int e2 = 0; e2 < 2; e2++) {
+            const int ii = 2 * r + e2;
             const float pr = fast_exp2(fmaf(s[8 * half + ii], kscale, -m_use));
             l_run += pr;
-            plo0 = fmaf(pr, e ? lo0.y : lo0.x, plo0);
-            plo1 = fmaf(pr, e ? lo1.y : lo1.x, plo1);
-            pb[half][ii] = movmatrix_trans(pack_half2_sat(pr * (e ? r0.y : r0.x), pr * (e ? r1.y : r1.x)));
+            plo0 = fmaf(pr, e2 ? lo0.y : lo0.x, plo0);
+            plo1 = fmaf(pr, e2 ? lo1.y : lo1.x, plo1);
+            pb[half][ii] = movmatrix_trans(pack_half2_sat(pr * (e2 ? r0.y : r0.x), pr * (e2 ? r1.y : r1.x)));
           }
         }
       }
@@ -545,7 +532,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
         q1 += __shfl_xor_sync(0xffffffffu, q1, sft);
       }
       float* rec = f.records + (int64_t)(gw + cu) * f.rec_stride + tig * (kRecHead + f.vs_max);
-      if (gid == 0) { rec[0] = m_run - boost; rec[1] = l; rec[2] = q0; rec[3] = q1; }
+      if (gid == 0) { rec[0] = m_ref; rec[1] = l; rec[2] = q0; rec[3] = q1; }
       const UnitDesc& d = f.desc[cu];
       store_class<Q8, 0, NACC>(rec, ws.head[16], d.vfirst[0], gid, acc_o);
       store_class<Q4, Q8, NACC>(rec, ws.head[17], d.vfirst[1], gid, acc_o);

@@ -783,3 +783,32 @@ def test_tensor_core_path_refuses_units_whose_widths_differ_from_the_host_copy(s
     torch.cuda.synchronize()
     assert int(status.item()) == sp.STATUS_BAD_LAYOUT
     assert torch.isfinite(out).all()
+
+
+def test_attention_with_value_outlier_tokens_that_carry_the_probability_mass(sp):
+    """A few late tokens whose value vectors are 30 times larger than the rest, one of them with the dominant score:
+    probability times value range is then far above what the first tiles suggested.  The kernel must follow
+    (its fp16 operand of the value contraction is rescaled when a tile needs more headroom), not saturate."""
+    wl = si.WORKLOADS["tiny"]
+    cfg = sp.default_config()
+    n = 900
+    q = si.draw_queries(wl, 0, 0)
+    S, caches = {}, {}
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        X = si.draw_unit(wl, 0, 0, side, 0, n_tokens=n).copy()
+        if side == si.SIDE_V:
+            X[700:705] *= 30.0
+        else:
+            X[702] = 2.0 * q[0]                                  # head 0 attends to token 702 almost exclusively
+        params = H.fit_params([X[:512]], 8.0)
+        off, total = H.cache_layout(params, 1, n)
+        c = np.zeros(total, np.uint8)
+        assert H.oracle_encode(params, side, X[None], [0], c, off) == 0
+        S[name] = dict(X=X, params=params, off=off, total=total)
+        caches[name] = c
+    ref_b, lse_b = _oracle_attention(4, q[None].astype(np.float64), [n], S["k"], S["v"], caches["k"], caches["v"])
+    ref_a, _ = _oracle_attention(4, q[None].astype(np.float64), [n], S["k"], S["v"], caches["k"], caches["v"], "A")
+    got, lse = _gpu_attention(sp, cfg, H.to_dev(q[None]), 1, 1, 4, [n], n, S["k"], S["v"], caches["k"], caches["v"])
+    assert np.abs(ref_b[0, 0]).max() > 5 * np.abs(ref_b[0, 1:]).max()     # head 0 did land on an outlier token
+    assert H.rel_err_per_vector(got[0], ref_b[0]) <= TOL and H.rel_err_per_vector(got[0], ref_a[0]) <= TOL
+    assert np.abs(lse[0] - lse_b[0]).max() <= 2e-3
