@@ -49,6 +49,10 @@
  *   - Then, for each scale group with a non-zero-width channel, ascending: lo16[128], R16[128]
  *     (little-endian fp16, token order).
  *   - tile bytes = 16 * sum_j b_j + 512 * (number of active scale groups); always a multiple of 16.
+ *   Paged caches.  Every call that addresses tiles takes an optional tile table (device int32) and its row stride:
+ *   with a table, unit_offset[u] is the base of a pool of tile-sized pages (spectra_tile_bytes each; units that share
+ *   a parameter set may share a pool) and tile t of unit u is page tile_table[u * table_stride + t] of that pool.
+ *   NULL means contiguous tiles as above.  The streaming cache of Sec. 3.3 then grows one page at a time.
  *   The K-side pairing puts two channels of one token 16 bits apart in a word, the V-side order
  *   puts two tokens of one channel 16 bits apart: what the tensor-core operand registers of the
  *   score and of the value contraction need, respectively.
@@ -187,8 +191,8 @@ int spectra_alloc_bits(const spectra_config* cfg, const float* var_alloc, int64_
 int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dtype, int flags, int64_t n_units,
                    int64_t n_param_sets, const int32_t* pos0, int32_t n_new, int64_t stride_unit,
                    int64_t stride_token, const float* w_enc, const float* mean_rot, const uint8_t* widths,
-                   uint8_t* cache, const int64_t* unit_offset, int32_t capacity_tokens, int32_t* status_word,
-                   void* stream);
+                   uint8_t* cache, const int64_t* unit_offset, int32_t capacity_tokens, const int32_t* tile_table,
+                   int64_t table_stride, int32_t* status_word, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * spectra_decode -- Sec. 3.3 (Mode A reconstruction): xhat = (yhat + m') W_dec for tokens [0, n_tokens[u])
@@ -203,7 +207,8 @@ int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dty
 int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
                    int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
                    const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out, int out_dtype,
-                   float* yhat_out, int64_t stride_unit, int64_t stride_token, int32_t* status_word, void* stream);
+                   float* yhat_out, int64_t stride_unit, int64_t stride_token, const int32_t* tile_table,
+                   int64_t table_stride, int32_t* status_word, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * spectra_decode_attention -- appendix "Latent-space attention and memory" (Mode B): one decode query per
@@ -241,8 +246,8 @@ int spectra_decode_attention(const spectra_config* cfg, const void* q, int q_dty
                              const float* mean_rot_k, const uint8_t* widths_k, const float* w_dec_v,
                              const float* mean_rot_v, const uint8_t* widths_v, const uint8_t* widths_k_host,
                              const uint8_t* widths_v_host, float softmax_scale, void* out, int out_dtype,
-                             float* lse, void* workspace, size_t workspace_bytes, int32_t* status_word,
-                             void* stream);
+                             float* lse, void* workspace, size_t workspace_bytes, const int32_t* tile_table_k,
+                             const int32_t* tile_table_v, int64_t table_stride, int32_t* status_word, void* stream);
 size_t spectra_attention_workspace_bytes(const spectra_config* cfg, int32_t batch, int32_t n_kv_heads,
                                          int32_t n_q_heads, int32_t max_seq_len);
 
@@ -266,8 +271,9 @@ int spectra_decode_step(const spectra_config* cfg, const void* q, int q_dtype, c
                         const float* w_dec_k, const float* mean_rot_k, const uint8_t* widths_k, const float* w_enc_v,
                         const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
                         const uint8_t* widths_k_host, const uint8_t* widths_v_host, float softmax_scale, void* out,
-                        int out_dtype, float* lse, void* workspace, size_t workspace_bytes, int32_t* status_word,
-                        void* stream);
+                        int out_dtype, float* lse, void* workspace, size_t workspace_bytes,
+                        const int32_t* tile_table_k, const int32_t* tile_table_v, int64_t table_stride,
+                        int32_t* status_word, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Helpers (host only, no device work).

@@ -168,31 +168,34 @@ def alloc_bits(cfg, var_alloc, n_units, ratio, widths):
 
 
 def encode(cfg, side, x, flags, n_units, n_param_sets, pos0, n_new, stride_unit, stride_token, w_enc, mean_rot,
-           widths, cache, unit_offset, status_word=None, capacity_tokens=0):
-    """capacity_tokens: tokens each unit-side's buffer holds (0: not checked)."""
+           widths, cache, unit_offset, status_word=None, capacity_tokens=0, tile_table=None, table_stride=0):
+    """capacity_tokens: tokens each unit-side's buffer holds (0: not checked).  tile_table: device int32
+    [n_units, table_stride] page indices of a paged cache (None: contiguous tiles)."""
     rc = lib().spectra_encode(C.byref(cfg), C.c_int(side), _ptr(x), C.c_int(_dtype_code(x)), C.c_int(flags),
                               C.c_int64(n_units), C.c_int64(n_param_sets), _ptr(pos0), C.c_int32(n_new),
                               C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(w_enc), _ptr(mean_rot),
                               _ptr(widths), _ptr(cache), _ptr(unit_offset), C.c_int32(capacity_tokens),
-                              _ptr(status_word), _stream())
+                              _ptr(tile_table), C.c_int64(table_stride), _ptr(status_word), _stream())
     _check(rc, "spectra_encode")
 
 
 def decode(cfg, side, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec, mean_rot, widths, out,
-           yhat_out, stride_unit, stride_token, status_word=None):
+           yhat_out, stride_unit, stride_token, status_word=None, tile_table=None, table_stride=0):
     out_code = _dtype_code(out) if out is not None else F32
     rc = lib().spectra_decode(C.byref(cfg), C.c_int(side), _ptr(cache), _ptr(unit_offset), C.c_int64(n_units),
                               C.c_int64(n_param_sets), _ptr(n_tokens), C.c_int32(max_tokens), _ptr(w_dec),
                               _ptr(mean_rot), _ptr(widths), _ptr(out), C.c_int(out_code), _ptr(yhat_out),
-                              C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(status_word), _stream())
+                              C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(tile_table), C.c_int64(table_stride),
+                              _ptr(status_word), _stream())
     _check(rc, "spectra_decode")
 
 
 def decode_attention(cfg, q, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k, cache_v,
                      unit_offset_v, n_param_sets, w_dec_k, mean_rot_k, widths_k, w_dec_v, mean_rot_v, widths_v,
-                     softmax_scale, out, lse, workspace, status_word=None, widths_k_host=None, widths_v_host=None):
+                     softmax_scale, out, lse, workspace, status_word=None, widths_k_host=None, widths_v_host=None,
+                     tile_table_k=None, tile_table_v=None, table_stride=0):
     """widths_*_host: optional numpy uint8 arrays [n_param_sets, 128] (host copies of the widths); they select the
-    tensor-core kernel."""
+    tensor-core kernel.  tile_table_*: device int32 [n_units, table_stride] page indices of paged caches."""
     wkh = wvh = C.c_void_p(0)
     if widths_k_host is not None:
         assert widths_k_host.dtype.name == "uint8" and widths_k_host.flags.c_contiguous
@@ -205,14 +208,15 @@ def decode_attention(cfg, q, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len,
         _ptr(seq_len), C.c_int32(max_seq_len), _ptr(cache_k), _ptr(unit_offset_k), _ptr(cache_v),
         _ptr(unit_offset_v), C.c_int64(n_param_sets), _ptr(w_dec_k), _ptr(mean_rot_k), _ptr(widths_k), _ptr(w_dec_v),
         _ptr(mean_rot_v), _ptr(widths_v), wkh, wvh, C.c_float(softmax_scale), _ptr(out), C.c_int(_dtype_code(out)), _ptr(lse),
-        _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()), _ptr(status_word), _stream())
+        _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()), _ptr(tile_table_k),
+        _ptr(tile_table_v), C.c_int64(table_stride), _ptr(status_word), _stream())
     _check(rc, "spectra_decode_attention")
 
 
 def decode_step(cfg, q, new_k, new_v, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k,
                 cache_v, unit_offset_v, n_param_sets, w_enc_k, w_dec_k, mean_rot_k, widths_k, w_enc_v, w_dec_v,
                 mean_rot_v, widths_v, softmax_scale, out, lse, workspace, status_word=None, widths_k_host=None,
-                widths_v_host=None):
+                widths_v_host=None, tile_table_k=None, tile_table_v=None, table_stride=0):
     """One decode step of a layer: appends new_k / new_v ([batch * n_kv_heads, 128], one vector per unit) at
     position seq_len - 1 and attends over seq_len tokens (seq_len already counts the new token)."""
     wkh = wvh = C.c_void_p(0)
@@ -229,5 +233,6 @@ def decode_step(cfg, q, new_k, new_v, batch, n_kv_heads, n_q_heads, seq_len, max
         _ptr(cache_k), _ptr(unit_offset_k), _ptr(cache_v), _ptr(unit_offset_v), C.c_int64(n_param_sets),
         _ptr(w_enc_k), _ptr(w_dec_k), _ptr(mean_rot_k), _ptr(widths_k), _ptr(w_enc_v), _ptr(w_dec_v), _ptr(mean_rot_v),
         _ptr(widths_v), wkh, wvh, C.c_float(softmax_scale), _ptr(out), C.c_int(_dtype_code(out)), _ptr(lse),
-        _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()), _ptr(status_word), _stream())
+        _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()), _ptr(tile_table_k),
+        _ptr(tile_table_v), C.c_int64(table_stride), _ptr(status_word), _stream())
     _check(rc, "spectra_decode_step")

@@ -72,13 +72,18 @@ WidthFacts width_facts(const uint8_t* wk, const uint8_t* wv, int64_t n_sets) {
   return F;
 }
 
-template <int Q8, int Q4, int Q2, int Q1>
-int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {
-  if (cudaFuncSetAttribute(attention_mma_kernel<Q8, Q4, Q2, Q1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <int Q8, int Q4, int Q2, int Q1, bool PAGED>
+int launch_fast_main_as(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {
+  if (cudaFuncSetAttribute(attention_mma_kernel<Q8, Q4, Q2, Q1, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem) != cudaSuccess)
     return SPECTRA_CUDA_ERROR;
-  attention_mma_kernel<Q8, Q4, Q2, Q1><<<grid, kFastWarps * 32, smem, st>>>(a, f);
+  attention_mma_kernel<Q8, Q4, Q2, Q1, PAGED><<<grid, kFastWarps * 32, smem, st>>>(a, f);
   return launch_status();
+}
+template <int Q8, int Q4, int Q2, int Q1>
+int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {
+  return a.map_k.table ? launch_fast_main_as<Q8, Q4, Q2, Q1, true>(a, f, grid, smem, st)
+                       : launch_fast_main_as<Q8, Q4, Q2, Q1, false>(a, f, grid, smem, st);
 }
 
 // Quota tuples (V blocks of 16 strips per class 8, 4, 2, 1) the main kernel is built for, smallest first.
@@ -149,7 +154,8 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
                    const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
                    const uint8_t* widths_k_host, const uint8_t* widths_v_host, float softmax_scale, void* out,
                    int out_dtype, float* lse, void* workspace, size_t workspace_bytes, int32_t* status_word,
-                   void* stream, const StepAppend* app) {
+                   void* stream, const StepAppend* app, const int32_t* tile_table_k, const int32_t* tile_table_v,
+                   int64_t table_stride) {
   int rc = check_config(cfg);
   if (rc) return rc;
   if (batch < 0 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || max_seq_len < 0 || n_param_sets < 1)
@@ -164,6 +170,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
     return SPECTRA_INVALID_ARG;
   if (lse && !mean_rot_k) return SPECTRA_INVALID_ARG;
   if ((widths_k_host == nullptr) != (widths_v_host == nullptr)) return SPECTRA_INVALID_ARG;
+  if ((tile_table_k == nullptr) != (tile_table_v == nullptr) || table_stride < 0) return SPECTRA_INVALID_ARG;
   // the kernels read the parameter matrices, the caches and the workspace with 16-byte accesses and bulk copies
   if ((((uintptr_t)w_dec_k | (uintptr_t)w_dec_v | (uintptr_t)cache_k | (uintptr_t)cache_v | (uintptr_t)workspace) & 15) != 0)
     return SPECTRA_INVALID_ARG;
@@ -184,6 +191,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
   a.n_splits = generic_splits((int)n_units, max_seq_len);
   a.status = status_word;
   a.max_seq_len = max_seq_len;
+  a.map_k = TileMap{tile_table_k, table_stride}; a.map_v = TileMap{tile_table_v, table_stride};
   cudaStream_t st = (cudaStream_t)stream;
 
   // ---- tensor-core path: scale group 64, host copy of the widths available; a GQA group of more than 4 query
@@ -219,10 +227,10 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       if (app) {
         AppendArgs ak{app->new_k, app->x_dtype, 0, SPECTRA_SIDE_K, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
                       app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, status_word, seq_len, n_kv_heads,
-                      max_seq_len};
+                      max_seq_len, a.map_k};
         AppendArgs av{app->new_v, app->x_dtype, 0, SPECTRA_SIDE_V, cfg->scale_group, n_param_sets, nullptr, 1, kD, kD,
                       app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, status_word, seq_len, n_kv_heads,
-                      max_seq_len};
+                      max_seq_len, a.map_v};
         decode_step_front_kernel<<<(unsigned)(n_vunits + 1 + 2 * n_units), kPrepThreads, kPrepDynSmem, st>>>(
             a, f, ak, av, (int)n_units);
       } else {
@@ -268,10 +276,12 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
     int32_t* pos = reinterpret_cast<int32_t*>(workspace);
     step_positions_kernel<<<(unsigned)((n_units + 255) / 256), 256, 0, st>>>(seq_len, n_kv_heads, (int)n_units, pos);
     rc = spectra_encode(cfg, SPECTRA_SIDE_K, app->new_k, app->x_dtype, 0, n_units, n_param_sets, pos, 1, kD, kD,
-                        app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, max_seq_len, status_word, stream);
+                        app->w_enc_k, mean_rot_k, widths_k, app->cache_k, unit_offset_k, max_seq_len, tile_table_k, table_stride,
+                        status_word, stream);
     if (rc) return rc;
     rc = spectra_encode(cfg, SPECTRA_SIDE_V, app->new_v, app->x_dtype, 0, n_units, n_param_sets, pos, 1, kD, kD,
-                        app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, max_seq_len, status_word, stream);
+                        app->w_enc_v, mean_rot_v, widths_v, app->cache_v, unit_offset_v, max_seq_len, tile_table_v, table_stride,
+                        status_word, stream);
     if (rc) return rc;
   }
   if (cudaFuncSetAttribute(attention_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -294,11 +304,13 @@ extern "C" int spectra_decode_attention(const spectra_config* cfg, const void* q
                                         const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
                                         const uint8_t* widths_k_host, const uint8_t* widths_v_host,
                                         float softmax_scale, void* out, int out_dtype, float* lse, void* workspace,
-                                        size_t workspace_bytes, int32_t* status_word, void* stream) {
+                                        size_t workspace_bytes, const int32_t* tile_table_k,
+                                        const int32_t* tile_table_v, int64_t table_stride, int32_t* status_word,
+                                        void* stream) {
   return attention_impl(cfg, q, q_dtype, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k,
                         cache_v, unit_offset_v, n_param_sets, w_dec_k, mean_rot_k, widths_k, w_dec_v, mean_rot_v,
                         widths_v, widths_k_host, widths_v_host, softmax_scale, out, out_dtype, lse, workspace,
-                        workspace_bytes, status_word, stream, nullptr);
+                        workspace_bytes, status_word, stream, nullptr, tile_table_k, tile_table_v, table_stride);
 }
 
 extern "C" int spectra_decode_step(const spectra_config* cfg, const void* q, int q_dtype, const void* new_k,
@@ -310,6 +322,7 @@ extern "C" int spectra_decode_step(const spectra_config* cfg, const void* q, int
                                    const float* w_dec_v, const float* mean_rot_v, const uint8_t* widths_v,
                                    const uint8_t* widths_k_host, const uint8_t* widths_v_host, float softmax_scale,
                                    void* out, int out_dtype, float* lse, void* workspace, size_t workspace_bytes,
+                                   const int32_t* tile_table_k, const int32_t* tile_table_v, int64_t table_stride,
                                    int32_t* status_word, void* stream) {
   if (!new_k || !new_v || !w_enc_k || !w_enc_v || !mean_rot_k || !mean_rot_v) return SPECTRA_INVALID_ARG;
   if (x_dtype != SPECTRA_F32 && x_dtype != SPECTRA_BF16) return SPECTRA_INVALID_ARG;
@@ -317,7 +330,7 @@ extern "C" int spectra_decode_step(const spectra_config* cfg, const void* q, int
   return attention_impl(cfg, q, q_dtype, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k,
                         cache_v, unit_offset_v, n_param_sets, w_dec_k, mean_rot_k, widths_k, w_dec_v, mean_rot_v,
                         widths_v, widths_k_host, widths_v_host, softmax_scale, out, out_dtype, lse, workspace,
-                        workspace_bytes, status_word, stream, &app);
+                        workspace_bytes, status_word, stream, &app, tile_table_k, tile_table_v, table_stride);
 }
 
 extern "C" int spectra_attention_path(const spectra_config* cfg, int32_t n_kv_heads, int32_t n_q_heads,

@@ -17,6 +17,7 @@ struct AttnArgs {
   const float* w_dec_k; const float* mean_rot_k; const uint8_t* widths_k;
   const float* w_dec_v; const float* mean_rot_v; const uint8_t* widths_v;
   float scale; void* out; int out_dtype; float* lse; float* partials; int n_splits; int32_t* status;
+  TileMap map_k, map_v;
   int max_seq_len;   // capacity of every sequence's buffers in tokens: a longer seq_len is reported and attends to nothing
 };
 
@@ -114,8 +115,8 @@ __global__ void __launch_bounds__(128) attention_generic_kernel(AttnArgs p) {
   for (int tile = tile_begin; tile < tile_end; tile++) {
     __syncthreads();
     {
-      const uint4* sk = reinterpret_cast<const uint4*>(base_k + (int64_t)tile * TK.tile_bytes);
-      const uint4* sv = reinterpret_cast<const uint4*>(base_v + (int64_t)tile * TV.tile_bytes);
+      const uint4* sk = reinterpret_cast<const uint4*>(base_k + p.map_k.page(u, tile) * TK.tile_bytes);
+      const uint4* sv = reinterpret_cast<const uint4*>(base_v + p.map_v.page(u, tile) * TV.tile_bytes);
       for (int i = tid; i < TK.tile_bytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(S.tile_k)[i] = sk[i];
       for (int i = tid; i < TV.tile_bytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(S.tile_v)[i] = sv[i];
     }

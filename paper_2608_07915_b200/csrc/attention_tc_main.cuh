@@ -265,10 +265,10 @@ __device__ __forceinline__ uint32_t pack_half2_sat(float a, float b) {
 // used, instead of sitting in registers through the whole tile) and the two producer cursors, which only lane 0
 // touches: the next tile to copy is the previous one plus the tile size until the unit's tiles run out.
 struct TileProducer {
-  uint64_t addr;         // global address of the next tile to copy
+  uint64_t base;         // global address of the unit's first tile (contiguous cache) or of its page pool (paged)
   uint32_t tb;           // tile bytes of the unit
   int32_t rem;           // tiles of the unit not yet copied
-  int32_t unit, pad;
+  int32_t unit, t;       // unit of the tensor path, logical index of the next tile to copy
 };
 struct WarpState {
   alignas(16) uint32_t head[20];   // UnitDesc words 0..5 (tbk, tbv, kmeta[2], vmeta[2]), two spare words, then words
@@ -303,7 +303,7 @@ __device__ __forceinline__ void fold_group(const unsigned char* meta, float qlo,
   }
 }
 
-template <int Q8, int Q4, int Q2, int Q1>
+template <int Q8, int Q4, int Q2, int Q1, bool PAGED>
 __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma_kernel(AttnArgs p, FastArgs f) {
   constexpr int NACC = Q8 + Q4 + Q2 + Q1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -328,6 +328,13 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
   int cu = start.x, ct = start.y, cnt = start.z;       // consumer: unit, tile, tiles of the unit
   // Copies are started by lane 0, whose cursors live in shared memory; every lane keeps the same counts of tiles
   // whose K / V copy has been started.  A unit's tiles are contiguous: its next tile is one tile size further.
+  // (lane 0 keeps the page of the next tile in a register, looked up one copy ahead, so that a paged cache costs
+  // no dependent global read at the time a copy is started)
+  int page_k = 0, page_v = 0;
+  auto page_of = [&](const TileProducer& q, int side) {
+    if constexpr (!PAGED) return q.t;
+    else return (int)(side ? p.map_v : p.map_k).page(q.unit / f.npass, q.t);
+  };
   auto next_unit = [&](TileProducer& q, int side) {    // the unit's tiles are used up: move to the next unit with tiles
     int u = q.unit + 1, n = 0;
     while (u < f.n_units) {
@@ -336,39 +343,35 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
       u++;
     }
     const UnitDesc& d = f.desc[min(u, f.n_units - 1)];
-    q.unit = u; q.rem = n;
+    q.unit = u; q.rem = n; q.t = 0;
     q.tb = side ? d.tbv : d.tbk;
-    q.addr = (uint64_t)(side ? p.cache_v + d.src_v : p.cache_k + d.src_k);
+    q.base = (uint64_t)(side ? p.cache_v + d.src_v : p.cache_k + d.src_k);
   };
   auto start_k = [&](int slot) {
-    if (ws.k.rem == 0) next_unit(ws.k, 0);
+    if (ws.k.rem == 0) { next_unit(ws.k, 0); page_k = page_of(ws.k, 0); }
     const uint32_t tb = ws.k.tb;
-    const uint64_t a = ws.k.addr;
     mbar_expect_tx(bars + 8 * slot, tb);
-    bulk_load(smem_u32(ring_k + slot * f.slot_k), (const void*)a, tb, bars + 8 * slot
-              , l2_evict_first_policy()
-              );
-    ws.k.addr = a + tb; ws.k.rem--;
+    bulk_load(smem_u32(ring_k + slot * f.slot_k), (const void*)(ws.k.base + (uint64_t)page_k * tb), tb, bars + 8 * slot,
+              l2_evict_first_policy());
+    ws.k.t++;
+    if (--ws.k.rem > 0) page_k = page_of(ws.k, 0);
   };
   auto start_v = [&](int slot) {
-    if (ws.v.rem == 0) next_unit(ws.v, 1);
+    if (ws.v.rem == 0) { next_unit(ws.v, 1); page_v = page_of(ws.v, 1); }
     const uint32_t tb = ws.v.tb;
-    const uint64_t a = ws.v.addr;
     mbar_expect_tx(bars + 8 * (4 + slot), tb);
-    bulk_load(smem_u32(ring_v + slot * f.slot_v), (const void*)a, tb, bars + 8 * (4 + slot)
-              , l2_evict_first_policy()
-              );
-    ws.v.addr = a + tb; ws.v.rem--;
+    bulk_load(smem_u32(ring_v + slot * f.slot_v), (const void*)(ws.v.base + (uint64_t)page_v * tb), tb,
+              bars + 8 * (4 + slot), l2_evict_first_policy());
+    ws.v.t++;
+    if (--ws.v.rem > 0) page_v = page_of(ws.v, 1);
   };
   int issued_k = min(D, count), issued_v = issued_k;
   int fill_k = issued_k % D, fill_v = fill_k;           // slots the next K / V copies go to
   if (lane == 0) {
     const UnitDesc& d = f.desc[cu];
-    const uint32_t tbk = d.tbk, tbv = d.tbv;
-    ws.k.unit = cu; ws.k.rem = cnt - ct; ws.k.tb = tbk;
-    ws.k.addr = (uint64_t)(p.cache_k + d.src_k + (int64_t)ct * tbk);
-    ws.v.unit = cu; ws.v.rem = cnt - ct; ws.v.tb = tbv;
-    ws.v.addr = (uint64_t)(p.cache_v + d.src_v + (int64_t)ct * tbv);
+    ws.k.unit = cu; ws.k.rem = cnt - ct; ws.k.t = ct; ws.k.tb = d.tbk; ws.k.base = (uint64_t)(p.cache_k + d.src_k);
+    ws.v.unit = cu; ws.v.rem = cnt - ct; ws.v.t = ct; ws.v.tb = d.tbv; ws.v.base = (uint64_t)(p.cache_v + d.src_v);
+    page_k = page_of(ws.k, 0); page_v = page_of(ws.v, 1);
     for (int j = 0; j < issued_k; j++) { start_k(j); start_v(j); }
   }
 
@@ -472,7 +475,8 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
       for (int r = 1; r < 8; r++)
         rm = __hmax2(rm, __hmax2(*reinterpret_cast<const __half2*>(&vr0[r]), *reinterpret_cast<const __half2*>(&vr1[r])));
       const float rmax = fmaxf(__low2float(rm), __high2float(rm));          // ranges are non-negative
-      const int e = (int)((__float_as_uint(rmax) >> 23) & 0xff) - 126;      // rmax < 2^e
+      // rmax < 2^e; ranges below fp16's normal range (or none at all) count as 2^-14, which keeps 2^(s - m_ref) finite
+      const int e = max((int)((__float_as_uint(rmax) >> 23) & 0xff) - 126, -14);
       float need = fmaf(mx, kscale, (float)(e - 13));                       // kscale is a positive power of two
       need = fmaxf(need, __shfl_xor_sync(0xffffffffu, need, 4));
       need = fmaxf(need, __shfl_xor_sync(0xffffffffu, need, 8));

@@ -55,7 +55,7 @@ struct EncodeArgs {
   const void* x; int x_dtype; int flags; int side; int scale_group;
   int64_t n_param_sets; const int32_t* pos0; int32_t n_new; int32_t capacity; int64_t stride_unit, stride_token;
   const float* w_enc; const float* mean_rot; const uint8_t* widths;
-  uint8_t* cache; const int64_t* unit_offset; int32_t* status;
+  uint8_t* cache; const int64_t* unit_offset; int32_t* status; TileMap map;
 };
 
 __global__ void __launch_bounds__(128, 1) encode_kernel(EncodeArgs p) {
@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(128, 1) encode_kernel(EncodeArgs p) {
   __syncthreads();
 
   // pack: one half-word of the payload at a time, in storage order
-  uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
+  uint8_t* tile_ptr = p.cache + p.unit_offset[u] + p.map.page(u, tile) * T.tile_bytes;
   const int payload = T.class_off[4];
   if (slot_lo == 0 && slot_hi == kTile) pack_full_tile(T, p.side, S.codes, kLdC, tile_ptr, tid, blockDim.x);
   else
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
 
   build_strip_table(S.tab, p.widths + (int64_t)ps * kD, p.scale_group);
   const StripTable& T = S.tab;
-  const uint8_t* tile_ptr = p.cache + p.unit_offset[u] + (int64_t)tile * T.tile_bytes;
+  const uint8_t* tile_ptr = p.cache + p.unit_offset[u] + p.map.page(u, tile) * T.tile_bytes;
   S.bias[tid] = p.mean_rot[(int64_t)ps * kD + tid];
 
   // unpack: thread t gathers the fields of token slot t
@@ -272,12 +272,14 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
                               int64_t n_units, int64_t n_param_sets, const int32_t* pos0, int32_t n_new,
                               int64_t stride_unit, int64_t stride_token, const float* w_enc, const float* mean_rot,
                               const uint8_t* widths, uint8_t* cache, const int64_t* unit_offset,
-                              int32_t capacity_tokens, int32_t* status_word, void* stream) {
+                              int32_t capacity_tokens, const int32_t* tile_table, int64_t table_stride,
+                              int32_t* status_word, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   if ((side != SPECTRA_SIDE_K && side != SPECTRA_SIDE_V) || n_units < 0 || n_new < 0 || n_param_sets < 1 ||
-      capacity_tokens < 0)
+      capacity_tokens < 0 || table_stride < 0)
     return SPECTRA_INVALID_ARG;
+  const TileMap map{tile_table, table_stride};
   if (x_dtype != SPECTRA_F32 && x_dtype != SPECTRA_BF16) return SPECTRA_INVALID_ARG;
   if (flags & ~SPECTRA_ROTATED_INPUT) return SPECTRA_INVALID_ARG;
   if ((flags & SPECTRA_ROTATED_INPUT) && x_dtype != SPECTRA_F32) return SPECTRA_INVALID_ARG;
@@ -288,7 +290,7 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   if (n_new <= kAppendMaxTokens) {   // decode-step appends: one light CTA per unit-side
     AppendArgs ap{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, stride_unit, stride_token,
-                  w_enc, mean_rot, widths, cache, unit_offset, status_word, nullptr, 1, capacity_tokens};
+                  w_enc, mean_rot, widths, cache, unit_offset, status_word, nullptr, 1, capacity_tokens, map};
     if (cudaFuncSetAttribute(encode_append_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAppendDynSmem) !=
         cudaSuccess)
       return SPECTRA_CUDA_ERROR;
@@ -299,7 +301,7 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
       stride_token % 8 == 0 && stride_unit % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
     // bf16 bulk encode: rotation on the tensor cores
     EncodeTcArgs ta{reinterpret_cast<const __nv_bfloat16*>(x), side, n_param_sets, pos0, n_new, capacity_tokens, stride_unit,
-                    stride_token, w_enc, mean_rot, widths, cache, unit_offset, status_word};
+                    stride_token, w_enc, mean_rot, widths, cache, unit_offset, status_word, map};
     // rotation on the 5th-generation tensor cores (accumulator tiles in tensor memory); the token tiles arrive by
     // TMA: a 3-D map over x [unit][token][channel] whose box is 8 channels x 128 tokens
     CUtensorMap xmap;
@@ -319,7 +321,7 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
     }
   }
   EncodeArgs a{x, x_dtype, flags, side, cfg->scale_group, n_param_sets, pos0, n_new, capacity_tokens, stride_unit, stride_token,
-               w_enc, mean_rot, widths, cache, unit_offset, status_word};
+               w_enc, mean_rot, widths, cache, unit_offset, status_word, map};
   if (cudaFuncSetAttribute(encode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CodecSmem)) !=
       cudaSuccess)
     return SPECTRA_CUDA_ERROR;
@@ -332,10 +334,11 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
                               int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
                               const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out,
                               int out_dtype, float* yhat_out, int64_t stride_unit, int64_t stride_token,
-                              int32_t* status_word, void* stream) {
+                              const int32_t* tile_table, int64_t table_stride, int32_t* status_word, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
-  if ((side != SPECTRA_SIDE_K && side != SPECTRA_SIDE_V) || n_units < 0 || max_tokens < 0 || n_param_sets < 1)
+  if ((side != SPECTRA_SIDE_K && side != SPECTRA_SIDE_V) || n_units < 0 || max_tokens < 0 || n_param_sets < 1 ||
+      table_stride < 0)
     return SPECTRA_INVALID_ARG;
   if (out_dtype != SPECTRA_F32 && out_dtype != SPECTRA_BF16) return SPECTRA_INVALID_ARG;
   if (n_units == 0 || max_tokens == 0) return SPECTRA_OK;
@@ -345,7 +348,7 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
   if (out && !w_dec) return SPECTRA_INVALID_ARG;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
-               out_dtype, yhat_out, stride_unit, stride_token, status_word};
+               out_dtype, yhat_out, stride_unit, stride_token, status_word, TileMap{tile_table, table_stride}};
   if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05), persistent grid
     const size_t dec_smem = sizeof(DecodeTcSmem) + 128;
     if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem) !=

@@ -298,6 +298,14 @@ __device__ inline void unpack_tile(const StripTable& T, int side, const uint8_t*
   }
 }
 
+// Where the tiles of a unit-side live.  Contiguous caches (table == NULL): tile t of unit u starts t tile sizes after
+// the unit's offset.  Paged caches: the unit's offset is the base of a pool of tile-sized pages and logical tile t
+// sits in page table[u * stride + t] of that pool (the append-only streaming cache of Sec. 3.3 grows a page at a time).
+struct TileMap {
+  const int32_t* table; int64_t stride;
+  __device__ __forceinline__ int64_t page(int64_t u, int t) const { return table ? (int64_t)table[u * stride + t] : (int64_t)t; }
+};
+
 // Asks the L2 for the 128-byte line that holds p; a later load then pays the L2's latency instead of the DRAM's.
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 

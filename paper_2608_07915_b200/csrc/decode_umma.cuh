@@ -35,7 +35,7 @@ struct DecodeArgs {
   const uint8_t* cache; const int64_t* unit_offset; int side; int scale_group; int64_t n_param_sets;
   const int32_t* n_tokens; const float* w_dec; const float* mean_rot; const uint8_t* widths;
   void* out; int out_dtype; float* yhat_out; int64_t stride_unit, stride_token;
-  int32_t* status;
+  int32_t* status; TileMap map;
 };
 
 struct DecodeTcSmem {
@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
           asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(tile_bytes) : "memory");
           asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                            um_smem_u32(S.half[h].raw)),
-                       "l"(unit_ptr + (int64_t)(ga + tt) * tile_bytes), "r"(tile_bytes), "r"(bar)
+                       "l"(unit_ptr + p.map.page(u, ga + tt) * tile_bytes), "r"(tile_bytes), "r"(bar)
                        : "memory");
         };
         if (staged) {
@@ -203,7 +203,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
         const int tile_pos = tile * kTile;
         const int n_here = min(n - tile_pos, kTile);
         const bool live = t < n_here;
-        const uint8_t* tile_ptr = unit_ptr + (int64_t)tile * tile_bytes;
+        const uint8_t* tile_ptr = unit_ptr + p.map.page(u, tile) * tile_bytes;
         if (staged) {
           ok = um_wait(um_smem_u32(&S.raw_full[hf]), (uint32_t)(i & 1));
           if (!ok) { status |= SPECTRA_STATUS_WAIT_TIMEOUT; break; }

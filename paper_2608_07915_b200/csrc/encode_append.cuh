@@ -17,6 +17,7 @@ struct AppendArgs {
   uint8_t* cache; const int64_t* unit_offset; int32_t* status;
   const int32_t* seq_len; int n_kv;      // with pos0 == NULL: the token goes to position seq_len[u / n_kv] - 1
   int32_t capacity;                      // tokens a unit-side's buffer holds (0: not checked)
+  TileMap map;
 };
 
 // Bounded wait for phase 0 of an mbarrier (each poll blocks for a bounded hardware interval).
@@ -138,7 +139,7 @@ __device__ inline void encode_append_body(const AppendArgs& p, int u, unsigned c
   for (int t = 0; t < n_new; t++) {
     const int pos = pos_first + t;
     const int slot = pos & (kTile - 1);
-    uint8_t* tile = base + (int64_t)(pos / kTile) * tile_bytes;
+    uint8_t* tile = base + p.map.page(u, pos / kTile) * tile_bytes;
     // the half-words the new fields go into (a tile's first token finds them cleared)
     unsigned old[4] = {0u, 0u, 0u, 0u};
     if (slot != 0) {

@@ -60,21 +60,23 @@ def test_bad_arguments_are_rejected_before_any_launch(lib):
     assert lib.spectra_fit_workspace_bytes(C.byref(bad), C.c_int64(1)) == 0
     bad = sp.default_config(b_max=9)
     assert lib.spectra_encode(C.byref(bad), 0, null, 0, 0, C.c_int64(1), C.c_int64(1), null, 1, C.c_int64(0),
-                              C.c_int64(0), null, null, null, null, null, 0, null, null) == sp.INVALID_ARG
+                              C.c_int64(0), null, null, null, null, null, 0, null, C.c_int64(0), null,
+                              null) == sp.INVALID_ARG
     # rotated input must be fp32; unknown flags; bad side
     args = (C.c_int64(1), C.c_int64(1), null, 1, C.c_int64(0), C.c_int64(0), null, null, null, null, null, 0, null,
-            null)
+            C.c_int64(0), null, null)
     assert lib.spectra_encode(C.byref(cfg), 0, null, sp.BF16, sp.ROTATED_INPUT, *args) == sp.INVALID_ARG
     assert lib.spectra_encode(C.byref(cfg), 0, null, sp.F32, 8, *args) == sp.INVALID_ARG
     assert lib.spectra_encode(C.byref(cfg), 2, null, sp.F32, 0, *args) == sp.INVALID_ARG
     assert lib.spectra_encode(C.byref(cfg), 0, null, sp.F32, 0, *args) == sp.INVALID_ARG     # null pointers
-    neg = (C.c_int64(1), C.c_int64(1), null, 1, C.c_int64(0), C.c_int64(0), null, null, null, null, null, -5, null, null)
+    neg = (C.c_int64(1), C.c_int64(1), null, 1, C.c_int64(0), C.c_int64(0), null, null, null, null, null, -5, null,
+           C.c_int64(0), null, null)
     assert lib.spectra_encode(C.byref(cfg), 0, null, sp.F32, 0, *neg) == sp.INVALID_ARG      # negative capacity
     # attention: query heads must be a multiple of kv heads; group size above 8 unsupported
     def attn(n_kv, n_q):
         return lib.spectra_decode_attention(C.byref(cfg), null, 0, 1, n_kv, n_q, null, 128, null, null, null, null,
                                             C.c_int64(1), null, null, null, null, null, null, C.c_float(0), null, 0,
-                                            null, null, C.c_size_t(0), null, null)
+                                            null, null, C.c_size_t(0), null, null, C.c_int64(0), null, null)
     assert attn(3, 8) == sp.INVALID_ARG
     assert attn(1, 16) == sp.UNSUPPORTED
     assert attn(2, 8) == sp.INVALID_ARG                                                      # null pointers
@@ -89,16 +91,18 @@ def test_misaligned_buffers_are_refused_on_the_host(lib):
     ok = 0x10000
     # spectra_encode: cache one byte off
     assert lib.spectra_encode(C.byref(cfg), 0, p(ok), sp.F32, 0, C.c_int64(1), C.c_int64(1), p(ok), 1, C.c_int64(128),
-                              C.c_int64(128), p(ok), p(ok), p(ok), p(ok + 1), p(ok), 0, null, null) == sp.INVALID_ARG
+                              C.c_int64(128), p(ok), p(ok), p(ok), p(ok + 1), p(ok), 0, null, C.c_int64(0), null,
+                              null) == sp.INVALID_ARG
     # spectra_decode: odd cache address
     assert lib.spectra_decode(C.byref(cfg), 0, p(ok + 1), p(ok), C.c_int64(1), C.c_int64(1), p(ok), 128, p(ok), p(ok),
-                              p(ok), p(ok), sp.F32, null, C.c_int64(128 * 128), C.c_int64(128), null,
-                              null) == sp.INVALID_ARG
+                              p(ok), p(ok), sp.F32, null, C.c_int64(128 * 128), C.c_int64(128), null, C.c_int64(0),
+                              null, null) == sp.INVALID_ARG
     # spectra_decode_attention: W_dec,K four bytes off
     big = C.c_size_t(1 << 30)
     assert lib.spectra_decode_attention(C.byref(cfg), p(ok), sp.F32, 1, 1, 4, p(ok), 128, p(ok), p(ok), p(ok), p(ok),
                                         C.c_int64(1), p(ok + 4), null, p(ok), p(ok), p(ok), p(ok), null, null,
-                                        C.c_float(0), p(ok), sp.F32, null, p(ok), big, null, null) == sp.INVALID_ARG
+                                        C.c_float(0), p(ok), sp.F32, null, p(ok), big, null, null, C.c_int64(0), null,
+                                        null) == sp.INVALID_ARG
 
 
 def test_cache_bytes_and_attention_path(lib):

@@ -812,3 +812,122 @@ def test_attention_with_value_outlier_tokens_that_carry_the_probability_mass(sp)
     assert np.abs(ref_b[0, 0]).max() > 5 * np.abs(ref_b[0, 1:]).max()     # head 0 did land on an outlier token
     assert H.rel_err_per_vector(got[0], ref_b[0]) <= TOL and H.rel_err_per_vector(got[0], ref_a[0]) <= TOL
     assert np.abs(lse[0] - lse_b[0]).max() <= 2e-3
+
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+def test_paged_caches_give_the_same_bytes_and_outputs_as_contiguous_ones(sp, dt):
+    """Paged caches (a page table over tile-sized pages of a pool shared by the sequences of a head): bulk encode,
+    appends, reconstruction, attention on both kernels and the fused step must produce, page by page, the bytes of
+    the contiguous layout, and the same outputs; the attention is also compared with the oracle on the gathered
+    bytes."""
+    wl = si.WORKLOADS["tiny"]
+    cfg = sp.default_config()
+    tdt = torch.float32 if dt == "f32" else torch.bfloat16
+    n_seq, n0, cap = 2, 600, 768                       # 600 cached tokens (4 full tiles + 88), room for 6 tiles
+    n_tiles = cap // 128
+    rng = np.random.default_rng(17)
+    perm = rng.permutation(2 * n_tiles + 3)            # pool of 15 pages, 12 used, interleaved between the sequences
+    table = np.stack([perm[:n_tiles], perm[n_tiles:2 * n_tiles]]).astype(np.int32)
+    tab_dev = H.to_dev(table)
+    zero_off = torch.zeros(n_seq, dtype=torch.int64, device="cuda")     # both sequences share the head's pool
+    S = {}
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        X = np.stack([si.draw_unit(wl, 0, 0, side, s, n_tokens=n0 + 2) for s in range(n_seq)])
+        if dt == "bf16":
+            X = si.to_bf16_f32(X)
+        params = H.fit_params([X[0, :512]], 8.0)
+        tb = int(params.tile_bytes[0])
+        off_c = np.array([0, n_tiles * tb], np.int64)
+        S[name] = dict(X=X, params=params, tb=tb, off=off_c, dp=H.dev_params(params),
+                       cont=torch.zeros(2 * n_tiles * tb, dtype=torch.uint8, device="cuda"),
+                       pool=torch.full((len(perm) * tb,), 0xEE, dtype=torch.uint8, device="cuda"))
+
+    def gathered(name):
+        c = S[name]
+        pool = c["pool"].cpu().numpy().reshape(len(perm), c["tb"])
+        return np.concatenate([pool[table[s, t]] for s in range(n_seq) for t in range(n_tiles)])
+
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    pos = torch.zeros(n_seq, dtype=torch.int32, device="cuda")
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        c = S[name]
+        x = H.to_dev(c["X"][:, :n0]).to(tdt)
+        for cache, off, kw in ((c["cont"], H.to_dev(c["off"]), {}),
+                               (c["pool"], zero_off, dict(tile_table=tab_dev, table_stride=n_tiles))):
+            sp.encode(cfg, side, x, 0, n_seq, 1, pos, n0, x.stride(0), 128, c["dp"]["w_enc"], c["dp"]["m_rot"],
+                      c["dp"]["widths"], cache, off, status, capacity_tokens=cap, **kw)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for name in ("k", "v"):
+        c = S[name]
+        g = gathered(name).reshape(n_seq, n_tiles, c["tb"])
+        r = c["cont"].cpu().numpy().reshape(n_seq, n_tiles, c["tb"])
+        assert np.array_equal(g[:, :5], r[:, :5])                       # the five tiles that hold tokens
+        pool = c["pool"].cpu().numpy().reshape(len(perm), c["tb"])
+        for pg in perm[2 * n_tiles:]:
+            assert (pool[pg] == 0xEE).all()                              # pages outside the tables stay untouched
+    # reconstruction
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        c = S[name]
+        outs = []
+        for cache, off, kw in ((c["cont"], H.to_dev(c["off"]), {}),
+                               (c["pool"], zero_off, dict(tile_table=tab_dev, table_stride=n_tiles))):
+            o = torch.zeros((n_seq, n0, 128), dtype=torch.float32, device="cuda")
+            y = torch.zeros((n_seq, n0, 128), dtype=torch.float32, device="cuda")
+            sp.decode(cfg, side, cache, off, n_seq, 1, torch.full((n_seq,), n0, dtype=torch.int32, device="cuda"), n0,
+                      c["dp"]["w_dec"], c["dp"]["m_rot"], c["dp"]["widths"], o, y, n0 * 128, 128, status, **kw)
+            torch.cuda.synchronize()
+            outs.append((o, y))
+        assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    # attention on both kernels, then two fused steps (the second crosses nothing; the tail tile grows in place)
+    k, v = S["k"], S["v"]
+    q = H.to_dev(np.stack([si.draw_queries(wl, 0, s) for s in range(n_seq)]))
+    ws = torch.zeros(sp.attention_workspace_bytes(cfg, n_seq, 1, 4, cap), dtype=torch.uint8, device="cuda")
+    seq = torch.full((n_seq,), n0, dtype=torch.int32, device="cuda")
+    for hw in (True, False):
+        res = []
+        for paged in (False, True):
+            o = torch.zeros((n_seq, 4, 128), dtype=torch.float32, device="cuda")
+            l = torch.zeros((n_seq, 4), dtype=torch.float32, device="cuda")
+            kw = dict(tile_table_k=tab_dev, tile_table_v=tab_dev, table_stride=n_tiles) if paged else {}
+            sp.decode_attention(cfg, q, n_seq, 1, 4, seq, cap, k["pool"] if paged else k["cont"],
+                                zero_off if paged else H.to_dev(k["off"]), v["pool"] if paged else v["cont"],
+                                zero_off if paged else H.to_dev(v["off"]), 1, k["dp"]["w_dec"], k["dp"]["m_rot"],
+                                k["dp"]["widths"], v["dp"]["w_dec"], v["dp"]["m_rot"], v["dp"]["widths"], 0.0, o, l, ws,
+                                status, k["params"].widths if hw else None, v["params"].widths if hw else None, **kw)
+            torch.cuda.synchronize()
+            res.append((o.cpu().numpy(), l.cpu().numpy()))
+        if hw:
+            assert np.array_equal(res[0][0], res[1][0]) and np.array_equal(res[0][1], res[1][1])
+        else:
+            assert np.allclose(res[0][0], res[1][0], rtol=1e-5, atol=1e-6)
+        gk, gv = gathered("k"), gathered("v")
+        ref, lse = oc.attention_units("B", q.cpu().numpy().astype(np.float64).reshape(n_seq, 4, 128), [n0] * n_seq, gk,
+                                      k["off"], [k["tb"]] * n_seq, gv, v["off"], [v["tb"]] * n_seq,
+                                      np.repeat(k["params"].w_dec, n_seq, 0), np.repeat(k["params"].m_rot, n_seq, 0),
+                                      np.repeat(k["params"].widths, n_seq, 0), np.repeat(v["params"].w_dec, n_seq, 0),
+                                      np.repeat(v["params"].m_rot, n_seq, 0), np.repeat(v["params"].widths, n_seq, 0),
+                                      64, 1.0 / np.sqrt(128.0))
+        assert H.rel_err_per_vector(res[1][0], ref) <= TOL
+    for step in range(2):
+        seq += 1
+        nk = H.to_dev(k["X"][:, n0 + step]).to(tdt).contiguous()
+        nv = H.to_dev(v["X"][:, n0 + step]).to(tdt).contiguous()
+        res = []
+        for paged in (False, True):
+            o = torch.zeros((n_seq, 4, 128), dtype=torch.float32, device="cuda")
+            kw = dict(tile_table_k=tab_dev, tile_table_v=tab_dev, table_stride=n_tiles) if paged else {}
+            sp.decode_step(cfg, q, nk, nv, n_seq, 1, 4, seq, cap, k["pool"] if paged else k["cont"],
+                           zero_off if paged else H.to_dev(k["off"]), v["pool"] if paged else v["cont"],
+                           zero_off if paged else H.to_dev(v["off"]), 1, k["dp"]["w_enc"], k["dp"]["w_dec"],
+                           k["dp"]["m_rot"], k["dp"]["widths"], v["dp"]["w_enc"], v["dp"]["w_dec"], v["dp"]["m_rot"],
+                           v["dp"]["widths"], 0.0, o, None, ws, status, k["params"].widths, v["params"].widths, **kw)
+            torch.cuda.synchronize()
+            res.append(o.cpu().numpy())
+        assert np.array_equal(res[0], res[1])
+    assert int(status.item()) == 0
+    for name in ("k", "v"):
+        c = S[name]
+        g = gathered(name).reshape(n_seq, n_tiles, c["tb"])
+        r = c["cont"].cpu().numpy().reshape(n_seq, n_tiles, c["tb"])
+        assert np.array_equal(g[:, :5], r[:, :5])
