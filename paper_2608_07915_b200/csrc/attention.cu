@@ -72,31 +72,23 @@ WidthFacts width_facts(const uint8_t* wk, const uint8_t* wv, int64_t n_sets) {
   return F;
 }
 
-template <int Q8, int Q4, int Q2, int Q1, bool PAGED>
+template <bool PAGED>
 int launch_fast_main_as(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {
-  if (cudaFuncSetAttribute(attention_mma_kernel<Q8, Q4, Q2, Q1, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)smem) != cudaSuccess)
+  if (cudaFuncSetAttribute(attention_mma_kernel<PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+      cudaSuccess)
     return SPECTRA_CUDA_ERROR;
-  attention_mma_kernel<Q8, Q4, Q2, Q1, PAGED><<<grid, kFastWarps * 32, smem, st>>>(a, f);
+  attention_mma_kernel<PAGED><<<grid, kFastWarps * 32, smem, st>>>(a, f);
   return launch_status();
 }
-template <int Q8, int Q4, int Q2, int Q1>
 int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {
-  return a.map_k.table ? launch_fast_main_as<Q8, Q4, Q2, Q1, true>(a, f, grid, smem, st)
-                       : launch_fast_main_as<Q8, Q4, Q2, Q1, false>(a, f, grid, smem, st);
+  return a.map_k.table ? launch_fast_main_as<true>(a, f, grid, smem, st) : launch_fast_main_as<false>(a, f, grid, smem, st);
 }
 
-// Quota tuples (V blocks of 16 strips per class 8, 4, 2, 1) the main kernel is built for, smallest first.
-// They cover the width profiles that reverse water-filling produces at 4x, 6x, 8x, 10x, 12x and 16x on decaying
-// spectra; anything else runs on the CUDA-core kernel.
-constexpr int kQuotas[][4] = {{0, 1, 8, 2}, {0, 1, 3, 6}, {0, 1, 6, 4}, {0, 8, 2, 2}, {0, 7, 3, 4}, {0, 1, 2, 7}, {0, 1, 8, 5}};
-constexpr int kNumQuotas = sizeof(kQuotas) / sizeof(kQuotas[0]);
-
-int pick_quota(const int (&vb)[4]);
+constexpr int kMaxVBlocks = kAccColumns / 4;   // V blocks of 16 strips a warp's share of tensor memory holds
 
 // Launch shape of the tensor-core path for a set of widths: shared-memory slot sizes, CTAs per SM, ring depth and
-// the kernel variant (quota < 0 or depth < 1: the widths fall outside the built variants).
-struct FastPlan { int slot_k, slot_v, ctas_per_sm, depth, quota; };
+// whether the V accumulators fit their tensor-memory columns (fits false or depth < 1: the CUDA-core kernel runs).
+struct FastPlan { int slot_k, slot_v, ctas_per_sm, depth; bool fits; };
 
 FastPlan plan_fast(const WidthFacts& F) {
   FastPlan P{};
@@ -110,17 +102,8 @@ FastPlan plan_fast(const WidthFacts& F) {
     P.ctas_per_sm--;
   P.depth = (int)(budget / ((size_t)P.ctas_per_sm * kFastWarps * pair));
   if (P.depth > 4) P.depth = 4;
-  P.quota = pick_quota(F.vb);
+  P.fits = F.max_vblocks <= kMaxVBlocks;
   return P;
-}
-
-int pick_quota(const int (&vb)[4]) {
-  for (int i = 0; i < kNumQuotas; i++) {
-    bool fits = true;
-    for (int c = 0; c < 4; c++) fits = fits && vb[c] <= kQuotas[i][c];
-    if (fits) return i;
-  }
-  return -1;
 }
 
 }  // namespace
@@ -204,9 +187,9 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
     const int sms = sm_count();
     if (sms <= 0) return SPECTRA_CUDA_ERROR;
     const FastPlan P = plan_fast(F);
-    const int slot_k = P.slot_k, slot_v = P.slot_v, ctas_per_sm = P.ctas_per_sm, depth = P.depth, quota = P.quota;
+    const int slot_k = P.slot_k, slot_v = P.slot_v, ctas_per_sm = P.ctas_per_sm, depth = P.depth;
     const size_t pair = (size_t)slot_k + slot_v;
-    if (depth >= 1 && quota >= 0) {
+    if (depth >= 1 && P.fits) {
       const int vs_max = (F.max_vstrips + 3) & ~3;     // records are fetched with bulk copies: 16-byte multiples
       FastLayout L = fast_layout(n_vunits, sms * ctas_per_sm * kFastWarps, vs_max);
       if (L.total > workspace_bytes) return SPECTRA_WORKSPACE_TOO_SMALL;
@@ -218,7 +201,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       f.records = reinterpret_cast<float*>(ws + L.rec_off);
       f.total_warps = L.total_warps; f.rec_stride = L.rec_stride; f.vs_max = vs_max;
       f.n_units = (int)n_vunits; f.npass = npass; f.depth = depth; f.slot_k = slot_k; f.slot_v = slot_v;
-      for (int c = 0; c < 4; c++) f.vq[c] = kQuotas[quota][c];
+      f.max_vblocks = kMaxVBlocks;
       if (cudaFuncSetAttribute(decode_step_front_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepDynSmem) !=
               cudaSuccess ||
           cudaFuncSetAttribute(attention_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepDynSmem) !=
@@ -241,15 +224,7 @@ int attention_impl(const spectra_config* cfg, const void* q, int q_dtype, int32_
       // (zero rows of B, unused accumulator rows): the pad keeps those reads inside the CTA's shared memory
       const size_t smem = (size_t)kFastWarps * depth * pair + kFastWarps * 64 + kFastWarps * kWarpStateBytes + 2048;
       const int grid = sms * ctas_per_sm;
-      switch (quota) {
-        case 0: rc = launch_fast_main<0, 1, 8, 2>(a, f, grid, smem, st); break;
-        case 1: rc = launch_fast_main<0, 1, 3, 6>(a, f, grid, smem, st); break;
-        case 2: rc = launch_fast_main<0, 1, 6, 4>(a, f, grid, smem, st); break;
-        case 3: rc = launch_fast_main<0, 8, 2, 2>(a, f, grid, smem, st); break;
-        case 4: rc = launch_fast_main<0, 7, 3, 4>(a, f, grid, smem, st); break;
-        case 5: rc = launch_fast_main<0, 1, 2, 7>(a, f, grid, smem, st); break;
-        default: rc = launch_fast_main<0, 1, 8, 5>(a, f, grid, smem, st); break;
-      }
+      rc = launch_fast_main(a, f, grid, smem, st);
       if (rc) return rc;
       if (cudaFuncSetAttribute(attention_mma_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kCombineDynSmem) != cudaSuccess)
@@ -342,7 +317,7 @@ extern "C" int spectra_attention_path(const spectra_config* cfg, int32_t n_kv_he
   const WidthFacts F = width_facts(widths_k_host, widths_v_host, n_param_sets);
   if (!F.ok) return -1;
   const FastPlan P = plan_fast(F);
-  return P.depth >= 1 && P.quota >= 0 ? SPECTRA_PATH_TENSOR_CORE : SPECTRA_PATH_CUDA_CORE;
+  return P.depth >= 1 && P.fits ? SPECTRA_PATH_TENSOR_CORE : SPECTRA_PATH_CUDA_CORE;
 }
 
 extern "C" size_t spectra_cache_bytes(const spectra_config* cfg, const uint8_t* widths_host, int64_t capacity_tokens) {

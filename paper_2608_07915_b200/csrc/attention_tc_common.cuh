@@ -31,7 +31,7 @@ constexpr int kFastGqa = 4;
 constexpr int kKcMax = 40;       // upper bound of B-table entries of a K tile: 384 strips in 8 (class, group) runs, each
                                  // run rounded up to whole chunks of 16 strips and a group-1 run starting on an even strip
 constexpr int kFastWarps = 4;    // warps per CTA of the main kernel
-constexpr int kFastCtasPerSm = 3; // CTAs of the main kernel per SM its register budget is set for
+constexpr int kFastCtasPerSm = 4; // CTAs of the main kernel per SM its register budget is set for
 constexpr int kRecHead = 4;      // floats of a record's per-head header: m, l, plo0, plo1
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -58,18 +58,18 @@ struct FastArgs {
   int n_units;       // units of the tensor path: (sequence, kv-head, pass); a pass takes up to 4 query heads of the group
   int npass;
   int depth; int slot_k, slot_v;
-  int vq[4];         // V blocks per class the launched main kernel is built for
+  int max_vblocks;   // V blocks of 16 strips whose accumulators fit the main kernel's tensor memory
 };
 
 // What the main kernel relies on for one unit, checked on the device against the widths the kernels actually read
 // (the host sized the shared-memory slots and picked the kernel variant from its own copy of the widths): tiles fit
-// their slots, every V class fits its quota of 16-strip blocks, the B table fits, and both tile streams start on a
+// their slots, the V blocks fit the tensor-memory columns of their accumulators, the B table fits, and both tile streams start on a
 // 16-byte boundary (bulk copies).
 __host__ __device__ inline bool fast_layout_ok(int tile_bytes_k, int tile_bytes_v, const int (&vblocks)[4],
                                                int k_entries, unsigned long long addr_k, unsigned long long addr_v,
-                                               int slot_k, int slot_v, const int (&vq)[4]) {
+                                               int slot_k, int slot_v, int max_vblocks) {
   bool ok = tile_bytes_k <= slot_k && tile_bytes_v <= slot_v && k_entries <= kKcMax;
-  for (int c = 0; c < 4; c++) ok = ok && vblocks[c] <= vq[c];
+  ok = ok && vblocks[0] + vblocks[1] + vblocks[2] + vblocks[3] <= max_vblocks;
   return ok && (addr_k & 15ull) == 0 && (addr_v & 15ull) == 0;
 }
 
@@ -428,7 +428,7 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
 #pragma unroll
   for (int c = 0; c < 4; c++) vblocks[c] = (TV.class_first[c + 1] - TV.class_first[c] + 15) >> 4;
   const unsigned long long addr_k = (unsigned long long)(p.cache_k + p.off_k[u]), addr_v = (unsigned long long)(p.cache_v + p.off_v[u]);
-  const bool ok = fast_layout_ok(TK.tile_bytes, TV.tile_bytes, vblocks, ent_base[8], addr_k, addr_v, f.slot_k, f.slot_v, f.vq);
+  const bool ok = fast_layout_ok(TK.tile_bytes, TV.tile_bytes, vblocks, ent_base[8], addr_k, addr_v, f.slot_k, f.slot_v, f.max_vblocks);
   if (tid == 64) {
     D.tbk = ok ? TK.tile_bytes : 16; D.tbv = ok ? TV.tile_bytes : 16;
     D.kmeta[0] = ok ? TK.meta_off[0] : -1; D.kmeta[1] = ok ? TK.meta_off[1] : -1;

@@ -12,9 +12,9 @@
 // The K tile is walked one scale group at a time (all classes of group 0, then all classes of group 1): a single
 // set of score accumulators is live, and each (class, group) run is a short loop whose body is compile-time code.
 //
-// The V accumulators live in registers, one 16-strip block per accumulator.  Their number and their class must be
-// compile-time facts, so the kernel is instantiated for a few "quota" tuples (blocks per class 8, 4, 2, 1); the
-// host picks the smallest tuple that covers the widths of the call.
+// The V accumulators live in tensor memory, one 16-strip block per 4 columns of the warp's lane quarter: a block is
+// fetched, updated and put back, so any number of blocks per class runs through the same code and no register holds
+// an accumulator across the score phase.
 #pragma once
 #include "attention_tc_common.cuh"
 
@@ -187,10 +187,8 @@ __device__ __forceinline__ void k_run(const unsigned char* ktile, uint32_t run, 
   kb += 64 * nch;
 }
 
-// One class of the V tile, at most Q blocks of 16 strips, accumulators acc_o[OFF .. OFF + Q).  The probabilities
-// first get the class's position scales; per half tile, MMA u of a block contracts the token pairs of B fragments
-// u and u + 4.  Rows past the end of the class read whatever follows in shared memory (finite after masking); their
-// accumulators are never stored.
+// One half tile of one V block (16 strips x 64 tokens) into the block's accumulators: MMA u contracts the token
+// pairs of B fragments u and u + 4.
 template <int W, int HP>
 __device__ __forceinline__ void v_block_half(const uint32_t (&xa)[W], const uint32_t (&xb)[W], const uint32_t (&pw)[8],
                                              float (&acc)[4]) {
@@ -205,51 +203,88 @@ __device__ __forceinline__ void v_block_half(const uint32_t (&xa)[W], const uint
   for (int u = 0; u < 4; u++)
     mma16816(acc, U::get(wa, was, u), U::get(wb, wbs, u), U::get(wa, was, u + 4), U::get(wb, wbs, u + 4), pw[u], pw[u + 4]);
 }
-template <int W, int Q, int OFF, int NACC>
+// The V accumulators (one 16-strip block = 4 registers per thread) live in tensor memory: each warp owns the 32
+// lanes of its quarter, a block takes 4 columns.  A block is fetched, updated by its 8 MMAs and put back, so the
+// number of blocks and their classes are run-time facts (any width profile runs here) and the registers they would
+// occupy through the score phase are free.
+__device__ __forceinline__ void tmem_put(uint32_t taddr, const float (&a)[4]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};" ::"r"(taddr), "f"(a[0]), "f"(a[1]), "f"(a[2]),
+               "f"(a[3])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_get(uint32_t taddr, float (&a)[4]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(a[0]), "=f"(a[1]), "=f"(a[2]), "=f"(a[3])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// One class of the V tile: blocks of 16 strips, accumulators at tensor-memory columns col, col + 4, ...  The
+// probabilities first get the class's position scales; per half tile, MMA u of a block contracts the token pairs of
+// B fragments u and u + 4.  Rows past the end of the class read whatever follows in shared memory (finite after
+// masking); their accumulator rows are never stored.  FRESH: the unit's first tile (accumulators start at zero);
+// otherwise what comes back from tensor memory is first multiplied by alpha, the rescaling a new reference owes.
+template <int W, bool FRESH>
 __device__ __forceinline__ void v_class(const unsigned char* vtile, uint32_t cls, int gid, int tig,
-                                        const uint32_t (&pb)[2][8], float (&acc_o)[NACC][4]) {
-  if constexpr (Q > 0) {
-    using U = Unpack<W>;
-    const int n = cls & 0xff;
-    if (n == 0) return;
-    uint32_t pw[2][8];
+                                        const uint32_t (&pb)[2][8], uint32_t& col, float alpha) {
+  using U = Unpack<W>;
+  const int n = cls & 0xff;
+  if (n == 0) return;
+  uint32_t pw[2][8];
 #pragma unroll
-    for (int hp = 0; hp < 2; hp++)
+  for (int hp = 0; hp < 2; hp++)
 #pragma unroll
-      for (int ii = 0; ii < 8; ii++) pw[hp][ii] = hmul2_pow2(pb[hp][ii], U::peff(ii));
-    const unsigned char* cbase = vtile + (cls >> 16) * 16 + 4 * W * tig + 16 * W * gid;
+    for (int ii = 0; ii < 8; ii++) pw[hp][ii] = hmul2_pow2(pb[hp][ii], U::peff(ii));
+  const unsigned char* px = vtile + (cls >> 16) * 16 + 4 * W * tig + 16 * W * gid;
+  const int nb = (n + 15) >> 4;
+  const bool rescale = alpha != 1.f;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  if (!FRESH) tmem_get(col, acc);
+#pragma unroll 1
+  for (int bi = 0; bi < nb; bi++, px += 256 * W, col += 4) {
     uint32_t xa[W], xb[W];
-    ld_tile_words<W>(cbase, xa);
-    ld_tile_words<W>(cbase + 16 * W * 8, xb);
+    ld_tile_words<W>(px, xa);
+    ld_tile_words<W>(px + 128 * W, xb);
+    float nxt[4] = {0.f, 0.f, 0.f, 0.f};
+    if (!FRESH) {
+      tmem_wait_ld();
+      if (rescale) {
 #pragma unroll
-    for (int bi = 0; bi < Q; bi++) {
-      if (16 * bi >= n) break;
-      uint32_t ya[W], yb[W];
-      if (bi + 1 < Q) {                       // the next block's words (whatever follows the class if this is its last)
-        ld_tile_words<W>(cbase + 16 * W * (16 * bi + 16), ya);
-        ld_tile_words<W>(cbase + 16 * W * (16 * bi + 24), yb);
+        for (int e = 0; e < 4; e++) acc[e] *= alpha;
       }
-      v_block_half<W, 0>(xa, xb, pw[0], acc_o[OFF + bi]);
-      v_block_half<W, 1>(xa, xb, pw[1], acc_o[OFF + bi]);
-      if (bi + 1 < Q) {
-#pragma unroll
-        for (int k = 0; k < W; k++) { xa[k] = ya[k]; xb[k] = yb[k]; }
-      }
+      if (bi + 1 < nb) tmem_get(col + 4, nxt);             // the next block's accumulators come while this one multiplies
     }
+    v_block_half<W, 0>(xa, xb, pw[0], acc);
+    v_block_half<W, 1>(xa, xb, pw[1], acc);
+    tmem_put(col, acc);
+#pragma unroll
+    for (int e = 0; e < 4; e++) acc[e] = nxt[e];
   }
+}
+template <bool FRESH>
+__device__ __forceinline__ void v_tile(const unsigned char* vtile, const uint4& vc, int gid, int tig,
+                                       const uint32_t (&pb)[2][8], uint32_t col, float alpha) {
+  v_class<8, FRESH>(vtile, vc.x, gid, tig, pb, col, alpha);
+  v_class<4, FRESH>(vtile, vc.y, gid, tig, pb, col, alpha);
+  v_class<2, FRESH>(vtile, vc.z, gid, tig, pb, col, alpha);
+  v_class<1, FRESH>(vtile, vc.w, gid, tig, pb, col, alpha);
 }
 
 // Writes one class's accumulators into a partial record: row r of the class goes to strip index first + r, taking
 // the column of the scale group the strip belongs to.
-template <int Q, int OFF, int NACC>
-__device__ __forceinline__ void store_class(float* rec, uint32_t cls, int first, int gid, const float (&acc_o)[NACC][4]) {
+__device__ __forceinline__ void store_class(float* rec, uint32_t cls, int first, int gid, uint32_t& col) {
   const int n = cls & 0xff, n_g0 = (cls >> 8) & 0xff;
-#pragma unroll
-  for (int bi = 0; bi < Q; bi++) {
+#pragma unroll 1
+  for (int r0 = 0; r0 < n; r0 += 16, col += 4) {
+    float acc[4];
+    tmem_get(col, acc);
+    tmem_wait_ld();
 #pragma unroll
     for (int half = 0; half < 2; half++) {
-      const int r = 16 * bi + gid + 8 * half;
-      if (r < n) rec[kRecHead + first + r] = r >= n_g0 ? acc_o[OFF + bi][2 * half + 1] : acc_o[OFF + bi][2 * half];
+      const int r = r0 + gid + 8 * half;
+      if (r < n) rec[kRecHead + first + r] = r >= n_g0 ? acc[2 * half + 1] : acc[2 * half];
     }
   }
 }
@@ -277,6 +312,7 @@ struct WarpState {
 };
 static_assert(sizeof(WarpState) == 128, "WarpState layout");
 constexpr int kWarpStateBytes = 128;
+constexpr int kAccColumns = 128;       // tensor-memory columns per CTA: 4 per V block of a warp, up to 32 blocks
 
 // Adds one scale group's share to the scores of this thread's 16 tokens, in units of 1 / kscale:
 // s'_t += R_t * (hi + lo partial sums) + lo_t * (sum of q' over the group's active channels / kscale).
@@ -303,9 +339,8 @@ __device__ __forceinline__ void fold_group(const unsigned char* meta, float qlo,
   }
 }
 
-template <int Q8, int Q4, int Q2, int Q1, bool PAGED>
+template <bool PAGED>
 __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma_kernel(AttnArgs p, FastArgs f) {
-  constexpr int NACC = Q8 + Q4 + Q2 + Q1;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gid = lane >> 2, tig = lane & 3;
@@ -320,11 +355,21 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
     for (int s = 0; s < 2 * 4; s++) mbar_init(bars + 8 * s, 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncwarp();
+  // tensor memory for the V accumulators: kAccColumns columns per CTA, allocated and freed by warp 0
+  __shared__ uint32_t tmem_base_s;
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)kAccColumns) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t acc_base = tmem_base_s + ((uint32_t)(warp & 3) << 21);   // this warp's lanes 32 * (warp % 4), column 0
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel may be scheduled as SMs free up
   const int4 start = f.warp_start[gw];                 // first unit, first tile in it, tiles of that unit, tiles of the share
   const int count = start.w;
-  if (count <= 0) return;
+  if (count > 0) {
   int cu = start.x, ct = start.y, cnt = start.z;       // consumer: unit, tile, tiles of the unit
   // Copies are started by lane 0, whose cursors live in shared memory; every lane keeps the same counts of tiles
   // whose K / V copy has been started.  A unit's tiles are contiguous: its next tile is one tile size further.
@@ -375,8 +420,9 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
     for (int j = 0; j < issued_k; j++) { start_k(j); start_v(j); }
   }
 
-  float acc_o[NACC][4];
   float m_ref = -INFINITY, l_run = 0.f, plo0 = 0.f, plo1 = 0.f;
+  float alpha_acc = 1.f;      // rescaling the accumulators in tensor memory still owe
+  bool acc_fresh = true;      // the unit's first tile: its accumulators start at zero
   float kscale = 0.f, qlo0 = 0.f, qlo1 = 0.f;
   int n_seq = 0;
   bool fresh = true, ok = true;
@@ -393,11 +439,8 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
       kscale = d.kscale[tig];                                  // a power of two: the divisions are exact
       qlo0 = d.qlo[tig][0] / kscale; qlo1 = d.qlo[tig][1] / kscale;
       n_seq = attended_tokens(p, (cu / f.npass) / p.n_kv);
-#pragma unroll
-      for (int mb = 0; mb < NACC; mb++)
-#pragma unroll
-        for (int e = 0; e < 4; e++) acc_o[mb][e] = 0.f;
       m_ref = -INFINITY; l_run = 0.f; plo0 = 0.f; plo1 = 0.f;
+      alpha_acc = 1.f; acc_fresh = true;
       fresh = false;
       __syncwarp();
     }
@@ -485,10 +528,7 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
         const float alpha = fast_exp2(m_ref - need);
         m_ref = need;
         l_run *= alpha; plo0 *= alpha; plo1 *= alpha;
-#pragma unroll
-        for (int mb = 0; mb < NACC; mb++)
-#pragma unroll
-          for (int e2 = 0; e2 < 4; e2++) acc_o[mb][e2] *= alpha;
+        alpha_acc *= alpha;                                   // applied to the accumulators when they are next fetched
       }
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
 #pragma unroll
@@ -514,10 +554,10 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
     // ------------------------------------------------------------ P~ x V codes
     {
       const uint4 vc = *reinterpret_cast<const uint4*>(&ws.head[16]);
-      v_class<8, Q8, 0, NACC>(vtile, vc.x, gid, tig, pb, acc_o);
-      v_class<4, Q4, Q8, NACC>(vtile, vc.y, gid, tig, pb, acc_o);
-      v_class<2, Q2, Q8 + Q4, NACC>(vtile, vc.z, gid, tig, pb, acc_o);
-      v_class<1, Q1, Q8 + Q4 + Q2, NACC>(vtile, vc.w, gid, tig, pb, acc_o);
+      if (acc_fresh) v_tile<true>(vtile, vc, gid, tig, pb, acc_base, 1.f);
+      else v_tile<false>(vtile, vc, gid, tig, pb, acc_base, alpha_acc);
+      tmem_wait_st();
+      alpha_acc = 1.f; acc_fresh = false;
     }
     if (issued_v < issued_k) {
       __syncwarp();
@@ -538,10 +578,11 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
       float* rec = f.records + (int64_t)(gw + cu) * f.rec_stride + tig * (kRecHead + f.vs_max);
       if (gid == 0) { rec[0] = m_ref; rec[1] = l; rec[2] = q0; rec[3] = q1; }
       const UnitDesc& d = f.desc[cu];
-      store_class<Q8, 0, NACC>(rec, ws.head[16], d.vfirst[0], gid, acc_o);
-      store_class<Q4, Q8, NACC>(rec, ws.head[17], d.vfirst[1], gid, acc_o);
-      store_class<Q2, Q8 + Q4, NACC>(rec, ws.head[18], d.vfirst[2], gid, acc_o);
-      store_class<Q1, Q8 + Q4 + Q2, NACC>(rec, ws.head[19], d.vfirst[3], gid, acc_o);
+      uint32_t col = acc_base;
+      store_class(rec, ws.head[16], d.vfirst[0], gid, col);
+      store_class(rec, ws.head[17], d.vfirst[1], gid, col);
+      store_class(rec, ws.head[18], d.vfirst[2], gid, col);
+      store_class(rec, ws.head[19], d.vfirst[3], gid, col);
       fresh = true;
     }
     // next tile of the flattened (unit, tile) space
@@ -561,6 +602,10 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
     // give copies that may still be in flight a bounded time to land before the shared memory is released
     for (int s = 0; s < D; s++) { mbar_wait(bars + 8 * s, 0); mbar_wait(bars + 8 * (4 + s), 0); }
   }
+  }   // count > 0
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base_s), "r"((uint32_t)kAccColumns) : "memory");
 }
 
 }  // namespace spectra

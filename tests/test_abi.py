@@ -107,8 +107,8 @@ def test_misaligned_buffers_are_refused_on_the_host(lib):
 
 def test_cache_bytes_and_attention_path(lib):
     """Host helpers: a unit-side's buffer size for a capacity in tokens, and which kernels an attention call will
-    run for a set of widths (the tensor-core kernel is built for a few tuples of V blocks per class; scale groups
-    other than 64, missing host widths and profiles outside the tuples take the CUDA-core kernel)."""
+    run for a set of widths (the tensor-core kernels take every width profile at scale group 64 when the host copy of
+    the widths is given; other scale groups and calls without host widths take the CUDA-core kernel)."""
     import numpy as np
     cfg = sp.default_config()
     w4 = [4] * 128
@@ -123,11 +123,11 @@ def test_cache_bytes_and_attention_path(lib):
     assert sp.attention_path(cfg, 4, 28, 1, two, two) == sp.PATH_TENSOR_CORE        # groups of 7 heads: two passes
     assert sp.attention_path(cfg, 8, 32, 1, None, None) == sp.PATH_CUDA_CORE        # no host widths
     assert sp.attention_path(sp.default_config(scale_group=32), 8, 32, 1, two, two) == sp.PATH_CUDA_CORE
-    eight = np.full((1, 128), 8, np.uint8)                                           # an 8-bit V class: no variant
-    assert sp.attention_path(cfg, 8, 32, 1, two, eight) == sp.PATH_CUDA_CORE
-    assert sp.attention_path(cfg, 8, 32, 1, eight, two) == sp.PATH_TENSOR_CORE      # the K side has no such limit
-    three = np.full((1, 128), 3, np.uint8)                                           # 8 + 8 blocks: beyond every tuple
-    assert sp.attention_path(cfg, 8, 32, 1, two, three) == sp.PATH_CUDA_CORE
+    eight = np.full((1, 128), 8, np.uint8)
+    assert sp.attention_path(cfg, 8, 32, 1, two, eight) == sp.PATH_TENSOR_CORE
+    assert sp.attention_path(cfg, 8, 32, 1, eight, two) == sp.PATH_TENSOR_CORE
+    seven = np.full((1, 128), 7, np.uint8)                                           # three sub-fields per channel
+    assert sp.attention_path(cfg, 8, 32, 1, seven, seven) == sp.PATH_TENSOR_CORE
     with pytest.raises(sp.SpectraError):
         sp.attention_path(cfg, 3, 8, 1, two, two)
     with pytest.raises(sp.SpectraError):

@@ -305,7 +305,7 @@ def _gpu_attention(sp, cfg, q_dev, batch, n_kv, n_q, seq_len, max_len, K, V, cac
 
 
 @pytest.mark.parametrize("host_widths", [True, False], ids=["tensor", "generic"])
-@pytest.mark.parametrize("ratio", [4.0, 6.0, 8.0, 12.0, 16.0])
+@pytest.mark.parametrize("ratio", [3.0, 4.0, 5.0, 6.0, 8.0, 12.0, 16.0])
 @pytest.mark.parametrize("n", [1024, 1000, 77])
 def test_tiny_attention_matches_oracle(sp, ratio, n, host_widths):
     wl, S = _tiny_setup(sp, ratio)
@@ -931,3 +931,33 @@ def test_paged_caches_give_the_same_bytes_and_outputs_as_contiguous_ones(sp, dt)
         g = gathered(name).reshape(n_seq, n_tiles, c["tb"])
         r = c["cont"].cpu().numpy().reshape(n_seq, n_tiles, c["tb"])
         assert np.array_equal(g[:, :5], r[:, :5])
+
+
+@pytest.mark.parametrize("widths", ["all8", "all7", "v8_k1", "odd_mix"])
+def test_tensor_core_attention_takes_any_width_profile(sp, widths):
+    """The tensor-core kernels keep the value accumulators in tensor memory, block by block, so no width profile is
+    special: 8-bit channels, three sub-fields per channel, one-bit keys with eight-bit values, and a mix with odd
+    class sizes all run there and match the oracle."""
+    wl = si.WORKLOADS["tiny"]
+    cfg = sp.default_config()
+    n = 700
+    rng = np.random.default_rng(3)
+    table = {"all8": (np.full(128, 8), np.full(128, 8)), "all7": (np.full(128, 7), np.full(128, 7)),
+             "v8_k1": (np.ones(128, np.int64), np.full(128, 8)),
+             "odd_mix": (rng.integers(0, 9, 128), rng.integers(0, 9, 128))}
+    wk, wv = (np.asarray(w, np.uint8) for w in table[widths])
+    S, caches = {}, {}
+    for side, name, w in ((si.SIDE_K, "k", wk), (si.SIDE_V, "v", wv)):
+        X = si.draw_unit(wl, 0, 0, side, 0, n_tokens=n)
+        params = H.fit_params([X], 4.0, widths_override=w)
+        off, total = H.cache_layout(params, 1, n)
+        c = np.zeros(total, np.uint8)
+        assert H.oracle_encode(params, side, X[None], [0], c, off) == 0
+        S[name] = dict(X=X, params=params, off=off, total=total)
+        caches[name] = c
+    assert sp.attention_path(cfg, 1, 4, 1, S["k"]["params"].widths, S["v"]["params"].widths) == sp.PATH_TENSOR_CORE
+    q = si.draw_queries(wl, 0, 0)
+    ref_b, lse_b = _oracle_attention(4, q[None].astype(np.float64), [n], S["k"], S["v"], caches["k"], caches["v"])
+    got, lse = _gpu_attention(sp, cfg, H.to_dev(q[None]), 1, 1, 4, [n], n, S["k"], S["v"], caches["k"], caches["v"])
+    assert H.rel_err_per_vector(got[0], ref_b[0]) <= TOL
+    assert np.abs(lse[0] - lse_b[0]).max() <= 2e-3
