@@ -145,9 +145,9 @@ __device__ __forceinline__ void k_chunk(const uint32_t (&xa)[W], const uint32_t 
 
 // One (class, scale group) run of the K tile: `run` = byte offset / 16 of its first pair | chunks << 16 |
 // slot of a strip stored alone in the last chunk << 24 | (such a strip exists) << 27.  A run has at most MAXC chunks
-// (64 channels per scale group; a group-1 run may start in the middle of a chunk).  The loop is unrolled with an
-// early exit, so that offsets are immediates and the next chunk's words are loaded while the current chunk is
-// multiplied.  The B table is walked in the same order; on entry b01, b23 hold the run's first entry and kb points
+// (64 channels per scale group; a group-1 run may start in the middle of a chunk).  The loop is kept rolled (the
+// sixteen warps of an SM run different parts of the kernel: its code has to stay small for the instruction cache)
+// and loads the next chunk's words while the current chunk is multiplied.  The B table is walked in the same order; on entry b01, b23 hold the run's first entry and kb points
 // at this lane's part of it; on exit they hold the entry after the run (the first of the next run; past the last
 // run a spare entry of the table, never used).
 template <int W, int MAXC>
@@ -160,31 +160,27 @@ __device__ __forceinline__ void k_run(const unsigned char* ktile, uint32_t run, 
   uint32_t xa[W], xb[W];
   ld_tile_words<W>(pa, xa);
   ld_tile_words<W>(pa + 128 * W, xb);
-#pragma unroll
-  for (int i = 0; i < MAXC; i++) {
-    if (i >= nch) break;
+#pragma unroll 1
+  for (int i = 0; i < nch; i++) {
+    pa += 256 * W;
+    kb += 64;
     uint32_t ya[W], yb[W];
-    if (i + 1 < MAXC) {                       // the next chunk's words (whatever follows the run if this is its last)
-      ld_tile_words<W>(pa + 256 * W * (i + 1), ya);
-      ld_tile_words<W>(pa + 256 * W * (i + 1) + 128 * W, yb);
-    }
+    ld_tile_words<W>(pa, ya);                 // the next chunk's words (whatever follows the run if this is its last)
+    ld_tile_words<W>(pa + 128 * W, yb);
     if (i == lone_i) {
       // the pair in slot `slot` of this chunk is one strip stored alone: the threads of that slot re-read it as
       // half-words (all threads load, a select keeps the result where it belongs)
       const int slot = (int)(run >> 24) & 7;
       uint32_t t[W];
-      ld_lone_words<W>(ktile + (run & 0xffffu) * 16 + 256 * W * i + 32 * W * slot + 2 * W * gid, t);
+      ld_lone_words<W>(pa - 256 * W - 32 * W * tig - 4 * W * gid + 32 * W * slot + 2 * W * gid, t);
       const bool mine_a = tig == slot, mine_b = tig + 4 == slot;
 #pragma unroll
       for (int k = 0; k < W; k++) { xa[k] = mine_a ? t[k] : xa[k]; xb[k] = mine_b ? t[k] : xb[k]; }
     }
-    k_chunk<W>(xa, xb, b01, b23, kb + 64 * (i + 1), acc);
-    if (i + 1 < MAXC) {
+    k_chunk<W>(xa, xb, b01, b23, kb, acc);
 #pragma unroll
-      for (int k = 0; k < W; k++) { xa[k] = ya[k]; xb[k] = yb[k]; }
-    }
+    for (int k = 0; k < W; k++) { xa[k] = ya[k]; xb[k] = yb[k]; }
   }
-  kb += 64 * nch;
 }
 
 // One half tile of one V block (16 strips x 64 tokens) into the block's accumulators: MMA u contracts the token
