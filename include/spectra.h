@@ -171,6 +171,22 @@ int spectra_alloc_bits(const spectra_config* cfg, const float* var_alloc, int64_
                        uint8_t* widths, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * spectra_alloc_bits_pooled -- the same rule with the budget pooled over pool_units consecutive units (Sec. 3.2 and
+ * the appendix's bit-profile figure: the paper's latent spans all KV heads of a layer, so a head with little energy
+ * gives its bits to the others; with cfg->width_group = 64 this is the paper's structure, one width per group of 64
+ * energy-ordered coordinates).  Every run of pool_units units gets pool_units * Btot bits over its pool_units * d
+ * channels; ties go to the lowest unit, then channel.  n_units must be a multiple of pool_units; at most 2048 width
+ * groups per pool (SPECTRA_UNSUPPORTED beyond).
+ * spectra_split_ratio -- the key/value budget split of Sec. 3.1 (last paragraph) and the appendix on hyperparameters:
+ * of the bits a nominal ratio gives keys and values together, the keys get the fraction kappa (0 < kappa < 1) and the
+ * values the rest: ratio_k = ratio / (2 kappa), ratio_v = ratio / (2 (1 - kappa)); kappa = 0.5 leaves both at ratio.
+ * Host only.
+ */
+int spectra_alloc_bits_pooled(const spectra_config* cfg, const float* var_alloc, int64_t n_units, int64_t pool_units,
+                              double ratio, uint8_t* widths, void* stream);
+int spectra_split_ratio(double ratio, double kappa, double* ratio_k, double* ratio_v);
+
+/* ------------------------------------------------------------------------------------------------
  * spectra_encode -- Sec. 3.2-3.3 (Mode A streaming: each token is down-projected, quantised per token at
  * the group widths and appended).  Appends n_new tokens to each of n_units unit-sides: unit u gets tokens
  * x[u*stride_unit + i*stride_token + 0..d) for i < n_new at cache positions pos0[u] + i.

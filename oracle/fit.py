@@ -149,6 +149,21 @@ def alloc_bits(v, btot, b_max=8, width_group=1):
     return np.repeat(b, width_group).astype(np.uint8)
 
 
+def alloc_bits_pooled(v_units, btot_per_unit, b_max=8, width_group=1):
+    """The same allocation with the budget pooled over several units (the KV heads of a layer: the paper's latent
+    spans all of them, Sec. 3.2 and the appendix's bit-profile figure).  v_units [n, d]; the n * d channels compete
+    for n * btot_per_unit bits under the rule of alloc_bits (index order: unit, then channel).  Returns [n, d]."""
+    v_units = np.asarray(v_units, dtype=np.float32)
+    n, d = v_units.shape
+    return alloc_bits(v_units.reshape(-1), n * btot_per_unit, b_max, width_group).reshape(n, d)
+
+
+def split_ratio(ratio, kappa):
+    """Key/value budget split (Sec. 3.1, last paragraph; appendix on hyperparameters): keys get the fraction kappa of
+    the bits that `ratio` gives keys and values together.  Returns (ratio_k, ratio_v)."""
+    return ratio / (2.0 * kappa), ratio / (2.0 * (1.0 - kappa))
+
+
 # ------------------------------------------------------------------ rate accounting
 
 def effective_bits_per_element(widths, scale_group):

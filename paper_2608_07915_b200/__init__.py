@@ -27,6 +27,7 @@ EXPORTS = [
     "spectra_fit_basis", "spectra_fit_basis_static", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
     "spectra_decode_attention", "spectra_decode_step", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
     "spectra_total_bits", "spectra_status_string", "spectra_cache_bytes", "spectra_attention_path",
+    "spectra_alloc_bits_pooled", "spectra_split_ratio",
 ]
 
 
@@ -165,6 +166,21 @@ def alloc_bits(cfg, var_alloc, n_units, ratio, widths):
     rc = lib().spectra_alloc_bits(C.byref(cfg), _ptr(var_alloc), C.c_int64(n_units), C.c_double(ratio), _ptr(widths),
                                   _stream())
     _check(rc, "spectra_alloc_bits")
+
+
+def alloc_bits_pooled(cfg, var_alloc, n_units, pool_units, ratio, widths):
+    """Allocation with the budget pooled over runs of pool_units consecutive units (the heads of a layer)."""
+    rc = lib().spectra_alloc_bits_pooled(C.byref(cfg), _ptr(var_alloc), C.c_int64(n_units), C.c_int64(pool_units),
+                                         C.c_double(ratio), _ptr(widths), _stream())
+    _check(rc, "spectra_alloc_bits_pooled")
+
+
+def split_ratio(ratio, kappa):
+    """(ratio_k, ratio_v): the keys get the fraction kappa of the bits of keys and values together."""
+    rk, rv = C.c_double(0), C.c_double(0)
+    _check(lib().spectra_split_ratio(C.c_double(ratio), C.c_double(kappa), C.byref(rk), C.byref(rv)),
+           "spectra_split_ratio")
+    return rk.value, rv.value
 
 
 def encode(cfg, side, x, flags, n_units, n_param_sets, pos0, n_new, stride_unit, stride_token, w_enc, mean_rot,

@@ -289,6 +289,55 @@ __global__ void __launch_bounds__(128) alloc_kernel(const float* __restrict__ va
   }
 }
 
+// Allocation with the budget pooled over `pool` consecutive units (the heads of one layer: the paper's latent spans
+// all of them): one CTA per pool, the groups' variances and widths in shared memory, the same greedy rule over all
+// pool * d / wg groups (index order = unit, then channel, so ties go to the lowest unit and channel).
+constexpr int kPoolMaxGroups = 2048;
+__global__ void __launch_bounds__(128) alloc_pooled_kernel(const float* __restrict__ var_alloc, int pool, int btot,
+                                                           int b_max, int wg, uint8_t* __restrict__ widths) {
+  __shared__ double v[kPoolMaxGroups];
+  __shared__ uint8_t b[kPoolMaxGroups];
+  __shared__ double red_v[4];
+  __shared__ int red_g[4];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ng = pool * kD / wg;
+  const float* src = var_alloc + (int64_t)blockIdx.x * pool * kD;
+  for (int g = tid; g < ng; g += 128) {
+    float acc = src[g * wg];
+    for (int j = 1; j < wg; j++) acc = __fadd_rn(acc, src[g * wg + j]);
+    v[g] = (double)(wg == 1 ? acc : __fdiv_rn(acc, (float)wg));
+    b[g] = 0;
+  }
+  __syncthreads();
+  long long steps = (long long)pool * btot / wg;
+  if (steps > (long long)ng * b_max) steps = (long long)ng * b_max;
+  for (long long it = 0; it < steps; it++) {
+    double best = -1.0; int best_g = 1 << 30;
+    for (int g = tid; g < ng; g += 128) {
+      if (b[g] < b_max) {
+        const double val = scalbn(v[g], -2 * (int)b[g]);
+        if (val > best || (val == best && g < best_g)) { best = val; best_g = g; }
+      }
+    }
+#pragma unroll
+    for (int s = 16; s; s >>= 1) {
+      const double ob = __shfl_xor_sync(0xffffffffu, best, s);
+      const int og = __shfl_xor_sync(0xffffffffu, best_g, s);
+      if (ob > best || (ob == best && og < best_g)) { best = ob; best_g = og; }
+    }
+    if (lane == 0) { red_v[warp] = best; red_g[warp] = best_g; }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < 4; w++)
+        if (red_v[w] > best || (red_v[w] == best && red_g[w] < best_g)) { best = red_v[w]; best_g = red_g[w]; }
+      if (best_g < ng) b[best_g]++;
+    }
+    __syncthreads();
+  }
+  uint8_t* dst = widths + (int64_t)blockIdx.x * pool * kD;
+  for (int j = tid; j < pool * kD; j += 128) dst[j] = b[j / wg];
+}
+
 }  // namespace spectra
 
 using namespace spectra;
@@ -374,4 +423,26 @@ extern "C" int spectra_alloc_bits(const spectra_config* cfg, const float* var_al
   alloc_kernel<<<(unsigned)((n_units + 3) / 4), 128, 0, (cudaStream_t)stream>>>(var_alloc, n_units, btot, cfg->b_max,
                                                                                 cfg->width_group, widths);
   return launch_status();
+}
+
+extern "C" int spectra_alloc_bits_pooled(const spectra_config* cfg, const float* var_alloc, int64_t n_units,
+                                         int64_t pool_units, double ratio, uint8_t* widths, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (n_units < 0 || pool_units < 1 || !(ratio > 0.0)) return SPECTRA_INVALID_ARG;
+  if (n_units == 0) return SPECTRA_OK;
+  if (n_units % pool_units) return SPECTRA_INVALID_ARG;
+  if (!var_alloc || !widths) return SPECTRA_INVALID_ARG;
+  if (pool_units * kD / cfg->width_group > kPoolMaxGroups) return SPECTRA_UNSUPPORTED;
+  const int btot = spectra_total_bits(cfg, ratio);
+  alloc_pooled_kernel<<<(unsigned)(n_units / pool_units), 128, 0, (cudaStream_t)stream>>>(
+      var_alloc, (int)pool_units, btot, cfg->b_max, cfg->width_group, widths);
+  return launch_status();
+}
+
+extern "C" int spectra_split_ratio(double ratio, double kappa, double* ratio_k, double* ratio_v) {
+  if (!(ratio > 0.0) || !(kappa > 0.0) || !(kappa < 1.0) || !ratio_k || !ratio_v) return SPECTRA_INVALID_ARG;
+  *ratio_k = ratio / (2.0 * kappa);
+  *ratio_v = ratio / (2.0 * (1.0 - kappa));
+  return SPECTRA_OK;
 }

@@ -961,3 +961,78 @@ def test_tensor_core_attention_takes_any_width_profile(sp, widths):
     got, lse = _gpu_attention(sp, cfg, H.to_dev(q[None]), 1, 1, 4, [n], n, S["k"], S["v"], caches["k"], caches["v"])
     assert H.rel_err_per_vector(got[0], ref_b[0]) <= TOL
     assert np.abs(lse[0] - lse_b[0]).max() <= 2e-3
+
+
+@pytest.mark.parametrize("width_group", [1, 64])
+def test_pooled_allocation_is_bit_exact(sp, width_group):
+    """spectra_alloc_bits_pooled against the oracle: budget pooled over the 8 heads of a layer, per channel and with
+    one width per group of 64 coordinates (the paper's structure), several ratios, ties included."""
+    rng = np.random.default_rng(23)
+    H, layers = 8, 3
+    v = ((np.arange(1, 129) ** -1.5)[None] * rng.uniform(0.02, 4.0, (layers * H, 1))).astype(np.float32)
+    v[5, 40:60] = v[5, 40]                               # ties inside a head
+    v[9] = v[8]                                          # and between heads
+    v[17, 100:] = 0.0                                    # a dead tail
+    cfg = sp.default_config(width_group=width_group)
+    for ratio in (4.0, 8.0, 12.0):
+        widths = torch.zeros((layers * H, 128), dtype=torch.uint8, device="cuda")
+        sp.alloc_bits_pooled(cfg, torch.from_numpy(v).cuda(), layers * H, H, ratio, widths)
+        torch.cuda.synchronize()
+        got = widths.cpu().numpy()
+        btot = ofit.total_bits(128, ratio)
+        for l in range(layers):
+            ref = ofit.alloc_bits_pooled(v[l * H:(l + 1) * H], btot, 8, width_group)
+            assert np.array_equal(got[l * H:(l + 1) * H], ref), (width_group, ratio, l)
+    rk, rv = sp.split_ratio(8.0, 0.25)
+    assert (rk, rv) == ofit.split_ratio(8.0, 0.25) == (16.0, 8.0 / 1.5)
+
+
+def test_paper_structure_allocation_end_to_end(sp):
+    """The paper's allocation structure through the whole path: one width per group of 64 energy-ordered coordinates,
+    the budget pooled over the KV heads of the layer (heads with little energy give their bits away, so tile sizes
+    differ per head) and split between keys and values with kappa = 0.25 (Sec. 3.1-3.2, appendix on hyperparameters).
+    Widths from the GPU equal the oracle's; encode, then attention on the tensor-core path, against the oracle."""
+    base = si.WORKLOADS["llama1"]
+    wl = dataclasses.replace(base, kv_heads=4, q_heads=16, n_fit=512)
+    cfg = sp.default_config(width_group=64)
+    n, Hk, G = 640, 4, 4
+    head_scale = np.array([3.0, 1.0, 0.3, 0.05], np.float32)          # very unequal heads
+    rk, rv = sp.split_ratio(8.0, 0.25)
+    S = {}
+    for side, name, ratio in ((si.SIDE_K, "k", rk), (si.SIDE_V, "v", rv)):
+        X = H.draw_units(wl, 0, side, 1, n) * head_scale[:, None, None]
+        fits = [ofit.fit_basis(X[h][:512].astype(np.float64), ofit.GAIN_SQRT) for h in range(Hk)]
+        v_alloc = np.stack([f["v_alloc"] for f in fits]).astype(np.float32)
+        ref_w = ofit.alloc_bits_pooled(v_alloc, ofit.total_bits(128, ratio), 8, 64)
+        widths = torch.zeros((Hk, 128), dtype=torch.uint8, device="cuda")
+        sp.alloc_bits_pooled(cfg, torch.from_numpy(v_alloc).cuda(), Hk, Hk, ratio, widths)
+        torch.cuda.synchronize()
+        assert np.array_equal(widths.cpu().numpy(), ref_w)
+        assert len(set(ref_w.sum(axis=1))) > 1                         # the heads did get different budgets
+        params = H.Params(np.stack([f["W_enc"] for f in fits]), np.stack([f["W_dec"] for f in fits]),
+                          np.stack([f["m_rot"] for f in fits]), ref_w, 64)
+        off, total = H.cache_layout(params, Hk, n)
+        cache = torch.zeros(total, dtype=torch.uint8, device="cuda")
+        st = _gpu_encode(sp, cfg, params, H.dev_params(params), side, H.to_dev(X).to(torch.bfloat16),
+                         torch.zeros(Hk, dtype=torch.int32, device="cuda"), cache, H.to_dev(off))
+        assert st == 0
+        ref = np.zeros(total, np.uint8)
+        assert H.oracle_encode(params, side, si.to_bf16_f32(X), [0] * Hk, ref, off) == 0
+        got = cache.cpu().numpy()
+        for u in range(Hk):
+            bad, tot, dmax, mmax, _ = H.compare_coded_units(ref[off[u]:], got[off[u]:], int(params.tile_bytes[u]), n,
+                                                            params.widths[u], 64, side)
+            assert dmax <= 1 and mmax <= 1 and bad <= max(2, MISMATCH_RATE * tot)
+        S[name] = dict(params=params, off=off, total=total, cache=got)
+    assert sp.attention_path(cfg, Hk, wl.q_heads, Hk, S["k"]["params"].widths, S["v"]["params"].widths) == \
+        sp.PATH_TENSOR_CORE
+    q = si.draw_queries(wl, 0, 0)[:wl.q_heads]
+    got, lse = _gpu_attention(sp, cfg, H.to_dev(q[None]), 1, Hk, wl.q_heads, [n], n, S["k"], S["v"], S["k"]["cache"],
+                              S["v"]["cache"])
+    K, V = S["k"], S["v"]
+    ref, lref = oc.attention_units("B", q.reshape(Hk, G, 128).astype(np.float64), [n] * Hk, K["cache"], K["off"],
+                                   K["params"].tile_bytes, V["cache"], V["off"], V["params"].tile_bytes,
+                                   K["params"].w_dec, K["params"].m_rot, K["params"].widths, V["params"].w_dec,
+                                   V["params"].m_rot, V["params"].widths, 64, 1.0 / np.sqrt(128.0))
+    assert H.rel_err_per_vector(got[0].reshape(Hk, G, 128), ref) <= TOL
+    assert np.abs(lse[0].reshape(Hk, G) - lref).max() <= 2e-3

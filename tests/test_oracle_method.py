@@ -334,3 +334,54 @@ def test_importance_allocation_beats_uniform_at_low_rate():
     wf = _attend(_coded_tiny(8.0, fit.GAIN_WHITEN, n), q, "A", n)[0]
     un = _attend(_coded_tiny(8.0, fit.GAIN_WHITEN, n, widths_override=2), q, "A", n)[0]
     assert np.linalg.norm(wf - dense) < np.linalg.norm(un - dense)
+
+
+# ----------------------------------------------------------------------------- pooled allocation, key/value split
+
+def _objective(v, b):
+    return float((np.asarray(v, np.float64) * 4.0 ** (-np.asarray(b, np.float64))).sum())
+
+
+def test_pooled_allocation_is_the_optimum_over_all_heads_together():
+    """Sec. 3.2 with the latent spanning all KV heads (appendix, bit-profile figure): the pooled allocation spends
+    exactly the pooled budget, never does worse than allocating head by head, equals it when the heads are
+    identical, moves bits from a weak head to a strong one, and still satisfies the discrete water level
+    D_i <= 4 D_j across heads (equal slope, Eq. 5)."""
+    rng = np.random.default_rng(5)
+    d, H, btot = 128, 4, 256
+    base = ((np.arange(1, d + 1) ** -1.5) * rng.uniform(0.9, 1.1, d)).astype(np.float32)   # no exact ties
+    same = np.stack([base] * H)
+    pooled = fit.alloc_bits_pooled(same, btot)
+    assert np.array_equal(pooled, np.stack([fit.alloc_bits(base, btot)] * H))
+    scales = np.array([4.0, 1.0, 0.25, 0.01], np.float32)
+    v = base[None] * scales[:, None] * rng.uniform(0.9, 1.1, (H, d)).astype(np.float32)
+    pooled = fit.alloc_bits_pooled(v, btot)
+    single = np.stack([fit.alloc_bits(v[h], btot) for h in range(H)])
+    assert pooled.sum() == H * btot == single.sum()
+    assert _objective(v, pooled) <= _objective(v, single)
+    per_head = pooled.sum(axis=1)
+    assert per_head[0] > per_head[1] > per_head[2] > per_head[3]
+    D = v.astype(np.float64) * 4.0 ** (-pooled.astype(np.float64))
+    assert D[pooled < 8].max() <= 4.0 * D[pooled > 0].min() * (1 + 1e-12)
+    # brute force on a tiny pool: 2 heads x 3 channels, 5 bits, widths up to 3
+    import itertools
+    vt = np.array([[9.0, 1.0, 0.1], [30.0, 0.5, 0.4]], np.float32)
+    got = fit.alloc_bits_pooled(vt, 5 // 2 + 0, b_max=3)          # 2 bits per head: 4 in the pool
+    best = min((b for b in itertools.product(range(4), repeat=6) if sum(b) == 4),
+               key=lambda b: _objective(vt.reshape(-1), b))
+    assert _objective(vt.reshape(-1), got.reshape(-1)) == _objective(vt.reshape(-1), best)
+    # one width per group of 64 coordinates, pooled over 8 heads: 16 groups compete (the paper's structure)
+    v8 = base[None] * rng.uniform(0.05, 3.0, (8, 1)).astype(np.float32)
+    g = fit.alloc_bits_pooled(v8, 256, width_group=64)
+    assert g.sum() == 8 * 256 and all(len(set(row[:64])) == 1 and len(set(row[64:])) == 1 for row in g)
+
+
+def test_key_value_budget_split():
+    """Sec. 3.1 (last paragraph): the keys get the fraction kappa of the joint budget.  kappa = 1/2 leaves both sides
+    at the nominal ratio; for any kappa the two budgets add up to the joint one."""
+    assert fit.split_ratio(8.0, 0.5) == (8.0, 8.0)
+    for kappa in (0.25, 0.4, 0.75):
+        rk, rv = fit.split_ratio(8.0, kappa)
+        bits_k, bits_v = 16 * 128 / rk, 16 * 128 / rv
+        assert abs(bits_k + bits_v - 2 * 16 * 128 / 8.0) < 1e-9
+        assert abs(bits_k / (bits_k + bits_v) - kappa) < 1e-12
