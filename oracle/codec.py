@@ -229,3 +229,37 @@ def encode_units(x, w_enc, m_rot, widths, gs, side, pos0, cache, unit_offset, ti
                                 C.c_int64(n_units), C.c_int64(pos0), C.c_int64(n_new), _p(cache),
                                 _p(_i64(unit_offset)), _p(_i64(tile_stride)))
     return int(st)
+
+
+def rope_rows(x, pos0, theta):
+    """Rotates row t of x ([n, d] fp64) at position pos0 + t (rotate-half pairing).  Returns a new array."""
+    x = _f64(x).copy()
+    n, d = x.shape
+    for t in range(n):
+        lib().spo_rope_row(_p(x[t]), C.c_int(d), C.c_double(pos0 + t), C.c_double(theta))
+    return x
+
+
+def decode_unit_rope(cache, tile_stride, n, w_dec, m_rot, widths, gs, side, pos0, theta):
+    cache = _u8(cache)
+    widths = _u8(widths)
+    d = widths.size
+    xhat = np.zeros((n, d), np.float64)
+    lib().spo_decode_unit_rope(_p(cache), C.c_int64(tile_stride), C.c_int64(n), _p(_f32(w_dec)), _p(_f32(m_rot)),
+                               _p(widths), C.c_int(d), C.c_int(gs), C.c_int(side), C.c_double(pos0), C.c_double(theta),
+                               _p(xhat))
+    return xhat
+
+
+def attention_rope_unit(mode, q, n, cache_k, stride_k, cache_v, stride_v, w_dec_k, m_rot_k, widths_k, w_dec_v, m_rot_v,
+                        widths_v, gs, scale, pos0, theta):
+    """One unit, q [G, d] (already rotated at the query's position).  mode 'A' or 'B'.  Returns out [G, d], lse [G]."""
+    q = _f64(q)
+    G, d = q.shape
+    out = np.zeros((G, d), np.float64)
+    lse = np.zeros(G, np.float64)
+    fn = lib().spo_attention_rope_mode_a if mode == "A" else lib().spo_attention_rope_mode_b
+    fn(_p(q), C.c_int(G), _p(_u8(cache_k)), C.c_int64(stride_k), _p(_u8(cache_v)), C.c_int64(stride_v), C.c_int64(n),
+       _p(_f32(w_dec_k)), _p(_f32(m_rot_k)), _p(_u8(widths_k)), _p(_f32(w_dec_v)), _p(_f32(m_rot_v)), _p(_u8(widths_v)),
+       C.c_int(d), C.c_int(gs), C.c_double(scale), C.c_double(pos0), C.c_double(theta), _p(out), _p(lse))
+    return out, lse

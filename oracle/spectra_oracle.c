@@ -16,6 +16,7 @@
  *   - attention over the coded cache, Mode A (reconstruct, then textbook softmax
  *     attention) and Mode B (latent-space attention, appendix "Latent-space attention
  *     and memory": q' = q W_up^T folded once, scores q' c^T, output lifted once)
+ *   - the same two with the rotary position embedding applied to the reconstructed keys (Sec. 3.3)
  *
  * Floating point: the quantiser is IEEE fp32, round-to-nearest-even, one rounding per
  * written operation, no fused multiply-add (compile with -ffp-contract=off).  Rotations,
@@ -426,6 +427,107 @@ void spo_attention_mode_b(const double* q, int G, const uint8_t* cache_k, int64_
       double acc = 0.0;
       for (int j = 0; j < d; j++) acc += qp[j] * (double)yk[t * d + j];
       s[t] = acc + cst;
+      if (s[t] > mx) mx = s[t];
+    }
+    double l = 0.0;
+    for (int64_t t = 0; t < n; t++) { s[t] = exp(s[t] - mx); l += s[t]; }
+    for (int j = 0; j < d; j++) {
+      double acc = 0.0;
+      for (int64_t t = 0; t < n; t++) acc += s[t] * (double)yv[t * d + j];
+      op[j] = acc / l + (double)mean_rot_v[j];
+    }
+    for (int i = 0; i < d; i++) {
+      double acc = 0.0;
+      for (int j = 0; j < d; j++) acc += op[j] * (double)w_dec_v[(int64_t)j * d + i];
+      out[h * d + i] = acc;
+    }
+    if (lse) lse[h] = mx + log(l);
+  }
+  free(yk); free(yv); free(s);
+}
+
+/* ---------------------------------------------------------------- rotary position embedding (RoPE)
+ * The paper's latent is taken before the position rotation: Mode A rebuilds K-hat and applies RoPE to it, per token
+ * position, before the scores (Sec. 3.3, "Streaming decode").  Convention: the two halves of a vector are paired,
+ * (x_i, x_{i + d/2}) is rotated by the angle pos * theta^(-2 i / d), i < d/2 (the "rotate-half" form).  The query
+ * handed to the attention functions below is already rotated at its own position. */
+void spo_rope_row(double* x, int d, double pos, double theta) {
+  const int h = d / 2;
+  for (int i = 0; i < h; i++) {
+    const double ang = pos * pow(theta, -2.0 * (double)i / (double)d);
+    const double c = cos(ang), sn = sin(ang);
+    const double a = x[i], b = x[i + h];
+    x[i] = a * c - b * sn;
+    x[i + h] = b * c + a * sn;
+  }
+}
+
+/* Reconstruct the keys of one unit and rotate token t at position pos0 + t: xhat [n, d] fp64. */
+void spo_decode_unit_rope(const uint8_t* cache, int64_t tile_stride, int64_t n, const float* w_dec,
+                          const float* mean_rot, const uint8_t* widths, int d, int gs, int side, double pos0,
+                          double theta, double* xhat_out) {
+  spo_decode_unit(cache, tile_stride, n, w_dec, mean_rot, widths, d, gs, side, NULL, xhat_out);
+  for (int64_t t = 0; t < n; t++) spo_rope_row(xhat_out + t * d, d, pos0 + (double)t, theta);
+}
+
+/* Mode A with RoPE: K-hat reconstructed, rotated per position, then textbook softmax attention with V-hat. */
+void spo_attention_rope_mode_a(const double* q, int G, const uint8_t* cache_k, int64_t stride_k,
+                               const uint8_t* cache_v, int64_t stride_v, int64_t n, const float* w_dec_k,
+                               const float* mean_rot_k, const uint8_t* widths_k, const float* w_dec_v,
+                               const float* mean_rot_v, const uint8_t* widths_v, int d, int gs, double scale,
+                               double pos0, double theta, double* out, double* lse) {
+  double* khat = (double*)malloc(sizeof(double) * (size_t)n * d);
+  double* vhat = (double*)malloc(sizeof(double) * (size_t)n * d);
+  double* s = (double*)malloc(sizeof(double) * (size_t)n);
+  spo_decode_unit_rope(cache_k, stride_k, n, w_dec_k, mean_rot_k, widths_k, d, gs, SPO_SIDE_K, pos0, theta, khat);
+  spo_decode_unit(cache_v, stride_v, n, w_dec_v, mean_rot_v, widths_v, d, gs, SPO_SIDE_V, NULL, vhat);
+  for (int h = 0; h < G; h++) {
+    double mx = -INFINITY;
+    for (int64_t t = 0; t < n; t++) {
+      double acc = 0.0;
+      for (int i = 0; i < d; i++) acc += q[h * d + i] * khat[t * d + i];
+      s[t] = acc * scale;
+      if (s[t] > mx) mx = s[t];
+    }
+    double l = 0.0;
+    for (int64_t t = 0; t < n; t++) { s[t] = exp(s[t] - mx); l += s[t]; }
+    for (int i = 0; i < d; i++) {
+      double acc = 0.0;
+      for (int64_t t = 0; t < n; t++) acc += s[t] * vhat[t * d + i];
+      out[h * d + i] = acc / l;
+    }
+    if (lse) lse[h] = mx + log(l);
+  }
+  free(khat); free(vhat); free(s);
+}
+
+/* Mode B with RoPE: no K-hat is formed.  The rotation is orthogonal, so q . R(p) k-hat = (R(-p) q) . k-hat: per
+ * token the query is rotated back by the token's position and folded through W_dec,K, q'_t = scale W_dec,K R(-p_t) q;
+ * the score is q'_t . (yhat_t + m'_K).  The value side is that of spo_attention_mode_b. */
+void spo_attention_rope_mode_b(const double* q, int G, const uint8_t* cache_k, int64_t stride_k,
+                               const uint8_t* cache_v, int64_t stride_v, int64_t n, const float* w_dec_k,
+                               const float* mean_rot_k, const uint8_t* widths_k, const float* w_dec_v,
+                               const float* mean_rot_v, const uint8_t* widths_v, int d, int gs, double scale,
+                               double pos0, double theta, double* out, double* lse) {
+  float* yk = (float*)malloc(sizeof(float) * (size_t)n * d);
+  float* yv = (float*)malloc(sizeof(float) * (size_t)n * d);
+  double* s = (double*)malloc(sizeof(double) * (size_t)n);
+  spo_decode_unit(cache_k, stride_k, n, w_dec_k, mean_rot_k, widths_k, d, gs, SPO_SIDE_K, yk, NULL);
+  spo_decode_unit(cache_v, stride_v, n, w_dec_v, mean_rot_v, widths_v, d, gs, SPO_SIDE_V, yv, NULL);
+  for (int h = 0; h < G; h++) {
+    double qr[SPO_MAX_D], qp[SPO_MAX_D], op[SPO_MAX_D];
+    double mx = -INFINITY;
+    for (int64_t t = 0; t < n; t++) {
+      for (int i = 0; i < d; i++) qr[i] = q[h * d + i];
+      spo_rope_row(qr, d, -(pos0 + (double)t), theta);
+      double acc_s = 0.0;
+      for (int j = 0; j < d; j++) {
+        double acc = 0.0;
+        for (int i = 0; i < d; i++) acc += (double)w_dec_k[(int64_t)j * d + i] * qr[i];
+        qp[j] = acc * scale;
+        acc_s += qp[j] * ((double)yk[t * d + j] + (double)mean_rot_k[j]);
+      }
+      s[t] = acc_s;
       if (s[t] > mx) mx = s[t];
     }
     double l = 0.0;

@@ -385,3 +385,64 @@ def test_key_value_budget_split():
         bits_k, bits_v = 16 * 128 / rk, 16 * 128 / rv
         assert abs(bits_k + bits_v - 2 * 16 * 128 / 8.0) < 1e-9
         assert abs(bits_k / (bits_k + bits_v) - kappa) < 1e-12
+
+
+# ----------------------------------------------------------------------------- rotary position embedding
+
+def test_rope_rows_against_closed_forms():
+    """The position rotation of Sec. 3.3 (applied to the reconstructed key): position 0 is the identity; d = 4 at
+    position 1 with theta = 10000 rotates the pair (x0, x2) by 1 rad and (x1, x3) by 0.01 rad (hand values); norms are
+    kept; and (R(a) q) . (R(b) k) depends on a - b only."""
+    x = np.array([[1.0, 2.0, 3.0, 4.0]])
+    assert np.array_equal(codec.rope_rows(x, 0, 10000.0), x)
+    y = codec.rope_rows(np.array([[1.0, 2.0, 3.0, 4.0], [1.0, 2.0, 3.0, 4.0]]), 0, 10000.0)[1]
+    want = [1 * math.cos(1.0) - 3 * math.sin(1.0), 2 * math.cos(0.01) - 4 * math.sin(0.01),
+            3 * math.cos(1.0) + 1 * math.sin(1.0), 4 * math.cos(0.01) + 2 * math.sin(0.01)]
+    assert np.abs(y - want).max() <= 1e-15
+    rng = np.random.default_rng(2)
+    q, k = rng.standard_normal((1, 128)), rng.standard_normal((1, 128))
+    for a, b in ((5, 3), (1005, 1003), (77, 75)):
+        ra = codec.rope_rows(q, a, 500000.0)[0]
+        rb = codec.rope_rows(k, b, 500000.0)[0]
+        assert abs(np.linalg.norm(ra) - np.linalg.norm(q)) <= 1e-12
+        if a == 5:
+            first = ra @ rb
+        assert abs(ra @ rb - first) <= 1e-9
+
+
+@pytest.mark.parametrize("gain_mode", [fit.GAIN_SQRT, fit.GAIN_WHITEN])
+def test_rope_latent_attention_equals_reconstruct_rotate_attend(gain_mode):
+    """With RoPE, Mode A (reconstruct the key, rotate it at its position, attend: Sec. 3.3) and the latent-space form
+    (rotate the query back per token and fold it through W_dec,K: the appendix's q' with the position rotation moved
+    to the query side) agree to 1e-10; without positions (theta large, all angles ~ 0 at pos0 = 0 for a tiny n) both
+    fall back to the plain functions; and the rotated reconstruction equals the rotation of the plain one."""
+    n = 200
+    c = _coded_tiny(6.0, gain_mode, n)
+    k, v = c["k"], c["v"]
+    q = si.draw_queries(si.WORKLOADS["tiny"], 0, 0).astype(np.float64)
+    theta, pos0 = 500000.0, 1234.0
+    q_rot = np.stack([codec.rope_rows(q[h][None], pos0 + n, theta)[0] for h in range(q.shape[0])])
+    args = (n, k["cache"], k["tb"], v["cache"], v["tb"], k["wd"], k["mr"], k["widths"], v["wd"], v["mr"], v["widths"], 64,
+            1.0 / np.sqrt(128.0), pos0, theta)
+    oa, la = codec.attention_rope_unit("A", q_rot, *args)
+    ob, lb = codec.attention_rope_unit("B", q_rot, *args)
+    assert np.abs(oa - ob).max() <= 1e-10 * np.abs(oa).max() and np.abs(la - lb).max() <= 1e-10
+    # the rotated reconstruction = rotation of the plain reconstruction; a dense check of Mode A on top of it
+    _, k_hat = codec.decode_unit(k["cache"], k["tb"], n, k["wd"], k["mr"], k["widths"], 64, codec.SIDE_K)
+    _, v_hat = codec.decode_unit(v["cache"], v["tb"], n, v["wd"], v["mr"], v["widths"], 64, codec.SIDE_V)
+    k_rot = codec.decode_unit_rope(k["cache"], k["tb"], n, k["wd"], k["mr"], k["widths"], 64, codec.SIDE_K, pos0, theta)
+    assert np.abs(k_rot - codec.rope_rows(k_hat, pos0, theta)).max() == 0.0
+    s = q_rot @ k_rot.T / np.sqrt(128.0)
+    p = np.exp(s - s.max(axis=1, keepdims=True))
+    p /= p.sum(axis=1, keepdims=True)
+    assert np.abs(oa - p @ v_hat).max() <= 1e-12 * np.abs(oa).max()
+    # relative positions only: shifting every position (query included) by the same amount changes nothing
+    q_rot2 = np.stack([codec.rope_rows(q[h][None], pos0 + 977 + n, theta)[0] for h in range(q.shape[0])])
+    oa2, _ = codec.attention_rope_unit("A", q_rot2, *args[:-2], pos0 + 977, theta)
+    assert np.abs(oa2 - oa).max() <= 1e-9 * np.abs(oa).max()
+    # and with all angles zero (position 0 only matters through pos * theta^..: use n = 1 at pos0 = 0)
+    o1, l1 = codec.attention_rope_unit("B", q, 1, *args[1:-2], 0.0, theta)
+    o0, l0 = codec.attention_units("B", q[None], [1], k["cache"], [0], [k["tb"]], v["cache"], [0], [v["tb"]],
+                                   k["wd"][None], k["mr"][None], k["widths"][None], v["wd"][None], v["mr"][None],
+                                   v["widths"][None], 64, 1.0 / np.sqrt(128.0))
+    assert np.abs(o1 - o0[0]).max() <= 1e-13 and np.abs(l1 - l0[0]).max() <= 1e-13
