@@ -227,6 +227,24 @@ int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, co
                    int64_t table_stride, int32_t* status_word, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * spectra_decode_rope -- Sec. 3.3: the latent is taken before the rotary position embedding, and the position
+ * rotation is applied to the key after its reconstruction.  spectra_decode for keys (tensor-core kernel) with that
+ * rotation in its epilogue: channels i and i + d/2 of token t of unit u are rotated by the angle of position
+ * position0[u] + t.  rope_cos, rope_sin: device fp32 [n_positions, d / 2], cos and sin of position * frequency_i
+ * (the tables a model keeps anyway), 16-byte aligned, n_positions > the largest position touched.  position0: device
+ * int32 [n_units] or NULL (all zero).  Other arguments as in spectra_decode (out must not be NULL).  The fused
+ * latent-space attention does not take positions: q . R(p) k-hat = (R(-p) q) . k-hat makes the folded query depend on
+ * the token, so a latent-space score needs the full d x d lift per token; callers with rotary models reconstruct
+ * (this call) and attend, as the paper's Mode A does.
+ */
+int spectra_decode_rope(const spectra_config* cfg, const uint8_t* cache, const int64_t* unit_offset, int64_t n_units,
+                        int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens, const float* w_dec,
+                        const float* mean_rot, const uint8_t* widths, void* out, int out_dtype, int64_t stride_unit,
+                        int64_t stride_token, const int32_t* tile_table, int64_t table_stride,
+                        const int32_t* position0, const float* rope_cos, const float* rope_sin, int32_t* status_word,
+                        void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * spectra_decode_attention -- appendix "Latent-space attention and memory" (Mode B): one decode query per
  * (sequence, query head) attends to the whole coded cache of its kv-head without reconstructing it:
  *     q' = softmax_scale * W_dec,K q      (the up-projection folded into the query, once per call)

@@ -27,7 +27,7 @@ EXPORTS = [
     "spectra_fit_basis", "spectra_fit_basis_static", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
     "spectra_decode_attention", "spectra_decode_step", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
     "spectra_total_bits", "spectra_status_string", "spectra_cache_bytes", "spectra_attention_path",
-    "spectra_alloc_bits_pooled", "spectra_split_ratio",
+    "spectra_alloc_bits_pooled", "spectra_split_ratio", "spectra_decode_rope",
 ]
 
 
@@ -204,6 +204,20 @@ def decode(cfg, side, cache, unit_offset, n_units, n_param_sets, n_tokens, max_t
                               C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(tile_table), C.c_int64(table_stride),
                               _ptr(status_word), _stream())
     _check(rc, "spectra_decode")
+
+
+def decode_rope(cfg, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec, mean_rot, widths, out,
+                stride_unit, stride_token, rope_cos, rope_sin, position0=None, status_word=None, tile_table=None,
+                table_stride=0):
+    """Reconstructs keys and applies the rotary position embedding (rotate-half pairing) from cos / sin tables
+    [positions, 64]; position0: device int32 [n_units] (None: 0)."""
+    rc = lib().spectra_decode_rope(C.byref(cfg), _ptr(cache), _ptr(unit_offset), C.c_int64(n_units),
+                                   C.c_int64(n_param_sets), _ptr(n_tokens), C.c_int32(max_tokens), _ptr(w_dec),
+                                   _ptr(mean_rot), _ptr(widths), _ptr(out), C.c_int(_dtype_code(out)),
+                                   C.c_int64(stride_unit), C.c_int64(stride_token), _ptr(tile_table),
+                                   C.c_int64(table_stride), _ptr(position0), _ptr(rope_cos), _ptr(rope_sin),
+                                   _ptr(status_word), _stream())
+    _check(rc, "spectra_decode_rope")
 
 
 def decode_attention(cfg, q, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k, cache_v,

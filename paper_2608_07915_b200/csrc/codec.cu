@@ -330,11 +330,13 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
   return launch_status();
 }
 
-extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
-                              int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
-                              const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out,
-                              int out_dtype, float* yhat_out, int64_t stride_unit, int64_t stride_token,
-                              const int32_t* tile_table, int64_t table_stride, int32_t* status_word, void* stream) {
+namespace {
+int decode_impl(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset, int64_t n_units,
+                int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens, const float* w_dec,
+                const float* mean_rot, const uint8_t* widths, void* out, int out_dtype, float* yhat_out,
+                int64_t stride_unit, int64_t stride_token, const int32_t* tile_table, int64_t table_stride,
+                const int32_t* rope_pos0, const float* rope_cos, const float* rope_sin, int32_t* status_word,
+                void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   if ((side != SPECTRA_SIDE_K && side != SPECTRA_SIDE_V) || n_units < 0 || max_tokens < 0 || n_param_sets < 1 ||
@@ -348,7 +350,8 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
   if (out && !w_dec) return SPECTRA_INVALID_ARG;
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
-               out_dtype, yhat_out, stride_unit, stride_token, status_word, TileMap{tile_table, table_stride}};
+               out_dtype, yhat_out, stride_unit, stride_token, status_word, TileMap{tile_table, table_stride},
+               rope_cos, rope_sin, rope_pos0};
   if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05), persistent grid
     const size_t dec_smem = sizeof(DecodeTcSmem) + 128;
     if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem) !=
@@ -368,4 +371,28 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
   dim3 grid((unsigned)((max_tokens + kTile - 1) / kTile), (unsigned)n_units);
   decode_kernel<<<grid, 128, sizeof(CodecSmem), (cudaStream_t)stream>>>(a);
   return launch_status();
+}
+}  // namespace
+
+extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
+                              int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
+                              const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out,
+                              int out_dtype, float* yhat_out, int64_t stride_unit, int64_t stride_token,
+                              const int32_t* tile_table, int64_t table_stride, int32_t* status_word, void* stream) {
+  return decode_impl(cfg, side, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec, mean_rot, widths,
+                     out, out_dtype, yhat_out, stride_unit, stride_token, tile_table, table_stride, nullptr, nullptr,
+                     nullptr, status_word, stream);
+}
+
+extern "C" int spectra_decode_rope(const spectra_config* cfg, const uint8_t* cache, const int64_t* unit_offset,
+                                   int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
+                                   const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out,
+                                   int out_dtype, int64_t stride_unit, int64_t stride_token, const int32_t* tile_table,
+                                   int64_t table_stride, const int32_t* position0, const float* rope_cos,
+                                   const float* rope_sin, int32_t* status_word, void* stream) {
+  if (!out || !rope_cos || !rope_sin) return SPECTRA_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(rope_cos) | reinterpret_cast<uintptr_t>(rope_sin)) & 15) return SPECTRA_INVALID_ARG;
+  return decode_impl(cfg, SPECTRA_SIDE_K, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec,
+                     mean_rot, widths, out, out_dtype, nullptr, stride_unit, stride_token, tile_table, table_stride,
+                     position0, rope_cos, rope_sin, status_word, stream);
 }

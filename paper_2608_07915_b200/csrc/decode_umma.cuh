@@ -36,6 +36,9 @@ struct DecodeArgs {
   const int32_t* n_tokens; const float* w_dec; const float* mean_rot; const uint8_t* widths;
   void* out; int out_dtype; float* yhat_out; int64_t stride_unit, stride_token;
   int32_t* status; TileMap map;
+  // rotary position embedding of the reconstructed vectors (NULL tables: none): cos and sin of position * frequency,
+  // [positions, d / 2] fp32, and the position of each unit's token 0 (NULL: 0)
+  const float* rope_cos; const float* rope_sin; const int32_t* rope_pos0;
 };
 
 struct DecodeTcSmem {
@@ -280,6 +283,60 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
         ok = um_wait(um_smem_u32(&S.acc_full[hf]), (uint32_t)(i & 1));
         if (!ok) { status |= SPECTRA_STATUS_WAIT_TIMEOUT; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (p.rope_cos) {
+          // Sec. 3.3: the position rotation is applied to the reconstructed key.  Channels i and i + 64 are a pair; any
+          // thread of a token's lane can read all of its columns, so this thread takes pairs 32 (ch0 / 64) .. + 31:
+          // 16 at a time, both halves, rotated by the angle of the token's position, stored as two pieces.
+          const uint32_t lane_acc = tb + 128u * hf + ((uint32_t)((warp & 3) * 32) << 16);
+          const int i0 = ch0 >> 1;
+          const int64_t pos = (int64_t)(p.rope_pos0 ? p.rope_pos0[u] : 0) + tile_pos + t;
+#pragma unroll 1
+          for (int part = 0; part < 2; part++) {
+            float ylo[16], yhi[16];
+            um_ld16(lane_acc + i0 + 16 * part, ylo); um_ld16(lane_acc + 64 + i0 + 16 * part, yhi);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (live) {
+              const float4* cs = reinterpret_cast<const float4*>(p.rope_cos + pos * (kD / 2) + i0 + 16 * part);
+              const float4* sn = reinterpret_cast<const float4*>(p.rope_sin + pos * (kD / 2) + i0 + 16 * part);
+#pragma unroll
+              for (int c = 0; c < 4; c++) {
+                const float4 cv = cs[c], sv = sn[c];
+                const float cc[4] = {cv.x, cv.y, cv.z, cv.w}, ss[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                  const float a = ylo[4 * c + e], b = yhi[4 * c + e];
+                  ylo[4 * c + e] = a * cc[e] - b * ss[e];
+                  yhi[4 * c + e] = b * cc[e] + a * ss[e];
+                }
+              }
+#pragma unroll
+              for (int half = 0; half < 2; half++) {
+                const float* y = half ? yhi : ylo;
+                const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + t) * p.stride_token + 64 * half + i0 + 16 * part;
+                const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out) + (uintptr_t)o * (p.out_dtype == SPECTRA_BF16 ? 2 : 4);
+                if ((addr & 15) == 0 && p.out_dtype == SPECTRA_BF16) {
+                  uint4* dst = reinterpret_cast<uint4*>(addr);
+#pragma unroll
+                  for (int c = 0; c < 2; c++) {
+                    __nv_bfloat162 h[4];
+#pragma unroll
+                    for (int e = 0; e < 4; e++) h[e] = __floats2bfloat162_rn(y[8 * c + 2 * e], y[8 * c + 2 * e + 1]);
+                    dst[c] = *reinterpret_cast<const uint4*>(h);
+                  }
+                } else if ((addr & 15) == 0) {
+                  float4* dst = reinterpret_cast<float4*>(addr);
+#pragma unroll
+                  for (int c = 0; c < 4; c++) dst[c] = make_float4(y[4 * c], y[4 * c + 1], y[4 * c + 2], y[4 * c + 3]);
+                } else {
+#pragma unroll
+                  for (int c = 0; c < 16; c++) store_from_float(p.out, p.out_dtype, o + c, y[c]);
+                }
+              }
+            }
+          }
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          continue;
+        }
         const uint32_t acc = tb + 128u * hf + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)ch0;
 #pragma unroll 1
         for (int part = 0; part < 2; part++) {

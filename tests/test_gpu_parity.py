@@ -1036,3 +1036,38 @@ def test_paper_structure_allocation_end_to_end(sp):
                                    V["params"].m_rot, V["params"].widths, 64, 1.0 / np.sqrt(128.0))
     assert H.rel_err_per_vector(got[0].reshape(Hk, G, 128), ref) <= TOL
     assert np.abs(lse[0].reshape(Hk, G) - lref).max() <= 2e-3
+
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+def test_reconstruction_with_rotary_positions_matches_oracle(sp, dt):
+    """Sec. 3.3, Mode A: keys are reconstructed and then rotated at their positions.  spectra_decode_rope against the
+    oracle's reconstruct-then-rotate, two units with different starting positions, ragged length."""
+    wl, S = _tiny_setup(sp, 8.0)
+    cfg = sp.default_config()
+    s = S["k"]
+    params = s["params"]
+    n, theta = 900, 500000.0
+    pos0 = np.array([0, 4000], np.int32)
+    ref_cache = np.zeros(s["total"], np.uint8)
+    H.oracle_encode(params, si.SIDE_K, s["X"][None, :n], [0], ref_cache, s["off"])
+    tb = int(params.tile_bytes[0])
+    want = [oc.decode_unit_rope(ref_cache, tb, n, params.w_dec[0], params.m_rot[0], params.widths[0], 64, si.SIDE_K,
+                                float(p0), theta) for p0 in pos0]
+    n_pos = int(pos0.max()) + 1024
+    ang = np.arange(n_pos, dtype=np.float64)[:, None] * theta ** (-2.0 * np.arange(64, dtype=np.float64) / 128.0)[None]
+    cos_t, sin_t = H.to_dev(np.cos(ang).astype(np.float32)), H.to_dev(np.sin(ang).astype(np.float32))
+    dp = H.dev_params(params)
+    cache2 = H.to_dev(np.concatenate([ref_cache, ref_cache]))
+    off2 = H.to_dev(np.array([0, ref_cache.size], np.int64))
+    tdt = torch.float32 if dt == "f32" else torch.bfloat16
+    out = torch.full((2, 1024, 128), 7.0, dtype=tdt, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sp.decode_rope(cfg, cache2, off2, 2, 1, torch.tensor([n, n - 100], dtype=torch.int32, device="cuda"), n, dp["w_dec"],
+                   dp["m_rot"], dp["widths"], out, 1024 * 128, 128, cos_t, sin_t, H.to_dev(pos0), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    tol = TOL if dt == "f32" else TOL + 2.0 ** -8
+    got = out.float().cpu().numpy()
+    assert H.rel_err_per_vector(got[0, :n], want[0]) <= tol
+    assert H.rel_err_per_vector(got[1, :n - 100], want[1][:n - 100]) <= tol
+    assert (got[0, n:] == 7.0).all() and (got[1, n - 100:] == 7.0).all()
