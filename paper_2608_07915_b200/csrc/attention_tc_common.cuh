@@ -254,6 +254,7 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
   const int ps = (int)(u % p.n_param_sets);
   const int G = min(kFastGqa, p.gqa - h0);                          // query heads of this pass
   // ---- all reads, issued together
+  const int64_t off_k = p.off_k[u], off_v = p.off_v[u];             // used at the very end: fetched with the first group
   const uint32_t wbar = smem_u32(&S.wbar);
   if (tid == 0) {
     mbar_init(wbar, 1);
@@ -427,14 +428,14 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
   int vblocks[4];
 #pragma unroll
   for (int c = 0; c < 4; c++) vblocks[c] = (TV.class_first[c + 1] - TV.class_first[c] + 15) >> 4;
-  const unsigned long long addr_k = (unsigned long long)(p.cache_k + p.off_k[u]), addr_v = (unsigned long long)(p.cache_v + p.off_v[u]);
+  const unsigned long long addr_k = (unsigned long long)(p.cache_k + off_k), addr_v = (unsigned long long)(p.cache_v + off_v);
   const bool ok = fast_layout_ok(TK.tile_bytes, TV.tile_bytes, vblocks, ent_base[8], addr_k, addr_v, f.slot_k, f.slot_v, f.max_vblocks);
   if (tid == 64) {
     D.tbk = ok ? TK.tile_bytes : 16; D.tbv = ok ? TV.tile_bytes : 16;
     D.kmeta[0] = ok ? TK.meta_off[0] : -1; D.kmeta[1] = ok ? TK.meta_off[1] : -1;
     D.vmeta[0] = ok ? TV.meta_off[0] : -1; D.vmeta[1] = ok ? TV.meta_off[1] : -1;
     D.n_vstrips = ok ? TV.n_strips : 0; D.pad0 = 0;
-    D.src_k = ok ? p.off_k[u] : 0; D.src_v = ok ? p.off_v[u] : 0;
+    D.src_k = ok ? off_k : 0; D.src_v = ok ? off_v : 0;
     if (!ok && p.status) atomicOr(p.status, SPECTRA_STATUS_BAD_LAYOUT);
   }
   if (!ok) {
