@@ -157,29 +157,23 @@ __device__ __forceinline__ void k_run(const unsigned char* ktile, uint32_t run, 
   if (nch == 0) return;
   const unsigned char* pa = ktile + (run & 0xffffu) * 16 + 32 * W * tig + 4 * W * gid;
   const int lone_i = (run >> 27) & 1u ? nch - 1 : -1;
-  uint32_t xa[W], xb[W];
-  ld_tile_words<W>(pa, xa);
-  ld_tile_words<W>(pa + 128 * W, xb);
 #pragma unroll 1
-  for (int i = 0; i < nch; i++) {
-    pa += 256 * W;
+  for (int i = 0; i < nch; i++, pa += 256 * W) {
+    uint32_t xa[W], xb[W];
+    ld_tile_words<W>(pa, xa);
+    ld_tile_words<W>(pa + 128 * W, xb);
     kb += 64;
-    uint32_t ya[W], yb[W];
-    ld_tile_words<W>(pa, ya);                 // the next chunk's words (whatever follows the run if this is its last)
-    ld_tile_words<W>(pa + 128 * W, yb);
     if (i == lone_i) {
       // the pair in slot `slot` of this chunk is one strip stored alone: the threads of that slot re-read it as
       // half-words (all threads load, a select keeps the result where it belongs)
       const int slot = (int)(run >> 24) & 7;
       uint32_t t[W];
-      ld_lone_words<W>(pa - 256 * W - 32 * W * tig - 4 * W * gid + 32 * W * slot + 2 * W * gid, t);
+      ld_lone_words<W>(pa - 32 * W * tig - 4 * W * gid + 32 * W * slot + 2 * W * gid, t);
       const bool mine_a = tig == slot, mine_b = tig + 4 == slot;
 #pragma unroll
       for (int k = 0; k < W; k++) { xa[k] = mine_a ? t[k] : xa[k]; xb[k] = mine_b ? t[k] : xb[k]; }
     }
     k_chunk<W>(xa, xb, b01, b23, kb, acc);
-#pragma unroll
-    for (int k = 0; k < W; k++) { xa[k] = ya[k]; xb[k] = yb[k]; }
   }
 }
 
@@ -236,27 +230,23 @@ __device__ __forceinline__ void v_class(const unsigned char* vtile, uint32_t cls
   const unsigned char* px = vtile + (cls >> 16) * 16 + 4 * W * tig + 16 * W * gid;
   const int nb = (n + 15) >> 4;
   const bool rescale = alpha != 1.f;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  if (!FRESH) tmem_get(col, acc);
 #pragma unroll 1
   for (int bi = 0; bi < nb; bi++, px += 256 * W, col += 4) {
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    if (!FRESH) tmem_get(col, acc);
     uint32_t xa[W], xb[W];
     ld_tile_words<W>(px, xa);
     ld_tile_words<W>(px + 128 * W, xb);
-    float nxt[4] = {0.f, 0.f, 0.f, 0.f};
     if (!FRESH) {
       tmem_wait_ld();
       if (rescale) {
 #pragma unroll
         for (int e = 0; e < 4; e++) acc[e] *= alpha;
       }
-      if (bi + 1 < nb) tmem_get(col + 4, nxt);             // the next block's accumulators come while this one multiplies
     }
     v_block_half<W, 0>(xa, xb, pw[0], acc);
     v_block_half<W, 1>(xa, xb, pw[1], acc);
     tmem_put(col, acc);
-#pragma unroll
-    for (int e = 0; e < 4; e++) acc[e] = nxt[e];
   }
 }
 template <bool FRESH>
