@@ -201,43 +201,80 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int kWarps = kPrepThreads / 32;
   if (bid == f.n_units) {
-    // ---- tile prefix sums over units and each worker warp's first unit
+    // ---- tile prefix sums over units and each worker warp's first unit.  One round of global reads (the lengths);
+    // counts, scan and the searches stay in shared memory when the call has at most 4096 units.
     const int n_units = f.n_units;
-    for (int b = tid; b < p.batch; b += kPrepThreads)
-      if (p.seq_len[b] > p.max_seq_len && p.status) atomicOr(p.status, SPECTRA_STATUS_CAPACITY);
-    const int per = (n_units + 127) / 128;
-    int local = 0;
-    if (tid < 128) {
-      for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (attended_tokens(p, (i / f.npass) / p.n_kv) + kTile - 1) / kTile;
-      S.scan[tid] = local;
-    }
-    __syncthreads();
-    if (tid == 0) {
-      int run = 0;
-      for (int i = 0; i < 128; i++) { const int v = S.scan[i]; S.scan[i] = run; run += v; }
-      f.tile_prefix[n_units] = run;
-    }
-    __syncthreads();
-    if (tid < 128) {
-      int run = S.scan[tid];
-      for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) {
-        f.tile_prefix[i] = run;
-        run += (attended_tokens(p, (i / f.npass) / p.n_kv) + kTile - 1) / kTile;
-      }
-    }
-    __syncthreads();
-    __threadfence_block();
     __shared__ int sprefix[4097];          // units of one call; larger calls search the global copy
     const bool in_smem = n_units <= 4096;
-    if (in_smem)
-      for (int i = tid; i <= n_units; i += kPrepThreads) sprefix[i] = f.tile_prefix[i];
-    __syncthreads();
+    const int per = (n_units + 127) / 128;
+    bool over = false;                     // a sequence longer than the buffers hold: reported, attended as empty
+    if (in_smem) {
+      for (int i = tid; i < n_units; i += kPrepThreads) {
+        const int n = p.seq_len[(i / f.npass) / p.n_kv];
+        over |= n > p.max_seq_len;
+        sprefix[i + 1] = n > p.max_seq_len ? 0 : (n + kTile - 1) / kTile;
+      }
+      if (tid == 0) sprefix[0] = 0;
+      __syncthreads();
+      if (tid < 128) {
+        int local = 0;
+        for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += sprefix[i + 1];
+        S.scan[tid] = local;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int run = 0;
+        for (int i = 0; i < 128; i++) { const int v = S.scan[i]; S.scan[i] = run; run += v; }
+      }
+      __syncthreads();
+      if (tid < 128) {
+        int run = S.scan[tid];
+        for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) { run += sprefix[i + 1]; sprefix[i + 1] = run; }
+      }
+      __syncthreads();
+      for (int i = tid; i <= n_units; i += kPrepThreads) f.tile_prefix[i] = sprefix[i];
+    } else {
+      for (int b = tid; b < p.batch; b += kPrepThreads) over |= p.seq_len[b] > p.max_seq_len;
+      int local = 0;
+      if (tid < 128) {
+        for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) local += (attended_tokens(p, (i / f.npass) / p.n_kv) + kTile - 1) / kTile;
+        S.scan[tid] = local;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int run = 0;
+        for (int i = 0; i < 128; i++) { const int v = S.scan[i]; S.scan[i] = run; run += v; }
+        f.tile_prefix[n_units] = run;
+      }
+      __syncthreads();
+      if (tid < 128) {
+        int run = S.scan[tid];
+        for (int i = tid * per; i < min((tid + 1) * per, n_units); i++) {
+          f.tile_prefix[i] = run;
+          run += (attended_tokens(p, (i / f.npass) / p.n_kv) + kTile - 1) / kTile;
+        }
+      }
+      __syncthreads();
+      __threadfence_block();
+    }
+    if (over && p.status) atomicOr(p.status, SPECTRA_STATUS_CAPACITY);
     const int* pre = in_smem ? sprefix : f.tile_prefix;
     const long long total = pre[n_units];
     // each worker warp's share of the flattened tile space: first unit with a tile of the share, first tile inside
     // that unit, tiles of that unit, tiles of the share
+    // floor(gw * total / W) without 64-bit divisions: total = q W + r, so it is gw q + floor(gw r / W); gw and r are
+    // below 2^16 whenever W is (the grids of this library are), else the plain form is used
+    const unsigned Wn = (unsigned)f.total_warps;
+    const unsigned tq = (unsigned)(total / Wn), tr = (unsigned)(total % Wn);
+    const bool small = Wn < 65536u;
     for (int gw = tid; gw < f.total_warps; gw += kPrepThreads) {
-      const long long g0 = (long long)gw * total / f.total_warps, g1 = (long long)(gw + 1) * total / f.total_warps;
+      long long g0, g1;
+      if (small) {
+        g0 = (long long)((unsigned)gw * tq) + ((unsigned)gw * tr) / Wn;
+        g1 = (long long)((unsigned)(gw + 1) * tq) + ((unsigned)(gw + 1) * tr) / Wn;
+      } else {
+        g0 = (long long)gw * total / f.total_warps; g1 = (long long)(gw + 1) * total / f.total_warps;
+      }
       int lo = 0, hi = n_units;             // first unit whose end is beyond g0
       while (lo < hi) {
         const int mid = (lo + hi) >> 1;
