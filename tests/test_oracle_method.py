@@ -446,3 +446,54 @@ def test_rope_latent_attention_equals_reconstruct_rotate_attend(gain_mode):
                                    k["wd"][None], k["mr"][None], k["widths"][None], v["wd"][None], v["mr"][None],
                                    v["widths"][None], 64, 1.0 / np.sqrt(128.0))
     assert np.abs(o1 - o0[0]).max() <= 1e-13 and np.abs(l1 - l0[0]).max() <= 1e-13
+
+
+# ---------------------------------------------------------------- many-query (prefill) attention, Mode A
+def test_prefill_on_the_handworked_case():
+    """Sec. 3.3, Mode A with a chunk of queries: query i sits at position pos0 + i and attends tokens 0 .. pos0 + i.
+    On the hand-worked cache (three tokens, pos0 = 1, two new queries): the first query sees two tokens, the second
+    all three.  With q = 0 the outputs are the plain means of the reconstructed values it may see; the second head
+    repeats the single-query case's scores 0.125, -0.625, -0.4375."""
+    from oracle import prefill
+    d, gs, k, v, k_hat, v_hat = _handworked_case()
+    q1 = [0.5, -0.25, 0, 1, 0, 0.125, 0, -0.0625]
+    q = np.array([[[0.0] * 8, q1], [[0.0] * 8, q1]])              # [n_new = 2, G = 2, d]
+    out, lse = prefill.prefill_mode_a(q, 1, k["cache"], k["tb"], v["cache"], v["tb"], k["wd"], k["m"], k["widths"],
+                                      v["wd"], v["m"], v["widths"], gs, 0.5)
+    assert np.abs(out[0, 0] - (v_hat[0] + v_hat[1]) / 2).max() <= 1e-14 and abs(lse[0, 0] - math.log(2.0)) <= 1e-14
+    assert np.abs(out[1, 0] - (v_hat[0] + v_hat[1] + v_hat[2]) / 3).max() <= 1e-14
+    e = [math.exp(0.125), math.exp(-0.625), math.exp(-0.4375)]
+    want0 = (e[0] * v_hat[0] + e[1] * v_hat[1]) / (e[0] + e[1])
+    want1 = (e[0] * v_hat[0] + e[1] * v_hat[1] + e[2] * v_hat[2]) / sum(e)
+    assert np.abs(out[0, 1] - want0).max() <= 1e-14 and abs(lse[0, 1] - math.log(e[0] + e[1])) <= 1e-14
+    assert np.abs(out[1, 1] - want1).max() <= 1e-14 and abs(lse[1, 1] - math.log(sum(e))) <= 1e-14
+
+
+def test_prefill_rows_equal_single_query_attention_at_their_lengths():
+    """Row i of the chunked computation is the single-query Mode A attention (the C oracle, pinned above) over the
+    first pos0 + i + 1 tokens: the causal limit is per row, off by one in neither direction."""
+    from oracle import prefill
+    n, pos0 = 300, 250
+    c = _coded_tiny(4.0, fit.GAIN_SQRT, n)
+    k, v = c["k"], c["v"]
+    rng = np.random.default_rng(5)
+    q = rng.standard_normal((n - pos0, 4, 128))
+    scale = 1.0 / np.sqrt(128.0)
+    out, lse = prefill.prefill_mode_a(q, pos0, k["cache"], k["tb"], v["cache"], v["tb"], k["wd"], k["mr"], k["widths"],
+                                      v["wd"], v["mr"], v["widths"], 64, scale)
+    for i in (0, 1, 5, 6, 49):                                     # 256 tokens (a tile edge) is row 5
+        oa, la = _attend(c, q[i], "A", pos0 + i + 1)
+        assert np.abs(out[i] - oa[0]).max() <= 1e-12 * max(1.0, np.abs(oa).max())
+        assert np.abs(lse[i] - la[0]).max() <= 1e-12
+
+
+def test_bf16_rounding_helper():
+    """Round to nearest, ties to even, on the 16 bits below bfloat16's mantissa."""
+    from oracle import prefill
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -7, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8 + 2.0 ** -20), 0.0,
+                  3.0e-5])
+    r = prefill.round_bf16(x)
+    # halfway cases go to the even mantissa: 1 + 2^-8 -> 1, 1 + 3 * 2^-8 -> 1 + 2^-6; just above halfway rounds away
+    assert r[0] == 1.0 and r[1] == 1.0 and r[2] == 1.0 + 2.0 ** -7 and r[3] == 1.0 + 2.0 ** -6
+    assert r[4] == -(1.0 + 2.0 ** -7) and r[5] == 0.0
+    assert abs(r[6] - 3.0e-5) <= 3.0e-5 * 2.0 ** -9
