@@ -245,6 +245,51 @@ int spectra_decode_rope(const spectra_config* cfg, const uint8_t* cache, const i
                         void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * spectra_decode_paged -- Sec. 3.3 (Mode A): reconstruction into a pool of pages of 128 tokens, the form a paged
+ * attention kernel reads.  out_pool: device, out_dtype SPECTRA_F32 or SPECTRA_BF16; token slot s (0..127) of tile t of
+ * unit u goes to out_pool[out_table[u * out_table_stride + t] * stride_page + s * stride_token + i], i = 0..d-1.
+ * out_table: device int32 [n_units, out_table_stride], out_table_stride >= ceil(max_tokens / 128) (SPECTRA_INVALID_ARG
+ * otherwise); the caller guarantees that every page index lies inside the pool.  It may be the same table as
+ * tile_table (the pages of the coded cache; NULL: contiguous).  Only tokens below n_tokens[u] are written.  rope_cos,
+ * rope_sin, position0: as in spectra_decode_rope, both tables NULL for no position rotation (keys only:
+ * SPECTRA_INVALID_ARG with side V).  Other arguments as in spectra_decode.
+ */
+int spectra_decode_paged(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
+                         int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
+                         const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out_pool, int out_dtype,
+                         int64_t stride_page, int64_t stride_token, const int32_t* tile_table, int64_t table_stride,
+                         const int32_t* out_table, int64_t out_table_stride, const int32_t* position0,
+                         const float* rope_cos, const float* rope_sin, int32_t* status_word, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * spectra_prefill_attention -- Sec. 3.3 (Mode A, reconstruct then attend) for a chunk of new queries: causal
+ * softmax attention of n_new queries per sequence over the reconstructed cache.  Query i of sequence b sits at
+ * position pos0[b] + i and attends tokens 0 .. pos0[b] + i; the pools must hold the reconstruction of all
+ * pos0[b] + n_new tokens (spectra_encode the chunk, then spectra_decode_paged both sides).  head_dim 128, bf16.
+ *   q, out    device bf16, element (b, i, h, c) at [b * stride_seq + i * stride_token + h * stride_head + c],
+ *             h = 0 .. n_q_heads - 1 (query head h uses KV head h / (n_q_heads / n_kv_heads)); 16-byte aligned,
+ *             strides multiples of 8 elements
+ *   k_pool, v_pool   device bf16 pools of n_pages pages [128 tokens][d]: token slot s of page g at
+ *             [g * stride_page + s * stride_token]; 16-byte aligned, strides multiples of 8 elements
+ *   page_table       device int32 [n_seqs * n_kv_heads, table_stride]: page of tile t of unit (b, kv head); NULL: the
+ *             page is unit * table_stride + t (table_stride = pages per unit, >= 1)
+ *   pos0      device int32 [n_seqs]; n_new: host value, the same for every sequence
+ *   scale     softmax scale (> 0), usually 1 / sqrt(d)
+ *   lse       device fp32 [n_seqs, n_new, n_q_heads] or NULL: natural logarithm of the sum of exp(scale q.k)
+ * Products run on the tensor cores with bf16 operands (probabilities are rounded to bf16 before P V, the row sum
+ * uses the rounded values) and fp32 accumulation.  Slots of the last page past the sequence's end may hold anything.
+ * status_word: SPECTRA_STATUS_WAIT_TIMEOUT if a bounded wait gave up (the output is then invalid).
+ * Returns SPECTRA_INVALID_ARG for NULL or misaligned arguments, SPECTRA_UNSUPPORTED if the grid would not fit.
+ */
+int spectra_prefill_attention(const void* q, const void* k_pool, const void* v_pool, int64_t n_pages,
+                              int64_t stride_page, int64_t stride_token, const int32_t* page_table,
+                              int64_t table_stride, int64_t n_seqs, int32_t n_kv_heads, int32_t n_q_heads,
+                              const int32_t* pos0, int32_t n_new, int64_t q_stride_seq, int64_t q_stride_token,
+                              int64_t q_stride_head, float scale, void* out, int64_t out_stride_seq,
+                              int64_t out_stride_token, int64_t out_stride_head, float* lse, int32_t* status_word,
+                              void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * spectra_decode_attention -- appendix "Latent-space attention and memory" (Mode B): one decode query per
  * (sequence, query head) attends to the whole coded cache of its kv-head without reconstructing it:
  *     q' = softmax_scale * W_dec,K q      (the up-projection folded into the query, once per call)

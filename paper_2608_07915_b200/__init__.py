@@ -27,7 +27,7 @@ EXPORTS = [
     "spectra_fit_basis", "spectra_fit_basis_static", "spectra_fit_workspace_bytes", "spectra_alloc_bits", "spectra_encode", "spectra_decode",
     "spectra_decode_attention", "spectra_decode_step", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
     "spectra_total_bits", "spectra_status_string", "spectra_cache_bytes", "spectra_attention_path",
-    "spectra_alloc_bits_pooled", "spectra_split_ratio", "spectra_decode_rope",
+    "spectra_alloc_bits_pooled", "spectra_split_ratio", "spectra_decode_rope", "spectra_decode_paged", "spectra_prefill_attention",
 ]
 
 
@@ -218,6 +218,34 @@ def decode_rope(cfg, cache, unit_offset, n_units, n_param_sets, n_tokens, max_to
                                    C.c_int64(table_stride), _ptr(position0), _ptr(rope_cos), _ptr(rope_sin),
                                    _ptr(status_word), _stream())
     _check(rc, "spectra_decode_rope")
+
+
+def decode_paged(cfg, side, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec, mean_rot, widths,
+                 out_pool, stride_page, stride_token, out_table, out_table_stride, tile_table=None, table_stride=0,
+                 position0=None, rope_cos=None, rope_sin=None, status_word=None):
+    """Reconstruction into a pool of 128-token pages: tile t of unit u goes to page out_table[u, t] (device int32)."""
+    rc = lib().spectra_decode_paged(C.byref(cfg), C.c_int(side), _ptr(cache), _ptr(unit_offset), C.c_int64(n_units),
+                                    C.c_int64(n_param_sets), _ptr(n_tokens), C.c_int32(max_tokens), _ptr(w_dec),
+                                    _ptr(mean_rot), _ptr(widths), _ptr(out_pool), C.c_int(_dtype_code(out_pool)),
+                                    C.c_int64(stride_page), C.c_int64(stride_token), _ptr(tile_table),
+                                    C.c_int64(table_stride), _ptr(out_table), C.c_int64(out_table_stride),
+                                    _ptr(position0), _ptr(rope_cos), _ptr(rope_sin), _ptr(status_word), _stream())
+    _check(rc, "spectra_decode_paged")
+
+
+def prefill_attention(q, k_pool, v_pool, n_pages, stride_page, stride_token, page_table, table_stride, n_seqs,
+                      n_kv_heads, n_q_heads, pos0, n_new, q_strides, softmax_scale, out, out_strides, lse=None,
+                      status_word=None):
+    """Causal attention of n_new queries per sequence over reconstructed bf16 page pools.  q_strides, out_strides:
+    (sequence, token, head) strides in elements."""
+    rc = lib().spectra_prefill_attention(_ptr(q), _ptr(k_pool), _ptr(v_pool), C.c_int64(n_pages),
+                                         C.c_int64(stride_page), C.c_int64(stride_token), _ptr(page_table),
+                                         C.c_int64(table_stride), C.c_int64(n_seqs), C.c_int32(n_kv_heads),
+                                         C.c_int32(n_q_heads), _ptr(pos0), C.c_int32(n_new), C.c_int64(q_strides[0]),
+                                         C.c_int64(q_strides[1]), C.c_int64(q_strides[2]), C.c_float(softmax_scale),
+                                         _ptr(out), C.c_int64(out_strides[0]), C.c_int64(out_strides[1]),
+                                         C.c_int64(out_strides[2]), _ptr(lse), _ptr(status_word), _stream())
+    _check(rc, "spectra_prefill_attention")
 
 
 def decode_attention(cfg, q, batch, n_kv_heads, n_q_heads, seq_len, max_seq_len, cache_k, unit_offset_k, cache_v,

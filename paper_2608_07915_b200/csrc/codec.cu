@@ -5,6 +5,7 @@
 #include "encode_append.cuh"
 #include "encode_umma.cuh"
 #include "decode_umma.cuh"
+#include "tensor_map.cuh"
 
 namespace spectra {
 
@@ -228,45 +229,13 @@ __global__ void __launch_bounds__(128, 1) decode_kernel(DecodeArgs p) {
   __syncthreads();
   for (int idx = tid; idx < n_here * kD; idx += blockDim.x) {
     const int tt = idx / kD, i = idx - tt * kD;
-    store_from_float(p.out, p.out_dtype, (int64_t)u * p.stride_unit + (int64_t)(tile_pos + tt) * p.stride_token + i,
-                     S.y[tt * kLdY + i]);
+    store_from_float(p.out, p.out_dtype, p.out_index(u, tile, tt) + i, S.y[tt * kLdY + i]);
   }
 }
 
 }  // namespace spectra
 
 using namespace spectra;
-
-namespace {
-
-// Tensor map over the bf16 input of a bulk encode: dimensions (channel, token, unit), box 8 channels x 128 tokens, no
-// swizzle, zeros outside.  The driver's encoder is looked up through the runtime (no link against the driver library).
-bool make_token_map(CUtensorMap* map, const void* x, int64_t n_tokens, int64_t n_units, int64_t stride_token,
-                    int64_t stride_unit) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static EncodeFn fn = nullptr;
-  if (!fn) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym ||
-        q != cudaDriverEntryPointSuccess)
-      return false;
-    fn = reinterpret_cast<EncodeFn>(sym);
-  }
-  if (n_tokens < 1 || n_units < 1) return false;
-  const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)n_tokens, (cuuint64_t)n_units};
-  // a single unit or token leaves its stride unused; the encoder still wants a legal value
-  const cuuint64_t strides[2] = {(cuuint64_t)(stride_token > 0 ? stride_token : kD) * 2,
-                                 (cuuint64_t)(stride_unit > 0 ? stride_unit : n_tokens * kD) * 2};
-  const cuuint32_t box[3] = {8, (cuuint32_t)kTile, 1}, estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-}  // namespace
 
 extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dtype, int flags,
                               int64_t n_units, int64_t n_param_sets, const int32_t* pos0, int32_t n_new,
@@ -335,8 +304,8 @@ int decode_impl(const spectra_config* cfg, int side, const uint8_t* cache, const
                 int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens, const float* w_dec,
                 const float* mean_rot, const uint8_t* widths, void* out, int out_dtype, float* yhat_out,
                 int64_t stride_unit, int64_t stride_token, const int32_t* tile_table, int64_t table_stride,
-                const int32_t* rope_pos0, const float* rope_cos, const float* rope_sin, int32_t* status_word,
-                void* stream) {
+                const int32_t* rope_pos0, const float* rope_cos, const float* rope_sin, const int32_t* out_table,
+                int64_t out_table_stride, int32_t* status_word, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   if ((side != SPECTRA_SIDE_K && side != SPECTRA_SIDE_V) || n_units < 0 || max_tokens < 0 || n_param_sets < 1 ||
@@ -351,7 +320,7 @@ int decode_impl(const spectra_config* cfg, int side, const uint8_t* cache, const
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
                out_dtype, yhat_out, stride_unit, stride_token, status_word, TileMap{tile_table, table_stride},
-               rope_cos, rope_sin, rope_pos0};
+               rope_cos, rope_sin, rope_pos0, TileMap{out_table, out_table_stride}};
   if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05), persistent grid
     const size_t dec_smem = sizeof(DecodeTcSmem) + 128;
     if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem) !=
@@ -381,7 +350,7 @@ extern "C" int spectra_decode(const spectra_config* cfg, int side, const uint8_t
                               const int32_t* tile_table, int64_t table_stride, int32_t* status_word, void* stream) {
   return decode_impl(cfg, side, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec, mean_rot, widths,
                      out, out_dtype, yhat_out, stride_unit, stride_token, tile_table, table_stride, nullptr, nullptr,
-                     nullptr, status_word, stream);
+                     nullptr, nullptr, 0, status_word, stream);
 }
 
 extern "C" int spectra_decode_rope(const spectra_config* cfg, const uint8_t* cache, const int64_t* unit_offset,
@@ -394,5 +363,21 @@ extern "C" int spectra_decode_rope(const spectra_config* cfg, const uint8_t* cac
   if ((reinterpret_cast<uintptr_t>(rope_cos) | reinterpret_cast<uintptr_t>(rope_sin)) & 15) return SPECTRA_INVALID_ARG;
   return decode_impl(cfg, SPECTRA_SIDE_K, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec,
                      mean_rot, widths, out, out_dtype, nullptr, stride_unit, stride_token, tile_table, table_stride,
-                     position0, rope_cos, rope_sin, status_word, stream);
+                     position0, rope_cos, rope_sin, nullptr, 0, status_word, stream);
+}
+
+extern "C" int spectra_decode_paged(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
+                                    int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,
+                                    const float* w_dec, const float* mean_rot, const uint8_t* widths, void* out_pool,
+                                    int out_dtype, int64_t stride_page, int64_t stride_token, const int32_t* tile_table,
+                                    int64_t table_stride, const int32_t* out_table, int64_t out_table_stride,
+                                    const int32_t* position0, const float* rope_cos, const float* rope_sin,
+                                    int32_t* status_word, void* stream) {
+  if (!out_pool || !out_table || out_table_stride < (max_tokens + kTile - 1) / kTile) return SPECTRA_INVALID_ARG;
+  if ((rope_cos == nullptr) != (rope_sin == nullptr)) return SPECTRA_INVALID_ARG;
+  if (rope_cos && side != SPECTRA_SIDE_K) return SPECTRA_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(rope_cos) | reinterpret_cast<uintptr_t>(rope_sin)) & 15) return SPECTRA_INVALID_ARG;
+  return decode_impl(cfg, side, cache, unit_offset, n_units, n_param_sets, n_tokens, max_tokens, w_dec, mean_rot, widths,
+                     out_pool, out_dtype, nullptr, stride_page, stride_token, tile_table, table_stride, position0,
+                     rope_cos, rope_sin, out_table, out_table_stride, status_word, stream);
 }

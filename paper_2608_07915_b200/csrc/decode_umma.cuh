@@ -39,6 +39,13 @@ struct DecodeArgs {
   // rotary position embedding of the reconstructed vectors (NULL tables: none): cos and sin of position * frequency,
   // [positions, d / 2] fp32, and the position of each unit's token 0 (NULL: 0)
   const float* rope_cos; const float* rope_sin; const int32_t* rope_pos0;
+  // paged output (table != NULL): token slot t of tile `tile` of unit u goes to page omap.page(u, tile) of a pool whose
+  // pages are stride_unit elements apart; otherwise unit u's tokens are stride_token apart from u * stride_unit on
+  TileMap omap;
+  __device__ __forceinline__ int64_t out_index(int64_t u, int tile, int t) const {
+    return omap.table ? omap.page(u, tile) * stride_unit + (int64_t)t * stride_token
+                      : u * stride_unit + ((int64_t)tile * kTile + t) * stride_token;
+  }
 };
 
 struct DecodeTcSmem {
@@ -312,7 +319,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
 #pragma unroll
               for (int half = 0; half < 2; half++) {
                 const float* y = half ? yhi : ylo;
-                const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + t) * p.stride_token + 64 * half + i0 + 16 * part;
+                const int64_t o = p.out_index(u, tile, t) + 64 * half + i0 + 16 * part;
                 const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out) + (uintptr_t)o * (p.out_dtype == SPECTRA_BF16 ? 2 : 4);
                 if ((addr & 15) == 0 && p.out_dtype == SPECTRA_BF16) {
                   uint4* dst = reinterpret_cast<uint4*>(addr);
@@ -344,7 +351,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
           um_ld16(acc + 32 * part, y); um_ld16(acc + 32 * part + 16, y + 16);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
           if (live) {
-            const int64_t o = (int64_t)u * p.stride_unit + (int64_t)(tile_pos + t) * p.stride_token + ch0 + 32 * part;
+            const int64_t o = p.out_index(u, tile, t) + ch0 + 32 * part;
             const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out) + (uintptr_t)o * (p.out_dtype == SPECTRA_BF16 ? 2 : 4);
             if ((addr & 15) == 0 && p.out_dtype == SPECTRA_BF16) {
               uint4* dst = reinterpret_cast<uint4*>(addr);

@@ -1,0 +1,160 @@
+"""GPU parity of the many-query path (Sec. 3.3, Mode A for a chunk of queries): reconstruction into paged bf16 pools
+(spectra_decode_paged) and causal attention over them (spectra_prefill_attention), against oracle/prefill.py.
+
+Tolerances.  The kernel reads bf16 keys and values (the storage the reconstruction is written in), rounds the
+probabilities to bf16 before P V, normalises with the sum of the rounded values and rounds the output to bf16:
+  * against the oracle run on bf16-rounded reconstructions, a weight's relative error is at most 2^-8 (two bf16
+    roundings, of its probability and through the sum) and the output's rounding adds 2^-9 of its size; errors of
+    independent tokens do not add up coherently, so 1e-2 of a vector's largest entry bounds what remains (measured:
+    a few 1e-3), and lse, which only sees the sum, stays within 5e-3;
+  * against the oracle on unrounded (fp64) reconstructions the bf16 storage itself enters: 2^-9 per key entry moves a
+    score by up to about 1e-2, hence 3e-2 on outputs and lse.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import spectra_inputs as si
+from oracle import codec as oc
+from oracle import prefill as opf
+from tests import helpers as H
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL_SAME_STORAGE = 1e-2
+TOL_LSE = 5e-3
+TOL_F64_STORAGE = 3e-2
+
+
+@pytest.fixture(scope="module")
+def sp():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a GPU")
+    import paper_2608_07915_b200 as sp_
+    sp_.lib()
+    return sp_
+
+
+def _setup(n_seq, kv_lens, ratio=4.0):
+    base = si.WORKLOADS["llama1"]
+    wl = dataclasses.replace(base, kv_heads=2, q_heads=2 * base.group, n_fit=512)
+    n_tok = max(kv_lens)
+    S = {}
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        X = H.draw_units(wl, 0, side, n_seq, max(n_tok, 512))
+        params = H.fit_params([X[h][:512] for h in range(wl.kv_heads)], ratio)
+        n_units = n_seq * wl.kv_heads
+        off, total = H.cache_layout(params, n_units, n_tok)
+        cache = np.zeros(total, np.uint8)
+        for u in range(n_units):
+            p = u % wl.kv_heads
+            one = H.Params(params.w_enc[[p]], params.w_dec[[p]], params.m_rot[[p]], params.widths[[p]], 64)
+            H.oracle_encode(one, side, X[u][None, :kv_lens[u // wl.kv_heads]], [0], cache[off[u]:], np.zeros(1, np.int64))
+        S[name] = dict(params=params, off=off, cache=cache)
+    return wl, S
+
+
+def _paged_reconstruction(sp, wl, S, n_seq, kv_lens, rng, fill):
+    """Both sides into bf16 pools through one shuffled page table; unused slots keep `fill`."""
+    cfg = sp.default_config()
+    n_units = n_seq * wl.kv_heads
+    max_len = max(kv_lens)
+    tiles = (max_len + 127) // 128
+    n_pages = n_units * tiles + 3
+    table = rng.permutation(n_pages)[:n_units * tiles].astype(np.int32).reshape(n_units, tiles)
+    table_d = H.to_dev(table)
+    n_tok_d = H.to_dev(np.array([kv_lens[u // wl.kv_heads] for u in range(n_units)], np.int32))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    pools = {}
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        s = S[name]
+        dp = H.dev_params(s["params"])
+        pool = torch.full((n_pages, 128, 128), fill, dtype=torch.bfloat16, device="cuda")
+        sp.decode_paged(cfg, side, H.to_dev(s["cache"]), H.to_dev(s["off"]), n_units, wl.kv_heads, n_tok_d, max_len,
+                        dp["w_dec"], dp["m_rot"], dp["widths"], pool, 128 * 128, 128, table_d, tiles,
+                        status_word=status)
+        pools[name] = pool
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return pools, table, table_d, tiles, n_pages
+
+
+def test_paged_reconstruction_matches_oracle(sp):
+    """spectra_decode_paged: every token lands in the page its table names, at its slot; nothing else is written."""
+    n_seq, kv_lens = 2, [350, 227]
+    wl, S = _setup(n_seq, kv_lens, 8.0)
+    pools, table, _, tiles, n_pages = _paged_reconstruction(sp, wl, S, n_seq, kv_lens, np.random.default_rng(1), 7.0)
+    for side, name in ((si.SIDE_K, "k"), (si.SIDE_V, "v")):
+        s = S[name]
+        got = pools[name].float().cpu().numpy()
+        written = np.zeros((n_pages, 128), bool)
+        for u in range(n_seq * wl.kv_heads):
+            p, n = u % wl.kv_heads, kv_lens[u // wl.kv_heads]
+            _, want = oc.decode_unit(s["cache"][s["off"][u]:], int(s["params"].tile_bytes[p]), n, s["params"].w_dec[p],
+                                     s["params"].m_rot[p], s["params"].widths[p], 64, side)
+            for t in range((n + 127) // 128):
+                m = min(128, n - 128 * t)
+                assert H.rel_err_per_vector(got[table[u, t], :m], want[128 * t:128 * t + m]) <= 2e-3 + 2.0 ** -8
+                written[table[u, t], :m] = True
+        assert (got[~written] == 7.0).all()
+
+
+@pytest.mark.parametrize("pos0,n_new", [([200, 77], 150), ([0], 1000), ([1000], 1), ([127, 128], 129)])
+def test_prefill_attention_matches_oracle(sp, pos0, n_new):
+    """Causal attention of a chunk of queries over the paged reconstruction against the oracle's Mode A, per row.
+    The pools start as NaN: slots past a sequence's end must not reach any output."""
+    n_seq = len(pos0)
+    kv_lens = [p + n_new for p in pos0]
+    wl, S = _setup(n_seq, kv_lens)
+    rng = np.random.default_rng(3)
+    pools, table, table_d, tiles, n_pages = _paged_reconstruction(sp, wl, S, n_seq, kv_lens, rng, float("nan"))
+    Hq, G = wl.q_heads, wl.group
+    q = (rng.standard_normal((n_seq, n_new, Hq, 128)) * 1.5).astype(np.float32)
+    q_d = H.to_dev(q).to(torch.bfloat16)
+    q_used = q_d.float().cpu().numpy().astype(np.float64)          # the queries are bf16 inputs: both sides read these
+    out = torch.full((n_seq, n_new, Hq, 128), 5.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros((n_seq, n_new, Hq), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scale = 1.0 / np.sqrt(128.0)
+    strides = (n_new * Hq * 128, Hq * 128, 128)
+    sp.prefill_attention(q_d, pools["k"], pools["v"], n_pages, 128 * 128, 128, table_d, tiles, n_seq, wl.kv_heads, Hq,
+                         H.to_dev(np.array(pos0, np.int32)), n_new, strides, scale, out, strides, lse, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = out.float().cpu().numpy()
+    got_lse = lse.cpu().numpy()
+    assert np.isfinite(got).all() and np.isfinite(got_lse).all()
+    K, V = S["k"], S["v"]
+    worst = worst64 = 0.0
+    for b in range(n_seq):
+        for kh in range(wl.kv_heads):
+            u = b * wl.kv_heads + kh
+            args = (q_used[b, :, kh * G:(kh + 1) * G], pos0[b], K["cache"][K["off"][u]:], int(K["params"].tile_bytes[kh]),
+                    V["cache"][V["off"][u]:], int(V["params"].tile_bytes[kh]), K["params"].w_dec[kh], K["params"].m_rot[kh],
+                    K["params"].widths[kh], V["params"].w_dec[kh], V["params"].m_rot[kh], V["params"].widths[kh], 64, scale)
+            ref, lref = opf.prefill_mode_a(*args, storage="bf16")
+            ref64, lref64 = opf.prefill_mode_a(*args, storage="f64")
+            g = got[b, :, kh * G:(kh + 1) * G]
+            worst = max(worst, H.rel_err_per_vector(g, ref))
+            worst64 = max(worst64, H.rel_err_per_vector(g, ref64))
+            assert np.abs(got_lse[b, :, kh * G:(kh + 1) * G] - lref).max() <= TOL_LSE
+            assert np.abs(got_lse[b, :, kh * G:(kh + 1) * G] - lref64).max() <= TOL_F64_STORAGE
+    assert worst <= TOL_SAME_STORAGE, worst
+    assert worst64 <= TOL_F64_STORAGE, worst64
+
+
+def test_prefill_attention_argument_checks(sp):
+    q = torch.zeros((1, 4, 2, 128), dtype=torch.bfloat16, device="cuda")
+    pool = torch.zeros((2, 128, 128), dtype=torch.bfloat16, device="cuda")
+    pos = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = (4 * 2 * 128, 2 * 128, 128)
+    with pytest.raises(sp.SpectraError):       # three query heads over two KV heads
+        sp.prefill_attention(q, pool, pool, 2, 128 * 128, 128, None, 1, 1, 2, 3, pos, 4, st, 0.1, q, st)
+    with pytest.raises(sp.SpectraError):       # a token stride that is not a multiple of 8 elements
+        sp.prefill_attention(q, pool, pool, 2, 128 * 128, 132, None, 1, 1, 2, 2, pos, 4, st, 0.1, q, st)
+    with pytest.raises(sp.SpectraError):       # no table and no pages-per-unit
+        sp.prefill_attention(q, pool, pool, 2, 128 * 128, 128, None, 0, 1, 2, 2, pos, 4, st, 0.1, q, st)
+    sp.prefill_attention(q, pool, pool, 2, 128 * 128, 128, None, 1, 0, 2, 2, pos, 4, st, 0.1, q, st)   # nothing to do
+    torch.cuda.synchronize()
