@@ -28,7 +28,7 @@ extern "C" int spectra_prefill_attention(const void* q, const void* k_pool, cons
        stride_token) & 7)
     return SPECTRA_INVALID_ARG;
   if (stride_token < kD || stride_page < stride_token) return SPECTRA_INVALID_ARG;
-  const int n_qblocks = (n_new + kTile - 1) / kTile;
+  const int n_qblocks = (n_new + kPfRows - 1) / kPfRows;
   const long long grid = (long long)n_qblocks * n_q_heads * n_seqs;
   if (grid > 0x7fffffffLL) return SPECTRA_UNSUPPORTED;
   CUtensorMap kmap, vmap;
