@@ -32,14 +32,14 @@ extern "C" int spectra_prefill_attention(const void* q, const void* k_pool, cons
   const long long grid = (long long)n_qblocks * n_q_heads * n_seqs;
   if (grid > 0x7fffffffLL) return SPECTRA_UNSUPPORTED;
   CUtensorMap kmap, vmap;
-  if (!make_token_map(&kmap, k_pool, kTile, n_pages, stride_token, stride_page) ||
-      !make_token_map(&vmap, v_pool, kTile, n_pages, stride_token, stride_page))
+  if (!make_token_map(&kmap, k_pool, kTile, n_pages, stride_token, stride_page, kPfSwizzle) ||
+      !make_token_map(&vmap, v_pool, kTile, n_pages, stride_token, stride_page, kPfSwizzle))
     return SPECTRA_CUDA_ERROR;
   PrefillArgs a{reinterpret_cast<const __nv_bfloat16*>(q), reinterpret_cast<__nv_bfloat16*>(out), lse,
                 q_stride_seq, q_stride_token, q_stride_head, out_stride_seq, out_stride_token, out_stride_head,
                 pos0, n_new, (int)n_seqs, n_kv_heads, n_q_heads / n_kv_heads, scale * 1.4426950408889634f,
                 page_table, table_stride, status_word, n_qblocks};
-  const size_t smem = sizeof(PrefillSmem) + 128;
+  const size_t smem = sizeof(PrefillSmem) + 1024;
   if (cudaFuncSetAttribute(prefill_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return SPECTRA_CUDA_ERROR;
   prefill_attention_kernel<<<(unsigned)grid, kPfThreads, smem, (cudaStream_t)stream>>>(a, kmap, vmap);

@@ -37,9 +37,18 @@ constexpr uint32_t kUmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | 
 // so a warp that waits long (the producer) does not spend issue slots on polling.
 __device__ __forceinline__ bool um_wait(uint32_t bar, uint32_t parity) {
   uint32_t done = 0;
+#ifdef UM_WAIT_SPIN
+  for (int it = 0; it < (1 << 26) && !done; ++it)
+    asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+#else
+#ifndef UM_WAIT_HINT
+#define UM_WAIT_HINT 1000u
+#endif
   for (int it = 0; it < (1 << 21) && !done; ++it)
     asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(done) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+                 : "=r"(done) : "r"(bar), "r"(parity), "r"(UM_WAIT_HINT) : "memory");
+#endif
   return done != 0;
 }
 
