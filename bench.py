@@ -45,6 +45,15 @@ def _peaks():
     return 6650.0, "fallback"
 
 
+def _tensor_peak():
+    """Dense bf16 TFLOP/s of a library GEMM timed alone on this machine (the burst figure), else the fallback."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
+
+
 class ClockSampler:
     """Samples SM clocks and clock-event reasons of one GPU in a background thread (NVML, read-only)."""
 
@@ -413,6 +422,7 @@ def run_ours(args, wl):
         del model, q_dev, nk_dev, nv_dev
         torch.cuda.empty_cache()
         line["other_workloads"] = _other_workloads(args, hbm_gbs)
+        line["prefill_attention"] = _prefill_attention()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         times, th, threads, desc = _oracle_rate(wl, 3, 1)
         line["cpu_baseline"] = {"value": th / float(np.mean(times)) / (wl.layers * wl.kv_heads), "unit": UNIT,
@@ -463,6 +473,44 @@ def _other_workloads(args, hbm_gbs):
         del m, q, nk, nv, o
         torch.cuda.empty_cache()
     return out
+
+
+def _prefill_attention():
+    """The many-query path (reconstruct, then attend): causal attention of one 32768-token chunk over reconstructed
+    bf16 page pools in the Llama-3.1-8B head shape, one layer, timed alone with CUDA events.  The pools hold seeded
+    random values (the kernel's speed does not depend on them); flops are the algorithmic ones of causal attention,
+    4 d per (query, visible token) pair, against the measured dense bf16 peak of a library GEMM."""
+    import torch
+
+    import paper_2608_07915_b200 as sp
+    n_seq, n_new, Hq, Hkv, d = 1, 32768, 32, 8, 128
+    tiles = (n_new + 127) // 128
+    n_pages = n_seq * Hkv * tiles
+    gen = torch.Generator(device="cuda").manual_seed(99)
+    kp = torch.randn((n_pages, 128, d), generator=gen, device="cuda").to(torch.bfloat16)
+    vp = torch.randn((n_pages, 128, d), generator=gen, device="cuda").to(torch.bfloat16)
+    q = torch.randn((n_seq, n_new, Hq, d), generator=gen, device="cuda").to(torch.bfloat16)
+    out = torch.empty_like(q)
+    pos0 = torch.zeros(n_seq, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    strides = (n_new * Hq * d, Hq * d, d)
+    ms = []
+    for i in range(8):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        sp.prefill_attention(q, kp, vp, n_pages, 128 * d, d, None, tiles, n_seq, Hkv, Hq, pos0, n_new, strides,
+                             1.0 / np.sqrt(d), out, strides, None, status)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            ms.append(e0.elapsed_time(e1))
+    t = float(np.median(ms))
+    flops = 4.0 * d * n_seq * Hq * (n_new * (n_new + 1) // 2)
+    peak, kind = _tensor_peak()
+    return {"workload": f"{n_seq} sequence x {n_new} new tokens, {Hq} query / {Hkv} KV heads, head_dim {d}, bf16 pools",
+            "kernel": "prefill_attention_kernel", "ms": t, "bound": "tensor", "achieved": flops / (t * 1e-3) / 1e12,
+            "peak": peak, "unit": "TFLOP/s", "frac": flops / (t * 1e-3) / 1e12 / peak, "peak_kind": kind,
+            "flops": flops, "status_word": int(status.item())}
 
 
 def main():
