@@ -118,7 +118,7 @@ typedef struct spectra_config {
  * spectra_fit_basis -- Sec. 3.1, Eq. 3-4 and the appendix "G-Weighted SVD", restated on cache vectors:
  * the right singular basis of the whitened weight is the eigenbasis of the uncentred second moment of
  * the produced keys, so per unit-side
- *     C = X^T X / N, mu = mean(X)            (fp32 products, fp64 accumulation)
+ *     C = X^T X / N, mu = mean(X)            (fp32 partial sums over at most 256 tokens, fp64 across them)
  *     C = U diag(lambda) U^T, lambda descending, each eigenvector's largest component positive (fp64 Jacobi)
  *     m = mu U, var_j = max(lambda_j - m_j^2, 0), gains gamma per cfg->gain_mode (floor 1e-12 lambda_1)
  *     W_enc = U diag(gamma), W_dec = diag(1/gamma) U^T, m' = m * gamma,
@@ -128,6 +128,10 @@ typedef struct spectra_config {
  * Outputs (device, fp32): w_enc, w_dec, basis_u [n_units, d, d] row-major; mean_rot, var_alloc, eigval
  *    [n_units, d].  basis_u and eigval may be NULL.
  * workspace: device, at least spectra_fit_workspace_bytes(cfg, n_units) bytes, 16-byte aligned.
+ * bf16 input with a 16-byte aligned x and strides that are multiples of 8 elements forms X^T X on the tensor cores,
+ * one CTA per unit-side with the partial sums added in token order: two calls on the same input give the same bits.
+ * Other inputs use a CUDA-core kernel whose fp64 atomic additions leave the last bits run-dependent.  Should a
+ * bounded wait of the tensor-core kernel give up, that unit's outputs are NaN.
  */
 int spectra_fit_basis(const spectra_config* cfg, const void* x, int x_dtype, int64_t n_units, int64_t n_tokens,
                       int64_t stride_unit, int64_t stride_token, float* w_enc, float* w_dec, float* mean_rot,

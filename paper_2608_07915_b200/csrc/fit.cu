@@ -1,6 +1,8 @@
 // spectra_fit_basis (second-moment accumulation + fp64 Jacobi eigensolver + transform assembly) and
 // spectra_alloc_bits (greedy integer reverse water-filling).
 #include "common.cuh"
+#include "moments_umma.cuh"
+#include "tensor_map.cuh"
 
 namespace spectra {
 
@@ -361,9 +363,24 @@ extern "C" int spectra_fit_basis(const spectra_config* cfg, const void* x, int x
   if (n_units > 65535) return SPECTRA_UNSUPPORTED;
   cudaStream_t st = (cudaStream_t)stream;
   FitWorkspace* ws = reinterpret_cast<FitWorkspace*>(workspace);
-  if (cudaMemsetAsync(ws, 0, sizeof(FitWorkspace) * (size_t)n_units, st) != cudaSuccess) return SPECTRA_CUDA_ERROR;
-  dim3 grid((unsigned)((n_tokens + kMomChunk - 1) / kMomChunk), (unsigned)n_units);
-  moments_kernel<<<grid, 256, 0, st>>>(x, x_dtype, n_tokens, stride_unit, stride_token, ws);
+  // bf16 inputs whose layout a tensor map can describe: X^T X on the tensor cores, one CTA per unit, sums in a fixed
+  // order (reproducible); anything else: the CUDA-core kernel with fp64 atomics
+  CUtensorMap xmap;
+  const bool tensor_path = x_dtype == SPECTRA_BF16 && (reinterpret_cast<uintptr_t>(x) & 15) == 0 && stride_token % 8 == 0 &&
+                           stride_unit % 8 == 0 && n_tokens < (1LL << 31) &&
+                           make_token_map(&xmap, x, n_tokens, n_units, stride_token, stride_unit, true);
+  if (tensor_path) {
+    const size_t smem = sizeof(MomentsSmem) + 1024;
+    if (cudaFuncSetAttribute(moments_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return SPECTRA_CUDA_ERROR;
+    double* base = reinterpret_cast<double*>(ws);
+    moments_umma_kernel<<<(unsigned)n_units, kMuThreads, smem, st>>>(xmap, n_tokens, base, base + kD * kD,
+                                                                     (int64_t)(sizeof(FitWorkspace) / sizeof(double)), nullptr);
+  } else {
+    if (cudaMemsetAsync(ws, 0, sizeof(FitWorkspace) * (size_t)n_units, st) != cudaSuccess) return SPECTRA_CUDA_ERROR;
+    dim3 grid((unsigned)((n_tokens + kMomChunk - 1) / kMomChunk), (unsigned)n_units);
+    moments_kernel<<<grid, 256, 0, st>>>(x, x_dtype, n_tokens, stride_unit, stride_token, ws);
+  }
   if (launch_status()) return SPECTRA_CUDA_ERROR;
   if (cudaFuncSetAttribute(eigen_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(EigSmem)) !=
       cudaSuccess)

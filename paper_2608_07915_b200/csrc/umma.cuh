@@ -52,4 +52,14 @@ __device__ __forceinline__ bool um_wait(uint32_t bar, uint32_t parity) {
   return done != 0;
 }
 
+// shared-memory matrix descriptor, 128-byte swizzle: rows of 128 bytes in groups of 8 (1024 bytes, sbo apart); lbo is
+// the distance between 64-element blocks along M/N of an MN-major operand (unused for K-major)
+__device__ __forceinline__ uint64_t um_desc_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)((lbo >> 4) & 0x3FFF) << 16) | ((uint64_t)((sbo >> 4) & 0x3FFF) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void um_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 }  // namespace spectra

@@ -1071,3 +1071,37 @@ def test_reconstruction_with_rotary_positions_matches_oracle(sp, dt):
     assert H.rel_err_per_vector(got[0, :n], want[0]) <= tol
     assert H.rel_err_per_vector(got[1, :n - 100], want[1][:n - 100]) <= tol
     assert (got[0, n:] == 7.0).all() and (got[1, n - 100:] == 7.0).all()
+
+
+@pytest.mark.parametrize("n_fit", [300, 1000, 4096])
+def test_fit_moments_on_tensor_cores_are_accurate_and_reproducible(sp, n_fit):
+    """bf16 inputs take the tensor-core moments (S = X^T X in fp32 per 256-token chunk, fp64 across chunks, fixed
+    order).  The sums left in the caller's workspace are compared with the fp64 sums of the same bf16 values (Sec. 3.1:
+    the basis is fitted from the second moments of the calibration tokens), for ragged token counts and inputs with a
+    mean; two calls give the same bits."""
+    wl = si.WORKLOADS["llama1"]
+    heads, n_all = 3, 4200
+    X = np.stack([si.draw_unit(wl, 0, h, si.SIDE_K, 0, n_tokens=n_all) for h in range(heads)])
+    X[1] += 0.75                                                     # a unit with a clear mean
+    cfg = sp.default_config()
+    xd = H.to_dev(X).to(torch.bfloat16)
+    Xb = xd.float().cpu().numpy().astype(np.float64)                 # the values the kernel reads
+    f32 = dict(dtype=torch.float32, device="cuda")
+    outs = []
+    for rep in range(2):
+        w_enc, w_dec = (torch.zeros((heads, 128, 128), **f32) for _ in range(2))
+        m_rot, var, lam = (torch.zeros((heads, 128), **f32) for _ in range(3))
+        ws = torch.full((sp.fit_workspace_bytes(cfg, heads),), 0xAB, dtype=torch.uint8, device="cuda")   # dirty
+        sp.fit_basis(cfg, xd, heads, n_fit, n_all * 128, 128, w_enc, w_dec, m_rot, var, lam, None, ws)
+        torch.cuda.synchronize()
+        outs.append((w_enc.cpu().numpy(), lam.cpu().numpy(), ws.cpu().numpy().copy()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    moments = outs[0][2].view(np.float64).reshape(heads, 128 * 128 + 128)
+    for h in range(heads):
+        S_ref = Xb[h, :n_fit].T @ Xb[h, :n_fit]
+        s_ref = Xb[h, :n_fit].sum(axis=0)
+        S = moments[h, :128 * 128].reshape(128, 128)
+        assert np.abs(S - S_ref).max() <= 2e-5 * np.abs(S_ref).max()
+        assert np.abs(moments[h, 128 * 128:] - s_ref).max() <= 1e-5 * max(1.0, np.abs(s_ref).max())
+        ref = ofit.fit_basis(Xb[h, :n_fit], ofit.GAIN_SQRT)
+        assert np.abs(outs[0][1][h] - ref["lam"]).max() <= 2e-6 * ref["lam"][0]
