@@ -77,7 +77,16 @@ int launch_fast_main_as(const AttnArgs& a, const FastArgs& f, int grid, size_t s
   if (cudaFuncSetAttribute(attention_mma_kernel<PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return SPECTRA_CUDA_ERROR;
-  attention_mma_kernel<PAGED><<<grid, kFastWarps * 32, smem, st>>>(a, f);
+  // programmatic dependent launch: the kernel's set-up (barriers, tensor-memory allocation) overlaps the preceding
+  // prep / front kernel; it waits for that kernel's completion before it reads the descriptors
+  cudaLaunchConfig_t lc{};
+  lc.gridDim = dim3((unsigned)grid); lc.blockDim = dim3(kFastWarps * 32);
+  lc.dynamicSmemBytes = smem; lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at; lc.numAttrs = 1;
+  if (cudaLaunchKernelEx(&lc, attention_mma_kernel<PAGED>, a, f) != cudaSuccess) return SPECTRA_CUDA_ERROR;
   return launch_status();
 }
 int launch_fast_main(const AttnArgs& a, const FastArgs& f, int grid, size_t smem, cudaStream_t st) {

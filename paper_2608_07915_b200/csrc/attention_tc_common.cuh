@@ -483,6 +483,9 @@ __device__ inline void attention_prep_body(const AttnArgs& p, const FastArgs& f,
 }
 
 __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p, FastArgs f) {
+  // the main kernel may be scheduled now: its set-up runs beside this grid, and it waits (griddepcontrol.wait) for this
+  // grid's completion before it reads anything written here
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   attention_prep_body(p, f, blockIdx.x);
 }
 
@@ -490,6 +493,7 @@ __global__ void __launch_bounds__(kPrepThreads) attention_prep_kernel(AttnArgs p
 // (the K side first).  The main kernel that follows reads what both parts wrote.
 __global__ void __launch_bounds__(kPrepThreads, 2) decode_step_front_kernel(AttnArgs p, FastArgs f, AppendArgs ak,
                                                                          AppendArgs av, int n_cache_units) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // as in attention_prep_kernel
   const int n_prep = f.n_units + 1;
   if ((int)blockIdx.x < n_prep) { attention_prep_body(p, f, blockIdx.x); return; }
   const int i = blockIdx.x - n_prep;

@@ -352,6 +352,8 @@ __global__ void __launch_bounds__(kFastWarps * 32, kFastCtasPerSm) attention_mma
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t acc_base = tmem_base_s + ((uint32_t)(warp & 3) << 21);   // this warp's lanes 32 * (warp % 4), column 0
 
+  // everything above ran beside the preceding launch (descriptors, appended tokens); from here on its results are read
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel may be scheduled as SMs free up
   const int4 start = f.warp_start[gw];                 // first unit, first tile in it, tiles of that unit, tiles of the share
   const int count = start.w;
