@@ -281,7 +281,7 @@ int spectra_decode_paged(const spectra_config* cfg, int side, const uint8_t* cac
  *   scale     softmax scale (> 0), usually 1 / sqrt(d)
  *   lse       device fp32 [n_seqs, n_new, n_q_heads] or NULL: natural logarithm of the sum of exp(scale q.k)
  * Products run on the tensor cores with bf16 operands (probabilities are rounded to bf16 before P V, the row sum
- * uses the rounded values) and fp32 accumulation.  Slots of the last page past the sequence's end may hold anything.
+ * is taken in fp32 before that rounding) and fp32 accumulation.  Slots of the last page past the sequence's end may hold anything.
  * status_word: SPECTRA_STATUS_WAIT_TIMEOUT if a bounded wait gave up (the output is then invalid).
  * Returns SPECTRA_INVALID_ARG for NULL or misaligned arguments, SPECTRA_UNSUPPORTED if the grid would not fit.
  */

@@ -2,9 +2,9 @@
 (spectra_decode_paged) and causal attention over them (spectra_prefill_attention), against oracle/prefill.py.
 
 Tolerances.  The kernel reads bf16 keys and values (the storage the reconstruction is written in), rounds the
-probabilities to bf16 before P V, normalises with the sum of the rounded values and rounds the output to bf16:
-  * against the oracle run on bf16-rounded reconstructions, a weight's relative error is at most 2^-8 (two bf16
-    roundings, of its probability and through the sum) and the output's rounding adds 2^-9 of its size; errors of
+probabilities to bf16 before P V, normalises with their fp32 sum and rounds the output to bf16:
+  * against the oracle run on bf16-rounded reconstructions, a weight is off by at most 2^-9 relative (the bf16
+    rounding of its probability; the sum is not rounded) and the output's rounding adds 2^-9 of its size; errors of
     independent tokens do not add up coherently, so 1e-2 of a vector's largest entry bounds what remains (measured:
     a few 1e-3), and lse, which only sees the sum, stays within 5e-3;
   * against the oracle on unrounded (fp64) reconstructions the bf16 storage itself enters: 2^-9 per key entry moves a
