@@ -158,3 +158,74 @@ def test_prefill_attention_argument_checks(sp):
         sp.prefill_attention(q, pool, pool, 2, 128 * 128, 128, None, 0, 1, 2, 2, pos, 4, st, 0.1, q, st)
     sp.prefill_attention(q, pool, pool, 2, 128 * 128, 128, None, 1, 0, 2, 2, pos, 4, st, 0.1, q, st)   # nothing to do
     torch.cuda.synchronize()
+
+
+def test_prefill_attention_at_the_benchmarked_size_on_sampled_rows(sp):
+    """The launch bench.py times (one 32768-token chunk, 32 query / 8 KV heads, seeded random bf16 pools): sampled
+    (row, head) outputs against the oracle's causal attention on the same bf16 values, row by row.  Rows at the start,
+    at tile and block edges, in the middle and at the end; every KV group is sampled."""
+    n_new, Hq, Hkv, d = 32768, 32, 8, 128
+    tiles = n_new // 128
+    n_pages = Hkv * tiles
+    gen = torch.Generator(device="cuda").manual_seed(99)
+    kp = torch.randn((n_pages, 128, d), generator=gen, device="cuda").to(torch.bfloat16)
+    vp = torch.randn((n_pages, 128, d), generator=gen, device="cuda").to(torch.bfloat16)
+    q = torch.randn((1, n_new, Hq, d), generator=gen, device="cuda").to(torch.bfloat16)
+    out = torch.empty_like(q)
+    lse = torch.zeros((1, n_new, Hq), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    strides = (n_new * Hq * d, Hq * d, d)
+    scale = 1.0 / np.sqrt(d)
+    sp.prefill_attention(q, kp, vp, n_pages, 128 * d, d, None, tiles, 1, Hkv, Hq, torch.zeros(1, dtype=torch.int32, device="cuda"),
+                         n_new, strides, scale, out, strides, lse, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rows = [0, 1, 127, 128, 255, 256, 257, 4095, 16384, 20000, 32639, 32640, 32767]
+    heads = [0, 5, 10, 15, 17, 22, 27, 31]                          # one per KV group
+    worst = 0.0
+    for h in heads:
+        kh = h // (Hq // Hkv)
+        K = kp[kh * tiles:(kh + 1) * tiles].reshape(-1, d).float().cpu().numpy().astype(np.float64)
+        V = vp[kh * tiles:(kh + 1) * tiles].reshape(-1, d).float().cpu().numpy().astype(np.float64)
+        for i in rows:
+            qi = q[0, i, h].float().cpu().numpy().astype(np.float64)[None, None]
+            ref, lref = opf.causal_attention(qi, K, V, i, scale)
+            got = out[0, i, h].float().cpu().numpy()
+            worst = max(worst, H.rel_err_per_vector(got[None], ref[0]))
+            assert abs(float(lse[0, i, h].item()) - lref[0, 0]) <= TOL_LSE
+    assert worst <= TOL_SAME_STORAGE, worst
+
+
+def test_paged_reconstruction_with_rotary_positions(sp):
+    """spectra_decode_paged with the position rotation of keys (Sec. 3.3: applied after reconstruction), fp32 pages."""
+    n_seq, kv_lens = 1, [300]
+    wl, S = _setup(n_seq, kv_lens, 8.0)
+    cfg = sp.default_config()
+    s = S["k"]
+    n_units, n, theta = wl.kv_heads, 300, 500000.0
+    tiles = 3
+    table = np.array([[4, 0, 2], [1, 5, 3]], np.int32)
+    pos0 = np.array([0, 1000], np.int32)
+    n_pos = 1000 + 384
+    ang = np.arange(n_pos, dtype=np.float64)[:, None] * theta ** (-2.0 * np.arange(64, dtype=np.float64) / 128.0)[None]
+    cos_t, sin_t = H.to_dev(np.cos(ang).astype(np.float32)), H.to_dev(np.sin(ang).astype(np.float32))
+    dp = H.dev_params(s["params"])
+    pool = torch.full((6, 128, 128), 7.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sp.decode_paged(cfg, si.SIDE_K, H.to_dev(s["cache"]), H.to_dev(s["off"]), n_units, wl.kv_heads,
+                    H.to_dev(np.full(n_units, n, np.int32)), n, dp["w_dec"], dp["m_rot"], dp["widths"], pool, 128 * 128, 128,
+                    H.to_dev(table), tiles, position0=H.to_dev(pos0), rope_cos=cos_t, rope_sin=sin_t, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = pool.cpu().numpy()
+    for u in range(n_units):
+        want = oc.decode_unit_rope(s["cache"][s["off"][u]:], int(s["params"].tile_bytes[u]), n, s["params"].w_dec[u],
+                                   s["params"].m_rot[u], s["params"].widths[u], 64, si.SIDE_K, float(pos0[u]), theta)
+        for t in range(tiles):
+            m = min(128, n - 128 * t)
+            assert H.rel_err_per_vector(got[table[u, t], :m], want[128 * t:128 * t + m]) <= 2e-3
+            assert (got[table[u, t], m:] == 7.0).all()
+    with pytest.raises(sp.SpectraError):                              # positions are for keys
+        sp.decode_paged(cfg, si.SIDE_V, H.to_dev(s["cache"]), H.to_dev(s["off"]), n_units, wl.kv_heads,
+                        H.to_dev(np.full(n_units, n, np.int32)), n, dp["w_dec"], dp["m_rot"], dp["widths"], pool, 128 * 128,
+                        128, H.to_dev(table), tiles, rope_cos=cos_t, rope_sin=sin_t)
