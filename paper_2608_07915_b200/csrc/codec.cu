@@ -5,6 +5,7 @@
 #include "encode_append.cuh"
 #include "encode_umma.cuh"
 #include "decode_umma.cuh"
+#include "decode_mma.cuh"
 #include "tensor_map.cuh"
 
 namespace spectra {
@@ -321,6 +322,21 @@ int decode_impl(const spectra_config* cfg, int side, const uint8_t* cache, const
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
                out_dtype, yhat_out, stride_unit, stride_token, status_word, TileMap{tile_table, table_stride},
                rope_cos, rope_sin, rope_pos0, TileMap{out_table, out_table_stride}};
+  const int esz = out_dtype == SPECTRA_BF16 ? 2 : 4;
+  if (out && !yhat_out && (reinterpret_cast<uintptr_t>(out) & (2 * esz - 1)) == 0 && stride_unit % 2 == 0 &&
+      stride_token % 2 == 0) {
+    // reconstruction with the packed fields as tensor-core operands (pairs of outputs are stored together: even strides)
+    const size_t smem = sizeof(DecodeMmaSmem) + 128;
+    if (cudaFuncSetAttribute(decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return SPECTRA_CUDA_ERROR;
+    const int tiles = (int)((max_tokens + kTile - 1) / kTile);
+    const long long n_slots = (long long)tiles * n_units;
+    const int sms = sm_count();
+    if (sms <= 0 || n_slots > 0x7fffffffLL) return SPECTRA_CUDA_ERROR;
+    const unsigned grid = (unsigned)(n_slots < sms ? n_slots : sms);
+    decode_mma_kernel<<<grid, kDmThreads, smem, (cudaStream_t)stream>>>(a, tiles, (int)n_slots);
+    return launch_status();
+  }
   if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05), persistent grid
     const size_t dec_smem = sizeof(DecodeTcSmem) + 128;
     if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem) !=
