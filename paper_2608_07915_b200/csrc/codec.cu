@@ -6,6 +6,7 @@
 #include "encode_umma.cuh"
 #include "decode_umma.cuh"
 #include "decode_mma.cuh"
+#include "decode_pairs.cuh"
 #include "tensor_map.cuh"
 
 namespace spectra {
@@ -325,16 +326,21 @@ int decode_impl(const spectra_config* cfg, int side, const uint8_t* cache, const
   const int esz = out_dtype == SPECTRA_BF16 ? 2 : 4;
   if (out && !yhat_out && (reinterpret_cast<uintptr_t>(out) & (2 * esz - 1)) == 0 && stride_unit % 2 == 0 &&
       stride_token % 2 == 0) {
-    // reconstruction with the packed fields as tensor-core operands (pairs of outputs are stored together: even strides)
-    const size_t smem = sizeof(DecodeMmaSmem) + 128;
-    if (cudaFuncSetAttribute(decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return SPECTRA_CUDA_ERROR;
+    // reconstruction with the packed fields themselves as tensor-core operands: the tcgen05 kernel takes the units it can
+    // hold (up to two scale groups and 192 strip positions), the mma.sync kernel behind it exactly the others
+    // (its outputs are stored in pairs: even strides)
     const int tiles = (int)((max_tokens + kTile - 1) / kTile);
     const long long n_slots = (long long)tiles * n_units;
     const int sms = sm_count();
     if (sms <= 0 || n_slots > 0x7fffffffLL) return SPECTRA_CUDA_ERROR;
     const unsigned grid = (unsigned)(n_slots < sms ? n_slots : sms);
-    decode_mma_kernel<<<grid, kDmThreads, smem, (cudaStream_t)stream>>>(a, tiles, (int)n_slots);
+    const size_t smem_p = sizeof(DecodePairSmem) + 128, smem_m = sizeof(DecodeMmaSmem) + 128;
+    if (cudaFuncSetAttribute(decode_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_p) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_m) != cudaSuccess)
+      return SPECTRA_CUDA_ERROR;
+    decode_pair_kernel<<<grid, kDpThreads, smem_p, (cudaStream_t)stream>>>(a, tiles, (int)n_slots);
+    if (launch_status()) return SPECTRA_CUDA_ERROR;
+    decode_mma_kernel<<<grid, kDmThreads, smem_m, (cudaStream_t)stream>>>(a, tiles, (int)n_slots, 1);
     return launch_status();
   }
   if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05), persistent grid

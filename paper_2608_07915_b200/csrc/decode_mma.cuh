@@ -21,9 +21,6 @@
 // Rows of B that belong to another scale group or lie past the end of a class are zero, and the unit index of such a
 // row is clamped for the load, so nothing is read outside the tile.  All waits are bounded.
 #pragma once
-#ifdef DM_TIMING
-#include <cstdio>
-#endif
 #include "decode_umma.cuh"
 
 namespace spectra {
@@ -43,7 +40,7 @@ struct DecodeMmaSmem {
   alignas(16) float u[kMaxGroups][kD];                // u_g
   alignas(16) float cvec[kD];                         // c
   DmRun run[kMaxGroups][4];
-  int n_ksteps, wexp;
+  int kg[kMaxGroups + 1], wexp;
   float red[16];
   alignas(8) uint64_t full[kDmSlots];
 };
@@ -55,7 +52,79 @@ __device__ __forceinline__ void dm_mma(float (&c)[4], uint32_t a0, uint32_t a1, 
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p, int n_slots_unit, int n_slots) {
+// The (group, class) runs of a unit-side's tile and their k-steps of 16 strips, by all threads of the CTA (ends with a
+// barrier).  Strips of class c whose channel lies in group g are the in-class indices [sa, sb); a K-side unit is a pair
+// of strips, a V-side unit one strip.  kg[g] = first k-step of group g, kg[n_groups..] = the total.
+__device__ inline void dm_build_runs(DmRun (*run)[4], int* kg, const StripTable& T, bool side_v, int gs) {
+  const int tid = threadIdx.x;
+  if (tid < 16) {
+    const int g = tid >> 2, c = tid & 3;
+    DmRun r{0, 0, 0, 0, -1};
+    if (g < T.n_groups) {
+      const int first = T.class_first[c], cnt = T.class_first[c + 1] - first;
+      int sa = 0, sb = 0;
+      for (int k = 0; k < cnt; k++) {
+        const int ch = T.chan[first + k];
+        sa += ch < g * gs;
+        sb += ch < (g + 1) * gs;
+      }
+      r.base = T.class_off[c];
+      if (sb > sa) {
+        if (side_v) { r.first = sa; r.n = sb - sa; }
+        else {
+          r.first = sa >> 1; r.n = ((sb - 1) >> 1) - r.first + 1;
+          if ((cnt & 1) && sb == cnt) r.lone = cnt >> 1;          // the class's odd last strip, stored alone
+        }
+      }
+    }
+    run[g][c] = r;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int ks = 0;
+    const int per = side_v ? 16 : 8;
+    for (int g = 0; g < kMaxGroups; g++) {
+      kg[g] = ks;
+      for (int c = 0; c < 4; c++) {
+        run[g][c].kstep0 = ks;
+        ks += (run[g][c].n + per - 1) / per;
+      }
+    }
+    kg[kMaxGroups] = ks;
+  }
+  __syncthreads();
+}
+
+// Entry (row of k-step ks, output channel nn) of W'' before the fp16 scale: 2^shift W_dec[chan] / L, zero for a row
+// outside its run's group or past the end of its class.
+__device__ inline float dm_b_value(const DmRun (*run)[4], const StripTable& T, const float* __restrict__ wsrc, bool side_v,
+                                   int gs, int ks, int row, int nn) {
+  int g = 0, c = 0;
+#pragma unroll
+  for (int gg = 0; gg < kMaxGroups; gg++)
+#pragma unroll
+    for (int cc = 0; cc < 4; cc++)
+      if (ks >= run[gg][cc].kstep0 && run[gg][cc].n > 0) { g = gg; c = cc; }
+  const DmRun r = run[g][c];
+  const int kk = ks - r.kstep0;
+  const int first = T.class_first[c], cnt = T.class_first[c + 1] - first;
+  const int s_in = side_v ? r.first + 16 * kk + row : 2 * (r.first + 8 * kk + (row >> 1)) + (row & 1);
+  if (s_in >= cnt) return 0.f;
+  const int k = first + s_in, ch = T.chan[k];
+  if (ch < g * gs || ch >= (g + 1) * gs) return 0.f;
+  const float L = (float)((1 << T.width[ch]) - 1);
+  return wsrc[ch * kD + nn] * (float)(1 << T.shift[k]) / L;
+}
+
+// Units the tcgen05 kernel of decode_pairs.cuh takes (the rest is this file's): at most two scale groups, at most
+// twelve k-steps, a tile that fits that kernel's slot, a source the bulk copy accepts.
+constexpr int kDpMaxKsteps = 12;
+__device__ __forceinline__ bool dm_pairs_eligible(const StripTable& T, int n_ksteps, const void* unit_ptr) {
+  return T.n_groups <= 2 && n_ksteps <= kDpMaxKsteps && T.tile_bytes <= kDecRawMax && (reinterpret_cast<uintptr_t>(unit_ptr) & 15) == 0;
+}
+
+// skip_pairs != 0: units that decode_pair_kernel takes are left to it
+__global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p, int n_slots_unit, int n_slots, int skip_pairs) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned char* smem_al = smem_raw + ((128u - (um_smem_u32(smem_raw) & 127u)) & 127u);
   DecodeMmaSmem& S = *reinterpret_cast<DecodeMmaSmem*>(smem_al);
@@ -69,12 +138,6 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   int loads_done = 0;                                    // bulk copies issued so far by this CTA (slot = count % 3)
-#ifdef DM_TIMING
-  long long dt[6] = {0, 0, 0, 0, 0, 0}, dprev = clock64(); int dtiles = 0;
-#define DM_T(i) { const long long tn = clock64(); dt[i] += tn - dprev; dprev = tn; }
-#else
-#define DM_T(i)
-#endif
   int status = 0;
   const int slot_end = (int)((long long)(blockIdx.x + 1) * n_slots / gridDim.x);
 
@@ -93,6 +156,13 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
     const int gs = p.scale_group, n_groups = T.n_groups;
     const int tile_bytes = T.tile_bytes;
     const uint8_t* unit_ptr = p.cache + p.unit_offset[u];
+    dm_build_runs(S.run, S.kg, T, side_v, gs);
+    const int n_ksteps = S.kg[kMaxGroups];
+    if (skip_pairs && dm_pairs_eligible(T, n_ksteps, unit_ptr)) continue;   // the other kernel's unit
+    if (n_ksteps > kDmMaxKsteps) {                       // cannot happen with 128 channels; never index past the table
+      status |= SPECTRA_STATUS_BAD_LAYOUT;
+      continue;
+    }
     // bulk copies need a 16-byte aligned source; a unit that is not is copied by the half's threads, two bytes at a time
     const bool bulk = (reinterpret_cast<uintptr_t>(unit_ptr) & 15) == 0;
     // the first copies go out while the tables are built
@@ -110,29 +180,6 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic reads of the slots are done
       for (int tt = 0; tt < min(n_tiles, kDmSlots); tt++) issue_load(tt);
     }
-    // ---- runs: strips of class c whose channel lies in group g are the in-class indices [sa, sb)
-    if (tid < 16) {
-      const int g = tid >> 2, c = tid & 3;
-      DmRun r{0, 0, 0, 0, -1};
-      if (g < n_groups) {
-        const int first = T.class_first[c], cnt = T.class_first[c + 1] - first;
-        int sa = 0, sb = 0;
-        for (int k = 0; k < cnt; k++) {
-          const int ch = T.chan[first + k];
-          sa += ch < g * gs;
-          sb += ch < (g + 1) * gs;
-        }
-        r.base = T.class_off[c];
-        if (sb > sa) {
-          if (side_v) { r.first = sa; r.n = sb - sa; }
-          else {
-            r.first = sa >> 1; r.n = ((sb - 1) >> 1) - r.first + 1;
-            if ((cnt & 1) && sb == cnt) r.lone = cnt >> 1;          // the class's odd last strip, stored alone
-          }
-        }
-      }
-      S.run[g][c] = r;
-    }
     // ---- largest |W_dec| (the scale that brings W'' into fp16's range)
     {
       float m = 0.f;
@@ -143,14 +190,6 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
     }
     __syncthreads();
     if (tid == 0) {
-      int ks = 0;
-      const int per = side_v ? 16 : 8;
-      for (int g = 0; g < kMaxGroups; g++)
-        for (int c = 0; c < 4; c++) {
-          S.run[g][c].kstep0 = ks;
-          ks += (S.run[g][c].n + per - 1) / per;
-        }
-      S.n_ksteps = ks;
       float m = 0.f;
       for (int i = 0; i < kDmThreads / 32; i++) m = fmaxf(m, S.red[i]);
       int e = 0;
@@ -158,41 +197,13 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
       S.wexp = e;
     }
     __syncthreads();
-    const int n_ksteps = S.n_ksteps;
     const int wexp = S.wexp;
-    if (n_ksteps > kDmMaxKsteps) {                       // cannot happen for 128 channels (host-checked bound); never index past the table
-      status |= SPECTRA_STATUS_BAD_LAYOUT;
-      // drain the copies already issued, then skip the run
-      if (bulk) {
-        for (int tt = 0; tt < min(n_tiles, kDmSlots); tt++) um_wait(um_smem_u32(&S.full[(load_base + tt) % kDmSlots]), (uint32_t)(((load_base + tt) / kDmSlots) & 1));
-        loads_done += min(n_tiles, kDmSlots);
-      }
-      continue;
-    }
     // ---- B table: W'' = 2^shift W_dec[chan] / L * 2^(15 - wexp), zero rows outside a run's group and class
     {
       const float wscale = exp2f((float)(15 - wexp));
       for (int idx = tid; idx < n_ksteps * 16 * kD; idx += kDmThreads) {
         const int nn = idx & (kD - 1), row = (idx >> 7) & 15, ks = idx >> 11;
-        // the run of this k-step
-        int g = 0, c = 0;
-#pragma unroll
-        for (int gg = 0; gg < kMaxGroups; gg++)
-#pragma unroll
-          for (int cc = 0; cc < 4; cc++)
-            if (ks >= S.run[gg][cc].kstep0 && S.run[gg][cc].n > 0) { g = gg; c = cc; }
-        const DmRun r = S.run[g][c];
-        const int kk = ks - r.kstep0;
-        const int first = T.class_first[c], cnt = T.class_first[c + 1] - first;
-        const int s_in = side_v ? r.first + 16 * kk + row : 2 * (r.first + 8 * kk + (row >> 1)) + (row & 1);
-        float v = 0.f;
-        if (s_in < cnt) {
-          const int k = first + s_in, ch = T.chan[k];
-          if (ch >= g * gs && ch < (g + 1) * gs) {
-            const float L = (float)((1 << T.width[ch]) - 1);
-            v = wsrc[ch * kD + nn] * (float)(1 << T.shift[k]) / L * wscale;
-          }
-        }
+        const float v = dm_b_value(S.run, T, wsrc, side_v, gs, ks, row, nn) * wscale;
         const int nb = nn >> 3, ln = (nn & 7) * 4 + ((row & 7) >> 1);
         reinterpret_cast<__half*>(&S.B[ks][nb][ln])[2 * (row >> 3) + (row & 1)] = __float2half_rn(v);
       }
@@ -212,7 +223,6 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
     }
     __syncthreads();
     const float rfac = exp2f((float)(24 - 15 + wexp));   // undoes 2^-24 of the fields and the scale of W''
-    DM_T(0)
 
     // ---- tiles of the run: this half takes tt = hf, hf + 2, ..
     bool ok = true;
@@ -233,7 +243,6 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
                      : "=r"(all) : "r"(mine), "r"(1 + hf), "n"(kDmHalf) : "memory");
         if (!all) { status |= SPECTRA_STATUS_WAIT_TIMEOUT; ok = false; break; }
       }
-      DM_T(1)
       const uint8_t* src = S.raw[s];
       // this thread's four token rows: row block rb (16 tokens), rows gid and gid + 8 of it
       const int t0 = 32 * wq + gid;                      // rows t0, t0 + 8, t0 + 16, t0 + 24
@@ -342,7 +351,6 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
             }
           }
         }
-        DM_T(2)
         // ---- + sum_g lo_g u_g + c, then (keys with positions) the rotary pairing, then the stores
 #pragma unroll 1
         for (int g = 0; g < n_groups; g++) {
@@ -396,13 +404,8 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
           }
         }
       }
-      DM_T(3)
       // ---- the half is done with the slot: refill it with the tile three further on
       asm volatile("bar.sync %0, %1;" ::"r"(1 + hf), "n"(kDmHalf) : "memory");
-      DM_T(4)
-#ifdef DM_TIMING
-      dtiles++;
-#endif
       if (bulk && (tid & (kDmHalf - 1)) == 0 && tt + kDmSlots < n_tiles) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         issue_load(tt + kDmSlots);
@@ -412,9 +415,6 @@ __global__ void __launch_bounds__(kDmThreads, 1) decode_mma_kernel(DecodeArgs p,
     // ---- end of the run: a timeout anywhere ends the CTA's work (the barrier phases are no longer known)
     if (__syncthreads_or(status & SPECTRA_STATUS_WAIT_TIMEOUT)) break;
   }
-#ifdef DM_TIMING
-  if (blockIdx.x == 0 && lane == 0 && (warp == 0 || warp == 4)) printf("DM warp %d tiles %d per tile: tables(total) %lld wait %lld mma %lld epilogue+store %lld halfsync %lld\n", warp, dtiles, dt[0], dt[1] / max(dtiles, 1), dt[2] / max(dtiles, 1), dt[3] / max(dtiles, 1), dt[4] / max(dtiles, 1));
-#endif
   if (status && p.status) atomicOr(p.status, status);
 }
 

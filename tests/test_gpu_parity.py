@@ -1105,3 +1105,51 @@ def test_fit_moments_on_tensor_cores_are_accurate_and_reproducible(sp, n_fit):
         assert np.abs(moments[h, 128 * 128:] - s_ref).max() <= 1e-5 * max(1.0, np.abs(s_ref).max())
         ref = ofit.fit_basis(Xb[h, :n_fit], ofit.GAIN_SQRT)
         assert np.abs(outs[0][1][h] - ref["lam"]).max() <= 2e-6 * ref["lam"][0]
+
+
+@pytest.mark.parametrize("case", ["fitted_8x", "fitted_4x", "all8", "all7", "all1", "odd_mix", "gs32", "gs128", "misaligned",
+                                  "one_group_empty"])
+def test_reconstruction_without_unpacked_codes_on_every_layout(sp, case):
+    """spectra_decode with no yhat output takes the kernels that feed the packed fields to the tensor cores (Sec. 3.3
+    Mode A reconstruction regrouped per scale group): the tcgen05 kernel where a unit fits it, the mma.sync kernel for
+    the rest (tiles above its slot, more than 192 strip positions, four scale groups, a source that is not 16-byte
+    aligned).  Both sides, fp32 and bf16 outputs, two units (one ragged), against the oracle's reconstruction."""
+    wl = si.WORKLOADS["tiny"]
+    gs = {"gs32": 32, "gs128": 128}.get(case, 64)
+    cfg = sp.default_config(scale_group=gs)
+    rng = np.random.default_rng(17)
+    n, n2 = 700, 389
+    shift = 6 if case == "misaligned" else 0
+    for side in (si.SIDE_K, si.SIDE_V):
+        X = si.draw_unit(wl, 0, 0, side, 0, n_tokens=n)
+        if case == "fitted_8x" or case == "gs32" or case == "gs128" or case == "misaligned":
+            params = H.fit_params([X], 8.0, gs=gs)
+        elif case == "fitted_4x":
+            params = H.fit_params([X], 4.0, gs=gs)
+        else:
+            w = {"all8": np.full(128, 8), "all7": np.full(128, 7), "all1": np.ones(128, np.int64),
+                 "odd_mix": rng.integers(0, 9, 128),
+                 "one_group_empty": np.concatenate([rng.integers(1, 5, 64), np.zeros(64, np.int64)])}[case]
+            params = H.fit_params([X], 4.0, gs=gs, widths_override=np.asarray(w, np.uint8))
+        tb = int(params.tile_bytes[0])
+        off = np.array([0, 6 * tb], np.int64)                      # two units of six tiles each
+        ref = np.zeros(12 * tb, np.uint8)
+        assert H.oracle_encode(params, side, X[None, :n], [0], ref, off[:1]) == 0
+        assert H.oracle_encode(params, side, X[None, 100:100 + n2], [0], ref, off[1:]) == 0
+        want = [oc.decode_unit(ref[off[u]:], tb, m, params.w_dec[0], params.m_rot[0], params.widths[0], gs, side)[1]
+                for u, m in ((0, n), (1, n2))]
+        dp = H.dev_params(params)
+        cache_dev = torch.zeros(ref.size + 16, dtype=torch.uint8, device="cuda")
+        cache_dev[shift:shift + ref.size] = H.to_dev(ref)
+        for dt in (torch.float32, torch.bfloat16):
+            out = torch.full((2, 768, 128), 7.0, dtype=dt, device="cuda")
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            sp.decode(cfg, side, cache_dev[shift:], H.to_dev(off), 2, 1, torch.tensor([n, n2], dtype=torch.int32, device="cuda"),
+                      n, dp["w_dec"], dp["m_rot"], dp["widths"], out, None, 768 * 128, 128, status_word=status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            tol = TOL if dt == torch.float32 else TOL + 2.0 ** -8
+            got = out.float().cpu().numpy()
+            assert H.rel_err_per_vector(got[0, :n], want[0]) <= tol
+            assert H.rel_err_per_vector(got[1, :n2], want[1]) <= tol
+            assert (got[0, n:] == 7.0).all() and (got[1, n2:] == 7.0).all()
