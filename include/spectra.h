@@ -219,10 +219,16 @@ int spectra_encode(const spectra_config* cfg, int side, const void* x, int x_dty
  * of every unit-side; fp32 accumulation.  out: device, out_dtype SPECTRA_F32 or SPECTRA_BF16, element
  * (u, t, i) at out[u*stride_unit + t*stride_token + i].  n_tokens: device int32 [n_units];
  * max_tokens (host value) bounds it.  yhat_out (device fp32, same strides, may be NULL) receives the
- * dequantised rotated coordinates.  cache must be 2-byte aligned (SPECTRA_INVALID_ARG otherwise).  Packed tiles are
- * fetched with bulk copies when cache + unit_offset[u] is 16-byte aligned (and a tile is at most 10 KB), else read in
- * place: same results, lower speed.  status_word: device int32 or NULL; a bounded wait of the tensor-core kernel that
- * gives up sets SPECTRA_STATUS_WAIT_TIMEOUT there (the reconstruction is then invalid).
+ * dequantised rotated coordinates.  cache must be 2-byte aligned (SPECTRA_INVALID_ARG otherwise).
+ * Speed, not the contract, depends on the call's shape.  With yhat_out NULL the sum is regrouped per scale group,
+ * xhat = sum_g R_g (fields x W_dec rows / L) + sum_g lo_g u_g + m' W_dec, and the packed sub-fields themselves are the
+ * tensor-core operand (exact as fp16 numbers; the W_dec rows enter as two fp16 parts: same accuracy as the
+ * element-wise path, about 1e-5 of a vector's largest entry): one tcgen05 kernel takes the units with at most two
+ * scale groups, at most 192 strip positions, tiles up to 10 KB and a 16-byte aligned cache + unit_offset[u]; the
+ * element-wise kernel, launched behind it, takes the other units.  With yhat_out the codes are dequantised one by one
+ * in the oracle's operation order (yhat bit-exact) and rotated with
+ * tcgen05.  status_word: device int32 or NULL; a bounded wait that gives up sets SPECTRA_STATUS_WAIT_TIMEOUT there
+ * (the reconstruction is then invalid).
  */
 int spectra_decode(const spectra_config* cfg, int side, const uint8_t* cache, const int64_t* unit_offset,
                    int64_t n_units, int64_t n_param_sets, const int32_t* n_tokens, int32_t max_tokens,

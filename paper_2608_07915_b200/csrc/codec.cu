@@ -5,7 +5,6 @@
 #include "encode_append.cuh"
 #include "encode_umma.cuh"
 #include "decode_umma.cuh"
-#include "decode_mma.cuh"
 #include "decode_pairs.cuh"
 #include "tensor_map.cuh"
 
@@ -323,24 +322,22 @@ int decode_impl(const spectra_config* cfg, int side, const uint8_t* cache, const
   DecodeArgs a{cache, unit_offset, side, cfg->scale_group, n_param_sets, n_tokens, w_dec, mean_rot, widths, out,
                out_dtype, yhat_out, stride_unit, stride_token, status_word, TileMap{tile_table, table_stride},
                rope_cos, rope_sin, rope_pos0, TileMap{out_table, out_table_stride}};
-  const int esz = out_dtype == SPECTRA_BF16 ? 2 : 4;
-  if (out && !yhat_out && (reinterpret_cast<uintptr_t>(out) & (2 * esz - 1)) == 0 && stride_unit % 2 == 0 &&
-      stride_token % 2 == 0) {
-    // reconstruction with the packed fields themselves as tensor-core operands: the tcgen05 kernel takes the units it can
-    // hold (up to two scale groups and 192 strip positions), the mma.sync kernel behind it exactly the others
-    // (its outputs are stored in pairs: even strides)
+  if (out && !yhat_out) {
+    // reconstruction with the packed fields themselves as the tensor-core operand: decode_pair_kernel takes the units it
+    // can hold (up to two scale groups and 192 strip positions, tiles up to 10 KB, aligned sources), decode_tc_kernel
+    // behind it exactly the others
     const int tiles = (int)((max_tokens + kTile - 1) / kTile);
     const long long n_slots = (long long)tiles * n_units;
     const int sms = sm_count();
     if (sms <= 0 || n_slots > 0x7fffffffLL) return SPECTRA_CUDA_ERROR;
     const unsigned grid = (unsigned)(n_slots < sms ? n_slots : sms);
-    const size_t smem_p = sizeof(DecodePairSmem) + 128, smem_m = sizeof(DecodeMmaSmem) + 128;
+    const size_t smem_p = sizeof(DecodePairSmem) + 128, smem_t = sizeof(DecodeTcSmem) + 128;
     if (cudaFuncSetAttribute(decode_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_p) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_m) != cudaSuccess)
+        cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_t) != cudaSuccess)
       return SPECTRA_CUDA_ERROR;
     decode_pair_kernel<<<grid, kDpThreads, smem_p, (cudaStream_t)stream>>>(a, tiles, (int)n_slots);
     if (launch_status()) return SPECTRA_CUDA_ERROR;
-    decode_mma_kernel<<<grid, kDmThreads, smem_m, (cudaStream_t)stream>>>(a, tiles, (int)n_slots, 1);
+    decode_tc_kernel<<<grid, kDecThreads, smem_t, (cudaStream_t)stream>>>(a, tiles, (int)n_slots, 1);
     return launch_status();
   }
   if (out) {   // reconstruction: inverse rotation on the tensor cores (tcgen05), persistent grid
@@ -353,7 +350,7 @@ int decode_impl(const spectra_config* cfg, int side, const uint8_t* cache, const
     const int sms = sm_count();
     if (sms <= 0 || n_slots > 0x7fffffffLL) return SPECTRA_CUDA_ERROR;
     const unsigned grid_tc = (unsigned)(n_slots < sms ? n_slots : sms);
-    decode_tc_kernel<<<grid_tc, kDecThreads, dec_smem, (cudaStream_t)stream>>>(a, tiles, (int)n_slots);
+    decode_tc_kernel<<<grid_tc, kDecThreads, dec_smem, (cudaStream_t)stream>>>(a, tiles, (int)n_slots, 0);
     return launch_status();
   }
   if (cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(CodecSmem)) !=

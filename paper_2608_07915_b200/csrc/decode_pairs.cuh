@@ -1,12 +1,13 @@
-// Fast reconstruction path of spectra_decode: the regrouping of decode_mma.cuh
+// Fast reconstruction path of spectra_decode: the regrouping of decode_runs.cuh
 //     xhat_t = sum_g R_g(t) [ sum_{strips k of group g} field_tk W''_k ] + sum_g lo_g(t) u_g + c
 // with the bracket as one tcgen05 product per scale group.  The A operand [128 tokens x K] holds the packed fields
 // themselves as fp16 numbers (a field shifted to bit 0 and masked is the subnormal field * 2^-24, which the tensor
 // core multiplies exactly): a worker thread takes one token and one pair of strips (K side: the 32-bit word of the
 // tile already holds both halves) and turns it into a 32-bit store of the K-major operand with one load, one shift
-// and one mask.  No code is assembled, dequantised or split into parts.  B = W'' as fp16 (scaled by a power of two),
-// rows in the order of the (group, class) runs, zero where a row belongs to another group or lies past its class.
-// Per tile: n_ksteps MMAs of 128 x 128 x 16 into one accumulator tile per group; the epilogue (thread = token and 64
+// and one mask.  No code is assembled, dequantised or split into parts.  B = W'' scaled by a power of two and split
+// into two fp16 parts (hi + lo: 22 bits; a single fp16 part left errors of 1e-3 of a vector's largest entry), rows in
+// the order of the (group, class) runs, zero where a row belongs to another group or lies past its class.
+// Per tile: 2 n_ksteps MMAs of 128 x 128 x 16 into one accumulator tile per group; the epilogue (thread = token and 64
 // channels) reads both, scales by the token's group ranges and adds the offset terms in fp32.
 //
 // Persistent CTAs over (unit, tile) slots; two buffers (packed tile, operand, accumulators, metadata) alternate between
@@ -15,9 +16,10 @@
 // per tile.  Barriers per buffer (bounded waits): raw_full, a_full (operand and metadata written), acc_full (MMAs
 // complete: accumulators ready, operand free), acc_free (epilogue done: accumulators and metadata free).  Units this kernel cannot
 // hold (more than two scale groups, more than twelve k-steps of 16 strips, tiles above its slot, a misaligned source)
-// are skipped: decode_mma_kernel, launched behind it, takes exactly those.
+// are skipped: decode_tc_kernel, launched behind it, takes exactly those.
 #pragma once
-#include "decode_mma.cuh"
+#include "decode_runs.cuh"
+#include "decode_umma.cuh"
 
 namespace spectra {
 
@@ -29,7 +31,7 @@ constexpr uint32_t kDpIdesc = (1u << 4) | (1u << 16) | ((128u >> 3) << 17) | ((1
 
 struct DecodePairSmem {
   StripTable tab;
-  alignas(128) uint8_t w[kDpK * kD * 2];               // W'': element (k, n) at (n / 8) * 16 K + (k / 8) * 128 + (k % 8) * 16 + (n % 8) * 2
+  alignas(128) uint8_t w[2][kDpK * kD * 2];            // W'' = hi + lo (two fp16 parts): element (k, n) at (n / 8) * 16 K + (k / 8) * 128 + (k % 8) * 16 + (n % 8) * 2
   struct Half {
     alignas(128) uint8_t a[kTile * kDpK * 2];          // fields: element (t, k) at (k / 8) * 2048 + t * 16 + (k % 8) * 2
     alignas(128) uint8_t raw[kDecRawMax];              // the packed tile
@@ -205,7 +207,7 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
     const uint8_t* unit_ptr = p.cache + p.unit_offset[u];
     dm_build_runs(S.run, S.kg, T, side_v, gs);
     const int n_ksteps = S.kg[kMaxGroups];
-    if (!dm_pairs_eligible(T, n_ksteps, unit_ptr)) continue;      // decode_mma_kernel takes this unit
+    if (!dm_pairs_eligible(T, n_ksteps, unit_ptr)) continue;      // decode_tc_kernel takes this unit
     const int tile_bytes = T.tile_bytes;
     // ---- largest |W_dec|: the power of two that brings W'' into fp16's range
     {
@@ -231,7 +233,10 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
         const int nn = idx & (kD - 1), row = (idx >> 7) & 15, ks = idx >> 11;
         const int k = 16 * ks + row;
         const float v = dm_b_value(S.run, T, wsrc, side_v, gs, ks, row, nn) * wscale;
-        *reinterpret_cast<__half*>(&S.w[(nn >> 3) * (16 * kDpK) + (k >> 3) * 128 + (k & 7) * 16 + (nn & 7) * 2]) = __float2half_rn(v);
+        const int wo = (nn >> 3) * (16 * kDpK) + (k >> 3) * 128 + (k & 7) * 16 + (nn & 7) * 2;
+        const __half hi = __float2half_rn(v);
+        *reinterpret_cast<__half*>(&S.w[0][wo]) = hi;
+        *reinterpret_cast<__half*>(&S.w[1][wo]) = __float2half_rn(v - __half2float(hi));
       }
       for (int idx = threadIdx.x; idx < 3 * kD; idx += kDpThreads) {     // u_0, u_1, c
         const int nn = idx & (kD - 1), g = idx >> 7;
@@ -268,7 +273,7 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
         load_raw(0);
         if (n_tiles > 1) load_raw(1);
         bool ok = true;
-        const uint32_t w0 = um_smem_u32(S.w);
+        const uint32_t w0 = um_smem_u32(S.w[0]), w1 = um_smem_u32(S.w[1]);
 #pragma unroll 1
         for (int tt = 0; tt < n_tiles && ok; tt++) {
           const int h = tt & 1, i = (h ? base1 : base0) + (tt >> 1);
@@ -281,14 +286,17 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
           const uint32_t a0 = um_smem_u32(S.half[h].a);
           // descriptors once; per k-step only the address fields move (the issuing thread's own instructions bound the
           // rate at which MMAs go out)
-          const uint64_t ad0 = um_desc(a0, 2048, 128), bd0 = um_desc(w0, 128, 16 * kDpK);
+          const uint64_t ad0 = um_desc(a0, 2048, 128), bh0 = um_desc(w0, 128, 16 * kDpK), bl0 = um_desc(w1, 128, 16 * kDpK);
 #pragma unroll
           for (int g = 0; g < 2; g++) {
             const int lo = g ? kg1 : 0, hi = g ? kg2 : kg1;
             const uint32_t d = tb + 128u * (2 * h + g);
-            if (lo < hi) um_mma_ss(d, ad0 + (uint64_t)(256 * lo), bd0 + (uint64_t)(16 * lo), kDpIdesc, 0);
+            // the fields against the high parts of W'', then against the low parts, into the same accumulator
+            if (lo < hi) um_mma_ss(d, ad0 + (uint64_t)(256 * lo), bh0 + (uint64_t)(16 * lo), kDpIdesc, 0);
 #pragma unroll 2
-            for (int ks = lo + 1; ks < hi; ks++) um_mma_ss(d, ad0 + (uint64_t)(256 * ks), bd0 + (uint64_t)(16 * ks), kDpIdesc, 1);
+            for (int ks = lo + 1; ks < hi; ks++) um_mma_ss(d, ad0 + (uint64_t)(256 * ks), bh0 + (uint64_t)(16 * ks), kDpIdesc, 1);
+#pragma unroll 2
+            for (int ks = lo; ks < hi; ks++) um_mma_ss(d, ad0 + (uint64_t)(256 * ks), bl0 + (uint64_t)(16 * ks), kDpIdesc, 1);
           }
           asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(um_smem_u32(&S.acc_full[h])) : "memory");
         }

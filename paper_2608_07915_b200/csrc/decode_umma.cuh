@@ -24,12 +24,12 @@
 //   acc_full   the MMAs are complete                 (workers wait)
 #pragma once
 #include "encode_umma.cuh"
+#include "decode_runs.cuh"
 
 namespace spectra {
 
 constexpr int kDecWorkers = 512;
 constexpr int kDecThreads = kDecWorkers + 32;
-constexpr int kDecRawMax = 10240;      // packed tiles up to this size are staged in shared memory, larger ones read in place
 
 struct DecodeArgs {
   const uint8_t* cache; const int64_t* unit_offset; int side; int scale_group; int64_t n_param_sets;
@@ -59,12 +59,15 @@ struct DecodeTcSmem {
   uint32_t field1[kD];                             // the channel's first (widest) sub-field: see field_desc()
   uint16_t sbase[4][kD];                           // per class: byte offset of the channel's strip; bit 15: stored alone
   uint8_t more[kD];                                // classes of the channel's further sub-fields (bit c), usually 0
+  DmRun run[kMaxGroups][4];                        // only to tell which units the packed-field kernel takes
+  int kg[kMaxGroups + 1];
   alignas(8) uint64_t raw_full[2], a_full[2], acc_full[2];
   uint32_t tmem_base;
 };
 static_assert(sizeof(DecodeTcSmem) + 128 <= 227 * 1024, "the reconstruction kernel's shared memory must fit one SM");
 
-__global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p, int n_slots_unit, int n_slots) {
+// skip_pairs != 0: units that decode_pair_kernel (decode_pairs.cuh) takes are left to it
+__global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p, int n_slots_unit, int n_slots, int skip_pairs) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned char* smem_al = smem_raw + ((128u - (um_smem_u32(smem_raw) & 127u)) & 127u);
   DecodeTcSmem& S = *reinterpret_cast<DecodeTcSmem*>(smem_al);
@@ -119,6 +122,10 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_tc_kernel(DecodeArgs p,
     if (n_tiles <= 0) continue;
     __syncthreads();                                     // the previous run is over
     build_strip_table(S.tab, p.widths + (int64_t)ps * kD, p.scale_group);
+    if (skip_pairs) {
+      dm_build_runs(S.run, S.kg, S.tab, p.side == SPECTRA_SIDE_V, p.scale_group);
+      if (dm_pairs_eligible(S.tab, S.kg[kMaxGroups], p.cache + p.unit_offset[u])) continue;
+    }
     const float* wsrc = p.w_dec + (int64_t)ps * kD * kD;
     for (int idx = threadIdx.x; idx < kD * kD; idx += kDecThreads) {
       const int k = idx / kD, nn = idx - k * kD;

@@ -1110,9 +1110,9 @@ def test_fit_moments_on_tensor_cores_are_accurate_and_reproducible(sp, n_fit):
 @pytest.mark.parametrize("case", ["fitted_8x", "fitted_4x", "all8", "all7", "all1", "odd_mix", "gs32", "gs128", "misaligned",
                                   "one_group_empty"])
 def test_reconstruction_without_unpacked_codes_on_every_layout(sp, case):
-    """spectra_decode with no yhat output takes the kernels that feed the packed fields to the tensor cores (Sec. 3.3
-    Mode A reconstruction regrouped per scale group): the tcgen05 kernel where a unit fits it, the mma.sync kernel for
-    the rest (tiles above its slot, more than 192 strip positions, four scale groups, a source that is not 16-byte
+    """spectra_decode with no yhat output feeds the packed fields to the tensor cores (Sec. 3.3 Mode A reconstruction
+    regrouped per scale group) for every unit that kernel can hold, and the element-wise kernel takes the rest in the
+    same call (tiles above the slot, more than 192 strip positions, four scale groups, a source that is not 16-byte
     aligned).  Both sides, fp32 and bf16 outputs, two units (one ragged), against the oracle's reconstruction."""
     wl = si.WORKLOADS["tiny"]
     gs = {"gs32": 32, "gs128": 128}.get(case, 64)
