@@ -26,7 +26,7 @@ import numpy as np
 METRIC = "coded_kv_decode_attention_kv_tokens_per_s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (one layer of the workload),
 # from the ncu capture summarised in profiles/attention_mma_kernel_llama32_2layer.md (same per-launch shape)
-NCU_TRAFFIC_BYTES = {"llama32": 173.5e6}
+NCU_TRAFFIC_BYTES = {"llama32": 172.8e6}
 # share of the dominant kernel (attention_mma_kernel) in the device time of a decode step, from the launch list of
 # this command summarised in profiles/decode_step_launch_list_llama32.md
 MAIN_KERNEL_SHARE = {"llama32": 0.778}
