@@ -104,12 +104,15 @@ def test_paged_reconstruction_matches_oracle(sp):
 SHAPES = [([200, 77], 150), ([0], 1000), ([1000], 1), ([127, 128], 129)]
 
 
+@pytest.mark.parametrize("Hkv,G", [(2, 4), (4, 7), (3, 1)], ids=["gqa4", "gqa7", "mha"])
 @pytest.mark.parametrize("pos0,n_new", SHAPES)
-def test_prefill_attention_kernel_on_seeded_pools(sp, pos0, n_new):
+def test_prefill_attention_kernel_on_seeded_pools(sp, pos0, n_new, Hkv, G):
     """The attention kernel alone: seeded bf16 keys and values laid out through a shuffled page table, every slot past
     a sequence's end NaN, against the oracle's causal attention on the same bf16 values, row by row (ragged chunk
     ends, a chunk that starts mid-tile, a single query, the diagonal crossing two tiles)."""
-    n_seq, Hkv, G, d = len(pos0), 2, 4, 128
+    n_seq, d = len(pos0), 128
+    if (Hkv, G) != (2, 4) and n_new == 1000:
+        pytest.skip("the long chunk is covered at one head shape")
     Hq = Hkv * G
     kv_lens = [p + n_new for p in pos0]
     tiles = (max(kv_lens) + 127) // 128
