@@ -132,6 +132,24 @@ def test_full_context_decode_step_matches_oracle(case):
                                     pk.widths, pv.w_dec, pv.m_rot, pv.widths, 64, 1.0 / np.sqrt(128.0))
         # bf16 queries on the GPU side are exactly the fp32 values the oracle used
         assert H.rel_err_per_vector(got[s, h], ref[0]) <= TOL, (case, s, h)
+    # ---- reconstruction of the whole layer in the launch bench.py times (every unit, bf16 out): the sampled units, which
+    #      hold the oracle's bytes now, against the oracle's reconstruction; every token
+    U = batch * Hk
+    n_rec = N + 1
+    if U * n_rec * d * 2 <= (6 << 30):
+        recon = torch.empty((U, n_rec, d), dtype=torch.bfloat16, device="cuda")
+        for side in (si.SIDE_K, si.SIDE_V):
+            ls = model.side[0][side]
+            sp.decode(model.cfg, side, ls.cache, ls.unit_offset, U, Hk, torch.full((U,), n_rec, dtype=torch.int32, device="cuda"),
+                      n_rec, ls.w_dec, ls.m_rot, ls.widths, recon, None, n_rec * d, d, status_word=model.status)
+            torch.cuda.synchronize()
+            assert int(model.status.item()) == 0
+            for (s, h) in sampled:
+                pr, tb, c = oracle_caches[(s, h)][side]
+                _, want = oc.decode_unit(c, tb, n_rec, pr.w_dec[0], pr.m_rot[0], pr.widths[0], 64, side, want_yhat=False)
+                got_r = recon[s * Hk + h].float().cpu().numpy()
+                assert H.rel_err_per_vector(got_r, want) <= TOL + 2.0 ** -8, (case, "reconstruction", side, s, h)
+        del recon
     # ---- a second step through the fused call (the one bench.py times)
     q2 = torch.randn((batch, wl.q_heads, d), generator=gen, device="cuda").to(torch.bfloat16)
     nk2 = torch.randn((batch * Hk, d), generator=gen, device="cuda").to(torch.bfloat16)
