@@ -275,8 +275,8 @@ extern "C" int spectra_encode(const spectra_config* cfg, int side, const void* x
     // rotation on the 5th-generation tensor cores (accumulator tiles in tensor memory); the token tiles arrive by
     // TMA: a 3-D map over x [unit][token][channel] whose box is 8 channels x 128 tokens
     CUtensorMap xmap;
-    if (make_token_map(&xmap, x, n_new, n_units, stride_token, stride_unit)) {
-      const size_t um_smem = sizeof(EncodeUmmaSmem) + 128;
+    if (make_token_map(&xmap, x, n_new, n_units, stride_token, stride_unit, true)) {
+      const size_t um_smem = sizeof(EncodeUmmaSmem) + 1024;
       if (cudaFuncSetAttribute(encode_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)um_smem) !=
           cudaSuccess)
         return SPECTRA_CUDA_ERROR;

@@ -207,6 +207,44 @@ def test_bulk_bf16_encode_with_ragged_starts_keeps_earlier_tokens(sp):
             assert not c_tail[end:].any() and not m_tail[end:].any()
 
 
+def test_bulk_bf16_encode_with_a_nan_and_an_out_of_range_token(sp):
+    """The bulk bf16 path on whole tiles with one token that holds a NaN and one whose rotated values leave fp16's
+    range: both are reported in the status word, every other token is stored exactly as without them, and the
+    out-of-range token is stored with its offset and range clipped and its codes saturated, as the oracle stores it."""
+    wl = si.WORKLOADS["tiny"]
+    cfg = sp.default_config()
+    n_units, n = 2, 512
+    X = [si.to_bf16_f32(si.draw_unit(wl, 0, u, si.SIDE_K, 0)[:n]) for u in range(n_units)]
+    params = H.fit_params(X, 8.0)
+    dp = H.dev_params(params)
+    off, total = H.cache_layout(params, n_units, n)
+    clean = np.stack(X)
+    bad = clean.copy()
+    bad[0, 130, 5] = np.nan
+    bad[1, 300] = si.to_bf16_f32(bad[1, 300] * 3.0e6)
+    zero = np.zeros(n_units, np.int64)
+    for side in (sp.SIDE_K, sp.SIDE_V):
+        caches = []
+        for x, want in ((clean, 0), (bad, sp.STATUS_NONFINITE | sp.STATUS_F16_RANGE)):
+            cache = torch.zeros(total, dtype=torch.uint8, device="cuda")
+            st = _gpu_encode(sp, cfg, params, dp, side, H.to_dev(x).to(torch.bfloat16), H.to_dev(zero.astype(np.int32)),
+                             cache, H.to_dev(off))
+            assert st == want
+            caches.append(cache.cpu().numpy())
+        ref = np.zeros(total, np.uint8)
+        assert H.oracle_encode(params, side, bad[:, :, :], zero, ref, off) == (sp.STATUS_NONFINITE | sp.STATUS_F16_RANGE)
+        for u, t_bad in ((0, 130), (1, 300)):
+            c0, m0 = H.unpack_codes(params, side, caches[0], off, u, n)
+            c1, m1 = H.unpack_codes(params, side, caches[1], off, u, n)
+            keep = np.arange(n) != t_bad
+            assert np.array_equal(c0[keep], c1[keep]) and np.array_equal(m0[keep], m1[keep])
+        c_ref, m_ref = H.unpack_codes(params, side, ref, off, 1, n)
+        c_got, m_got = H.unpack_codes(params, side, caches[1], off, 1, n)
+        assert np.abs(c_got[300].astype(np.int64) - c_ref[300].astype(np.int64)).max() <= 1
+        assert np.abs(H.f16_ordinal(m_got[300]) - H.f16_ordinal(m_ref[300])).max() <= 1
+        assert c_got[300].max() > 0                        # the token is stored, not dropped
+
+
 # ----------------------------------------------------------------------------- config 0 end to end
 
 def _tiny_setup(sp, ratio=4.0, gain_mode=ofit.GAIN_SQRT, n=1024, gs=64):
