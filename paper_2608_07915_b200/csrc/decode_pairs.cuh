@@ -145,7 +145,18 @@ __device__ __forceinline__ void dp_chunk(const DecodePairSmem& S, uint32_t acc0,
 }
 __device__ __forceinline__ void dp_store16(const DecodeArgs& p, int64_t o, const float (&y)[16]) {
   const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out) + (uintptr_t)o * (p.out_dtype == SPECTRA_BF16 ? 2 : 4);
-  if (p.out_dtype == SPECTRA_BF16 && (addr & 15) == 0) {
+  if (p.out_dtype == SPECTRA_BF16 && (addr & 31) == 0) {
+    // one 32-byte store: the token's 16 channels fill a whole sector
+    uint32_t h[8];
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+      const __nv_bfloat162 v = __floats2bfloat162_rn(y[2 * k], y[2 * k + 1]);
+      h[k] = *reinterpret_cast<const uint32_t*>(&v);
+    }
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(addr), "r"(h[0]), "r"(h[1]), "r"(h[2]),
+                 "r"(h[3]), "r"(h[4]), "r"(h[5]), "r"(h[6]), "r"(h[7])
+                 : "memory");
+  } else if (p.out_dtype == SPECTRA_BF16 && (addr & 15) == 0) {
     uint4* dst = reinterpret_cast<uint4*>(addr);
 #pragma unroll
     for (int c = 0; c < 2; c++) {
@@ -154,6 +165,13 @@ __device__ __forceinline__ void dp_store16(const DecodeArgs& p, int64_t o, const
       for (int k = 0; k < 4; k++) h[k] = __floats2bfloat162_rn(y[8 * c + 2 * k], y[8 * c + 2 * k + 1]);
       dst[c] = *reinterpret_cast<const uint4*>(h);
     }
+  } else if (p.out_dtype == SPECTRA_F32 && (addr & 31) == 0) {
+#pragma unroll
+    for (int c = 0; c < 2; c++)
+      asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(addr + 32 * c), "f"(y[8 * c]),
+                   "f"(y[8 * c + 1]), "f"(y[8 * c + 2]), "f"(y[8 * c + 3]), "f"(y[8 * c + 4]), "f"(y[8 * c + 5]),
+                   "f"(y[8 * c + 6]), "f"(y[8 * c + 7])
+                   : "memory");
   } else if (p.out_dtype == SPECTRA_F32 && (addr & 15) == 0) {
     float4* dst = reinterpret_cast<float4*>(addr);
 #pragma unroll
