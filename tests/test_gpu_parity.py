@@ -1191,3 +1191,38 @@ def test_reconstruction_without_unpacked_codes_on_every_layout(sp, case):
             assert H.rel_err_per_vector(got[0, :n], want[0]) <= tol
             assert H.rel_err_per_vector(got[1, :n2], want[1]) <= tol
             assert (got[0, n:] == 7.0).all() and (got[1, n2:] == 7.0).all()
+
+
+@pytest.mark.parametrize("skew", [16, 8, 1])
+def test_reconstruction_into_outputs_of_any_alignment(sp, skew):
+    """The packed-field reconstruction stores 32 bytes per instruction where the output allows it; an output that
+    starts `skew` elements into a 32-byte-aligned buffer takes the 16-byte or the element-wise stores instead.  All of
+    them write the same values, and nothing outside the unit's tokens."""
+    wl = si.WORKLOADS["tiny"]
+    cfg = sp.default_config()
+    n = 300
+    for side in (si.SIDE_K, si.SIDE_V):
+        X = si.draw_unit(wl, 0, 0, side, 0, n_tokens=n)
+        params = H.fit_params([X], 8.0)
+        tb = int(params.tile_bytes[0])
+        ref = np.zeros(3 * tb, np.uint8)
+        assert H.oracle_encode(params, side, X[None, :n], [0], ref, np.zeros(1, np.int64)) == 0
+        dp = H.dev_params(params)
+        cache_dev = H.to_dev(ref)
+        off = H.to_dev(np.zeros(1, np.int64))
+        n_dev = torch.tensor([n], dtype=torch.int32, device="cuda")
+        for dt in (torch.bfloat16, torch.float32):
+            outs = []
+            for s in (0, skew):
+                buf = torch.full((384 * 128 + 64,), 7.0, dtype=dt, device="cuda")
+                out = buf[s:s + 384 * 128].view(1, 384, 128)
+                assert out.data_ptr() % 32 == (s * buf.element_size()) % 32
+                status = torch.zeros(1, dtype=torch.int32, device="cuda")
+                sp.decode(cfg, side, cache_dev, off, 1, 1, n_dev, n, dp["w_dec"], dp["m_rot"], dp["widths"], out, None,
+                          384 * 128, 128, status_word=status)
+                torch.cuda.synchronize()
+                assert int(status.item()) == 0
+                full = buf.float().cpu().numpy()
+                assert (full[:s] == 7.0).all() and (full[s + n * 128:] == 7.0).all()
+                outs.append(full[s:s + n * 128])
+            assert np.array_equal(outs[0], outs[1])
