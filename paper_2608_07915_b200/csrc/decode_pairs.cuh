@@ -79,10 +79,30 @@ __device__ __forceinline__ int dp_run(const DmRun& r, const uint8_t* __restrict_
       for (int G = 0; G < 16; G++)
         v[G] = mine ? (uint32_t)*reinterpret_cast<const uint16_t*>(lp + 2 * ((8 * G * W) >> 4))
                     : *reinterpret_cast<const uint32_t*>(cp + 4 * ((8 * G * W) >> 4));
-    } else {
+    } else if (V) {
 #pragma unroll
       for (int G = 0; G < 16; G++)
-        v[G] = *reinterpret_cast<const uint32_t*>(cp + (V ? 4 * ((G >> 2) * W + (((8 * (G & 1)) * W) >> 4)) : 4 * ((8 * G * W) >> 4)));
+        v[G] = *reinterpret_cast<const uint32_t*>(cp + 4 * ((G >> 2) * W + (((8 * (G & 1)) * W) >> 4)));
+    } else {
+      // K side: the four units of a step sit a multiple of 64 bytes apart, so their words of one token group share
+      // banks.  Lane pr therefore walks the sixteen token groups in blocks of four in the order blk ^ pr: at every
+      // step the four units read different banks, and the stores (row = token) stay conflict-free in any order.
+      const uint8_t* cpb[4];
+      uint8_t* dstb[4];
+#pragma unroll
+      for (int blk = 0; blk < 4; blk++) {
+        const int gb = 4 * (blk ^ pr);
+        cpb[blk] = cp + 4 * ((8 * gb * W) >> 4);
+        dstb[blk] = dst + gb * 128;
+      }
+#pragma unroll
+      for (int G = 0; G < 16; G++) v[G] = *reinterpret_cast<const uint32_t*>(cpb[G >> 2] + 4 * ((8 * (G & 3) * W) >> 4));
+#pragma unroll
+      for (int G = 0; G < 16; G++) {
+        const int sh = (8 * (G & 3) * W) & 15;
+        *reinterpret_cast<uint32_t*>(dstb[G >> 2] + (G & 3) * 128) = (v[G] >> (sh + shq)) & FM;
+      }
+      continue;
     }
 #pragma unroll
     for (int G = 0; G < 16; G++) {
