@@ -207,6 +207,43 @@ def test_bulk_bf16_encode_with_ragged_starts_keeps_earlier_tokens(sp):
             assert not c_tail[end:].any() and not m_tail[end:].any()
 
 
+@pytest.mark.parametrize("kind", ["mixed", "dead_group", "odd_classes", "8", "7", "1", "3"])
+def test_bulk_bf16_encode_on_every_width_profile(sp, kind):
+    """The bulk bf16 path (rotation on tcgen05, channel-major code tile, gathered half-words) on width profiles that
+    use every class, every sub-field shift, classes with an odd number of strips and an empty scale group: whole and
+    partly filled tiles, both sides, against the oracle's encode of the same bf16 vectors up to rare rounding ties."""
+    wl = si.WORKLOADS["tiny"]
+    cfg = sp.default_config()
+    rng = np.random.default_rng(23)
+    n = 300                                               # two whole tiles and a ragged one
+    X = si.to_bf16_f32(si.draw_unit(wl, 0, 0, si.SIDE_K, 0)[:n])
+    params = H.fit_params([X], 4.0, widths_override=_random_widths(rng, kind))
+    dp = H.dev_params(params)
+    off, total = H.cache_layout(params, 1, n)
+    zero = np.zeros(1, np.int64)
+    for side in (sp.SIDE_K, sp.SIDE_V):
+        ref = np.zeros(total, np.uint8)
+        assert H.oracle_encode(params, side, X[None], zero, ref, off) == 0
+        cache = torch.zeros(total, dtype=torch.uint8, device="cuda")
+        st = _gpu_encode(sp, cfg, params, dp, side, H.to_dev(X[None]).to(torch.bfloat16), H.to_dev(zero.astype(np.int32)),
+                         cache, H.to_dev(off))
+        assert st == 0
+        got = cache.cpu().numpy()
+        c_ref, m_ref = H.unpack_codes(params, side, ref, off, 0, n)
+        c_got, m_got = H.unpack_codes(params, side, got, off, 0, n)
+        diff = np.abs(c_got.astype(np.int64) - c_ref.astype(np.int64))
+        assert diff.max() <= 1 and (diff != 0).sum() <= 6
+        meta = np.abs(H.f16_ordinal(m_got) - H.f16_ordinal(m_ref))
+        assert meta.max() <= 1 and (meta.max(axis=1) != 0).sum() <= 3
+        # where codes and metadata agree the bytes do too: a token-wise comparison of the packed tiles' unpacked
+        # content is the whole content, so nothing else may differ
+        tb = int(params.tile_bytes[0])
+        same_tiles = [t for t in range((n + 127) // 128)
+                      if not diff[t * 128:(t + 1) * 128].any() and not meta[t * 128:(t + 1) * 128].any()]
+        for t in same_tiles:
+            assert np.array_equal(got[off[0] + t * tb: off[0] + (t + 1) * tb], ref[off[0] + t * tb: off[0] + (t + 1) * tb])
+
+
 def test_bulk_bf16_encode_with_a_nan_and_an_out_of_range_token(sp):
     """The bulk bf16 path on whole tiles with one token that holds a NaN and one whose rotated values leave fp16's
     range: both are reported in the status word, every other token is stored exactly as without them, and the
