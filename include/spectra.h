@@ -375,6 +375,14 @@ int spectra_decode_step(const spectra_config* cfg, const void* q, int q_dtype, c
  *   SPECTRA_GAIN_SQRT, layout 1.
  * spectra_total_bits: Btot = floor(16 d / ratio) clamped to b_max * d.
  * spectra_status_string: name of a return code.
+ *
+ * spectra_selftest_quotients (device work): the bulk bf16 encoder takes the quotients (2^b - 1) / R16, b = 1..8, of
+ *   the quantiser (Sec. 3.2: code = round((y - lo) (2^b - 1) / R)) from one shared reciprocal and fused
+ *   multiply-add corrections instead of eight divisions.  This call runs that computation for every positive finite
+ *   fp16 value of R16 and every b on the device and writes to mismatches[0] (device pointer, one int64) how many of
+ *   the 8 x 31 743 quotients differ in any bit from the IEEE single-precision division; 0 is the only acceptable
+ *   answer.  Enqueued on `stream`; returns SPECTRA_INVALID_ARG for a NULL pointer, SPECTRA_CUDA_ERROR if the launch
+ *   failed.
  */
 size_t spectra_tile_bytes(const spectra_config* cfg, const uint8_t* widths_host);
 size_t spectra_cache_bytes(const spectra_config* cfg, const uint8_t* widths_host, int64_t capacity_tokens);
@@ -383,6 +391,7 @@ int spectra_attention_path(const spectra_config* cfg, int32_t n_kv_heads, int32_
 void spectra_config_default(spectra_config* cfg);
 int32_t spectra_total_bits(const spectra_config* cfg, double ratio);
 const char* spectra_status_string(int code);
+int spectra_selftest_quotients(int64_t* mismatches, void* stream);
 
 #ifdef __cplusplus
 }

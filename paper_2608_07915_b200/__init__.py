@@ -28,6 +28,7 @@ EXPORTS = [
     "spectra_decode_attention", "spectra_decode_step", "spectra_attention_workspace_bytes", "spectra_tile_bytes", "spectra_config_default",
     "spectra_total_bits", "spectra_status_string", "spectra_cache_bytes", "spectra_attention_path",
     "spectra_alloc_bits_pooled", "spectra_split_ratio", "spectra_decode_rope", "spectra_decode_paged", "spectra_prefill_attention",
+    "spectra_selftest_quotients",
 ]
 
 
@@ -68,6 +69,13 @@ def default_config(**overrides):
 
 def status_string(code):
     return lib().spectra_status_string(C.c_int(code)).decode()
+
+
+def selftest_quotients(mismatches):
+    """mismatches: int64 device tensor of one element; receives how many quotients (2^b - 1) / R16 of the bulk
+    encoder differ from the IEEE division over every positive finite fp16 R16 and b = 1..8 (0 is the only
+    acceptable answer).  Runs on the current stream."""
+    _check(lib().spectra_selftest_quotients(_ptr(mismatches), _stream()), "spectra_selftest_quotients")
 
 
 def _check(rc, what):

@@ -400,3 +400,11 @@ extern "C" int spectra_decode_paged(const spectra_config* cfg, int side, const u
                      out_pool, out_dtype, nullptr, stride_page, stride_token, tile_table, table_stride, position0,
                      rope_cos, rope_sin, out_table, out_table_stride, status_word, stream);
 }
+
+extern "C" int spectra_selftest_quotients(int64_t* mismatches, void* stream) {
+  if (!mismatches) return SPECTRA_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemsetAsync(mismatches, 0, sizeof(int64_t), st) != cudaSuccess) return SPECTRA_CUDA_ERROR;
+  selftest_quotients_kernel<<<0x7c00 / 256, 256, 0, st>>>(reinterpret_cast<unsigned long long*>(mismatches));
+  return launch_status();
+}

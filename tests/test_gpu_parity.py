@@ -1263,3 +1263,12 @@ def test_reconstruction_into_outputs_of_any_alignment(sp, skew):
                 assert (full[:s] == 7.0).all() and (full[s + n * 128:] == 7.0).all()
                 outs.append(full[s:s + n * 128])
             assert np.array_equal(outs[0], outs[1])
+
+
+def test_quotients_from_a_shared_reciprocal_equal_the_division(sp):
+    """The bulk encoder's L_b / R16 (one reciprocal, fused multiply-add corrections) against the IEEE division for
+    every positive finite fp16 R16 and every width: not one bit may differ, or its codes would not be the oracle's."""
+    bad = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    sp.selftest_quotients(bad)
+    torch.cuda.synchronize()
+    assert int(bad.item()) == 0
