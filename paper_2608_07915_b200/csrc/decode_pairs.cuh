@@ -40,6 +40,8 @@ struct DecodePairSmem {
   alignas(16) float cvec[kD];
   uint16_t meta[4][4][kTile];                          // lo16 and R16 of both groups of the last four tiles, kept for the epilogue
   DmRun run[kMaxGroups][4];
+  float row_coef[kDpK];                                // per operand row: 2^shift / L of its strip
+  int16_t row_chan[kDpK];                              // its channel; -1: a zero row (another group's strip, or past its class)
   int kg[kMaxGroups + 1], wexp;
   float red[17];
   alignas(8) uint64_t raw_full[2], a_full[2], acc_full[2], acc_free[2];
@@ -247,6 +249,29 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
     const int n_ksteps = S.kg[kMaxGroups];
     if (!dm_pairs_eligible(T, n_ksteps, unit_ptr)) continue;      // decode_tc_kernel takes this unit
     const int tile_bytes = T.tile_bytes;
+    // ---- the operand rows: row (k-step, slot) -> channel and 2^shift / L of its strip, or a zero row (another
+    // group's strip, or past the end of its class).  Done once per row, not once per entry of W''.
+    for (int k = threadIdx.x; k < n_ksteps * 16; k += kDpThreads) {
+      const int ks = k >> 4, row = k & 15;
+      int g = 0, c = 0;
+      for (int gg = 0; gg < kMaxGroups; gg++)
+        for (int cc = 0; cc < 4; cc++)
+          if (ks >= S.run[gg][cc].kstep0 && S.run[gg][cc].n > 0) { g = gg; c = cc; }
+      const DmRun r = S.run[g][c];
+      const int kk = ks - r.kstep0;
+      const int first = T.class_first[c], cnt = T.class_first[c + 1] - first;
+      const int s_in = side_v ? r.first + 16 * kk + row : 2 * (r.first + 8 * kk + (row >> 1)) + (row & 1);
+      int ch = -1;
+      float coef = 0.f;
+      if (s_in < cnt) {
+        const int kx = first + s_in, chx = T.chan[kx];
+        if (chx >= g * gs && chx < (g + 1) * gs) {
+          ch = chx;
+          coef = (float)(1 << T.shift[kx]) / (float)((1 << T.width[chx]) - 1);
+        }
+      }
+      S.row_chan[k] = (int16_t)ch; S.row_coef[k] = coef;
+    }
     // ---- largest |W_dec|: the power of two that brings W'' into fp16's range
     {
       float m = 0.f;
@@ -268,9 +293,9 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
     {
       const float wscale = exp2f((float)(15 - wexp));
       for (int idx = threadIdx.x; idx < n_ksteps * 16 * kD; idx += kDpThreads) {
-        const int nn = idx & (kD - 1), row = (idx >> 7) & 15, ks = idx >> 11;
-        const int k = 16 * ks + row;
-        const float v = dm_b_value(S.run, T, wsrc, side_v, gs, ks, row, nn) * wscale;
+        const int nn = idx & (kD - 1), k = idx >> 7;       // operand row k = 16 k-step + slot
+        const int rch = S.row_chan[k];                   // (written before the two barriers above)
+        const float v = rch < 0 ? 0.f : wsrc[rch * kD + nn] * S.row_coef[k] * wscale;
         const int wo = (nn >> 3) * (16 * kDpK) + (k >> 3) * 128 + (k & 7) * 16 + (nn & 7) * 2;
         const __half hi = __float2half_rn(v);
         *reinterpret_cast<__half*>(&S.w[0][wo]) = hi;

@@ -56,27 +56,6 @@ __device__ inline void dm_build_runs(DmRun (*run)[4], int* kg, const StripTable&
   __syncthreads();
 }
 
-// Entry (row of k-step ks, output channel nn) of W'' before the fp16 scale: 2^shift W_dec[chan] / L, zero for a row
-// outside its run's group or past the end of its class.
-__device__ inline float dm_b_value(const DmRun (*run)[4], const StripTable& T, const float* __restrict__ wsrc, bool side_v,
-                                   int gs, int ks, int row, int nn) {
-  int g = 0, c = 0;
-#pragma unroll
-  for (int gg = 0; gg < kMaxGroups; gg++)
-#pragma unroll
-    for (int cc = 0; cc < 4; cc++)
-      if (ks >= run[gg][cc].kstep0 && run[gg][cc].n > 0) { g = gg; c = cc; }
-  const DmRun r = run[g][c];
-  const int kk = ks - r.kstep0;
-  const int first = T.class_first[c], cnt = T.class_first[c + 1] - first;
-  const int s_in = side_v ? r.first + 16 * kk + row : 2 * (r.first + 8 * kk + (row >> 1)) + (row & 1);
-  if (s_in >= cnt) return 0.f;
-  const int k = first + s_in, ch = T.chan[k];
-  if (ch < g * gs || ch >= (g + 1) * gs) return 0.f;
-  const float L = (float)((1 << T.width[ch]) - 1);
-  return wsrc[ch * kD + nn] * (float)(1 << T.shift[k]) / L;
-}
-
 // Units the tcgen05 kernel of decode_pairs.cuh takes (decode_tc_kernel takes the rest): at most two scale groups, at
 // most twelve k-steps, a tile that fits that kernel's slot, a source the bulk copy accepts.
 constexpr int kDpMaxKsteps = 12;
