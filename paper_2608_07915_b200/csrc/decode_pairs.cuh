@@ -29,6 +29,11 @@ constexpr int kDpK = kDpMaxKsteps * 16;               // strip positions of the 
 // fp16 A and B, fp32 D, A K-major, B MN-major, N = 128, M = 128
 constexpr uint32_t kDpIdesc = (1u << 4) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
+// An item of a builder warp's list (a unit's tiles all have the same items, so the list is made once per unit; see
+// dp_item): x = byte offset of the class in the tile | class << 14 | (unit stored alone + 1) << 16,
+// y = first unit | last unit of the run << 8 | first operand position << 16.
+constexpr int kDpMaxItems = 24;
+
 struct DecodePairSmem {
   StripTable tab;
   alignas(128) uint8_t w[2][kDpK * kD * 2];            // W'' = hi + lo (two fp16 parts): element (k, n) at (n / 8) * 16 K + (k / 8) * 128 + (k % 8) * 16 + (n % 8) * 2
@@ -40,6 +45,8 @@ struct DecodePairSmem {
   alignas(16) float cvec[kD];
   uint16_t meta[4][4][kTile];                          // lo16 and R16 of both groups of the last four tiles, kept for the epilogue
   DmRun run[kMaxGroups][4];
+  uint2 items[8][kDpMaxItems];                         // the builder warps' items (see dp_item)
+  int n_items[8];
   float row_coef[kDpK];                                // per operand row: 2^shift / L of its strip
   int16_t row_chan[kDpK];                              // its channel; -1: a zero row (another group's strip, or past its class)
   int kg[kMaxGroups + 1], wexp;
@@ -57,69 +64,63 @@ static_assert(sizeof(DecodePairSmem) + 128 <= 227 * 1024, "the reconstruction ke
 // Units past the end of the run (the padding of its last k-step) repeat the last unit: they meet zero rows of W'',
 // and the operand never holds anything but fields.
 template <int W, bool V>
-__device__ __forceinline__ int dp_run(const DmRun& r, const uint8_t* __restrict__ src, uint8_t* __restrict__ a, int first_item, int lane) {
+__device__ __forceinline__ void dp_item(int base, int u0, int last, int kpos0, int lone, const uint8_t* __restrict__ src,
+                                        uint8_t* __restrict__ a, int lane) {
   constexpr uint32_t FM = ((1u << W) - 1u) * (V ? 1u : 0x00010001u);
-  constexpr int PER_STEP = V ? 16 : 8;                       // units per k-step
   const int q = lane >> 2, pr = lane & 3;
-  const int nk = (r.n + PER_STEP - 1) / PER_STEP, last = r.first + r.n - 1;
-  const uint8_t* cb = src + r.base + 4 * ((q * W) >> 4);
+  const uint8_t* cb = src + base + 4 * ((q * W) >> 4);
   const int shq = (q * W) & 15;
   constexpr int US = V ? 16 * W : 32 * W;                    // bytes of a unit's stretch
-#pragma unroll 1
-  for (int item = first_item; item < nk * (PER_STEP / 4); item += 8) {
-    const int unit = min(r.first + 4 * item + pr, last);
-    const uint8_t* cp = cb + US * unit;
-    // operand position of the unit: K side 2 strips per unit
-    const int kpos = 16 * r.kstep0 + (V ? 1 : 2) * (4 * item + pr);
-    uint8_t* dst = a + (kpos >> 3) * 2048 + (kpos & 7) * 2 + q * 16;
-    uint32_t v[16];
-    if (!V && __any_sync(0xffffffffu, unit == r.lone)) {
-      // a strip stored alone sits among these four units: its words are half-words, the partner's half is zero
-      const bool mine = unit == r.lone;
-      const uint8_t* lp = src + r.base + US * unit + 2 * ((q * W) >> 4);
+  const int unit = min(u0 + pr, last);
+  const uint8_t* cp = cb + US * unit;
+  // operand position of the unit: K side 2 strips per unit
+  const int kpos = kpos0 + (V ? 1 : 2) * pr;
+  uint8_t* dst = a + (kpos >> 3) * 2048 + (kpos & 7) * 2 + q * 16;
+  uint32_t v[16];
+  if (!V && __any_sync(0xffffffffu, unit == lone)) {
+    // a strip stored alone sits among these four units: its words are half-words, the partner's half is zero
+    const bool mine = unit == lone;
+    const uint8_t* lp = src + base + US * unit + 2 * ((q * W) >> 4);
 #pragma unroll
-      for (int G = 0; G < 16; G++)
-        v[G] = mine ? (uint32_t)*reinterpret_cast<const uint16_t*>(lp + 2 * ((8 * G * W) >> 4))
-                    : *reinterpret_cast<const uint32_t*>(cp + 4 * ((8 * G * W) >> 4));
-    } else if (V) {
+    for (int G = 0; G < 16; G++)
+      v[G] = mine ? (uint32_t)*reinterpret_cast<const uint16_t*>(lp + 2 * ((8 * G * W) >> 4))
+                  : *reinterpret_cast<const uint32_t*>(cp + 4 * ((8 * G * W) >> 4));
+  } else if (V) {
 #pragma unroll
-      for (int G = 0; G < 16; G++)
-        v[G] = *reinterpret_cast<const uint32_t*>(cp + 4 * ((G >> 2) * W + (((8 * (G & 1)) * W) >> 4)));
-    } else {
-      // K side: the four units of a step sit a multiple of 64 bytes apart, so their words of one token group share
-      // banks.  Lane pr therefore walks the sixteen token groups in blocks of four in the order blk ^ pr: at every
-      // step the four units read different banks, and the stores (row = token) stay conflict-free in any order.
-      const uint8_t* cpb[4];
-      uint8_t* dstb[4];
+    for (int G = 0; G < 16; G++)
+      v[G] = *reinterpret_cast<const uint32_t*>(cp + 4 * ((G >> 2) * W + (((8 * (G & 1)) * W) >> 4)));
+  } else {
+    // K side: the four units of a step sit a multiple of 64 bytes apart, so their words of one token group share
+    // banks.  Lane pr therefore walks the sixteen token groups in blocks of four in the order blk ^ pr: at every
+    // step the four units read different banks, and the stores (row = token) stay conflict-free in any order.
+    const uint8_t* cpb[4];
+    uint8_t* dstb[4];
 #pragma unroll
-      for (int blk = 0; blk < 4; blk++) {
-        const int gb = 4 * (blk ^ pr);
-        cpb[blk] = cp + 4 * ((8 * gb * W) >> 4);
-        dstb[blk] = dst + gb * 128;
-      }
-#pragma unroll
-      for (int G = 0; G < 16; G++) v[G] = *reinterpret_cast<const uint32_t*>(cpb[G >> 2] + 4 * ((8 * (G & 3) * W) >> 4));
-#pragma unroll
-      for (int G = 0; G < 16; G++) {
-        const int sh = (8 * (G & 3) * W) & 15;
-        *reinterpret_cast<uint32_t*>(dstb[G >> 2] + (G & 3) * 128) = (v[G] >> (sh + shq)) & FM;
-      }
-      continue;
+    for (int blk = 0; blk < 4; blk++) {
+      const int gb = 4 * (blk ^ pr);
+      cpb[blk] = cp + 4 * ((8 * gb * W) >> 4);
+      dstb[blk] = dst + gb * 128;
     }
+#pragma unroll
+    for (int G = 0; G < 16; G++) v[G] = *reinterpret_cast<const uint32_t*>(cpb[G >> 2] + 4 * ((8 * (G & 3) * W) >> 4));
 #pragma unroll
     for (int G = 0; G < 16; G++) {
-      if (V) {
-        const int sh = 16 * ((G >> 1) & 1) + (((8 * (G & 1)) * W) & 15);
-        *reinterpret_cast<uint16_t*>(dst + G * 128) = (uint16_t)((v[G] >> (sh + shq)) & FM);
-      } else {
-        const int sh = (8 * G * W) & 15;
-        *reinterpret_cast<uint32_t*>(dst + G * 128) = (v[G] >> (sh + shq)) & FM;
-      }
+      const int sh = (8 * (G & 3) * W) & 15;
+      *reinterpret_cast<uint32_t*>(dstb[G >> 2] + (G & 3) * 128) = (v[G] >> (sh + shq)) & FM;
+    }
+    return;
+  }
+#pragma unroll
+  for (int G = 0; G < 16; G++) {
+    if (V) {
+      const int sh = 16 * ((G >> 1) & 1) + (((8 * (G & 1)) * W) & 15);
+      *reinterpret_cast<uint16_t*>(dst + G * 128) = (uint16_t)((v[G] >> (sh + shq)) & FM);
+    } else {
+      const int sh = (8 * G * W) & 15;
+      *reinterpret_cast<uint32_t*>(dst + G * 128) = (v[G] >> (sh + shq)) & FM;
     }
   }
-  return nk * (PER_STEP / 4);
 }
-
 // Bounded wait that sleeps between polls: the waiting warps share their schedulers with the working ones.
 __device__ __forceinline__ bool dp_wait(uint32_t bar, uint32_t parity) {
   uint32_t done = 0;
@@ -249,6 +250,27 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
     const int n_ksteps = S.kg[kMaxGroups];
     if (!dm_pairs_eligible(T, n_ksteps, unit_ptr)) continue;      // decode_tc_kernel takes this unit
     const int tile_bytes = T.tile_bytes;
+    // ---- the builder warps' item lists: four units (half a k-step on the K side, a quarter on the V side) per item,
+    // handed out round robin across the runs so that every warp gets the same number of them, give or take one
+    if (threadIdx.x < 8) {
+      const int w = threadIdx.x, per = side_v ? 16 : 8;
+      int done = 0, cnt = 0;
+      for (int g = 0; g < 2; g++)
+        for (int c = 0; c < 4; c++) {
+          const DmRun r = S.run[g][c];
+          if (r.n == 0) continue;
+          const int nit = (r.n + per - 1) / per * (per / 4);
+          for (int item = (w - done) & 7; item < nit; item += 8)
+            if (cnt < kDpMaxItems) {
+              S.items[w][cnt] = make_uint2((uint32_t)r.base | (uint32_t)c << 14 | (uint32_t)(r.lone + 1) << 16,
+                                           (uint32_t)(r.first + 4 * item) | (uint32_t)(r.first + r.n - 1) << 8 |
+                                               (uint32_t)(16 * r.kstep0 + (side_v ? 1 : 2) * 4 * item) << 16);
+              cnt++;
+            }
+          done += nit;
+        }
+      S.n_items[w] = cnt;
+    }
     // ---- the operand rows: row (k-step, slot) -> channel and 2^shift / L of its strip, or a zero row (another
     // group's strip, or past the end of its class).  Done once per row, not once per entry of W''.
     for (int k = threadIdx.x; k < n_ksteps * 16; k += kDpThreads) {
@@ -378,24 +400,22 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
         if (ok && i >= 1) ok = dp_wait(um_smem_u32(&S.acc_full[bf]), (uint32_t)((i - 1) & 1));
         if (!ok) { status |= SPECTRA_STATUS_WAIT_TIMEOUT; break; }
         const uint8_t* src = Hs.raw;
-        int done = 0;                                    // items handed out so far: the next run starts with the next warp
+        const int my_items = S.n_items[warp];
 #pragma unroll 1
-        for (int g = 0; g < 2; g++) {
-#pragma unroll 1
-          for (int c = 0; c < 4; c++) {
-            const DmRun r = S.run[g][c];
-            if (r.n == 0) continue;
-            if (side_v) {
-              if (c == 0) done += dp_run<8, true>(r, src, Hs.a, (warp - done) & 7, lane);
-              else if (c == 1) done += dp_run<4, true>(r, src, Hs.a, (warp - done) & 7, lane);
-              else if (c == 2) done += dp_run<2, true>(r, src, Hs.a, (warp - done) & 7, lane);
-              else done += dp_run<1, true>(r, src, Hs.a, (warp - done) & 7, lane);
-            } else {
-              if (c == 0) done += dp_run<8, false>(r, src, Hs.a, (warp - done) & 7, lane);
-              else if (c == 1) done += dp_run<4, false>(r, src, Hs.a, (warp - done) & 7, lane);
-              else if (c == 2) done += dp_run<2, false>(r, src, Hs.a, (warp - done) & 7, lane);
-              else done += dp_run<1, false>(r, src, Hs.a, (warp - done) & 7, lane);
-            }
+        for (int it = 0; it < my_items; it++) {
+          const uint2 e = S.items[warp][it];
+          const int base = (int)(e.x & 0x3fffu), c = (int)(e.x >> 14) & 3, lone = (int)(e.x >> 16) - 1;
+          const int u0 = (int)(e.y & 0xffu), last = (int)(e.y >> 8) & 0xff, kpos0 = (int)(e.y >> 16);
+          if (side_v) {
+            if (c == 0) dp_item<8, true>(base, u0, last, kpos0, lone, src, Hs.a, lane);
+            else if (c == 1) dp_item<4, true>(base, u0, last, kpos0, lone, src, Hs.a, lane);
+            else if (c == 2) dp_item<2, true>(base, u0, last, kpos0, lone, src, Hs.a, lane);
+            else dp_item<1, true>(base, u0, last, kpos0, lone, src, Hs.a, lane);
+          } else {
+            if (c == 0) dp_item<8, false>(base, u0, last, kpos0, lone, src, Hs.a, lane);
+            else if (c == 1) dp_item<4, false>(base, u0, last, kpos0, lone, src, Hs.a, lane);
+            else if (c == 2) dp_item<2, false>(base, u0, last, kpos0, lone, src, Hs.a, lane);
+            else dp_item<1, false>(base, u0, last, kpos0, lone, src, Hs.a, lane);
           }
         }
         // the tokens' group offsets and ranges, kept for the epilogue (the packed tile is handed back now)
@@ -435,8 +455,11 @@ __global__ void __launch_bounds__(kDpThreads, 1) decode_pair_kernel(DecodeArgs p
         const int bf = tt & 1, i = (bf ? base1 : base0) + (tt >> 1);
         const int tile = ga + tt, tile_pos = tile * kTile;
         const int n_here = min(n - tile_pos, kTile);
-        // a_full: the metadata of this tile are in place (the MMAs follow it, so this wait costs nothing)
-        ok = dp_wait(um_smem_u32(&S.a_full[bf]), (uint32_t)(i & 1)) && dp_wait(um_smem_u32(&S.acc_full[bf]), (uint32_t)(i & 1));
+        // The MMAs of this tile were issued after its operand and metadata were complete (a_full), so their completion
+        // says that the metadata are in place too.  a_full itself is not waited for here: the builders may already
+        // have completed it once more (for the tile after next, which only needs this tile's MMAs) before this
+        // warp looks, and a phase parity cannot tell that from "not yet".
+        ok = dp_wait(um_smem_u32(&S.acc_full[bf]), (uint32_t)(i & 1));
         if (!ok) { status |= SPECTRA_STATUS_WAIT_TIMEOUT; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int ms = (tiles_done + tt) & 3;
