@@ -32,6 +32,8 @@ constexpr uint32_t kDpIdesc = (1u << 4) | (1u << 16) | ((128u >> 3) << 17) | ((1
 // An item of a builder warp's list (a unit's tiles all have the same items, so the list is made once per unit; see
 // dp_item): x = byte offset of the class in the tile | class << 14 | (unit stored alone + 1) << 16,
 // y = first unit | last unit of the run << 8 | first operand position << 16.
+// A unit this kernel takes has at most twelve k-steps, i.e. 48 items (values side), handed out round robin over at most
+// eight runs: a warp gets at most 48 / 8 + 8 = 14 of them.
 constexpr int kDpMaxItems = 24;
 
 struct DecodePairSmem {
